@@ -1,0 +1,207 @@
+"""Pins for the oracle's log-prob gather, clipped surrogate (Eq. 1) and value loss (Eq. 4-5)."""
+import numpy as np
+import pytest
+import torch
+from scipy.special import logsumexp
+
+import oracle
+
+
+def make(rng, R=7, V=13, scale=2.0):
+    x = (scale * rng.standard_normal((R, V))).astype(np.float32)
+    y = rng.integers(0, V, R).astype(np.int32)
+    adv = rng.standard_normal(R).astype(np.float32)
+    lp = x[np.arange(R), y] - logsumexp(x.astype(np.float64), axis=1)
+    old = (lp + 0.25 * rng.standard_normal(R)).astype(np.float32)
+    return x, y, adv, old
+
+
+def test_logprob_against_scipy_and_normalisation():
+    rng = np.random.default_rng(0)
+    x, y, _, _ = make(rng, 9, 1001, 3.0)
+    lp = oracle.logprob(x, y)
+    ref = x[np.arange(9), y] - logsumexp(x.astype(np.float64), axis=1)
+    np.testing.assert_allclose(lp, ref, rtol=0, atol=1e-12)
+    # every column as target: probabilities sum to one
+    for r in range(2):
+        allp = [oracle.logprob(x[r:r + 1], np.array([v], np.int32))[0] for v in range(0, 1001)]
+        assert abs(np.exp(allp).sum() - 1.0) < 1e-12
+    # shift invariance and rows / strides
+    lp2 = oracle.logprob(x + np.float32(8.0), y)
+    np.testing.assert_allclose(lp2, lp, atol=1e-5)
+    rows = np.array([5, 0, 8], np.int32)
+    np.testing.assert_allclose(oracle.logprob(x, y, rows), ref[rows], atol=1e-12)
+    big = np.zeros((9, 1100), np.float32)
+    big[:, :1001] = x
+    np.testing.assert_allclose(oracle.logprob(big[:, :1001], y), ref, atol=1e-12)
+
+
+def test_logprob_bf16_and_extremes():
+    rng = np.random.default_rng(1)
+    xb = torch.from_numpy(2 * rng.standard_normal((4, 64)).astype(np.float32)).to(torch.bfloat16)
+    bits = xb.view(torch.int16).numpy().view(np.uint16)
+    y = rng.integers(0, 64, 4).astype(np.int32)
+    ref = torch.log_softmax(xb.double(), dim=1)[torch.arange(4), torch.from_numpy(y).long()]
+    np.testing.assert_allclose(oracle.logprob(bits, y), ref.numpy(), atol=1e-12)
+    x = np.full((1, 10), -1e4, np.float32)
+    x[0, 3] = 1e4
+    assert oracle.logprob(x, np.array([3], np.int32))[0] == pytest.approx(0.0, abs=1e-12)
+    assert oracle.logprob(x, np.array([4], np.int32))[0] == pytest.approx(-2e4)
+
+
+def torch_policy_loss(x, y, old, adv, el, eh, denom):
+    """Eq. 1 restated with autograd as an independent comparator (float64)."""
+    xt = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+    lp = torch.log_softmax(xt, dim=1)[torch.arange(len(y)), torch.tensor(y).long()]
+    rho = torch.exp(lp - torch.tensor(old, dtype=torch.float64))
+    A = torch.tensor(adv, dtype=torch.float64)
+    obj = torch.minimum(rho * A, torch.clamp(rho, 1 - el, 1 + eh) * A)
+    loss = -(obj.sum() / denom)
+    loss.backward()
+    return loss.item(), xt.grad.numpy(), (-obj).detach().numpy()
+
+
+@pytest.mark.parametrize("el,eh", [(0.2, 0.2), (0.2, 0.28), (1e9, 1e9)])
+def test_policy_loss_matches_autograd(el, eh):
+    rng = np.random.default_rng(2)
+    x, y, adv, old = make(rng, 40, 17)
+    out = oracle.policy_loss(x, y, None, None, old, adv, el, eh)
+    loss, grad, tl = torch_policy_loss(x, y, old, adv, el, eh, 40)
+    assert out["loss"] == pytest.approx(loss, rel=1e-12)
+    np.testing.assert_allclose(out["token_loss"], tl, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(out["dlogits"], grad, rtol=1e-10, atol=1e-14)
+    np.testing.assert_allclose(out["dlogits"].sum(axis=1), 0, atol=1e-14)
+    if el < 1:
+        assert out["clip_lo"] + out["clip_hi"] > 0          # the case does exercise the clip
+        rho = np.exp(out["logp"] - old)
+        lo = (rho < 1 - el) & (adv < 0)
+        hi = (rho > 1 + eh) & (adv > 0)
+        assert out["clip_lo"] == lo.sum() and out["clip_hi"] == hi.sum()
+        assert np.all(out["dlogits"][lo | hi] == 0)
+    else:
+        assert out["clip_lo"] == out["clip_hi"] == 0
+
+
+def test_policy_loss_finite_differences():
+    rng = np.random.default_rng(3)
+    x, y, adv, old = make(rng, 5, 8)
+    x = x.astype(np.float32)
+    out = oracle.policy_loss(x, y, None, None, old, adv, 0.2, 0.28)
+    rho = np.exp(out["logp"] - old)
+    assert np.all(np.abs(rho - 0.8) > 1e-3) and np.all(np.abs(rho - 1.28) > 1e-3)
+    h = 2.0 ** -10          # exactly representable perturbation of fp32 inputs
+    for r in range(5):
+        for v in range(8):
+            xp, xm = x.copy(), x.copy()
+            xp[r, v] += h
+            xm[r, v] -= h
+            assert xp[r, v] - xm[r, v] == 2 * h
+            lp = oracle.policy_loss(xp, y, None, None, old, adv, 0.2, 0.28, want_dlogits=False)["loss"]
+            lm = oracle.policy_loss(xm, y, None, None, old, adv, 0.2, 0.28, want_dlogits=False)["loss"]
+            fd = (lp - lm) / (2 * h)
+            assert out["dlogits"][r, v] == pytest.approx(fd, abs=2e-6)
+
+
+def test_policy_loss_on_policy_special_case_and_indexing():
+    rng = np.random.default_rng(4)
+    x, y, adv, _ = make(rng, 6, 11)
+    lp = oracle.logprob(x, y)
+    # old == new (to fp32 rounding): ratio 1, loss = -mean(A), gradient (A/n)(p - onehot)
+    out = oracle.policy_loss(x, y, None, None, lp.astype(np.float32), adv, 0.2, 0.2)
+    assert out["loss"] == pytest.approx(-adv.astype(float).mean(), rel=1e-6)
+    p = np.exp(x.astype(float) - logsumexp(x.astype(float), axis=1, keepdims=True))
+    onehot = np.eye(11)[y]
+    np.testing.assert_allclose(out["dlogits"], adv[:, None] / 6 * (p - onehot), rtol=1e-6, atol=1e-9)
+    # rows / aux_idx / denom
+    rows = np.array([4, 1], np.int32)
+    aux = np.array([9, 2], np.int32)
+    old_big = np.zeros(12, np.float32)
+    adv_big = np.zeros(12, np.float32)
+    old_big[aux] = lp[rows] + 0.1
+    adv_big[aux] = adv[rows]
+    o2 = oracle.policy_loss(x, y, rows, aux, old_big, adv_big, 0.2, 0.2, denom=10.0)
+    l, g, _ = torch_policy_loss(x[rows], y[rows], old_big[aux], adv_big[aux], 0.2, 0.2, 10.0)
+    assert o2["loss"] == pytest.approx(l, rel=1e-12)
+    np.testing.assert_allclose(o2["dlogits"], g, rtol=1e-10, atol=1e-14)
+
+
+def test_policy_loss_tie_on_clip_edge_keeps_gradient():
+    x = np.zeros((1, 4), np.float32)
+    y = np.array([0], np.int32)
+    lp = float(oracle.logprob(x, y)[0])
+    old = np.array([lp], np.float32)
+    # ratio is exp(lp - fp32(lp)): make eps so that the edge equals the ratio exactly
+    rho = np.exp(lp - float(old[0]))
+    out = oracle.policy_loss(x, y, None, None, old, np.array([1.0], np.float32), 1 - rho, rho - 1)
+    assert out["clip_lo"] == out["clip_hi"] == 0 and np.any(out["dlogits"] != 0)
+    out = oracle.policy_loss(x, y, None, None, old, np.zeros(1, np.float32), 0.2, 0.2)
+    assert out["loss"] == 0 and np.all(out["dlogits"] == 0)
+    out = oracle.policy_loss(x[:0], y[:0], None, None, old, old, 0.2, 0.2)
+    assert out["loss"] == 0.0
+
+
+def torch_value_loss(v, vo, R, idx, xl, xh, denom):
+    vt = torch.tensor(v, dtype=torch.float64, requires_grad=True)
+    vo = torch.tensor(vo, dtype=torch.float64)
+    R = torch.tensor(R, dtype=torch.float64)
+    ix = torch.tensor(idx).long()
+    vc = torch.maximum(torch.minimum(vt, vo + xh), vo - xl)
+    l = 0.5 * torch.maximum((vt - R) ** 2, (vc - R) ** 2)
+    loss = l[ix].sum() / denom
+    loss.backward()
+    return loss.item(), vt.grad.numpy()
+
+
+@pytest.mark.parametrize("xl,xh", [(0.5, 0.6), (0.05, 0.02), (1e9, 1e9)])
+def test_value_loss_matches_autograd_and_fd(xl, xh):
+    rng = np.random.default_rng(5)
+    N = 60
+    v = rng.standard_normal(N).astype(np.float32)
+    vo = (v + 0.3 * rng.standard_normal(N)).astype(np.float32)
+    R = rng.choice([-1.0, 1.0], N).astype(np.float32)
+    idx = np.sort(rng.choice(N, 25, replace=False)).astype(np.int32)
+    loss, dv = oracle.value_loss(v, vo, R, idx, xl, xh)
+    l, g = torch_value_loss(v, vo, R, idx, xl, xh, 25)
+    assert loss == pytest.approx(l, rel=1e-12)
+    np.testing.assert_allclose(dv, g, rtol=1e-12, atol=1e-15)
+    off = np.ones(N, bool)
+    off[idx] = False
+    assert np.all(dv[off] == 0)
+    if xl > 1e8:
+        assert loss == pytest.approx(0.5 * np.mean((v[idx].astype(float) - R[idx]) ** 2), rel=1e-12)
+        np.testing.assert_allclose(dv[idx], (v[idx].astype(float) - R[idx]) / 25, rtol=1e-12)
+    h = 2.0 ** -12
+    for p in idx[:8]:
+        vp, vm = v.copy(), v.copy()
+        vp[p] += h
+        vm[p] -= h
+        fd = (oracle.value_loss(vp, vo, R, idx, xl, xh)[0] - oracle.value_loss(vm, vo, R, idx, xl, xh)[0]) / (vp[p] - vm[p])
+        kink = min(abs(v[p] - (vo[p] - xl)), abs(v[p] - (vo[p] + xh)))
+        if kink > 2 * h:
+            assert dv[p] == pytest.approx(fd, abs=1e-4)
+
+
+def test_value_loss_empty_and_denominator():
+    v = np.array([0.3, -0.2], np.float32)
+    loss, dv = oracle.value_loss(v, v, v, np.zeros(0, np.int32), 0.5, 0.6)
+    assert loss == 0 and np.all(dv == 0)
+    loss, dv = oracle.value_loss(v, v, np.zeros(2, np.float32), np.array([1], np.int32), 0.5, 0.6, denom=4.0)
+    assert loss == pytest.approx(0.5 * float(v[1]) ** 2 / 4) and dv[1] == pytest.approx(float(v[1]) / 4)
+
+
+def test_lmhead_rows_equal_matmul():
+    rng = np.random.default_rng(6)
+    M, K, V = 5, 24, 40
+    H = torch.from_numpy(rng.standard_normal((M, K)).astype(np.float32)).to(torch.bfloat16)
+    W = torch.from_numpy(0.1 * rng.standard_normal((K, V)).astype(np.float32)).to(torch.bfloat16)
+    hb = H.view(torch.int16).numpy().view(np.uint16)
+    wb = W.view(torch.int16).numpy().view(np.uint16)
+    rows = np.array([3, 0], np.int32)
+    x = oracle.lmhead_logits_rows(hb, wb, rows)
+    ref = (H.double() @ W.double()).numpy()
+    np.testing.assert_allclose(x, ref[rows], rtol=1e-13, atol=1e-13)
+    dx = rng.standard_normal((M, V))
+    np.testing.assert_allclose(oracle.lmhead_dhidden_rows(dx, wb), dx @ W.double().numpy().T, rtol=1e-12, atol=1e-13)
+    cols = [7, 1, 39]
+    np.testing.assert_allclose(oracle.lmhead_dweight_cols(hb, dx[:, cols]),
+                               (H.double().numpy().T @ dx)[:, cols], rtol=1e-12, atol=1e-13)
