@@ -1,0 +1,223 @@
+/*
+ * tppo.h -- C ABI of the B200 (sm_100a) T-PPO token-selective update library.
+ *
+ * The library computes the part of a Truncated-PPO training step that the paper's method changes:
+ * EGAE advantages over possibly truncated responses (Section 3.1, Eq. 6), the policy / value
+ * token filter (Section 3.2), and the two losses restricted to the surviving tokens (Eq. 1 and
+ * Eq. 4-5, Algorithm 1 lines 6, 8, 9).
+ *
+ * Conventions that hold for every entry point
+ *   - Every array pointer is a DEVICE pointer unless the comment says "host".  The caller owns all
+ *     buffers, the workspace included; the library allocates nothing and keeps no state between
+ *     calls.  Scalars are passed by value.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work and return; they never
+ *     synchronise the stream or the device.
+ *   - Return value: a tppo_status.  Anything the host can detect (null pointer, negative size,
+ *     workspace too small, misalignment, unsupported shape) is reported before any kernel is
+ *     launched and leaves all outputs untouched.  Problems only the device can see (a target id
+ *     outside [0,V), an index outside its array, a scan wait that ran out) set bits of a status
+ *     word in the call's output and the affected outputs are written as 0 -- never NaN, never a
+ *     trap.
+ *   - Packed token layout: sequence i occupies positions [seq_begin[i], seq_begin[i+1]) laid out
+ *     prompt | response tokens of earlier windows | response tokens of this window.
+ *   - Workspace: query tppo_workspace_bytes() with the same sizes, pass at least that many bytes,
+ *     256-byte aligned.  Contents need no initialisation and are garbage afterwards.  Two calls
+ *     that may overlap on the GPU need different workspaces.
+ */
+#ifndef TPPO_H
+#define TPPO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TPPO_OK = 0,
+    TPPO_ERR_INVALID_ARG = 1, /* null / negative / inconsistent argument, bad alignment      */
+    TPPO_ERR_WORKSPACE = 2,   /* workspace pointer null, misaligned or smaller than required */
+    TPPO_ERR_UNSUPPORTED = 3, /* valid request this build cannot serve                       */
+    TPPO_ERR_CUDA = 4         /* a CUDA runtime call failed (launch error, wrong device)     */
+} tppo_status;
+
+/* bits of the device status word */
+enum {
+    TPPO_DEV_BAD_TARGET = 1,  /* targets[row] outside [0, V): that row contributes nothing   */
+    TPPO_DEV_WAIT_TIMEOUT = 2,/* a bounded look-back wait gave up: outputs incomplete        */
+    TPPO_DEV_BAD_INDEX = 4,   /* a row / token index outside its array: entry skipped        */
+    TPPO_DEV_BAD_SEGMENT = 8  /* segment bounds outside [0, N] or not ascending: skipped     */
+};
+
+typedef enum {
+    TPPO_OP_EGAE = 0,
+    TPPO_OP_SELECT_TOKENS = 1,
+    TPPO_OP_POLICY_LOSS = 2,
+    TPPO_OP_VALUE_LOSS = 3,
+    TPPO_OP_LMHEAD = 4
+} tppo_op;
+
+/* logits element types */
+enum { TPPO_BF16 = 0, TPPO_F32 = 1 };
+
+/* where the gradient with respect to the logits goes */
+enum {
+    TPPO_DLOGITS_NONE = 0,    /* forward only (e.g. old-policy log-probs, Algorithm 1 line 3) */
+    TPPO_DLOGITS_FULL = 1,    /* [R, ld] like the logits; rows that are not selected are     */
+                              /* zero-filled; may be the logits buffer itself (in place)     */
+    TPPO_DLOGITS_COMPACT = 2  /* [n_max, V] dense, row j belongs to the j-th selected row    */
+};
+
+/* Library version (major*10000 + minor*100 + patch). Host call. */
+int tppo_version(void);
+
+/* Human-readable name of a status code (static string, host). */
+const char *tppo_status_string(int status);
+
+/*
+ * Workspace bytes needed by one call of `op`.  N = packed tokens, B = sequences / segments,
+ * n_max = capacity of the selected-token list, V = vocabulary (0 where it does not apply).
+ * Returns 0 for an unknown op.  Host call, launches nothing.
+ */
+size_t tppo_workspace_bytes(int op, int64_t N, int32_t B, int64_t n_max, int32_t V);
+
+/*
+ * EGAE advantages and Monte-Carlo returns (Section 3.1, Eq. 6 with the TD residual of Eq. 3;
+ * R_t as defined after Eq. 5; Algorithm 1 line 6).
+ *
+ * For each response segment [seg_begin[i], seg_end[i]) of the packed arrays, backwards in t:
+ *     delta_t = rewards[t] + gamma * V(s_{t+1}) - values[t]
+ *     A_t     = delta_t + gamma*lambda * A_{t+1},   A_end = 0
+ *     R_t     = rewards[t] + gamma * R_{t+1},       R_end = 0
+ * where V(s_{t+1}) = values[t+1] inside the segment and, after the last token, 0 if the response
+ * finished, else bootstrap[i] -- or, when bootstrap is NULL, values[seg_end[i]-1], the paper's
+ * assumption V(s_l) = V(s_{l-1}) for a response cut at the window length l.
+ *
+ *   rewards, values  [N] fp32      seg_begin, seg_end  [B] int32, ascending, disjoint,
+ *   truncated        [B] u8                            0 <= begin <= end <= N (empty allowed)
+ *   bootstrap        [B] fp32 or NULL
+ *   advantages       [N] fp32 out; returns [N] fp32 out or NULL.  Positions outside every
+ *                    segment are written 0.
+ *   status           [1] int32 out: device status bits (0 = clean).
+ * Sums are carried in fp64 and rounded once to fp32 on store.  N < 2^31.
+ */
+int tppo_egae(const float *rewards, const float *values,
+              const int32_t *seg_begin, const int32_t *seg_end,
+              const uint8_t *truncated, const float *bootstrap,
+              int32_t B, int64_t N, float gamma, float lambda,
+              float *advantages, float *returns, int32_t *status,
+              void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Token filter and compaction (Section 3.2; "selective filtering of prompt and truncated tokens").
+ * With o = p - seq_begin[i] for the sequence i that holds position p:
+ *   policy token  iff  prompt_len[i]+prev_len[i] <= o < prompt_len[i]+prev_len[i]+new_len[i]
+ *                                                       - (truncated[i] ? tail_drop : 0)
+ *                      (response tokens generated in the current step, finished or not, minus
+ *                      the last tail_drop tokens of an unfinished sequence)
+ *   value token   iff  !truncated[i] and prompt_len[i] <= o < prompt_len[i]+prev_len[i]+new_len[i]
+ *                      (all generated tokens of finished sequences)
+ * each ANDed with the optional byte masks (non-zero = keep).  Prompt tokens are in neither set.
+ *
+ *   seq_begin [B+1] int32 ascending; prompt_len, prev_len, new_len [B] int32 >= 0; truncated [B] u8
+ *   extra_policy_mask, extra_value_mask  [N] u8 or NULL
+ *   policy_idx, value_idx  [N] int32 out: selected positions in ascending order (bit-exact,
+ *                          run-to-run deterministic); entries past the count are untouched
+ *   counts   [4] int32 out: n_policy, n_value, device status bits, 0
+ * The counts stay on the device so that the loss calls can consume them without a host round trip.
+ */
+int tppo_select_tokens(const int32_t *seq_begin, const int32_t *prompt_len,
+                       const int32_t *prev_len, const int32_t *new_len,
+                       const uint8_t *truncated, int32_t tail_drop,
+                       const uint8_t *extra_policy_mask, const uint8_t *extra_value_mask,
+                       int32_t B, int64_t N,
+                       int32_t *policy_idx, int32_t *value_idx, int32_t *counts,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Fused per-token log-softmax gather + clipped PPO surrogate, forward and backward to the logits
+ * (Eq. 1 with decoupled eps_low / eps_high; token-level mean and no KL term per Section 4.1.1;
+ * Algorithm 1 line 8).  For the j-th selected row r = rows[j] (j < n), a = aux_idx[j]:
+ *     logp_j = x[r, y] - log sum_v exp(x[r, v]),            y = targets[r]
+ *     rho    = exp(logp_j - old_logp[a])
+ *     l_j    = -min(rho*adv[a], clip(rho, 1-eps_low, 1+eps_high)*adv[a])
+ *     loss   = (1/denom) * sum_j l_j
+ *     dlogits[., v] = (adv[a]*rho*active/denom) * (softmax_v - 1[v == y])
+ * with active = 0 exactly when the clipped term is strictly the smaller one (the gradient is then
+ * zero), and n = min(*n_sel, n_max).  Each selected logits row is read once from HBM.
+ *
+ *   logits    [R, ld] elements of logits_dtype (TPPO_BF16 or TPPO_F32), row stride ld >= V
+ *   targets   [R] int32: the token scored by logits row r (the caller applies the next-token shift)
+ *   rows      [n_max] int32 distinct row indices, or NULL for 0..n_max-1
+ *   n_sel     [1] int32 device count (e.g. counts+0 of tppo_select_tokens) or NULL for n_max
+ *   aux_idx   [n_max] int32 index into old_logp / adv, or NULL to use the row index
+ *   old_logp, adv   fp32, length aux_len (bounds-checked against it)
+ *   denom     > 0: divisor of the mean (gradient accumulation / several GPUs); <= 0: n
+ *   logp, token_loss  [n_max] fp32 out, compact, either may be NULL
+ *   loss      [1] fp32 out
+ *   stats     [4] int32 out: n, rows clipped at the lower edge, at the upper edge, status bits
+ *   dlogits   per dlogits_mode (same element type as the logits); FULL mode may alias `logits`
+ *   kernel_hint  0 = choose automatically; other values select a specific kernel for tuning and
+ *                testing and never change the result beyond rounding (see tppo_policy_kernels)
+ * Zero selected rows give loss 0 and no gradient writes beyond FULL mode's zero fill.
+ * Reductions are done in a fixed order: results are run-to-run identical.
+ */
+int tppo_policy_loss_fwd_bwd(const void *logits, int32_t logits_dtype,
+                             int64_t R, int32_t V, int64_t ld,
+                             const int32_t *targets,
+                             const int32_t *rows, const int32_t *n_sel, int64_t n_max,
+                             const int32_t *aux_idx,
+                             const float *old_logp, const float *adv, int64_t aux_len,
+                             float eps_low, float eps_high, float denom,
+                             float *logp, float *token_loss, float *loss, int32_t *stats,
+                             void *dlogits, int32_t dlogits_mode, int32_t kernel_hint,
+                             void *workspace, size_t workspace_bytes, void *stream);
+
+/* kernel_hint values of tppo_policy_loss_fwd_bwd */
+enum {
+    TPPO_POLICY_AUTO = 0,
+    TPPO_POLICY_TWO_PASS = 1,     /* any shape / dtype: row read twice from global memory      */
+    TPPO_POLICY_CLUSTER_SMEM = 2  /* bf16, V % 8 == 0, 16-byte aligned rows: row held in the    */
+                                  /* shared memory of a thread-block cluster, read once         */
+};
+
+/*
+ * Clipped value regression on the value tokens, forward and backward (Eq. 4-5; Algorithm 1
+ * line 9).  For p = value_idx[j], j < n = min(*n_sel, n_max):
+ *     Vc = clip(values[p], old_values[p] - xi_low, old_values[p] + xi_high)
+ *     l  = 1/2 * max((values[p]-returns[p])^2, (Vc-returns[p])^2),   loss = (1/denom) sum l
+ *     dvalues[p] = (values[p]-returns[p])/denom  if the unclipped term is the max (ties included),
+ *                  else (Vc-returns[p])/denom if Vc == values[p], else 0
+ *   values, old_values, returns [N] fp32; value_idx [n_max] int32 (distinct) or NULL for 0..n_max-1
+ *   loss [1] fp32 out; dvalues [N] fp32 out (zero off the value tokens) or NULL
+ *   stats [2] int32 out: n, status bits
+ */
+int tppo_value_loss(const float *values, const float *old_values, const float *returns,
+                    int64_t N, const int32_t *value_idx, const int32_t *n_sel, int64_t n_max,
+                    float xi_low, float xi_high, float denom,
+                    float *loss, float *dvalues, int32_t *stats,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * LM-head variant of the fused policy loss: the logits x = hidden * weight are a dense
+ * [M,K] x [K,V] contraction on the tensor cores and are never written to memory; outputs are the
+ * loss, the log-probs and the gradients dhidden = dX * weight^T and dweight = hidden^T * dX.
+ * (Math as tppo_policy_loss_fwd_bwd with all M rows selected.)  Returns TPPO_ERR_UNSUPPORTED in
+ * builds without the tensor-core kernel.
+ *   hidden [M,K] bf16, weight [K,V] bf16, targets [M], aux_idx [M] or NULL, old_logp/adv fp32
+ *   dhidden [M,K] bf16 out, dweight [K,V] bf16 out
+ */
+int tppo_lmhead_logprob_fwd_bwd(const void *hidden, const void *weight,
+                                int64_t M, int32_t K, int32_t V,
+                                const int32_t *targets, const int32_t *aux_idx,
+                                const float *old_logp, const float *adv, int64_t aux_len,
+                                float eps_low, float eps_high, float denom,
+                                float *logp, float *token_loss, float *loss, int32_t *stats,
+                                void *dhidden, void *dweight,
+                                void *workspace, size_t workspace_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TPPO_H */

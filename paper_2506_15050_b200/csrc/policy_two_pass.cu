@@ -1,0 +1,192 @@
+// General-shape policy-loss kernel: one thread block per selected row, the row is read twice from
+// global memory (the second read usually hits L2).  Serves fp32 logits, vocabulary sizes and row
+// strides that the shared-memory-resident kernel cannot take, and small problems.
+//   pass 1: per-thread online max / sum-of-exponentials, block combine  -> log-sum-exp
+//   scalar: Eq. 1 ratio, clip, loss term, gradient factor
+//   pass 2: gradient factor * (softmax - onehot) written in the logits' element type
+#include "policy_common.cuh"
+
+namespace tppo {
+
+constexpr int kTwoPassThreads = 512;
+
+template <int DT> struct ElemT;
+template <> struct ElemT<TPPO_BF16> { using type = uint16_t; };
+template <> struct ElemT<TPPO_F32> { using type = float; };
+
+__device__ __forceinline__ float load_elem(const uint16_t* p) { return __uint_as_float(uint32_t(*p) << 16); }
+__device__ __forceinline__ float load_elem(const float* p) { return *p; }
+__device__ __forceinline__ void store_elem(uint16_t* p, float v) {
+    *p = uint16_t(pack_bf16x2(v, 0.f) & 0xffffu);
+}
+__device__ __forceinline__ void store_elem(float* p, float v) { *p = v; }
+
+// 8 consecutive elements from a 16-byte aligned address
+__device__ __forceinline__ void load8(const uint16_t* p, float (&x)[8]) {
+    const uint4 w = *reinterpret_cast<const uint4*>(p);
+    x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);
+    x[4] = bf16_lo(w.z); x[5] = bf16_hi(w.z); x[6] = bf16_lo(w.w); x[7] = bf16_hi(w.w);
+}
+__device__ __forceinline__ void load8(const float* p, float (&x)[8]) {
+    const float4 a = *reinterpret_cast<const float4*>(p);
+    const float4 b = *reinterpret_cast<const float4*>(p + 4);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+}
+__device__ __forceinline__ void store8(uint16_t* p, const float (&g)[8]) {
+    uint4 w;
+    w.x = pack_bf16x2(g[0], g[1]); w.y = pack_bf16x2(g[2], g[3]);
+    w.z = pack_bf16x2(g[4], g[5]); w.w = pack_bf16x2(g[6], g[7]);
+    *reinterpret_cast<uint4*>(p) = w;
+}
+__device__ __forceinline__ void store8(float* p, const float (&g)[8]) {
+    *reinterpret_cast<float4*>(p) = make_float4(g[0], g[1], g[2], g[3]);
+    *reinterpret_cast<float4*>(p + 4) = make_float4(g[4], g[5], g[6], g[7]);
+}
+
+// running (max, sum of 2^(x*log2e - max*log2e)) update with n new values
+template <int N>
+__device__ __forceinline__ void online_update(float& m, float& s, const float (&x)[N]) {
+    float mx = x[0];
+#pragma unroll
+    for (int k = 1; k < N; ++k) mx = fmaxf(mx, x[k]);
+    const float m_new = fmaxf(m, mx);
+    const float off = m_new * kLog2e;
+    float acc = s * ex2(fmaf(m, kLog2e, -off));
+#pragma unroll
+    for (int k = 0; k < N; ++k) acc += ex2(fmaf(x[k], kLog2e, -off));
+    m = m_new;
+    s = acc;
+}
+
+template <int DT, bool VEC>
+__global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const PolicyArgs a) {
+    using T = typename ElemT<DT>::type;
+    __shared__ float s_m[kTwoPassThreads / 32], s_s[kTwoPassThreads / 32];
+    __shared__ float s_lse, s_coef;
+
+    const int64_t n = policy_n(a);
+    const float inv_denom = policy_inv_denom(a, n);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const T* logits = static_cast<const T*>(a.logits);
+    T* dl = static_cast<T*>(a.dlogits);
+
+    for (int64_t j = blockIdx.x; j < n; j += gridDim.x) {
+        const RowMeta meta = policy_row_meta(a, j);
+        const T* x_row = logits + (meta.row_ok ? meta.row : 0) * a.ld;
+        T* g_row = nullptr;
+        if (a.mode == TPPO_DLOGITS_FULL && meta.row_ok) g_row = dl + meta.row * a.ld;
+        if (a.mode == TPPO_DLOGITS_COMPACT) g_row = dl + j * int64_t(a.V);
+
+        float coef = 0.f, lse = 0.f;
+        if (meta.ok) {
+            // ---- pass 1 -------------------------------------------------------------------
+            float m = -1.0e30f, s = 0.f;
+            if (VEC) {
+                const int nu = a.V >> 3;
+                for (int u = tid; u < nu; u += kTwoPassThreads) {
+                    float x[8];
+                    load8(x_row + (int64_t(u) << 3), x);
+                    online_update<8>(m, s, x);
+                }
+                for (int v = (nu << 3) + tid; v < a.V; v += kTwoPassThreads) {
+                    float x[1] = {load_elem(x_row + v)};
+                    online_update<1>(m, s, x);
+                }
+            } else {
+                for (int v = tid; v < a.V; v += kTwoPassThreads) {
+                    float x[1] = {load_elem(x_row + v)};
+                    online_update<1>(m, s, x);
+                }
+            }
+            const float wm = warp_max(m);
+            s = warp_sum(s * ex2((m - wm) * kLog2e));
+            if (lane == 0) { s_m[warp] = wm; s_s[warp] = s; }
+            __syncthreads();
+            if (tid == 0) {
+                float M = s_m[0];
+                for (int w = 1; w < kTwoPassThreads / 32; ++w) M = fmaxf(M, s_m[w]);
+                float S = 0.f;
+                for (int w = 0; w < kTwoPassThreads / 32; ++w) S += s_s[w] * ex2((s_m[w] - M) * kLog2e);
+                const float l = M + logf(S);
+                const RowLoss rl = ppo_row(load_elem(x_row + meta.y), l, __ldg(a.old_logp + meta.aux),
+                                           __ldg(a.adv + meta.aux), a.eps_low, a.eps_high, inv_denom);
+                if (a.logp) a.logp[j] = rl.logp;
+                if (a.token_loss) a.token_loss[j] = rl.loss;
+                a.row_loss[j] = rl.loss;
+                a.row_clip[j] = uint8_t(rl.clip);
+                s_lse = l;
+                s_coef = rl.coef;
+            }
+            __syncthreads();
+            coef = s_coef;
+            lse = s_lse;
+        } else if (tid == 0) {
+            atomicOr(a.stats + 3, policy_bad_bits(meta, a));
+            if (a.logp) a.logp[j] = 0.f;
+            if (a.token_loss) a.token_loss[j] = 0.f;
+            a.row_loss[j] = 0.f;
+            a.row_clip[j] = 0;
+        }
+
+        // ---- pass 2 -----------------------------------------------------------------------
+        if (g_row) {
+            const float off = lse * kLog2e;
+            if (coef == 0.f) {   // clipped, zero advantage or invalid entry: the gradient row is zero
+                if (VEC) {
+                    const int nu = a.V >> 3;
+                    const float z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                    for (int u = tid; u < nu; u += kTwoPassThreads) store8(g_row + (int64_t(u) << 3), z);
+                    for (int v = (nu << 3) + tid; v < a.V; v += kTwoPassThreads) store_elem(g_row + v, 0.f);
+                } else {
+                    for (int v = tid; v < a.V; v += kTwoPassThreads) store_elem(g_row + v, 0.f);
+                }
+            } else if (VEC) {
+                const int nu = a.V >> 3;
+                const int yu = meta.y >> 3, yk = meta.y & 7;
+                for (int u = tid; u < nu; u += kTwoPassThreads) {
+                    float x[8], g[8];
+                    load8(x_row + (int64_t(u) << 3), x);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) g[k] = coef * ex2(fmaf(x[k], kLog2e, -off));
+                    if (u == yu) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) if (k == yk) g[k] -= coef;
+                    }
+                    store8(g_row + (int64_t(u) << 3), g);
+                }
+                for (int v = (nu << 3) + tid; v < a.V; v += kTwoPassThreads) {
+                    float g = coef * ex2(fmaf(load_elem(x_row + v), kLog2e, -off));
+                    if (v == meta.y) g -= coef;
+                    store_elem(g_row + v, g);
+                }
+            } else {
+                for (int v = tid; v < a.V; v += kTwoPassThreads) {
+                    float g = coef * ex2(fmaf(load_elem(x_row + v), kLog2e, -off));
+                    if (v == meta.y) g -= coef;
+                    store_elem(g_row + v, g);
+                }
+            }
+        }
+        __syncthreads();   // s_lse / s_coef are reused by the next row
+    }
+}
+
+int launch_policy_two_pass(const PolicyArgs& a, int dtype, cudaStream_t s) {
+    int64_t blocks = a.n_max < 1 ? 1 : a.n_max;
+    if (blocks > kNumSms * 3) blocks = kNumSms * 3;
+    const size_t esz = dtype == TPPO_BF16 ? 2 : 4;
+    bool vec = aligned(a.logits, 16) && (a.ld * esz) % 16 == 0;
+    if (a.mode == TPPO_DLOGITS_FULL) vec = vec && aligned(a.dlogits, 16);
+    if (a.mode == TPPO_DLOGITS_COMPACT)
+        vec = vec && aligned(a.dlogits, 16) && (int64_t(a.V) * esz) % 16 == 0;
+    if (dtype == TPPO_BF16) {
+        if (vec) policy_two_pass_kernel<TPPO_BF16, true><<<int(blocks), kTwoPassThreads, 0, s>>>(a);
+        else policy_two_pass_kernel<TPPO_BF16, false><<<int(blocks), kTwoPassThreads, 0, s>>>(a);
+    } else {
+        if (vec) policy_two_pass_kernel<TPPO_F32, true><<<int(blocks), kTwoPassThreads, 0, s>>>(a);
+        else policy_two_pass_kernel<TPPO_F32, false><<<int(blocks), kTwoPassThreads, 0, s>>>(a);
+    }
+    return cudaGetLastError() == cudaSuccess ? TPPO_OK : TPPO_ERR_CUDA;
+}
+
+}  // namespace tppo

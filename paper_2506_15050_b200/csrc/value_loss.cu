@@ -1,0 +1,110 @@
+// Clipped value regression on the value tokens, forward and backward (Eq. 4-5 of the paper;
+// Algorithm 1 line 9).  A gather over value_idx: 3 fp32 reads + 1 index read + 1 gradient write
+// per value token.  The mean is reduced in a fixed order (per-thread strided partials in fp64,
+// fixed shuffle tree, per-block partials summed by one block), so results are run-to-run
+// identical.
+#include "common.cuh"
+
+namespace tppo {
+
+constexpr int kValThreads = 256;
+constexpr int kValMaxBlocks = kNumSms * 4;
+
+struct ValueArgs {
+    const float* values;
+    const float* old_values;
+    const float* returns;
+    const int32_t* value_idx;
+    const int32_t* n_sel;
+    int64_t n_max;
+    int64_t N;
+    float xi_low, xi_high, denom;
+    float* loss;
+    float* dvalues;
+    int32_t* stats;       // [2]: n, status bits
+    double* partial;      // [gridDim.x]
+    uint32_t* done;       // [1] blocks finished
+};
+
+__global__ void __launch_bounds__(kValThreads) value_loss_kernel(const ValueArgs a) {
+    __shared__ double s_red[kValThreads / 32];
+    __shared__ bool s_last;
+    int64_t n = a.n_max;
+    if (a.n_sel) { const int64_t c = *a.n_sel; n = c < 0 ? 0 : (c < n ? c : n); }
+    const double d = a.denom > 0.f ? double(a.denom) : double(n > 0 ? n : 1);
+    const float inv_d = float(1.0 / d);
+
+    double acc = 0.0;
+    bool bad = false;
+    for (int64_t j = int64_t(blockIdx.x) * kValThreads + threadIdx.x; j < n;
+         j += int64_t(gridDim.x) * kValThreads) {
+        const int64_t p = a.value_idx ? int64_t(__ldg(a.value_idx + j)) : j;
+        if (p < 0 || p >= a.N) { bad = true; continue; }
+        const float v = __ldg(a.values + p), vo = __ldg(a.old_values + p), R = __ldg(a.returns + p);
+        const float vc = fminf(fmaxf(v, vo - a.xi_low), vo + a.xi_high);
+        const float e1 = (v - R) * (v - R), e2 = (vc - R) * (vc - R);
+        float g;
+        if (e1 >= e2) { acc += 0.5 * double(e1); g = v - R; }
+        else { acc += 0.5 * double(e2); g = (vc == v) ? (vc - R) : 0.f; }
+        if (a.dvalues) a.dvalues[p] = g * inv_d;
+    }
+    if (bad) atomicOr(a.stats + 1, TPPO_DEV_BAD_INDEX);
+    acc = warp_sum(acc);
+    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < kValThreads / 32; ++w) t += s_red[w];
+        a.partial[blockIdx.x] = t;
+        __threadfence();
+        s_last = atomicAdd(a.done, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (s_last && threadIdx.x == 0) {   // the last block to finish adds the partials in order
+        __threadfence();
+        double t = 0.0;
+        for (unsigned b = 0; b < gridDim.x; ++b) t += reinterpret_cast<volatile double*>(a.partial)[b];
+        *a.loss = n > 0 ? float(t / d) : 0.f;
+        a.stats[0] = int32_t(n);
+    }
+}
+
+size_t value_workspace_bytes() {
+    return align_up(sizeof(uint32_t), kWsAlign) + align_up(sizeof(double) * kValMaxBlocks, kWsAlign);
+}
+
+}  // namespace tppo
+
+using namespace tppo;
+
+TPPO_API int tppo_value_loss(const float* values, const float* old_values, const float* returns,
+                             int64_t N, const int32_t* value_idx, const int32_t* n_sel,
+                             int64_t n_max, float xi_low, float xi_high, float denom, float* loss,
+                             float* dvalues, int32_t* stats, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    if (N < 0 || n_max < 0 || N >= (int64_t(1) << 31) || !loss || !stats)
+        return TPPO_ERR_INVALID_ARG;
+    if (n_max > 0 && (!values || !old_values || !returns)) return TPPO_ERR_INVALID_ARG;
+    if (!value_idx && n_max > N) return TPPO_ERR_INVALID_ARG;
+    if (!(xi_low >= 0.f) || !(xi_high >= 0.f)) return TPPO_ERR_INVALID_ARG;
+    const size_t need = value_workspace_bytes();
+    if (!workspace || workspace_bytes < need || !aligned(workspace, kWsAlign))
+        return TPPO_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    TPPO_CUDA_CHECK(cudaMemsetAsync(stats, 0, 2 * sizeof(int32_t), s));
+    TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0, sizeof(uint32_t), s));
+    if (dvalues && N > 0) TPPO_CUDA_CHECK(cudaMemsetAsync(dvalues, 0, size_t(N) * sizeof(float), s));
+    ValueArgs a;
+    a.values = values; a.old_values = old_values; a.returns = returns; a.value_idx = value_idx;
+    a.n_sel = n_sel; a.n_max = n_max; a.N = N; a.xi_low = xi_low; a.xi_high = xi_high;
+    a.denom = denom; a.loss = loss; a.dvalues = dvalues; a.stats = stats;
+    a.done = static_cast<uint32_t*>(workspace);
+    a.partial = reinterpret_cast<double*>(static_cast<char*>(workspace) +
+                                          align_up(sizeof(uint32_t), kWsAlign));
+    int64_t blocks = (n_max + kValThreads - 1) / kValThreads;
+    if (blocks < 1) blocks = 1;
+    if (blocks > kValMaxBlocks) blocks = kValMaxBlocks;
+    value_loss_kernel<<<int(blocks), kValThreads, 0, s>>>(a);
+    TPPO_CUDA_CHECK(cudaGetLastError());
+    return TPPO_OK;
+}

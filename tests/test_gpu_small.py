@@ -1,0 +1,404 @@
+"""GPU parity: CUDA path (through the C ABI) against the float64 oracle, element by element, on
+small seeded inputs that still span several tiles, ragged tails and the edge cases."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_15050_b200 import synth
+from gpu_util import DEV, adv_close, dev, run_egae, run_policy, run_select, run_value
+
+pytestmark = pytest.mark.gpu
+
+LOGP_ATOL = 2e-3       # per-token log-probs and losses from bf16 logits, fp32 accumulation
+ADV_RTOL = 1e-5        # fp32 advantages
+
+
+def f32(x):
+    return float(np.float32(x))
+
+
+# ------------------------------------------------------------------------------------------------
+# selection
+# ------------------------------------------------------------------------------------------------
+def check_select(c, tail_drop=0, pm=None, vm=None):
+    pol, val, cn = run_select(c, tail_drop, pm, vm)
+    rp, rv = oracle.select_tokens(c["seq_begin"], c["prompt_len"], c["prev_len"], c["new_len"],
+                                  c["truncated"], tail_drop, pm, vm)
+    assert cn[2] == 0
+    assert cn[0] == len(rp) and cn[1] == len(rv)
+    assert np.array_equal(pol, rp) and np.array_equal(val, rv)
+    return cn
+
+
+def test_select_config1():
+    cn = check_select(synth.config1())
+    assert cn[0] == 170 and cn[1] == 42
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_select_random_multi_tile(seed):
+    rng = np.random.default_rng(seed)
+    B = int(rng.integers(1, 60))
+    prompt = rng.integers(0, 300, B)
+    prev = rng.integers(0, 500, B) * rng.integers(0, 2, B)
+    new = rng.integers(0, 700, B)
+    trunc = rng.integers(0, 2, B).astype(np.uint8)
+    sb, _, _ = synth.pack(prompt, prev, new)
+    c = dict(seq_begin=sb, prompt_len=prompt, prev_len=prev, new_len=new, truncated=trunc)
+    N = int(sb[-1])
+    check_select(c, tail_drop=int(rng.integers(0, 40)))
+    pm = rng.integers(0, 2, max(N, 1)).astype(np.uint8)
+    vm = rng.integers(0, 2, max(N, 1)).astype(np.uint8)
+    check_select(c, 3, pm, vm)
+    check_select(c, 0, pm, None)
+
+
+def test_select_edge_cases():
+    z = np.zeros(1, np.int32)
+    # one sequence, everything selected; all truncated; all prompt; empty sequences; tile-aligned end
+    for prompt, prev, new, trunc in [([0], [0], [4096], [0]), ([0], [0], [8192], [1]),
+                                     ([5000], [0], [0], [0]), ([0, 0, 3], [0, 0, 0], [0, 0, 1], [0, 1, 0]),
+                                     ([1], [4094], [1], [0]), ([7], [0], [1], [1])]:
+        sb, _, _ = synth.pack(prompt, prev, new)
+        c = dict(seq_begin=sb, prompt_len=np.array(prompt), prev_len=np.array(prev),
+                 new_len=np.array(new), truncated=np.array(trunc, np.uint8))
+        check_select(c)
+        check_select(c, tail_drop=2)
+
+
+def test_select_run_to_run_identical_and_config4():
+    c = synth.config4(B=600, hi=32768)
+    a1 = run_select(c, 16, c["extra_policy_mask"], c["extra_value_mask"])
+    a2 = run_select(c, 16, c["extra_policy_mask"], c["extra_value_mask"])
+    assert np.array_equal(a1[0], a2[0]) and np.array_equal(a1[1], a2[1])
+    check_select(c, 16, c["extra_policy_mask"], c["extra_value_mask"])
+    check_select(c, 0)
+
+
+# ------------------------------------------------------------------------------------------------
+# EGAE
+# ------------------------------------------------------------------------------------------------
+def check_egae(B, r, v, sb, se, tr, boot, gamma, lam):
+    adv, ret, status = run_egae(B, r, v, sb, se, tr, boot, gamma, lam)
+    ra, rr = oracle.egae(r, v, sb, se, tr, boot, f32(gamma), f32(lam))
+    assert status == 0
+    assert adv_close(adv, ra, sb, se, ADV_RTOL) <= 1.0
+    assert adv_close(ret, rr, sb, se, ADV_RTOL) <= 1.0
+    return adv, ret
+
+
+def test_egae_config1_and_truncated_tail_is_zero():
+    c = synth.config1()
+    adv, ret = check_egae(c["B"], c["rewards"], c["values"], c["seg_begin"], c["seg_end"],
+                          c["truncated"], None, c["gamma"], c["lam"])
+    for i in (1, 3):   # gamma=1, no reward: the last token of a truncated response has A = 0
+        assert adv[c["seg_end"][i] - 1] == 0.0
+
+
+@pytest.mark.parametrize("gamma,lam", [(1.0, 0.95), (1.0, 1.0), (0.99, 0.9), (0.999, 1.0), (0.9, 0.0)])
+def test_egae_random_ragged(gamma, lam):
+    rng = np.random.default_rng(5)
+    B = 37
+    lens = rng.integers(0, 9000, B)
+    lens[3] = 2048          # tile-aligned lengths and a length-1 segment
+    lens[4] = 4096
+    lens[5] = 1
+    gaps = rng.integers(0, 50, B)
+    sb = np.cumsum(gaps + np.concatenate([[0], lens[:-1]])).astype(np.int32)
+    se = (sb + lens).astype(np.int32)
+    N = int(se[-1]) + 13
+    r = rng.standard_normal(N).astype(np.float32)      # dense (process) rewards
+    v = rng.standard_normal(N).astype(np.float32)
+    tr = rng.integers(0, 2, B).astype(np.uint8)
+    boot = rng.standard_normal(B).astype(np.float32)
+    check_egae(B, r, v, sb, se, tr, boot, gamma, lam)
+    check_egae(B, r, v, sb, se, tr, None, gamma, lam)
+
+
+def test_egae_edge_cases():
+    rng = np.random.default_rng(6)
+    r = rng.standard_normal(5000).astype(np.float32)
+    v = rng.standard_normal(5000).astype(np.float32)
+    one = lambda *a: np.array(a, np.int32)
+    check_egae(1, r, v, one(0), one(5000), np.array([1], np.uint8), None, 1.0, 0.95)   # B = 1
+    check_egae(1, r, v, one(0), one(5000), np.array([0], np.uint8), None, 1.0, 1.0)
+    check_egae(1, r[:1], v[:1], one(0), one(1), np.array([1], np.uint8), None, 1.0, 0.95)
+    check_egae(3, r, v, one(10, 10, 4000), one(10, 2048, 4001), np.array([0, 1, 0], np.uint8), None, 0.97, 0.9)
+    adv, ret, st = run_egae(0, r[:100], v[:100], np.zeros(0, np.int32), np.zeros(0, np.int32),
+                            np.zeros(0, np.uint8), None, 1.0, 0.95)
+    assert st == 0 and np.all(adv == 0) and np.all(ret == 0)
+    a1 = run_egae(1, r, v, one(3), one(4999), np.array([1], np.uint8), None, 1.0, 0.95)
+    a2 = run_egae(1, r, v, one(3), one(4999), np.array([1], np.uint8), None, 1.0, 0.95)
+    assert np.array_equal(a1[0], a2[0]) and np.array_equal(a1[1], a2[1])     # run-to-run identical
+    _, _, st = run_egae(1, r, v, one(3), one(6000), np.array([1], np.uint8), None, 1.0, 0.95)
+    assert st == 8      # segment end beyond N is reported, not followed
+
+
+@pytest.mark.parametrize("lam", [0.9, 0.95, 1.0])
+def test_egae_config4_reduced(lam):
+    c = synth.config4(B=400)
+    check_egae(c["B"], c["rewards"], c["values"], c["seg_begin"], c["seg_end"], c["truncated"],
+               c["bootstrap"], 1.0, lam)
+
+
+# ------------------------------------------------------------------------------------------------
+# policy loss
+# ------------------------------------------------------------------------------------------------
+def grad_close(gpu, ref, coef_abs, bf16):
+    """dlogits tolerance: one rounding of the result (2^-8 relative for bf16, generous for fp32) plus
+    the propagated log-prob error, relative to the row's gradient factor."""
+    rel = 2.0 ** -7 if bf16 else 1e-4
+    tol = rel * np.abs(ref) + 1e-3 * coef_abs[:, None] + 1e-12
+    err = np.abs(gpu.astype(np.float64) - ref)
+    return float(np.max(err / tol))
+
+
+def check_policy(logits_t, targets, rows, aux_idx, old_logp, adv, el, eh, denom=0.0, mode=2, hint=0,
+                 inplace=False):
+    is_bf16 = logits_t.dtype == torch.bfloat16
+    host = synth.bf16_bits(logits_t) if is_bf16 else logits_t.cpu().numpy()
+    R, V = host.shape
+    ref = oracle.policy_loss(host, targets, rows, aux_idx, old_logp, adv, f32(el), f32(eh), f32(denom))
+    out = run_policy(logits_t.clone() if inplace else logits_t, targets, rows, aux_idx, old_logp, adv,
+                     el, eh, denom, mode, hint, inplace=inplace)
+    n = R if rows is None else len(rows)
+    assert out["status"] == 0 and out["n"] == n
+    np.testing.assert_allclose(out["logp"][:n], ref["logp"], rtol=0, atol=LOGP_ATOL)
+    np.testing.assert_allclose(out["token_loss"][:n], ref["token_loss"], rtol=0,
+                               atol=LOGP_ATOL * max(1.0, float(np.max(np.abs(adv))) * 2))
+    assert abs(out["loss"] - ref["loss"]) <= LOGP_ATOL * max(1.0, float(np.max(np.abs(adv))))
+    # clip decisions may differ only for ratios within rounding of an edge
+    rho = np.exp(ref["logp"] - np.asarray(old_logp, np.float64)[aux_idx if aux_idx is not None else (rows if rows is not None else np.arange(R))])
+    near = int(np.sum((np.abs(rho - (1 - f32(el))) < 1e-3) | (np.abs(rho - (1 + f32(eh))) < 1e-3)))
+    assert abs(out["clip_lo"] - ref["clip_lo"]) <= near and abs(out["clip_hi"] - ref["clip_hi"]) <= near
+    if mode != 0:
+        g = out["dlogits"].float().cpu().numpy()
+        d = f32(denom) if denom > 0 else max(n, 1)
+        a_idx = aux_idx if aux_idx is not None else (rows if rows is not None else np.arange(R))
+        coef = np.abs(np.asarray(adv, np.float64)[a_idx] * rho / d)
+        if mode == 2:
+            assert g.shape == (max(n, 1), V)
+            if near == 0:
+                assert grad_close(g[:n], ref["dlogits"], coef, is_bf16) <= 1.0
+        else:
+            sel = np.arange(R) if rows is None else np.asarray(rows)
+            if near == 0:
+                assert grad_close(g[sel][:, :V], ref["dlogits"], coef, is_bf16) <= 1.0
+            unsel = np.setdiff1d(np.arange(R), sel)
+            assert np.all(g[unsel][:, :V] == 0)          # rows that are not selected: exact zeros
+        inactive = np.where(np.all(ref["dlogits"] == 0, axis=1))[0]
+        if near == 0 and len(inactive):
+            gi = g[:n][inactive] if mode == 2 else g[sel][inactive][:, :V]
+            assert np.all(gi == 0)                        # clipped rows: exact zeros
+    return out, ref
+
+
+def policy_inputs(rng, R, V, dtype, scale, n_aux=None):
+    x = (scale * rng.standard_normal((R, V))).astype(np.float32)
+    xt = torch.from_numpy(x).to(dtype).to(DEV)
+    host = synth.bf16_bits(xt) if dtype == torch.bfloat16 else x
+    y = rng.integers(0, V, R).astype(np.int32)
+    y[0], y[-1] = 0, V - 1
+    lp = oracle.logprob(host, y)
+    n_aux = R if n_aux is None else n_aux
+    return xt, y, lp
+
+
+def test_policy_config1_fp32():
+    c = synth.config1()
+    xt = torch.from_numpy(c["logits"]).to(DEV)
+    pol, _ = oracle.select_tokens(c["seq_begin"], c["prompt_len"], c["prev_len"], c["new_len"], c["truncated"])
+    adv, _ = oracle.egae(c["rewards"], c["values"], c["seg_begin"], c["seg_end"], c["truncated"], None, 1.0, f32(0.95))
+    old = (oracle.logprob(c["logits"], c["targets"]) + c["old_logp_noise"]).astype(np.float32)
+    for mode in (0, 1, 2):
+        out, ref = check_policy(xt, c["targets"], pol, None, old, adv.astype(np.float32), 0.2, 0.2, mode=mode)
+    assert out["n"] == 170
+    check_policy(xt, c["targets"], pol, None, old, adv.astype(np.float32), 0.2, 0.2, mode=1, inplace=True)
+
+
+@pytest.mark.parametrize("hint", [1, 2])
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_policy_bf16_qwen_vocab(hint, mode):
+    """V = 152064 with few rows: several rows per cluster, every cluster rank, both kernels."""
+    rng = np.random.default_rng(10 + mode)
+    R, V = 330, 152064
+    xt, y, lp = policy_inputs(rng, R, V, torch.bfloat16, 2.0)
+    rows = np.sort(rng.choice(R, 301, replace=False)).astype(np.int32)
+    y[rows[1]] = 38016          # first element of the second slice of a 4-CTA cluster
+    y[rows[2]] = 38015
+    lp = oracle.logprob(synth.bf16_bits(xt), y)
+    old = (lp + 0.15 * rng.standard_normal(R)).astype(np.float32)       # some ratios leave the clip range
+    adv = rng.standard_normal(R).astype(np.float32)
+    out, ref = check_policy(xt, y, rows, None, old, adv, 0.2, 0.28, mode=mode, hint=hint)
+    assert ref["clip_lo"] > 0 and ref["clip_hi"] > 0
+
+
+@pytest.mark.parametrize("variant", [2, 4, 8, 4 | (1 << 4), 4 | (2 << 4)])
+def test_policy_cluster_variants_inplace(variant):
+    rng = np.random.default_rng(20)
+    R, V = 200, 152064
+    xt, y, lp = policy_inputs(rng, R, V, torch.bfloat16, 2.0)
+    old = (lp + 0.05 * rng.standard_normal(R)).astype(np.float32)
+    adv = rng.standard_normal(R).astype(np.float32)
+    check_policy(xt, y, None, None, old, adv, 0.2, 0.2, mode=1, hint=2 | (variant << 8), inplace=True)
+
+
+@pytest.mark.parametrize("V,ld,dtype,hint", [(1001, 1001, torch.bfloat16, 0), (1001, 1008, torch.float32, 0),
+                                             (4096, 4096, torch.bfloat16, 2), (32000, 32768, torch.bfloat16, 2),
+                                             (32000, 32768, torch.bfloat16, 1), (50264, 50264, torch.bfloat16, 0),
+                                             (1000, 1000, torch.float32, 1)])
+def test_policy_shapes(V, ld, dtype, hint):
+    rng = np.random.default_rng(30)
+    R = 70
+    x = (2 * rng.standard_normal((R, ld))).astype(np.float32)
+    full = torch.from_numpy(x).to(dtype).to(DEV)
+    xt = full[:, :V]
+    host = (synth.bf16_bits(full) if dtype == torch.bfloat16 else x)[:, :V]
+    y = rng.integers(0, V, R).astype(np.int32)
+    y[0], y[1] = 0, V - 1
+    rows = np.sort(rng.choice(R, 50, replace=False)).astype(np.int32)
+    aux = rng.permutation(90)[:50].astype(np.int32)
+    lp = oracle.logprob(host, y, rows)
+    old = np.zeros(90, np.float32)
+    adv = np.zeros(90, np.float32)
+    old[aux] = lp + 0.1 * rng.standard_normal(50)
+    adv[aux] = rng.standard_normal(50)
+    for mode in (1, 2):
+        is_bf16 = dtype == torch.bfloat16
+        ref = oracle.policy_loss(host, y, rows, aux, old, adv, f32(0.2), f32(0.2), f32(64.0))
+        out = run_policy(xt, y, rows, aux, old, adv, 0.2, 0.2, 64.0, mode, hint, V=V)
+        assert out["status"] == 0 and out["n"] == 50
+        np.testing.assert_allclose(out["logp"][:50], ref["logp"], atol=LOGP_ATOL)
+        assert abs(out["loss"] - ref["loss"]) <= LOGP_ATOL
+        g = out["dlogits"].float().cpu().numpy()
+        rho = np.exp(ref["logp"] - old[aux])
+        coef = np.abs(adv[aux] * rho / 64.0)
+        gsel = g[:50] if mode == 2 else g[rows][:, :V]
+        near = np.sum((np.abs(rho - 0.8) < 1e-3) | (np.abs(rho - 1.2) < 1e-3))
+        if near == 0:
+            assert grad_close(gsel, ref["dlogits"], coef, is_bf16) <= 1.0
+
+
+def test_policy_overflow_safety_and_onehot_row():
+    V = 8192
+    x = np.zeros((4, V), np.float32)
+    x[0, :] = 3.0e38          # huge equal logits: uniform distribution, no overflow
+    x[1, 5] = 1.0e4
+    x[1, 6:] = -1.0e4         # one dominant logit: logp -> 0
+    x[2, :] = -3.0e38
+    x[3, :] = np.linspace(-80, 80, V)
+    xt = torch.from_numpy(x).to(torch.bfloat16).to(DEV)
+    y = np.array([7, 5, 0, V - 1], np.int32)
+    host = synth.bf16_bits(xt)
+    lp = oracle.logprob(host, y)
+    assert abs(lp[0] + np.log(V)) < 1e-9 and abs(lp[1]) < 1e-9
+    old = lp.astype(np.float32)
+    adv = np.array([1.0, -1.0, 0.5, 2.0], np.float32)
+    for hint in (1, 2):
+        out, ref = check_policy(xt, y, None, None, old, adv, 0.2, 0.2, mode=2, hint=hint)
+        assert np.all(np.isfinite(out["dlogits"].float().cpu().numpy()))
+
+
+@pytest.mark.parametrize("hint", [1, 2])
+def test_policy_zero_selected_and_device_count(hint):
+    rng = np.random.default_rng(40)
+    R, V = 40, 8192
+    xt, y, lp = policy_inputs(rng, R, V, torch.bfloat16, 2.0)
+    old = lp.astype(np.float32)
+    adv = rng.standard_normal(R).astype(np.float32)
+    rows = np.arange(0, R, 2).astype(np.int32)
+    out = run_policy(xt, y, rows, None, old, adv, 0.2, 0.2, 0.0, 1, hint, n_sel=0)
+    assert out["n"] == 0 and out["loss"] == 0.0 and out["status"] == 0
+    assert np.all(out["dlogits"].float().cpu().numpy() == 0)     # FULL mode: every row zero-filled
+    # device-side count smaller than the list capacity
+    out = run_policy(xt, y, rows, None, old, adv, 0.2, 0.2, 0.0, 1, hint, n_sel=7)
+    ref = oracle.policy_loss(synth.bf16_bits(xt), y, rows[:7], None, old, adv, f32(0.2), f32(0.2))
+    assert out["n"] == 7 and abs(out["loss"] - ref["loss"]) < LOGP_ATOL
+    g = out["dlogits"].float().cpu().numpy()
+    assert np.all(g[np.setdiff1d(np.arange(R), rows[:7])] == 0)
+    # bad target / bad row are reported and skipped
+    y2 = y.copy()
+    y2[rows[2]] = V
+    rows2 = rows.copy()
+    rows2[4] = R + 5
+    out = run_policy(xt, y2, rows2, None, old, adv, 0.2, 0.2, 0.0, 2, hint)
+    assert out["status"] == (1 | 4)
+    keep = np.array([k for k in range(len(rows)) if k not in (2, 4)])
+    ref = oracle.policy_loss(synth.bf16_bits(xt), y, rows[keep], None, old, adv, f32(0.2), f32(0.2), f32(len(rows)))
+    assert abs(out["loss"] - ref["loss"]) < LOGP_ATOL
+    g = out["dlogits"].float().cpu().numpy()
+    assert np.all(g[2] == 0) and np.all(g[4] == 0) and np.all(np.isfinite(g))
+
+
+def test_policy_run_to_run_identical():
+    rng = np.random.default_rng(41)
+    R, V = 300, 152064
+    xt, y, lp = policy_inputs(rng, R, V, torch.bfloat16, 2.0)
+    old = (lp + 0.05 * rng.standard_normal(R)).astype(np.float32)
+    adv = rng.standard_normal(R).astype(np.float32)
+    a = run_policy(xt, y, None, None, old, adv, 0.2, 0.2, 0.0, 2, 0)
+    b = run_policy(xt, y, None, None, old, adv, 0.2, 0.2, 0.0, 2, 0)
+    assert a["loss"] == b["loss"] and np.array_equal(a["logp"], b["logp"])
+    assert torch.equal(a["dlogits"], b["dlogits"])
+
+
+def test_policy_rejects_bad_arguments():
+    from paper_2506_15050_b200 import binding as b
+    xt = torch.zeros((4, 64), dtype=torch.bfloat16, device=DEV)
+    y = np.zeros(4, np.int32)
+    z = np.zeros(4, np.float32)
+    with pytest.raises(b.TppoError) as e:
+        run_policy(xt, y, None, None, z, z, -0.1, 0.2)
+    assert e.value.status == 1
+    with pytest.raises(b.TppoError) as e:
+        run_policy(xt, y, None, None, z, z, 0.2, 0.2, hint=2)       # V too small for the cluster kernel
+    assert e.value.status == 3
+    ws = torch.empty(16, dtype=torch.uint8, device=DEV)
+    with pytest.raises(b.TppoError) as e:
+        b.tppo_policy_loss_fwd_bwd(xt, dev(y), None, None, 4, None, dev(z), dev(z), 0.2, 0.2, 0.0, None, None,
+                                   torch.zeros(1, device=DEV), torch.zeros(4, dtype=torch.int32, device=DEV),
+                                   None, 0, ws)
+    assert e.value.status == 2
+
+
+# ------------------------------------------------------------------------------------------------
+# value loss
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("xl,xh", [(0.5, 0.6), (0.05, 0.02)])
+def test_value_loss(xl, xh):
+    rng = np.random.default_rng(50)
+    N = 70000
+    v = rng.standard_normal(N).astype(np.float32)
+    vo = (v + 0.3 * rng.standard_normal(N)).astype(np.float32)
+    R = rng.choice([-1.0, 1.0], N).astype(np.float32)
+    idx = np.sort(rng.choice(N, 41234, replace=False)).astype(np.int32)
+    loss, dv, n, st = run_value(v, vo, R, idx, xl, xh)
+    rl, rdv = oracle.value_loss(v, vo, R, idx, f32(xl), f32(xh))
+    assert n == len(idx) and st == 0
+    assert abs(loss - rl) <= 1e-5 * max(1.0, abs(rl))
+    # the clip bound is rounded in fp32 on the GPU: tokens within an ulp of a bound may switch branch
+    edge = (np.abs(v - (vo - f32(xl))) < 1e-6) | (np.abs(v - (vo + f32(xh))) < 1e-6)
+    np.testing.assert_allclose(dv[~edge], rdv[~edge], rtol=1e-5, atol=1e-9)
+    loss2, dv2, _, _ = run_value(v, vo, R, idx, xl, xh)
+    assert loss2 == loss and np.array_equal(dv, dv2)
+    loss3, dv3, n3, _ = run_value(v, vo, R, idx, xl, xh, denom=1000.0, n_sel=100)
+    rl3, rdv3 = oracle.value_loss(v, vo, R, idx[:100], f32(xl), f32(xh), 1000.0)
+    assert n3 == 100 and abs(loss3 - rl3) <= 1e-6
+    np.testing.assert_allclose(dv3[~edge], rdv3[~edge], rtol=1e-5, atol=1e-9)
+    loss4, dv4, n4, _ = run_value(v, vo, R, idx, xl, xh, n_sel=0)
+    assert loss4 == 0 and n4 == 0 and np.all(dv4 == 0)
+    bad = idx.copy()
+    bad[5] = N + 3
+    _, dv5, _, st5 = run_value(v, vo, R, bad, xl, xh)
+    assert st5 == 4 and np.all(np.isfinite(dv5))
+
+
+def test_value_loss_config1():
+    c = synth.config1()
+    _, ret = oracle.egae(c["rewards"], c["values"], c["seg_begin"], c["seg_end"], c["truncated"], None, 1.0, f32(0.95))
+    _, val = oracle.select_tokens(c["seq_begin"], c["prompt_len"], c["prev_len"], c["new_len"], c["truncated"])
+    loss, dv, n, st = run_value(c["values"], c["old_values"], ret.astype(np.float32), val, 0.5, 0.6)
+    rl, rdv = oracle.value_loss(c["values"], c["old_values"], ret.astype(np.float32), val, f32(0.5), f32(0.6))
+    assert n == 42 and abs(loss - rl) < 1e-6
+    np.testing.assert_allclose(dv, rdv, rtol=1e-5, atol=1e-9)
