@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of the T-PPO token-selective update path on B200.
+
+One "step" is one pass of the whole hot path over one synthetic batch shaped like the paper's
+Qwen2.5-32B long-CoT step: EGAE + Monte-Carlo returns over the full batch of 512 ragged responses,
+policy / value token selection, the fused log-prob + clipped-surrogate loss forward/backward over a
+[16384, 152064] bf16 logits micro-batch (gradient written to a second buffer), and the value loss
+on 16384 value tokens.  The metric is selected (policy) tokens per second.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W]            CUDA path (this repo)
+  python bench.py --impl reference ...                           float64 CPU oracle on host cores
+
+Prints one JSON line.  With N > 1 (torchrun) every rank runs the same per-GPU workload (the path
+shards by sequence with no data-path collective); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2506_15050_b200 import synth  # noqa: E402
+
+METRIC = "selected tokens/s, fused logprob+PPO loss fwd+bwd, V=152064 bf16; % HBM peak"
+UNIT = "selected tokens/s"
+ALGO_BYTES_PER_TOKEN = 2 * 2 * synth.V_QWEN       # bf16 row read once + bf16 gradient row written once
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_setup(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    return rank, world, local
+
+
+class Step:
+    """Device-resident state of the workload and the four C-ABI calls of one step."""
+
+    def __init__(self, dev, seed=2, rows=16384):
+        from paper_2506_15050_b200 import binding as b
+        self.b, self.dev = b, dev
+        c = synth.config3(dev, seed=seed, n_tokens=rows)
+        self.c = c
+        t = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).to(dev)
+        self.N, self.B, self.V, self.n = c["N"], c["B"], c["V"], c["n_tokens"]
+        self.host = {k: c[k] for k in ("rewards", "values", "old_values", "seg_begin", "seg_end",
+                                       "truncated", "seq_begin", "prompt_len", "prev_len", "new_len",
+                                       "extra_policy_mask", "extra_value_mask", "targets")}
+        self.rewards, self.values = t(c["rewards"], torch.float32), t(c["values"], torch.float32)
+        self.old_values = t(c["old_values"], torch.float32)
+        self.seg_b, self.seg_e = t(c["seg_begin"], torch.int32), t(c["seg_end"], torch.int32)
+        self.trunc = t(c["truncated"], torch.uint8)
+        self.seq_begin = t(c["seq_begin"], torch.int32)
+        self.prompt, self.prev, self.new = (t(c[k], torch.int32) for k in ("prompt_len", "prev_len", "new_len"))
+        self.pmask, self.vmask = t(c["extra_policy_mask"], torch.uint8), t(c["extra_value_mask"], torch.uint8)
+        self.targets = t(c["targets"], torch.int32)
+        self.logits = c["logits"]
+        N, n = self.N, self.n
+        self.adv, self.ret = torch.zeros(N, device=dev), torch.zeros(N, device=dev)
+        self.pol = torch.zeros(N, dtype=torch.int32, device=dev)
+        self.val = torch.zeros(N, dtype=torch.int32, device=dev)
+        self.counts = torch.zeros(4, dtype=torch.int32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.logp, self.tok_loss = torch.zeros(n, device=dev), torch.zeros(n, device=dev)
+        self.loss, self.vloss = torch.zeros(1, device=dev), torch.zeros(1, device=dev)
+        self.stats = torch.zeros(4, dtype=torch.int32, device=dev)
+        self.vstats = torch.zeros(2, dtype=torch.int32, device=dev)
+        self.dlogits = torch.empty_like(self.logits)
+        self.dvalues = torch.zeros(N, device=dev)
+        self.old_logp = torch.zeros(N, device=dev)
+        self.ws_egae = b.workspace(b.OP_EGAE, N, self.B, 0, 0, dev)
+        self.ws_sel = b.workspace(b.OP_SELECT_TOKENS, N, self.B, 0, 0, dev)
+        self.ws_pol = b.workspace(b.OP_POLICY_LOSS, n, 0, n, self.V, dev)
+        self.ws_val = b.workspace(b.OP_VALUE_LOSS, N, 0, N, 0, dev)
+        self.ev = None
+        self.hint = 0
+        # old-policy log-probs (Algorithm 1 line 3): forward-only pass of the same kernel, plus noise
+        self.egae()
+        self.select()
+        self.policy(forward_only=True)
+        torch.cuda.synchronize()
+        idx = self.pol[:n].long()
+        self.old_logp[idx] = self.logp + t(c["old_logp_noise"], torch.float32)[idx]
+
+    def egae(self):
+        c = self.c
+        self.b.tppo_egae(self.rewards, self.values, self.seg_b, self.seg_e, self.trunc, None,
+                         c["gamma"], c["lam"], self.adv, self.ret, self.status, self.ws_egae)
+
+    def select(self):
+        self.b.tppo_select_tokens(self.seq_begin, self.prompt, self.prev, self.new, self.trunc, 0,
+                                  self.pmask, self.vmask, self.N, self.pol, self.val, self.counts,
+                                  self.ws_sel)
+
+    def policy(self, forward_only=False):
+        c, b = self.c, self.b
+        b.tppo_policy_loss_fwd_bwd(
+            self.logits, self.targets, None, self.counts[0:1], self.n, self.pol, self.old_logp,
+            self.adv, c["eps_low"], c["eps_high"], 0.0, self.logp, self.tok_loss, self.loss,
+            self.stats, None if forward_only else self.dlogits,
+            b.DLOGITS_NONE if forward_only else b.DLOGITS_COMPACT, self.ws_pol, kernel_hint=self.hint)
+
+    def value(self):
+        c = self.c
+        self.b.tppo_value_loss(self.values, self.old_values, self.ret, self.val, self.counts[1:2],
+                               self.N, c["xi_low"], c["xi_high"], 0.0, self.vloss, self.dvalues,
+                               self.vstats, self.ws_val)
+
+    def run(self, events=None):
+        self.egae()
+        self.select()
+        if events is not None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            self.policy()
+            e1.record()
+            events.append((e0, e1))
+        else:
+            self.policy()
+        self.value()
+
+    KERNELS_PER_STEP = 6   # egae scan, select, policy prepare + sweep + finish, value loss
+
+
+def cpu_oracle_step_seconds(c, n_tokens, sample_rows):
+    """Times the oracle, as it stands, on host cores: EGAE and selection on the full batch, policy
+    loss forward+backward on `sample_rows` rows of the micro-batch (scaled to n_tokens), value loss."""
+    import oracle
+    f32 = lambda x: float(np.float32(x))
+    t0 = time.perf_counter()
+    adv, ret = oracle.egae(c["rewards"], c["values"], c["seg_begin"], c["seg_end"], c["truncated"],
+                           None, f32(c["gamma"]), f32(c["lam"]))
+    t1 = time.perf_counter()
+    pol, val = oracle.select_tokens(c["seq_begin"], c["prompt_len"], c["prev_len"], c["new_len"],
+                                    c["truncated"], 0, c["extra_policy_mask"], c["extra_value_mask"])
+    t2 = time.perf_counter()
+    logits = c["logits_sample"]
+    rows = np.arange(sample_rows, dtype=np.int32)
+    old = np.zeros(c["N"], np.float32)
+    out = oracle.policy_loss(logits, c["targets"], rows, pol[:sample_rows], old,
+                             adv.astype(np.float32), f32(c["eps_low"]), f32(c["eps_high"]),
+                             float(n_tokens))
+    t3 = time.perf_counter()
+    oracle.value_loss(c["values"], c["old_values"], ret.astype(np.float32), val, f32(c["xi_low"]),
+                      f32(c["xi_high"]))
+    t4 = time.perf_counter()
+    del out
+    t_policy = (t3 - t2) * (n_tokens / sample_rows)
+    return (t1 - t0) + (t2 - t1) + t_policy + (t4 - t3), oracle.num_threads(), \
+        {"egae_s": t1 - t0, "select_s": t2 - t1, "policy_sample_s": t3 - t2, "value_s": t4 - t3}
+
+
+def run_reference(args, rank):
+    """The oracle on the host cores: same metric, bounded sample per step."""
+    if rank != 0:
+        return
+    c = synth.config3("cpu", with_logits=False)
+    sample_rows = args.ref_rows
+    c["logits_sample"] = synth.bf16_bits(synth.randn_bf16((sample_rows, synth.V_QWEN), 2.0, 2, "cpu"))
+    times = []
+    for i in range(args.warmup + args.steps):
+        t, cores, parts = cpu_oracle_step_seconds(c, c["n_tokens"], sample_rows)
+        if i >= args.warmup:
+            times.append(t)
+    t = float(np.mean(times))
+    value = c["n_tokens"] / t
+    sample = (f"EGAE+selection+value loss on the full batch, policy loss fwd+bwd on {sample_rows} of "
+              f"{c['n_tokens']} rows (V=152064) scaled to the full micro-batch")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "cfg3: 512-response EGAE batch + [16384,152064] bf16 loss micro-batch"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-rows", type=int, default=512, help="oracle sample rows per step")
+    ap.add_argument("--cpu-rows", type=int, default=1024, help="rows of the cpu_baseline sample")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--hint", type=int, default=0, help="kernel_hint passed to the policy loss")
+    ap.add_argument("--rows", type=int, default=16384,
+                    help="rows of the loss micro-batch (smaller only for profiler captures)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    rank, world, local = dist_setup(args.gpus)
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA path has no CPU fallback")
+    warmup = max(args.warmup, 3)
+    dev = f"cuda:{local}"
+    torch.cuda.set_device(local)
+    st = Step(dev, rows=args.rows)
+    st.hint = args.hint
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        st.run()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    events = []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        st.run(events)
+    t1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = t0.elapsed_time(t1)
+    if world > 1:
+        import torch.distributed as dist
+        tt = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    ms_step = ms_total / args.steps
+    n_tok = int(st.counts[0].item())
+    assert n_tok == st.n and int(st.stats[3].item()) == 0 and int(st.status.item()) == 0
+    value = world * n_tok / (ms_step * 1e-3)
+    pol_ms = float(np.mean([a.elapsed_time(b) for a, b in events]))
+    peak, peak_kind = measured_peaks()
+    achieved = n_tok * ALGO_BYTES_PER_TOKEN / (pol_ms * 1e-3) / 1e9
+
+    # ---- end to end: host buffers in, losses out, copies inside the timed region ---------------
+    e2e = None
+    if not args.no_e2e:
+        pin = lambda x: x.cpu().pin_memory()
+        h_logits = pin(st.logits)
+        small = [st.rewards, st.values, st.old_values, st.seg_b, st.seg_e, st.trunc, st.seq_begin,
+                 st.prompt, st.prev, st.new, st.pmask, st.vmask, st.targets, st.old_logp]
+        h_small = [pin(x) for x in small]
+        h_out = torch.empty(2, dtype=torch.float32).pin_memory()
+        h_cnt = torch.empty(4, dtype=torch.int32).pin_memory()
+        h2d = h_logits.numel() * 2 + sum(x.numel() * x.element_size() for x in h_small)
+        d2h = 2 * 4 + 4 * 4
+
+        def e2e_step():
+            st.logits.copy_(h_logits, non_blocking=True)
+            for d, h in zip(small, h_small):
+                d.copy_(h, non_blocking=True)
+            st.run()
+            h_out[0:1].copy_(st.loss, non_blocking=True)
+            h_out[1:2].copy_(st.vloss, non_blocking=True)
+            h_cnt.copy_(st.counts, non_blocking=True)
+            torch.cuda.synchronize()
+
+        e2e_step()
+        barrier()
+        w0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        barrier()
+        e2e_s = (time.perf_counter() - w0) / args.e2e_steps
+        if world > 1:
+            import torch.distributed as dist
+            tt = torch.tensor([e2e_s], device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_s = float(tt.item())
+        e2e = {"value": world * n_tok / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_s * 1e3, "steps": args.e2e_steps}
+        del h_logits
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        c = dict(st.c)
+        c["logits_sample"] = synth.bf16_bits(st.logits[:args.cpu_rows])
+        t, cores, parts = cpu_oracle_step_seconds(c, n_tok, args.cpu_rows)
+        cpu = {"value": n_tok / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": (f"EGAE+selection+value loss on the full batch, policy loss fwd+bwd on "
+                          f"{args.cpu_rows} of {n_tok} rows scaled to the micro-batch"),
+               "seconds": {k: round(v, 4) for k, v in parts.items()}}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
+            "config": {"workload": "cfg3: EGAE over 512 ragged responses (N=%d tokens), selection, "
+                                   "[%d,152064] bf16 fused log-prob+PPO loss fwd+bwd, value loss "
+                                   "on %d tokens" % (st.N, st.n, int(st.counts[1].item())),
+                       "l2": "inputs larger than L2 (%.2f GB logits per step)" % (st.n * st.V * 2 / 1e9),
+                       "dlogits": "compact, separate buffer", "kernel_hint": args.hint},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_kind": peak_kind,
+                         "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": None,
+                         "kernel": "policy_cluster_kernel", "kernel_ms": pol_ms,
+                         "algorithmic_bytes_per_launch": n_tok * ALGO_BYTES_PER_TOKEN},
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": Step.KERNELS_PER_STEP * args.steps,
+            "clocks": clocks}))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

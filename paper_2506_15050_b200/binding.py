@@ -121,7 +121,11 @@ def tppo_policy_loss_fwd_bwd(logits, targets, rows, n_sel, n_max, aux_idx, old_l
     R, ld = logits.shape[0], logits.stride(0)
     V = logits.shape[1] if V is None else V
     if dlogits is not None:
-        assert dlogits.dtype == logits.dtype and dlogits.is_cuda
+        assert dlogits.dtype == logits.dtype and dlogits.is_cuda and dlogits.stride(-1) == 1
+        if dlogits_mode == DLOGITS_FULL:
+            assert dlogits.stride(0) == ld, "FULL mode: dlogits must have the logits' row stride"
+        else:
+            assert dlogits.is_contiguous(), "COMPACT mode: dlogits must be dense [n_max, V]"
     _check(_lib.tppo_policy_loss_fwd_bwd(
         logits.data_ptr(), dt, R, V, ld, _ptr(targets, torch.int32), _ptr(rows, torch.int32),
         _ptr(n_sel, torch.int32), n_max, _ptr(aux_idx, torch.int32),

@@ -6,15 +6,28 @@
 // the next rows are in flight while the current row is being worked on.  The 15 compute warps pull
 // their 16-byte units of the slice into registers, form a thread-local maximum and the
 // exponentials relative to it (one ex2 per logit, kept in registers as fp32), and reduce
-// (max, sum, target logit) over the warp, the CTA and -- through distributed shared memory and a
-// cluster-scope mbarrier -- the cluster.  With the row's log-sum-exp known every thread evaluates
+// (max, sum, target logit) over the warp and -- through asynchronous distributed-shared-memory
+// stores that count bytes on the receiver's mbarrier -- the cluster.  With the row's log-sum-exp known every thread evaluates
 // Eq. 1 of the paper (ratio, clip, loss term, gradient factor), rescales its stored exponentials
-// into  factor * (softmax - onehot),  rounds once to bf16 and writes the result over its slice in
-// shared memory; the producer warp sends it to global memory with bulk stores and reuses the
-// buffer once the store has drained.  Each logit crosses the HBM interface exactly once in each
-// direction.  No multicast is used: every CTA issues plain copies of its own slice.
+// into  factor * (softmax - onehot),  rounds once to bf16 and stores the result: either straight
+// from registers with 128-bit global stores (default; the stage buffer is then free as soon as
+// the row is in registers), or over its slice in shared memory, from where the producer warp sends
+// it out with bulk stores.  Each logit crosses the HBM interface exactly once in each direction.
+// No multicast is used: every CTA issues plain copies of its own slice.
 #include "policy_common.cuh"
 #include "ptx.cuh"
+
+#ifdef TPPO_TIMELINE
+// Debug builds only: per-row phase timestamps (SM clock) of cluster 0, read back by a test driver.
+__device__ unsigned long long g_timeline[8][64][16];
+#define TL(rank, it, slot) \
+    do { if (cid == 0 && (it) < 64) g_timeline[rank][it][slot] = clock64(); } while (0)
+extern "C" int tppo_debug_timeline(void* host_out) {
+    return int(cudaMemcpyFromSymbol(host_out, g_timeline, sizeof(g_timeline)));
+}
+#else
+#define TL(rank, it, slot) do {} while (0)
+#endif
 
 namespace tppo {
 
@@ -24,19 +37,17 @@ constexpr int kClThreads = kClComputeThreads + 32;           // + producer warp
 constexpr int kClMaxUnits = 10;                              // 16-byte units per thread per slice
 constexpr int kClMaxStages = 4;
 constexpr int kClMaxCluster = 8;
-constexpr uint32_t kClCtlBytes = 1024;                       // control block ahead of the stages
-constexpr uint32_t kClCopyChunk = 16384;                     // bytes per bulk copy instruction
+constexpr int kClMaxParts = kClMaxCluster * kClComputeWarps; // warp partials a CTA receives per row
+constexpr uint32_t kClCtlBytes = 4096;                       // control block ahead of the stages
+constexpr uint32_t kClCopyChunk = 1u << 17;                  // bytes per bulk copy instruction
 constexpr uint32_t kNegInfPair = 0xff80ff80u;                // two bf16 -inf
 
 struct ClusterCtl {
     unsigned long long full[kClMaxStages];   // slice landed in shared memory (tx-count barrier)
     unsigned long long done[kClMaxStages];   // compute warps are finished with the stage
-    unsigned long long xchg[2];              // C partials arrived from the cluster
-    unsigned long long wready;               // every compute warp has published its partial
-    float4 part[2][kClMaxCluster];           // (max, sum, target logit, -) of each CTA
-    float2 wpart[kClComputeWarps];           // (max, sum) of each warp
-    float wxy;                               // target logit if it lies in this CTA's slice
-    int abort;
+    unsigned long long xchg[2];              // all (max, sum) partials of the row have arrived
+    float2 part[2][kClMaxParts];             // (max, sum) of every compute warp of the cluster
+    float xy[2];                             // the row's target logit, sent by the thread that owns it
 };
 static_assert(sizeof(ClusterCtl) <= kClCtlBytes, "control block too large");
 
@@ -45,7 +56,8 @@ struct ClusterLaunch {
     uint32_t stage_stride;   // bytes between stage buffers (multiple of 128)
 };
 
-template <int C, bool GRAD>
+// OUT: 0 = forward only, 1 = gradient via shared memory + bulk stores, 2 = gradient straight from registers
+template <int C, int OUT>
 __global__ void __launch_bounds__(kClThreads, 1)
 policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -53,10 +65,12 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
     const uint32_t stage0 = ptx::smem_addr(smem) + kClCtlBytes;
 
     const uint32_t rank = ptx::cluster_ctarank();
-    const int64_t cid = ptx::cluster_id_x(), ncl = ptx::num_clusters_x();
-    const int64_t n = policy_n(a);
-    const int64_t n_it = n > cid ? (n - cid + ncl - 1) / ncl : 0;   // rows j = cid + it * ncl
+    const int32_t cid = int32_t(ptx::cluster_id_x()), ncl = int32_t(ptx::num_clusters_x());
+    const int32_t n = int32_t(policy_n(a));
+    const int32_t n_it = n > cid ? (n - cid + ncl - 1) / ncl : 0;   // rows j = cid + it * ncl
     const uint32_t S = cfg.stages;
+    constexpr bool GRAD = OUT != 0;
+    constexpr bool STAGED = OUT == 1;   // the stage buffer also stages the gradient
 
     // this CTA's slice of every row, in 16-byte units
     const uint32_t units_total = uint32_t(a.V) >> 3;
@@ -71,14 +85,11 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
             ptx::mbar_init(ptx::smem_addr(&ctl->full[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->done[s]), kClComputeWarps);
         }
-        ptx::mbar_init(ptx::smem_addr(&ctl->xchg[0]), C);
-        ptx::mbar_init(ptx::smem_addr(&ctl->xchg[1]), C);
-        ptx::mbar_init(ptx::smem_addr(&ctl->wready), kClComputeWarps);
-        ctl->abort = 0;
-        ctl->wxy = 0.f;
+        ptx::mbar_init(ptx::smem_addr(&ctl->xchg[0]), 1);
+        ptx::mbar_init(ptx::smem_addr(&ctl->xchg[1]), 1);
         ptx::fence_mbar_init_cluster();
     }
-    ptx::cluster_sync_all();   // barriers of every CTA are initialised before any remote arrive
+    ptx::cluster_sync_all();   // barriers of every CTA are initialised before any remote signal
 
     const uint8_t* logits = static_cast<const uint8_t*>(a.logits);
     uint8_t* dl = static_cast<uint8_t*>(a.dlogits);
@@ -86,13 +97,13 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
     if (tid >= kClComputeThreads) {
         // ===================== producer warp: all bulk copies of this CTA =====================
         if (tid == kClComputeThreads) {
-            int64_t issued = 0;
-            auto issue_load = [&](int64_t it) {
-                const uint32_t st = uint32_t(it % S);
-                const int64_t j = cid + it * ncl;
-                const int64_t r = a.rows ? int64_t(__ldg(a.rows + j)) : j;
+            int32_t issued = 0;
+            auto issue_load = [&](int32_t it) {
+                const uint32_t st = uint32_t(it) % S;
+                const int64_t j = int64_t(cid) + int64_t(it) * ncl;
+                const int64_t r = __ldg(&a.rec[j].row);
                 const uint32_t bar = ptx::smem_addr(&ctl->full[st]);
-                if (r >= 0 && r < a.R && slice_bytes > 0) {
+                if (r >= 0 && slice_bytes > 0) {
                     ptx::mbar_arrive_expect_tx(bar, slice_bytes);
                     const uint8_t* src = logits + (r * a.ld) * 2 + uint64_t(u0) * 16u;
                     const uint32_t dst = stage0 + st * cfg.stage_stride;
@@ -105,22 +116,23 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
                 }
                 issued = it + 1;
             };
-            const int64_t pro = n_it < int64_t(S) ? n_it : int64_t(S);
-            for (int64_t it = 0; it < pro; ++it) issue_load(it);
+            const int32_t pro = n_it < int32_t(S) ? n_it : int32_t(S);
+            for (int32_t it = 0; it < pro; ++it) issue_load(it);
 
             bool ok = true;
-            for (int64_t it = 0; it < n_it && ok; ++it) {
-                const uint32_t st = uint32_t(it % S);
-                ok = ptx::mbar_wait<false>(ptx::smem_addr(&ctl->done[st]), uint32_t(it / S) & 1u);
+            uint32_t st = 0, ph = 0;
+            for (int32_t it = 0; it < n_it; ++it) {
+                ok = ptx::mbar_wait<false>(ptx::smem_addr(&ctl->done[st]), ph);
                 if (!ok) break;
-                if (GRAD) {
-                    const int64_t j = cid + it * ncl;
+                TL(rank, it, 8);
+                if (STAGED) {
+                    const int64_t j = int64_t(cid) + int64_t(it) * ncl;
                     uint8_t* dst = nullptr;
                     if (a.mode == TPPO_DLOGITS_COMPACT) {
                         dst = dl + (j * int64_t(a.V)) * 2;
                     } else {
-                        const int64_t r = a.rows ? int64_t(__ldg(a.rows + j)) : j;
-                        if (r >= 0 && r < a.R) dst = dl + (r * a.ld) * 2;
+                        const int64_t r = __ldg(&a.rec[j].row);
+                        if (r >= 0) dst = dl + (r * a.ld) * 2;
                     }
                     if (dst && slice_bytes > 0) {
                         dst += uint64_t(u0) * 16u;
@@ -131,21 +143,27 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
                         }
                     }
                     ptx::bulk_commit();
-                    if (it >= 1) {
+                    TL(rank, it, 9);
+                    if (S == 1) {
+                        ptx::bulk_wait_read<0>();             // single buffer: drain, then refill
+                        if (it + 1 < n_it) issue_load(it + 1);
+                    } else if (it >= 1) {
                         ptx::bulk_wait_read<1>();             // the store of row it-1 has left smem
-                        if (it - 1 + S < n_it) issue_load(it - 1 + S);
+                        TL(rank, it, 10);
+                        if (it - 1 + int32_t(S) < n_it) issue_load(it - 1 + int32_t(S));
+                        TL(rank, it, 11);
                     }
                 } else {
-                    if (it + S < n_it) issue_load(it + S);    // registers hold the row: reuse now
+                    if (it + int32_t(S) < n_it) issue_load(it + int32_t(S));   // the row is in registers
                 }
+                if (++st == S) { st = 0; ph ^= 1u; }
             }
             if (!ok) {
-                ctl->abort = 1;
                 atomicOr(a.stats + 3, TPPO_DEV_WAIT_TIMEOUT);
                 // let the copies that are still in flight into this CTA's shared memory land
-                const int64_t first = issued > int64_t(S) ? issued - int64_t(S) : 0;
-                for (int64_t it = first; it < issued; ++it)
-                    ptx::mbar_wait<false>(ptx::smem_addr(&ctl->full[it % S]), uint32_t(it / S) & 1u);
+                const int32_t first = issued > int32_t(S) ? issued - int32_t(S) : 0;
+                for (int32_t it = first; it < issued; ++it)
+                    ptx::mbar_wait<false>(ptx::smem_addr(&ctl->full[uint32_t(it) % S]), (uint32_t(it) / S) & 1u);
             }
             ptx::bulk_wait<0>();
         }
@@ -154,23 +172,23 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
         // ================================ compute warps ======================================
         const int lane = tid & 31, warp = tid >> 5;
         const float inv_denom = policy_inv_denom(a, n);
-        RowMeta meta_next;
-        float A_next = 0.f, old_next = 0.f;
-        if (n_it > 0) {
-            meta_next = policy_row_meta(a, cid);
-            if (meta_next.ok) { A_next = __ldg(a.adv + meta_next.aux); old_next = __ldg(a.old_logp + meta_next.aux); }
-        }
+        constexpr uint32_t kPartBytes = uint32_t(C) * kClComputeWarps * 8u;   // partials per row
+        RowRec rec_next;
+        rec_next.row = -1; rec_next.y = -1; rec_next.adv = 0.f; rec_next.old_logp = 0.f;
+        if (n_it > 0) rec_next = load_rec(a.rec + cid);
         bool ok = true;
-        for (int64_t it = 0; it < n_it; ++it) {
-            const uint32_t st = uint32_t(it % S);
-            const int64_t j = cid + it * ncl;
-            const RowMeta meta = meta_next;
-            const float A = A_next, old_lp = old_next;
-            if (it + 1 < n_it) {   // fetch the next row's scalars one row ahead
-                meta_next = policy_row_meta(a, j + ncl);
-                if (meta_next.ok) { A_next = __ldg(a.adv + meta_next.aux); old_next = __ldg(a.old_logp + meta_next.aux); }
-            }
-            if (!ptx::mbar_wait<false>(ptx::smem_addr(&ctl->full[st]), uint32_t(it / S) & 1u)) { ok = false; break; }
+        uint32_t st = 0, ph = 0;
+        for (int32_t it = 0; it < n_it; ++it) {
+            const int64_t j = int64_t(cid) + int64_t(it) * ncl;
+            const RowRec rec = rec_next;
+            const bool row_ok = rec.row >= 0, rec_ok = rec.y >= 0;
+            const uint32_t par = uint32_t(it) & 1u, xph = (uint32_t(it) >> 1) & 1u;
+            if (tid == 0)   // this row's exchange: C*15 warp partials (+ the target logit)
+                ptx::mbar_arrive_expect_tx(ptx::smem_addr(&ctl->xchg[par]), kPartBytes + (rec_ok ? 4u : 0u));
+            if (it + 1 < n_it) rec_next = load_rec(a.rec + j + ncl);   // one row ahead, used next turn
+            if (tid == 0) TL(rank, it, 0);
+            if (!ptx::mbar_wait<false>(ptx::smem_addr(&ctl->full[st]), ph)) { ok = false; break; }
+            if (tid == 0) TL(rank, it, 1);
 
             // ---- slice -> registers ------------------------------------------------------
             const uint32_t sbase = stage0 + st * cfg.stage_stride;
@@ -178,10 +196,17 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
 #pragma unroll
             for (int k = 0; k < kClMaxUnits; ++k) {
                 const uint32_t u = uint32_t(tid) + uint32_t(k) * kClComputeThreads;
-                xw[k] = (u < nu && meta.row_ok) ? ptx::lds128(sbase + u * 16u)
+                xw[k] = (u < nu && row_ok) ? ptx::lds128(sbase + u * 16u)
                                                 : make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
             }
-            if (!GRAD) {   // the stage can be refilled as soon as every warp holds its units
+            // the target logit, if it lies in one of this thread's units
+            const int32_t yu = (rec.y >> 3) - int32_t(u0);
+            const bool y_mine = rec_ok && yu >= 0 && yu < int32_t(nu) && (yu % kClComputeThreads) == tid;
+            const uint32_t y_off = uint32_t(yu) * 16u + uint32_t(rec.y & 7) * 2u;   // within the slice
+            const uint32_t y_addr = sbase + y_off;
+            float x_y = 0.f;
+            if (y_mine) x_y = __uint_as_float(uint32_t(ptx::lds_u16(y_addr)) << 16);
+            if (!STAGED) {   // the stage can be refilled as soon as every warp holds its units
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->done[st]));
             }
@@ -194,101 +219,113 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
             }
             float m_t = fmaxf(bf16_lo(pm), bf16_hi(pm));
             m_t = fmaxf(m_t, -1.0e30f);                 // a thread with no unit: keep finite
+            if (tid == 0) TL(rank, it, 12);
             // ---- exponentials relative to the thread-local max, kept in registers ---------
             const float off_t = m_t * kLog2e;
-            float e[kClMaxUnits][8];
-            float s_t = 0.f;
+            // (two fp32 lanes per instruction: packed FMA / ADD / MUL halve the issue slots)
+            uint64_t e2[kClMaxUnits][4];
+            uint64_t s2 = ptx::pack_f32x2(0.f, 0.f);
+            const uint64_t k2 = ptx::pack_f32x2(kLog2e, kLog2e), o2 = ptx::pack_f32x2(-off_t, -off_t);
 #pragma unroll
             for (int k = 0; k < kClMaxUnits; ++k) {
                 const uint32_t w[4] = {xw[k].x, xw[k].y, xw[k].z, xw[k].w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    e[k][2 * q] = ex2(fmaf(bf16_lo(w[q]), kLog2e, -off_t));
-                    e[k][2 * q + 1] = ex2(fmaf(bf16_hi(w[q]), kLog2e, -off_t));
-                    s_t += e[k][2 * q] + e[k][2 * q + 1];
+                    float t0, t1;
+                    ptx::unpack_f32x2(ptx::fma_f32x2(ptx::pack_f32x2(bf16_lo(w[q]), bf16_hi(w[q])), k2, o2), t0, t1);
+                    e2[k][q] = ptx::pack_f32x2(ex2(t0), ex2(t1));
+                    s2 = ptx::add_f32x2(s2, e2[k][q]);
                 }
             }
-            // ---- the target logit, if one of this thread's elements -------------------------
-            const int32_t yu = (meta.y >> 3) - int32_t(u0);
-            const bool y_here = meta.ok && yu >= 0 && yu < int32_t(nu);     // in this CTA's slice
-            const bool y_mine = y_here && (yu % kClComputeThreads) == tid;
-            const int yk = yu / kClComputeThreads, ye = meta.y & 7;
-            if (y_mine) {
-                uint32_t word = 0;
-#pragma unroll
-                for (int k = 0; k < kClMaxUnits; ++k) {
-                    if (k == yk) {
-                        const uint32_t w[4] = {xw[k].x, xw[k].y, xw[k].z, xw[k].w};
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) if (q == (ye >> 1)) word = w[q];
-                    }
-                }
-                ctl->wxy = (ye & 1) ? bf16_hi(word) : bf16_lo(word);
+            float s_t;
+            {
+                float sa, sb;
+                ptx::unpack_f32x2(s2, sa, sb);
+                s_t = sa + sb;
             }
-            // ---- warp, CTA and cluster reduction of (max, sum) ------------------------------
+            if (tid == 0) TL(rank, it, 2);
+            // ---- warp partial -> every CTA of the cluster (asynchronous remote stores that count
+            //      bytes on the receiver's barrier: no fence, no second hop) ----------------------
             const float wm = warp_max(m_t);
             const float ws = warp_sum(s_t * ex2((m_t - wm) * kLog2e));
-            if (lane == 0) ctl->wpart[warp] = make_float2(wm, ws);
-            __syncwarp();        // the target-logit write of any lane precedes lane 0's arrive
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->wready));
-            const uint32_t par = uint32_t(it) & 1u;
-            if (warp == 0) {
-                if (!ptx::mbar_wait<false>(ptx::smem_addr(&ctl->wready), par)) { ok = false; break; }
-                const float2 p = lane < kClComputeWarps ? ctl->wpart[lane] : make_float2(-1.0e30f, 0.f);
-                const float cm = warp_max(p.x);
-                const float cs = warp_sum(p.y * ex2((p.x - cm) * kLog2e));
-                const float xy = y_here ? ctl->wxy : 0.f;
-                __syncwarp();     // every lane has read the shared partials before any is released
-                if (lane < C) {   // lane c delivers this CTA's partial to CTA c
-                    const uint32_t dst = ptx::map_to_cta(ptx::smem_addr(&ctl->part[par][rank]), lane);
-                    ptx::st_cluster_f32x4(dst, cm, cs, xy, 0.f);
-                    ptx::mbar_arrive_remote(ptx::map_to_cta(ptx::smem_addr(&ctl->xchg[par]), lane));
+            if (lane < C) {
+                const uint32_t slot = ptx::smem_addr(&ctl->part[par][rank * kClComputeWarps + warp]);
+                ptx::st_async_f32x2(ptx::map_to_cta(slot, lane), wm, ws,
+                                    ptx::map_to_cta(ptx::smem_addr(&ctl->xchg[par]), lane));
+            }
+            if (y_mine) {
+#pragma unroll
+                for (int c = 0; c < C; ++c)
+                    ptx::st_async_f32(ptx::map_to_cta(ptx::smem_addr(&ctl->xy[par]), c), x_y,
+                                      ptx::map_to_cta(ptx::smem_addr(&ctl->xchg[par]), c));
+            }
+            if (tid == 0) TL(rank, it, 4);
+            if (!ptx::mbar_wait<true>(ptx::smem_addr(&ctl->xchg[par]), xph)) { ok = false; break; }
+            if (tid == 0) TL(rank, it, 5);
+            // every warp combines the cluster's partials on its own
+            float pmx = -1.0e30f, psum = 0.f;
+            {
+                float2 p[(kClMaxParts + 31) / 32];
+#pragma unroll
+                for (int i = 0; i < (C * kClComputeWarps + 31) / 32; ++i) {
+                    const int idx = lane + i * 32;
+                    p[i] = idx < C * kClComputeWarps ? ctl->part[par][idx] : make_float2(-1.0e30f, 0.f);
+                    pmx = fmaxf(pmx, p[i].x);
                 }
-            }
-            if (!ptx::mbar_wait<true>(ptx::smem_addr(&ctl->xchg[par]), uint32_t(it >> 1) & 1u)) { ok = false; break; }
-            float Mx = -1.0e30f;
+                pmx = warp_max(pmx);
 #pragma unroll
-            for (int c = 0; c < C; ++c) Mx = fmaxf(Mx, ctl->part[par][c].x);
-            float Ssum = 0.f, xy = 0.f;
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                const float4 p = ctl->part[par][c];
-                Ssum += p.y * ex2((p.x - Mx) * kLog2e);
-                xy += p.z;
+                for (int i = 0; i < (C * kClComputeWarps + 31) / 32; ++i)
+                    psum += p[i].y * ex2((p[i].x - pmx) * kLog2e);
+                psum = warp_sum(psum);
             }
+            const float Mx = pmx, Ssum = psum;
+            if (tid == 0) TL(rank, it, 7);
             RowLoss rl;
             rl.logp = 0.f; rl.loss = 0.f; rl.coef = 0.f; rl.clip = 0;
-            if (meta.ok) rl = ppo_row(xy, Mx + logf(Ssum), old_lp, A, a.eps_low, a.eps_high, inv_denom);
+            if (rec_ok) rl = ppo_row(ctl->xy[par] - Mx, logf(Ssum), rec.old_logp, rec.adv, a.eps_low, a.eps_high, inv_denom);
             if (rank == 0 && tid == 0) {
-                if (!meta.ok) atomicOr(a.stats + 3, policy_bad_bits(meta, a));
                 if (a.logp) a.logp[j] = rl.logp;
                 if (a.token_loss) a.token_loss[j] = rl.loss;
                 a.row_loss[j] = rl.loss;
                 a.row_clip[j] = uint8_t(rl.clip);
             }
             if (GRAD) {
-                // ---- factor * (softmax - onehot), one rounding to bf16, back into the slice --
-                const float scale = meta.ok ? rl.coef * ex2((m_t - Mx) * kLog2e) / Ssum : 0.f;
+                // ---- factor * (softmax - onehot), one rounding to bf16 ---------------------------
+                const float scale = rec_ok ? rl.coef * ex2((m_t - Mx) * kLog2e) / Ssum : 0.f;   // skipped row: zeros
+                uint8_t* grow = nullptr;      // this CTA's slice of the gradient row (direct stores)
+                if (!STAGED) {
+                    if (a.mode == TPPO_DLOGITS_COMPACT) grow = dl + (j * int64_t(a.V)) * 2 + uint64_t(u0) * 16u;
+                    else if (row_ok) grow = dl + (int64_t(rec.row) * a.ld) * 2 + uint64_t(u0) * 16u;
+                }
+                const uint64_t sc2 = ptx::pack_f32x2(scale, scale);
 #pragma unroll
                 for (int k = 0; k < kClMaxUnits; ++k) {
                     const uint32_t u = uint32_t(tid) + uint32_t(k) * kClComputeThreads;
-                    float g[8];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) g[q] = meta.ok ? e[k][q] * scale : 0.f;
-                    if (y_mine && k == yk) {
-#pragma unroll
-                        for (int q = 0; q < 8; ++q) if (q == ye) g[q] -= rl.coef;
-                    }
                     if (u < nu) {
-                        ptx::sts128(sbase + u * 16u,
-                                    make_uint4(pack_bf16x2(g[0], g[1]), pack_bf16x2(g[2], g[3]),
-                                               pack_bf16x2(g[4], g[5]), pack_bf16x2(g[6], g[7])));
+                        uint4 g;
+                        g.x = ptx::pack_bf16x2_from_f32x2(ptx::mul_f32x2(e2[k][0], sc2));
+                        g.y = ptx::pack_bf16x2_from_f32x2(ptx::mul_f32x2(e2[k][1], sc2));
+                        g.z = ptx::pack_bf16x2_from_f32x2(ptx::mul_f32x2(e2[k][2], sc2));
+                        g.w = ptx::pack_bf16x2_from_f32x2(ptx::mul_f32x2(e2[k][3], sc2));
+                        if (STAGED) ptx::sts128(sbase + u * 16u, g);
+                        else if (grow) ptx::stg128(grow + u * 16u, g);
                     }
                 }
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->done[st]));
+                if (y_mine) {   // the one-hot term, applied before the single rounding
+                    const float g = ex2(fmaf(x_y, kLog2e, -off_t)) * scale - rl.coef;
+                    const uint16_t gb = uint16_t(pack_bf16x2(g, 0.f) & 0xffffu);
+                    if (STAGED) ptx::sts_u16(y_addr, gb);
+                    else if (grow) *reinterpret_cast<uint16_t*>(grow + y_off) = gb;   // after this thread's own 16-byte store
+                }
+                if (tid == 0) TL(rank, it, 3);
+                if (STAGED) {
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->done[st]));
+                }
+                if (tid == 0) TL(rank, it, 6);
             }
+            if (++st == S) { st = 0; ph ^= 1u; }
         }
         if (!ok && (tid & 31) == 0) atomicOr(a.stats + 3, TPPO_DEV_WAIT_TIMEOUT);
     }
@@ -304,7 +341,7 @@ struct ClusterPlan {
     int max_clusters;
 };
 
-template <int C, bool GRAD>
+template <int C, int OUT>
 static int plan_and_launch(const PolicyArgs& a, cudaStream_t s, int forced_stages) {
     const uint32_t units_total = uint32_t(a.V) >> 3;
     const uint32_t max_units = (units_total + C - 1) / C;     // largest slice, 16-byte units
@@ -321,7 +358,7 @@ static int plan_and_launch(const PolicyArgs& a, cudaStream_t s, int forced_stage
     if (forced_stages > 0 && uint32_t(forced_stages) < stages) stages = uint32_t(forced_stages);
     const uint32_t smem_bytes = kClCtlBytes + stages * stride;
 
-    auto kern = policy_cluster_kernel<C, GRAD>;
+    auto kern = policy_cluster_kernel<C, OUT>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes)) != cudaSuccess)
         return TPPO_ERR_CUDA;
     cudaLaunchConfig_t lc = {};
@@ -347,15 +384,23 @@ static int plan_and_launch(const PolicyArgs& a, cudaStream_t s, int forced_stage
     return TPPO_OK;
 }
 
-// variant: bits 0-3 cluster size (0 = default 4), bits 4-7 stage cap (0 = as many as fit)
+// variant: bits 0-3 cluster size (0 = default 4), bits 4-6 stage cap (0 = as many as fit),
+// bit 7: store the gradient straight from registers instead of staging it in shared memory for
+// bulk stores (measured slower: the 128-bit global stores stall the compute warps)
 int launch_policy_cluster(const PolicyArgs& a, cudaStream_t s, int variant) {
     const int c = (variant & 15) ? (variant & 15) : 4;
-    const int st = (variant >> 4) & 15;
-    const bool grad = a.mode != TPPO_DLOGITS_NONE;
-    switch (c) {
-        case 2: return grad ? plan_and_launch<2, true>(a, s, st) : plan_and_launch<2, false>(a, s, st);
-        case 4: return grad ? plan_and_launch<4, true>(a, s, st) : plan_and_launch<4, false>(a, s, st);
-        case 8: return grad ? plan_and_launch<8, true>(a, s, st) : plan_and_launch<8, false>(a, s, st);
+    const int st = (variant >> 4) & 7;
+    const int out = a.mode == TPPO_DLOGITS_NONE ? 0 : ((variant & 128) ? 2 : 1);
+    switch (c * 4 + out) {
+        case 2 * 4 + 0: return plan_and_launch<2, 0>(a, s, st);
+        case 2 * 4 + 1: return plan_and_launch<2, 1>(a, s, st);
+        case 2 * 4 + 2: return plan_and_launch<2, 2>(a, s, st);
+        case 4 * 4 + 0: return plan_and_launch<4, 0>(a, s, st);
+        case 4 * 4 + 1: return plan_and_launch<4, 1>(a, s, st);
+        case 4 * 4 + 2: return plan_and_launch<4, 2>(a, s, st);
+        case 8 * 4 + 0: return plan_and_launch<8, 0>(a, s, st);
+        case 8 * 4 + 1: return plan_and_launch<8, 1>(a, s, st);
+        case 8 * 4 + 2: return plan_and_launch<8, 2>(a, s, st);
         default: return TPPO_ERR_UNSUPPORTED;
     }
 }

@@ -29,7 +29,23 @@ struct PolicyArgs {
     float* row_loss;     // workspace [n_max]: per-row loss term, 0 for skipped rows
     uint8_t* row_clip;   // workspace [n_max]: 0 none, 1 lower edge, 2 upper edge
     uint8_t* row_flag;   // workspace [R]: 1 = row is selected (FULL mode with a row list)
+    struct RowRec* rec;  // workspace [n_max]: per-entry scalars gathered ahead of the vocabulary sweep
 };
+
+// Everything the vocabulary sweep needs to know about the j-th selected entry, gathered once by a
+// small kernel so that the sweep reads one 16-byte record per row instead of chasing indices.
+struct __align__(16) RowRec {
+    int32_t row;        // logits row, or -1 when the row index is out of range
+    int32_t y;          // target id, or -1 when the entry is to be skipped (bad row, aux or target)
+    float adv;          // adv[aux]
+    float old_logp;     // old_logp[aux]
+};
+__device__ __forceinline__ RowRec load_rec(const RowRec* p) {
+    const int4 v = __ldg(reinterpret_cast<const int4*>(p));
+    RowRec r;
+    r.row = v.x; r.y = v.y; r.adv = __int_as_float(v.z); r.old_logp = __int_as_float(v.w);
+    return r;
+}
 
 __device__ __forceinline__ int64_t policy_n(const PolicyArgs& a) {
     int64_t n = a.n_max;
@@ -80,10 +96,12 @@ struct RowLoss {
     float logp, loss, coef;
     int clip;
 };
-__device__ __forceinline__ RowLoss ppo_row(float x_y, float lse, float old_lp, float A,
+// x_y_rel = x_y - max_v x_v and log_sum = log sum_v exp(x_v - max) are passed separately so that
+// the log-prob keeps full precision when the logits are large.
+__device__ __forceinline__ RowLoss ppo_row(float x_y_rel, float log_sum, float old_lp, float A,
                                            float eps_low, float eps_high, float inv_denom) {
     RowLoss r;
-    r.logp = x_y - lse;
+    r.logp = x_y_rel - log_sum;
     const float rho = expf(r.logp - old_lp);
     const float lo = 1.f - eps_low, hi = 1.f + eps_high;
     const float rc = fminf(fmaxf(rho, lo), hi);

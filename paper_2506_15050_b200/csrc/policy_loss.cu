@@ -5,13 +5,24 @@
 namespace tppo {
 
 // ---- helper kernels -----------------------------------------------------------------------
-__global__ void policy_mark_rows_kernel(const PolicyArgs a) {
+// Gathers the per-entry scalars (row, target, advantage, old log-prob) into 16-byte records, checks
+// every index once, and in FULL mode marks the selected rows.
+__global__ void policy_prepare_kernel(const PolicyArgs a) {
     const int64_t n = policy_n(a);
+    int bad = 0;
     for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n;
          j += int64_t(gridDim.x) * blockDim.x) {
-        const int64_t r = __ldg(a.rows + j);
-        if (r >= 0 && r < a.R) a.row_flag[r] = 1;
+        const RowMeta m = policy_row_meta(a, j);
+        RowRec r;
+        r.row = m.row_ok ? int32_t(m.row) : -1;
+        r.y = m.ok ? m.y : -1;
+        r.adv = m.ok ? __ldg(a.adv + m.aux) : 0.f;
+        r.old_logp = m.ok ? __ldg(a.old_logp + m.aux) : 0.f;
+        a.rec[j] = r;
+        if (!m.ok) bad |= policy_bad_bits(m, a);
+        if (m.row_ok && a.rows && a.mode == TPPO_DLOGITS_FULL) a.row_flag[m.row] = 1;
     }
+    if (bad) atomicOr(a.stats + 3, bad);
 }
 
 // FULL mode: rows of dlogits that are not selected get zeros in their V columns.
@@ -72,13 +83,14 @@ __global__ void __launch_bounds__(1024) policy_finish_kernel(const PolicyArgs a)
 }
 
 
-int launch_policy_two_pass(const PolicyArgs& a, int dtype, cudaStream_t s);
+int launch_policy_two_pass(const PolicyArgs& a, int dtype, cudaStream_t s, int variant);
 int launch_policy_cluster(const PolicyArgs& a, cudaStream_t s, int variant);
 bool policy_cluster_supported(const PolicyArgs& a, int dtype);
 
 size_t policy_workspace_bytes(int64_t R, int64_t n_max) {
-    return align_up(size_t(n_max > 0 ? n_max : 1) * sizeof(float), kWsAlign) +
-           align_up(size_t(n_max > 0 ? n_max : 1), kWsAlign) + align_up(size_t(R > 0 ? R : 1), kWsAlign);
+    const size_t n = size_t(n_max > 0 ? n_max : 1);
+    return align_up(n * sizeof(float), kWsAlign) + align_up(n, kWsAlign) +
+           align_up(size_t(R > 0 ? R : 1), kWsAlign) + align_up(n * sizeof(RowRec), kWsAlign);
 }
 }  // namespace tppo
 
@@ -122,6 +134,8 @@ TPPO_API int tppo_policy_loss_fwd_bwd(const void* logits, int32_t logits_dtype, 
     a.row_clip = reinterpret_cast<uint8_t*>(w);
     w += align_up(size_t(n_max > 0 ? n_max : 1), kWsAlign);
     a.row_flag = reinterpret_cast<uint8_t*>(w);
+    w += align_up(size_t(R > 0 ? R : 1), kWsAlign);
+    a.rec = reinterpret_cast<RowRec*>(w);
 
     const int base_hint = kernel_hint & 0xff;
     const bool can_cluster = policy_cluster_supported(a, logits_dtype);
@@ -131,23 +145,23 @@ TPPO_API int tppo_policy_loss_fwd_bwd(const void* logits, int32_t logits_dtype, 
         return TPPO_ERR_INVALID_ARG;
 
     TPPO_CUDA_CHECK(cudaMemsetAsync(stats, 0, 4 * sizeof(int32_t), s));
+    const bool fill_rows = dlogits_mode == TPPO_DLOGITS_FULL && R > 0;
+    if (fill_rows && rows) TPPO_CUDA_CHECK(cudaMemsetAsync(a.row_flag, 0, size_t(R), s));
     if (n_max > 0) {
-        const bool use_cluster =
-            base_hint == TPPO_POLICY_CLUSTER_SMEM || (base_hint == TPPO_POLICY_AUTO && can_cluster);
+        const int pb = int((n_max + 255) / 256 < 1184 ? (n_max + 255) / 256 : 1184);
+        policy_prepare_kernel<<<pb, 256, 0, s>>>(a);
+        // The cluster kernel wins when a gradient is written; a forward-only sweep reads each row
+        // once in either kernel and the plain one keeps more rows in flight.
+        const bool use_cluster = base_hint == TPPO_POLICY_CLUSTER_SMEM ||
+                                 (base_hint == TPPO_POLICY_AUTO && can_cluster &&
+                                  dlogits_mode != TPPO_DLOGITS_NONE);
         int rc = TPPO_ERR_UNSUPPORTED;
         if (use_cluster) rc = launch_policy_cluster(a, s, (kernel_hint >> 8) & 0xff);
-        if (rc == TPPO_ERR_UNSUPPORTED && base_hint == TPPO_POLICY_AUTO) rc = TPPO_ERR_UNSUPPORTED + 100;
-        if (!use_cluster || rc == TPPO_ERR_UNSUPPORTED + 100) rc = launch_policy_two_pass(a, logits_dtype, s);
+        if (!use_cluster || (rc == TPPO_ERR_UNSUPPORTED && base_hint == TPPO_POLICY_AUTO))
+            rc = launch_policy_two_pass(a, logits_dtype, s, (kernel_hint >> 8) & 0xff);
         if (rc != TPPO_OK) return rc;
     }
-    if (dlogits_mode == TPPO_DLOGITS_FULL && R > 0) {
-        if (rows) {
-            TPPO_CUDA_CHECK(cudaMemsetAsync(a.row_flag, 0, size_t(R), s));
-            if (n_max > 0) {
-                const int blocks = int((n_max + 255) / 256 < 1184 ? (n_max + 255) / 256 : 1184);
-                policy_mark_rows_kernel<<<blocks, 256, 0, s>>>(a);
-            }
-        }
+    if (fill_rows) {
         const int zb = int(R < 1184 ? R : 1184);
         if (logits_dtype == TPPO_BF16) policy_zero_rows_kernel<uint16_t><<<zb, 256, 0, s>>>(a);
         else policy_zero_rows_kernel<float><<<zb, 256, 0, s>>>(a);

@@ -62,7 +62,7 @@ template <int DT, bool VEC>
 __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const PolicyArgs a) {
     using T = typename ElemT<DT>::type;
     __shared__ float s_m[kTwoPassThreads / 32], s_s[kTwoPassThreads / 32];
-    __shared__ float s_lse, s_coef;
+    __shared__ float s_max, s_logsum, s_coef;
 
     const int64_t n = policy_n(a);
     const float inv_denom = policy_inv_denom(a, n);
@@ -71,14 +71,15 @@ __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const 
     T* dl = static_cast<T*>(a.dlogits);
 
     for (int64_t j = blockIdx.x; j < n; j += gridDim.x) {
-        const RowMeta meta = policy_row_meta(a, j);
-        const T* x_row = logits + (meta.row_ok ? meta.row : 0) * a.ld;
+        const RowRec rec = load_rec(a.rec + j);
+        const bool row_ok = rec.row >= 0, rec_ok = rec.y >= 0;
+        const T* x_row = logits + int64_t(row_ok ? rec.row : 0) * a.ld;
         T* g_row = nullptr;
-        if (a.mode == TPPO_DLOGITS_FULL && meta.row_ok) g_row = dl + meta.row * a.ld;
+        if (a.mode == TPPO_DLOGITS_FULL && row_ok) g_row = dl + int64_t(rec.row) * a.ld;
         if (a.mode == TPPO_DLOGITS_COMPACT) g_row = dl + j * int64_t(a.V);
 
-        float coef = 0.f, lse = 0.f;
-        if (meta.ok) {
+        float coef = 0.f, row_max = 0.f, log_sum = 0.f;
+        if (rec_ok) {
             // ---- pass 1 -------------------------------------------------------------------
             float m = -1.0e30f, s = 0.f;
             if (VEC) {
@@ -107,21 +108,22 @@ __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const 
                 for (int w = 1; w < kTwoPassThreads / 32; ++w) M = fmaxf(M, s_m[w]);
                 float S = 0.f;
                 for (int w = 0; w < kTwoPassThreads / 32; ++w) S += s_s[w] * ex2((s_m[w] - M) * kLog2e);
-                const float l = M + logf(S);
-                const RowLoss rl = ppo_row(load_elem(x_row + meta.y), l, __ldg(a.old_logp + meta.aux),
-                                           __ldg(a.adv + meta.aux), a.eps_low, a.eps_high, inv_denom);
+                const float log_s = logf(S);
+                const RowLoss rl = ppo_row(load_elem(x_row + rec.y) - M, log_s, rec.old_logp, rec.adv,
+                                           a.eps_low, a.eps_high, inv_denom);
                 if (a.logp) a.logp[j] = rl.logp;
                 if (a.token_loss) a.token_loss[j] = rl.loss;
                 a.row_loss[j] = rl.loss;
                 a.row_clip[j] = uint8_t(rl.clip);
-                s_lse = l;
+                s_max = M;
+                s_logsum = log_s;
                 s_coef = rl.coef;
             }
             __syncthreads();
             coef = s_coef;
-            lse = s_lse;
+            row_max = s_max;
+            log_sum = s_logsum;
         } else if (tid == 0) {
-            atomicOr(a.stats + 3, policy_bad_bits(meta, a));
             if (a.logp) a.logp[j] = 0.f;
             if (a.token_loss) a.token_loss[j] = 0.f;
             a.row_loss[j] = 0.f;
@@ -130,7 +132,7 @@ __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const 
 
         // ---- pass 2 -----------------------------------------------------------------------
         if (g_row) {
-            const float off = lse * kLog2e;
+            const float off = log_sum * kLog2e;   // exponent of softmax_v = (x_v - max)*log2e - off
             if (coef == 0.f) {   // clipped, zero advantage or invalid entry: the gradient row is zero
                 if (VEC) {
                     const int nu = a.V >> 3;
@@ -142,12 +144,12 @@ __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const 
                 }
             } else if (VEC) {
                 const int nu = a.V >> 3;
-                const int yu = meta.y >> 3, yk = meta.y & 7;
+                const int yu = rec.y >> 3, yk = rec.y & 7;
                 for (int u = tid; u < nu; u += kTwoPassThreads) {
                     float x[8], g[8];
                     load8(x_row + (int64_t(u) << 3), x);
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) g[k] = coef * ex2(fmaf(x[k], kLog2e, -off));
+                    for (int k = 0; k < 8; ++k) g[k] = coef * ex2(fmaf(x[k] - row_max, kLog2e, -off));
                     if (u == yu) {
 #pragma unroll
                         for (int k = 0; k < 8; ++k) if (k == yk) g[k] -= coef;
@@ -155,25 +157,27 @@ __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const 
                     store8(g_row + (int64_t(u) << 3), g);
                 }
                 for (int v = (nu << 3) + tid; v < a.V; v += kTwoPassThreads) {
-                    float g = coef * ex2(fmaf(load_elem(x_row + v), kLog2e, -off));
-                    if (v == meta.y) g -= coef;
+                    float g = coef * ex2(fmaf(load_elem(x_row + v) - row_max, kLog2e, -off));
+                    if (v == rec.y) g -= coef;
                     store_elem(g_row + v, g);
                 }
             } else {
                 for (int v = tid; v < a.V; v += kTwoPassThreads) {
-                    float g = coef * ex2(fmaf(load_elem(x_row + v), kLog2e, -off));
-                    if (v == meta.y) g -= coef;
+                    float g = coef * ex2(fmaf(load_elem(x_row + v) - row_max, kLog2e, -off));
+                    if (v == rec.y) g -= coef;
                     store_elem(g_row + v, g);
                 }
             }
         }
-        __syncthreads();   // s_lse / s_coef are reused by the next row
+        __syncthreads();   // the shared row scalars are reused by the next row
     }
 }
 
-int launch_policy_two_pass(const PolicyArgs& a, int dtype, cudaStream_t s) {
+// variant: blocks per SM (0 = default 3)
+int launch_policy_two_pass(const PolicyArgs& a, int dtype, cudaStream_t s, int variant) {
+    const int per_sm = (variant & 15) ? (variant & 15) : 3;
     int64_t blocks = a.n_max < 1 ? 1 : a.n_max;
-    if (blocks > kNumSms * 3) blocks = kNumSms * 3;
+    if (blocks > kNumSms * per_sm) blocks = kNumSms * per_sm;
     const size_t esz = dtype == TPPO_BF16 ? 2 : 4;
     bool vec = aligned(a.logits, 16) && (a.ld * esz) % 16 == 0;
     if (a.mode == TPPO_DLOGITS_FULL) vec = vec && aligned(a.dlogits, 16);

@@ -76,7 +76,10 @@ def run_policy(logits_t, targets, rows, aux_idx, old_logp, adv, eps_low, eps_hig
     if mode == b.DLOGITS_NONE:
         dl = None
     elif mode == b.DLOGITS_FULL:
-        dl = logits_t if inplace else torch.full_like(logits_t, float("nan"))
+        if inplace:
+            dl = logits_t
+        else:   # FULL mode shares the logits' row stride
+            dl = torch.full((R, logits_t.stride(0)), float("nan"), dtype=logits_t.dtype, device=DEV)[:, :logits_t.shape[1]]
     else:
         dl = torch.full((max(n_max, 1), V), float("nan"), dtype=logits_t.dtype, device=DEV)
     ws = b.workspace(b.OP_POLICY_LOSS, R, 0, n_max, V, DEV)
