@@ -35,6 +35,9 @@ from paper_2506_15050_b200 import synth  # noqa: E402
 METRIC = "selected tokens/s, fused logprob+PPO loss fwd+bwd, V=152064 bf16; % HBM peak"
 UNIT = "selected tokens/s"
 ALGO_BYTES_PER_TOKEN = 2 * 2 * synth.V_QWEN       # bf16 row read once + bf16 gradient row written once
+# dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the sweep kernel at 2048 rows
+# (1194.38 MB; the full workload is too large to capture), per row; traffic is proportional to rows.
+NCU_TRAFFIC_BYTES_PER_TOKEN = 1194.38e6 / 2048
 
 
 def measured_peaks():
@@ -366,7 +369,9 @@ def main():
                        "dlogits": "compact, separate buffer", "kernel_hint": args.hint},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": peak_kind,
-                         "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": None,
+                         "frac_of_nominal_8TBs": achieved / 8000.0,
+                         "traffic": n_tok * NCU_TRAFFIC_BYTES_PER_TOKEN if st.V == synth.V_QWEN else None,
+                         "traffic_note": "ncu DRAM bytes of a 2048-row capture scaled by rows",
                          "kernel": "policy_cluster_kernel", "kernel_ms": pol_ms,
                          "algorithmic_bytes_per_launch": n_tok * ALGO_BYTES_PER_TOKEN},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": Step.KERNELS_PER_STEP * args.steps,
