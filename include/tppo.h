@@ -39,7 +39,8 @@ typedef enum {
     TPPO_ERR_INVALID_ARG = 1, /* null / negative / inconsistent argument, bad alignment      */
     TPPO_ERR_WORKSPACE = 2,   /* workspace pointer null, misaligned or smaller than required */
     TPPO_ERR_UNSUPPORTED = 3, /* valid request this build cannot serve                       */
-    TPPO_ERR_CUDA = 4         /* a CUDA runtime call failed (launch error, wrong device)     */
+    TPPO_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch error, wrong device)     */
+    TPPO_ERR_TOO_LARGE = 5    /* problem exceeds a fixed built-in capacity (see *_static)    */
 } tppo_status;
 
 /* bits of the device status word */
@@ -108,6 +109,36 @@ int tppo_egae(const float *rewards, const float *values,
               int32_t B, int64_t N, float gamma, float lambda,
               float *advantages, float *returns, int32_t *status,
               void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * tppo_egae without a caller workspace and without any allocation.  (The paper has no counterpart:
+ * this is a packaging variant of tppo_egae, same arithmetic, same outputs.)
+ *
+ * Who needs it: code that runs where device memory cannot be requested -- a plug-in inside a
+ * training or serving runtime that has already reserved the whole device for its own pool (a raw
+ * cudaMalloc there fails or fragments the pool), or a latency-critical section that must not pay
+ * cudaMalloc's device-wide synchronisation -- and that has no spare buffer of its own to lend as
+ * workspace.  The scan's tile descriptors live in a fixed array compiled into the library
+ * (TPPO_EGAE_STATIC_MAX_TOKENS / 2048 descriptors of 64 bytes plus one counter, about 128 KB); every
+ * GPU that loads the library holds that array until the process exits.
+ *
+ * Arguments and results are those of tppo_egae minus the workspace pair.  Differences:
+ *   - N > TPPO_EGAE_STATIC_MAX_TOKENS returns TPPO_ERR_TOO_LARGE before anything is launched.
+ *   - The first call on each device looks up the device address of the built-in array (the device
+ *     must be current, as for every call) and caches it; make that first call outside any stream
+ *     capture.  Later calls only enqueue a clear of the array and the kernel.
+ *   - All calls on a device share the one array, which still holds the previous call's contents:
+ *     each call clears it on `stream` before the scan.  Two calls that can overlap on the GPU
+ *     (different streams without an ordering between them) race on it and give undefined results;
+ *     order them, or use tppo_egae with separate workspaces.
+ * The function calls no cudaMalloc / cudaFree and no allocating library routine.
+ */
+#define TPPO_EGAE_STATIC_MAX_TOKENS 4194304
+int tppo_egae_static(const float *rewards, const float *values,
+                     const int32_t *seg_begin, const int32_t *seg_end,
+                     const uint8_t *truncated, const float *bootstrap,
+                     int32_t B, int64_t N, float gamma, float lambda,
+                     float *advantages, float *returns, int32_t *status, void *stream);
 
 /*
  * Token filter and compaction (Section 3.2; "selective filtering of prompt and truncated tokens").

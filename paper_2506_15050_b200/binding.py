@@ -36,6 +36,8 @@ _lib.tppo_workspace_bytes.argtypes = [C.c_int, _i64, _i32, _i64, _i32]
 _lib.tppo_egae.restype = C.c_int
 _lib.tppo_egae.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _f32, _vp, _vp, _vp,
                            _vp, _sz, _vp]
+_lib.tppo_egae_static.restype = C.c_int
+_lib.tppo_egae_static.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _f32, _vp, _vp, _vp, _vp]
 _lib.tppo_select_tokens.restype = C.c_int
 _lib.tppo_select_tokens.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _i32, _i64, _vp, _vp,
                                     _vp, _vp, _sz, _vp]
@@ -99,6 +101,23 @@ def tppo_egae(rewards, values, seg_begin, seg_end, truncated, bootstrap, gamma, 
                           B, N, gamma, lam, _ptr(advantages, torch.float32),
                           _ptr(returns, torch.float32), _ptr(status, torch.int32),
                           _ptr(ws), ws.numel(), _stream()))
+
+
+EGAE_STATIC_MAX_TOKENS = 4194304
+
+
+def tppo_egae_static(rewards, values, seg_begin, seg_end, truncated, bootstrap, gamma, lam,
+                     advantages, returns, status):
+    """tppo_egae for callers that cannot allocate device memory and have no workspace to lend
+    (e.g. a plug-in inside a runtime that owns the device's whole memory pool): the scan's scratch
+    is a fixed array inside the library.  At most EGAE_STATIC_MAX_TOKENS tokens; calls on one device
+    share that array, so calls that may overlap on the GPU must be ordered by the caller."""
+    N, B = rewards.numel(), seg_begin.numel()
+    _check(_lib.tppo_egae_static(_ptr(rewards, torch.float32), _ptr(values, torch.float32),
+                                 _ptr(seg_begin, torch.int32), _ptr(seg_end, torch.int32),
+                                 _ptr(truncated, torch.uint8), _ptr(bootstrap, torch.float32),
+                                 B, N, gamma, lam, _ptr(advantages, torch.float32),
+                                 _ptr(returns, torch.float32), _ptr(status, torch.int32), _stream()))
 
 
 def tppo_select_tokens(seq_begin, prompt_len, prev_len, new_len, truncated, tail_drop,

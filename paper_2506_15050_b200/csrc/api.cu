@@ -18,6 +18,7 @@ TPPO_API const char* tppo_status_string(int status) {
         case TPPO_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case TPPO_ERR_UNSUPPORTED: return "unsupported";
         case TPPO_ERR_CUDA: return "CUDA runtime error";
+        case TPPO_ERR_TOO_LARGE: return "problem larger than the built-in capacity of this entry point";
         default: return "unknown status";
     }
 }

@@ -248,3 +248,70 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
     TPPO_CUDA_CHECK(cudaGetLastError());
     return TPPO_OK;
 }
+
+// ---- allocation-free variant ------------------------------------------------------------------
+// For callers that can neither allocate device memory nor lend a workspace (a plug-in inside a
+// runtime that owns the whole device's memory pool; a latency-critical section that must avoid
+// cudaMalloc's device-wide synchronisation).  The tile descriptors and the ticket counter live in
+// this fixed device array; each GPU that loads the library keeps it until the process ends.
+namespace tppo {
+constexpr int64_t kStaticMaxTokens = TPPO_EGAE_STATIC_MAX_TOKENS;
+constexpr size_t kStaticTiles = size_t((kStaticMaxTokens + kScanTile - 1) / kScanTile);
+constexpr size_t kStaticScratchBytes = 256 + kStaticTiles * sizeof(TileState);
+static_assert(sizeof(TileState) == 64, "tile descriptor is 64 bytes");
+}  // namespace tppo
+
+static __device__ __align__(256) unsigned char g_egae_static_scratch[tppo::kStaticScratchBytes];
+
+namespace tppo {
+constexpr int kMaxDevices = 64;
+// Device address of g_egae_static_scratch per device ordinal.  In host code the array's name is
+// only a handle for the runtime, never a device address: the address comes from
+// cudaGetSymbolAddress, asked once per device with that device current.
+static void* g_static_scratch_addr[kMaxDevices] = {};
+
+static int static_scratch_for_current_device(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TPPO_ERR_CUDA;
+    void* p = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        if (cudaGetSymbolAddress(&p, g_egae_static_scratch) != cudaSuccess || !p) return TPPO_ERR_CUDA;
+        __atomic_store_n(&g_static_scratch_addr[dev], p, __ATOMIC_RELEASE);   // same value from any thread
+    }
+    *out = p;
+    return TPPO_OK;
+}
+}  // namespace tppo
+
+TPPO_API int tppo_egae_static(const float* rewards, const float* values, const int32_t* seg_begin,
+                              const int32_t* seg_end, const uint8_t* truncated,
+                              const float* bootstrap, int32_t B, int64_t N, float gamma,
+                              float lambda, float* advantages, float* returns, int32_t* status,
+                              void* stream) {
+    if (B < 0 || N < 0 || !status) return TPPO_ERR_INVALID_ARG;
+    if (N > kStaticMaxTokens) return TPPO_ERR_TOO_LARGE;
+    if (N > 0 && (!rewards || !values || !advantages)) return TPPO_ERR_INVALID_ARG;
+    if (B > 0 && (!seg_begin || !seg_end || !truncated)) return TPPO_ERR_INVALID_ARG;
+    if (!(gamma >= 0.f && gamma <= 1.f) || !(lambda >= 0.f && lambda <= 1.f))
+        return TPPO_ERR_INVALID_ARG;
+    void* scratch = nullptr;
+    const int rc = static_scratch_for_current_device(&scratch);
+    if (rc != TPPO_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
+    if (N == 0) return TPPO_OK;
+    EgaeArgs a;
+    a.rewards = rewards; a.values = values; a.seg_begin = seg_begin; a.seg_end = seg_end;
+    a.truncated = truncated; a.bootstrap = bootstrap; a.B = B; a.N = int32_t(N);
+    a.num_tiles = int32_t((N + kScanTile - 1) / kScanTile);
+    a.gamma = double(gamma);
+    a.gl = double(gamma) * double(lambda);
+    a.adv = advantages; a.ret = returns; a.status = status;
+    a.ticket = static_cast<uint32_t*>(scratch);
+    a.state = reinterpret_cast<TileState*>(static_cast<char*>(scratch) + 256);
+    // the array still holds the previous call's flags and ticket: clear the part this call uses
+    TPPO_CUDA_CHECK(cudaMemsetAsync(scratch, 0, 256 + size_t(a.num_tiles) * sizeof(TileState), s));
+    egae_scan_kernel<<<a.num_tiles, kScanThreads, 0, s>>>(a);
+    TPPO_CUDA_CHECK(cudaGetLastError());
+    return TPPO_OK;
+}
