@@ -231,13 +231,27 @@ int tppo_value_loss(const float *values, const float *old_values, const float *r
                     void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * LM-head variant of the fused policy loss: the logits x = hidden * weight are a dense
- * [M,K] x [K,V] contraction on the tensor cores and are never written to memory; outputs are the
- * loss, the log-probs and the gradients dhidden = dX * weight^T and dweight = hidden^T * dX.
- * (Math as tppo_policy_loss_fwd_bwd with all M rows selected.)  Returns TPPO_ERR_UNSUPPORTED in
- * builds without the tensor-core kernel.
- *   hidden [M,K] bf16, weight [K,V] bf16, targets [M], aux_idx [M] or NULL, old_logp/adv fp32
- *   dhidden [M,K] bf16 out, dweight [K,V] bf16 out
+ * LM-head variant of the fused policy loss (Eq. 1 as in tppo_policy_loss_fwd_bwd, every one of the
+ * M rows selected): the logits x = hidden * weight are a dense [M,K] x [K,V] bf16 contraction on
+ * the tensor cores (fp32 accumulation) and are never written to memory.  Outputs are the loss, the
+ * per-row log-probs and losses, and the gradients
+ *     dhidden = dX * weight^T,   dweight = hidden^T * dX,   dX = (adv*rho*active/denom)(softmax - onehot).
+ * The vocabulary is swept twice (statistics, then gradients with the logits recomputed); dX exists
+ * only as a bf16 buffer for one chunk of vocabulary columns at a time inside the workspace.
+ *
+ *   hidden   [M, K] bf16 row-major     weight  [K, V] bf16 row-major     (16-byte aligned)
+ *   targets  [M] int32                 aux_idx [M] int32 index into old_logp / adv, or NULL (= row)
+ *   old_logp, adv   fp32, length aux_len
+ *   logp, token_loss [M] fp32 out or NULL;  loss [1] fp32 out;  stats [4] int32 out as in
+ *   tppo_policy_loss_fwd_bwd (n = M)
+ *   dhidden  [M, K] bf16 out or NULL;  dweight [K, V] bf16 out or NULL (both NULL: forward only)
+ *   chunk_tiles  0 = choose automatically; otherwise the number of 256-column vocabulary tiles per
+ *                chunk, clamped to the automatic choice (which sizes the workspace).  For tuning
+ *                and testing; changes the result only by the rounding order of dhidden's sum.
+ *   workspace    tppo_workspace_bytes(TPPO_OP_LMHEAD, M, K, 0, V) bytes
+ * K and V must be multiples of 8 (TPPO_ERR_UNSUPPORTED otherwise).  A row with a target outside
+ * [0, V) or an aux index outside [0, aux_len) contributes nothing and raises the status bit.
+ * The first call on a device looks up the driver's tensor-map encoder (TPPO_ERR_CUDA if absent).
  */
 int tppo_lmhead_logprob_fwd_bwd(const void *hidden, const void *weight,
                                 int64_t M, int32_t K, int32_t V,
@@ -245,7 +259,7 @@ int tppo_lmhead_logprob_fwd_bwd(const void *hidden, const void *weight,
                                 const float *old_logp, const float *adv, int64_t aux_len,
                                 float eps_low, float eps_high, float denom,
                                 float *logp, float *token_loss, float *loss, int32_t *stats,
-                                void *dhidden, void *dweight,
+                                void *dhidden, void *dweight, int32_t chunk_tiles,
                                 void *workspace, size_t workspace_bytes, void *stream);
 
 #ifdef __cplusplus

@@ -59,8 +59,10 @@ def _logits_view(logits):
         code = 0
     elif a.dtype == np.float32:
         code = 1
+    elif a.dtype == np.float64:
+        code = 2
     else:
-        raise TypeError("logits must be uint16 (bf16 bits) or float32")
+        raise TypeError("logits must be uint16 (bf16 bits), float32 or float64")
     return a, code, a.strides[0] // a.itemsize
 
 

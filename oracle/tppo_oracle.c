@@ -41,11 +41,14 @@ static double widen_bf16(uint16_t h)
     return (double)f;
 }
 
-/* dtype: 0 = bf16 (uint16 storage), 1 = fp32 */
+/* dtype: 0 = bf16 (uint16 storage), 1 = fp32, 2 = double (logits the oracle formed itself from
+ * hidden states and the LM-head weight) */
 static double logit_at(const void *logits, int dtype, int64_t ld, int64_t row, int64_t v)
 {
     if (dtype == 0)
         return widen_bf16(((const uint16_t *)logits)[row * ld + v]);
+    if (dtype == 2)
+        return ((const double *)logits)[row * ld + v];
     return (double)((const float *)logits)[row * ld + v];
 }
 

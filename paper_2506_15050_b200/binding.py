@@ -50,8 +50,8 @@ _lib.tppo_value_loss.argtypes = [_vp, _vp, _vp, _i64, _vp, _vp, _i64, _f32, _f32
                                  _vp, _vp, _sz, _vp]
 _lib.tppo_lmhead_logprob_fwd_bwd.restype = C.c_int
 _lib.tppo_lmhead_logprob_fwd_bwd.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _i64,
-                                             _f32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
-                                             _sz, _vp]
+                                             _f32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, _i32,
+                                             _vp, _sz, _vp]
 
 
 class TppoError(RuntimeError):
@@ -167,8 +167,9 @@ def tppo_value_loss(values, old_values, returns, value_idx, n_sel, n_max, xi_low
 
 def tppo_lmhead_logprob_fwd_bwd(hidden, weight, targets, aux_idx, old_logp, adv, eps_low,
                                 eps_high, denom, logp, token_loss, loss, stats, dhidden, dweight,
-                                ws):
+                                ws, chunk_tiles=0):
     M, K = hidden.shape
+    assert weight.shape[0] == K
     V = weight.shape[1]
     _check(_lib.tppo_lmhead_logprob_fwd_bwd(
         _ptr(hidden, torch.bfloat16), _ptr(weight, torch.bfloat16), M, K, V,
@@ -176,4 +177,4 @@ def tppo_lmhead_logprob_fwd_bwd(hidden, weight, targets, aux_idx, old_logp, adv,
         _ptr(adv, torch.float32), old_logp.numel(), eps_low, eps_high, denom,
         _ptr(logp, torch.float32), _ptr(token_loss, torch.float32), _ptr(loss, torch.float32),
         _ptr(stats, torch.int32), _ptr(dhidden, torch.bfloat16), _ptr(dweight, torch.bfloat16),
-        _ptr(ws), ws.numel(), _stream()))
+        chunk_tiles, _ptr(ws), ws.numel(), _stream()))

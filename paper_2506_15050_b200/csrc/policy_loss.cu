@@ -82,6 +82,19 @@ __global__ void __launch_bounds__(1024) policy_finish_kernel(const PolicyArgs a)
     }
 }
 
+// Host launchers of the two helper kernels for other translation units (the LM-head variant).
+int launch_policy_prepare(const PolicyArgs& a, cudaStream_t s) {
+    if (a.n_max <= 0) return TPPO_OK;
+    const int pb = int((a.n_max + 255) / 256 < 1184 ? (a.n_max + 255) / 256 : 1184);
+    policy_prepare_kernel<<<pb, 256, 0, s>>>(a);
+    TPPO_CUDA_CHECK(cudaGetLastError());
+    return TPPO_OK;
+}
+int launch_policy_finish(const PolicyArgs& a, cudaStream_t s) {
+    policy_finish_kernel<<<1, 1024, 0, s>>>(a);
+    TPPO_CUDA_CHECK(cudaGetLastError());
+    return TPPO_OK;
+}
 
 int launch_policy_two_pass(const PolicyArgs& a, int dtype, cudaStream_t s, int variant);
 int launch_policy_cluster(const PolicyArgs& a, cudaStream_t s, int variant);

@@ -1,0 +1,186 @@
+"""GPU parity of the LM-head variant (logits = hidden x weight on the tensor cores, never stored)
+against the oracle, which forms the logits in float64 from the same bf16 inputs and then applies
+its ordinary policy-loss routine and the plain definitions dH = dX W^T, dW = H^T dX.
+
+Tolerances: log-probs, per-token losses and the loss 2e-3 absolute; gradients 1e-2 of the largest
+reference magnitude per tensor, plus a per-element worst-case rounding bound: dX is rounded to bf16
+(unit roundoff 2^-8) before the second contraction and the result once more, so
+|gpu - ref| <= 2^-8 * (sum |a||b| + |ref|), the sum of absolute products coming from the oracle's own
+contraction routines applied to the operands with their sign bits cleared."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_15050_b200 import binding as b
+from paper_2506_15050_b200 import synth
+from gpu_util import DEV
+
+pytestmark = pytest.mark.gpu
+f32 = lambda x: float(np.float32(x))
+LOGP_ATOL = 2e-3
+GRAD_RTOL = 1e-2
+
+
+def t(a, dt):
+    return None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(dt).to(DEV)
+
+
+def run_lmhead(hidden, weight, targets, old_logp, adv, eps_low, eps_high, denom=0.0, aux=None,
+               want_dh=True, want_dw=True, chunk_tiles=0):
+    M, K = hidden.shape
+    V = weight.shape[1]
+    logp = torch.full((M,), float("nan"), device=DEV)
+    tl = torch.full((M,), float("nan"), device=DEV)
+    loss = torch.full((1,), float("nan"), device=DEV)
+    stats = torch.full((4,), -1, dtype=torch.int32, device=DEV)
+    dh = torch.full((M, K), float("nan"), dtype=torch.bfloat16, device=DEV) if want_dh else None
+    dw = torch.full((K, V), float("nan"), dtype=torch.bfloat16, device=DEV) if want_dw else None
+    ws = b.workspace(b.OP_LMHEAD, M, K, 0, V, DEV)
+    b.tppo_lmhead_logprob_fwd_bwd(hidden, weight, t(targets, torch.int32), t(aux, torch.int32),
+                                  t(old_logp, torch.float32), t(adv, torch.float32), eps_low,
+                                  eps_high, denom, logp, tl, loss, stats, dh, dw, ws,
+                                  chunk_tiles=chunk_tiles)
+    torch.cuda.synchronize()
+    return dict(logp=logp.cpu().numpy(), token_loss=tl.cpu().numpy(), loss=float(loss),
+                stats=stats.cpu().numpy(), dh=None if dh is None else dh.float().cpu().numpy(),
+                dw=None if dw is None else dw.float().cpu().numpy(), dh_t=dh, dw_t=dw)
+
+
+def oracle_lmhead(hb, wb, rows, targets, old_logp, adv, eps_low, eps_high, denom):
+    """Oracle results for the given rows: float64 logits, then Eq. 1 on them."""
+    x = oracle.lmhead_logits_rows(hb, wb, np.asarray(rows, np.int32))
+    ref = oracle.policy_loss(x, np.asarray(targets)[rows], None, None, np.asarray(old_logp)[rows],
+                             np.asarray(adv)[rows], eps_low, eps_high, denom=denom)
+    return x, ref
+
+
+def grad_close(gpu, ref, abs_sum, what):
+    scale = float(np.max(np.abs(ref)))
+    err = np.abs(gpu - ref)
+    assert np.all(np.isfinite(gpu)), what
+    assert float(err.max()) <= GRAD_RTOL * scale + 1e-30, (what, float(err.max()), scale)
+    bound = 1.05 * 2.0 ** -8 * (abs_sum + np.abs(ref)) + 1e-30
+    assert np.all(err <= bound), (what, float((err / bound).max()))
+
+
+def magnitude(bits):
+    return np.asarray(bits) & np.uint16(0x7FFF)
+
+
+def ref_dhidden(dx, wb):
+    return oracle.lmhead_dhidden_rows(dx, wb), oracle.lmhead_dhidden_rows(np.abs(dx), magnitude(wb))
+
+
+def ref_dweight(hb, dx):
+    return oracle.lmhead_dweight_cols(hb, dx), oracle.lmhead_dweight_cols(magnitude(hb), np.abs(dx))
+
+
+def make_case(M, K, V, seed, w_std=0.05):
+    hidden = synth.randn_bf16((M, K), 1.0, seed, DEV)
+    weight = synth.randn_bf16((K, V), w_std, seed + 1000, DEV)
+    rng = np.random.default_rng(seed)
+    targets = rng.integers(0, V, M).astype(np.int32)
+    adv = rng.standard_normal(M).astype(np.float32)
+    noise = (0.05 * rng.standard_normal(M)).astype(np.float32)
+    return hidden, weight, targets, adv, noise
+
+
+def old_logp_from_oracle(hb, wb, targets, noise):
+    M = hb.shape[0]
+    x = oracle.lmhead_logits_rows(hb, wb, np.arange(M, dtype=np.int32))
+    lp = oracle.logprob(x, targets)
+    return x, (lp + noise).astype(np.float32)
+
+
+@pytest.mark.parametrize("M,K,V,chunk", [(300, 320, 2000, 0), (300, 320, 2000, 3),
+                                         (1024, 512, 8200, 5), (128, 64, 256, 0)])
+def test_lmhead_matches_oracle(M, K, V, chunk):
+    hidden, weight, targets, adv, noise = make_case(M, K, V, seed=40 + M % 7)
+    hb, wb = synth.bf16_bits(hidden), synth.bf16_bits(weight)
+    x, old_logp = old_logp_from_oracle(hb, wb, targets, noise)
+    eps_low, eps_high = 0.2, 0.28
+    ref = oracle.policy_loss(x, targets, None, None, old_logp, adv, f32(eps_low), f32(eps_high))
+    out = run_lmhead(hidden, weight, targets, old_logp, adv, eps_low, eps_high, chunk_tiles=chunk)
+    assert out["stats"][3] == 0 and out["stats"][0] == M
+    assert np.max(np.abs(out["logp"] - ref["logp"])) <= LOGP_ATOL
+    # rows whose ratio sits on a clip edge may take the other branch in fp32
+    rho = np.exp(ref["logp"] - old_logp)
+    edge = (np.abs(rho - (1 - eps_low)) < 1e-3) | (np.abs(rho - (1 + eps_high)) < 1e-3)
+    assert np.max(np.abs(out["token_loss"] - ref["token_loss"])[~edge]) <= LOGP_ATOL
+    assert abs(out["loss"] - ref["loss"]) <= LOGP_ATOL
+    assert abs(int(out["stats"][1]) - ref["clip_lo"]) <= int(edge.sum())
+    assert abs(int(out["stats"][2]) - ref["clip_hi"]) <= int(edge.sum())
+    dx = ref["dlogits"]
+    dx[edge] = 0.0
+    keep = ~edge
+    ref_dh, abs_dh = ref_dhidden(dx, wb)
+    grad_close(out["dh"][keep], ref_dh[keep], abs_dh[keep], "dhidden")
+    if not edge.any():
+        grad_close(out["dw"], *ref_dweight(hb, dx), "dweight")
+    # clipped rows have a zero gradient
+    clipped = (ref["dlogits"] == 0).all(axis=1) & keep
+    assert np.all(out["dh"][clipped] == 0)
+
+
+def test_lmhead_forward_only_and_denominator():
+    M, K, V = 256, 128, 1024
+    hidden, weight, targets, adv, noise = make_case(M, K, V, seed=7)
+    hb, wb = synth.bf16_bits(hidden), synth.bf16_bits(weight)
+    x, old_logp = old_logp_from_oracle(hb, wb, targets, noise)
+    ref = oracle.policy_loss(x, targets, None, None, old_logp, adv, f32(0.2), f32(0.2), denom=1000.0)
+    fwd = run_lmhead(hidden, weight, targets, old_logp, adv, 0.2, 0.2, denom=1000.0, want_dh=False,
+                     want_dw=False)
+    assert abs(fwd["loss"] - ref["loss"]) <= LOGP_ATOL
+    assert np.max(np.abs(fwd["logp"] - ref["logp"])) <= LOGP_ATOL
+    full = run_lmhead(hidden, weight, targets, old_logp, adv, 0.2, 0.2, denom=1000.0)
+    assert full["loss"] == fwd["loss"] and np.array_equal(full["logp"], fwd["logp"])
+    grad_close(full["dh"], *ref_dhidden(ref["dlogits"], wb), "dhidden")
+
+
+def test_lmhead_aux_index_and_bad_rows():
+    M, K, V = 200, 64, 512
+    hidden, weight, targets, adv, noise = make_case(M, K, V, seed=11)
+    hb, wb = synth.bf16_bits(hidden), synth.bf16_bits(weight)
+    x, old_logp = old_logp_from_oracle(hb, wb, targets, noise)
+    rng = np.random.default_rng(3)
+    perm = rng.permutation(M).astype(np.int32)              # row j reads adv / old_logp at perm[j]
+    adv_p = np.empty_like(adv); adv_p[perm] = adv
+    old_p = np.empty_like(old_logp); old_p[perm] = old_logp
+    bad_t = targets.copy(); bad_t[5] = V; bad_t[17] = -1
+    aux = perm.copy(); aux[40] = M + 3
+    good = np.ones(M, bool); good[[5, 17, 40]] = False
+    out = run_lmhead(hidden, weight, bad_t, old_p, adv_p, 0.2, 0.2, aux=aux)
+    assert out["stats"][3] == (b.DEV_BAD_TARGET | b.DEV_BAD_INDEX)
+    # the mean still divides by M; the three bad rows contribute nothing
+    rows = np.nonzero(good)[0].astype(np.int32)
+    ref = oracle.policy_loss(x, targets, rows, None, old_logp, adv, f32(0.2), f32(0.2), denom=float(M))
+    assert abs(out["loss"] - ref["loss"]) <= LOGP_ATOL
+    assert np.max(np.abs(out["logp"][good] - ref["logp"])) <= LOGP_ATOL
+    assert np.all(out["logp"][~good] == 0) and np.all(out["token_loss"][~good] == 0)
+    assert np.all(out["dh"][~good] == 0)
+    grad_close(out["dh"][good], *ref_dhidden(ref["dlogits"], wb), "dhidden")
+    dx_all = np.zeros((M, V)); dx_all[good] = ref["dlogits"]
+    grad_close(out["dw"], *ref_dweight(hb, dx_all), "dweight")
+
+
+def test_lmhead_host_errors_and_determinism():
+    M, K, V = 128, 64, 512
+    hidden, weight, targets, adv, noise = make_case(M, K, V, seed=5)
+    old = np.full(M, -6.0, np.float32)
+    a = run_lmhead(hidden, weight, targets, old, adv, 0.2, 0.2)
+    c = run_lmhead(hidden, weight, targets, old, adv, 0.2, 0.2)
+    assert a["loss"] == c["loss"] and torch.equal(a["dh_t"], c["dh_t"]) and torch.equal(a["dw_t"], c["dw_t"])
+    ws = b.workspace(b.OP_LMHEAD, M, K, 0, V, DEV)
+    loss = torch.zeros(1, device=DEV)
+    stats = torch.zeros(4, dtype=torch.int32, device=DEV)
+    args = lambda h, w, wsp: (h, w, t(targets, torch.int32), None, t(old, torch.float32),
+                              t(adv, torch.float32), 0.2, 0.2, 0.0, None, None, loss, stats, None,
+                              None, wsp)
+    with pytest.raises(b.TppoError) as e:
+        b.tppo_lmhead_logprob_fwd_bwd(*args(hidden, weight, ws[:256]))
+    assert e.value.status == 2
+    w_odd = synth.randn_bf16((K, 508), 0.05, 1, DEV)          # V not a multiple of 8
+    with pytest.raises(b.TppoError) as e:
+        b.tppo_lmhead_logprob_fwd_bwd(*args(hidden, w_odd, ws))
+    assert e.value.status == 3
