@@ -184,3 +184,89 @@ def test_lmhead_host_errors_and_determinism():
     with pytest.raises(b.TppoError) as e:
         b.tppo_lmhead_logprob_fwd_bwd(*args(hidden, w_odd, ws))
     assert e.value.status == 3
+
+
+# ---------------------------------------------------------------------------------------------
+# config 5 at full size: [16384, 5120] x [5120, 152064], the launch configuration that is timed.
+# The oracle forms one vocabulary row of logits at a time, so it checks sampled rows in full and,
+# for dweight (which sums over all rows), a run whose advantages are zero outside the sampled
+# rows: every other row then has dX = 0 and the reference sum has only the sampled terms.
+# ---------------------------------------------------------------------------------------------
+LOG_V_MODEL = -13.0      # typical log-prob of a random token under these logits (an input, not a result)
+
+
+def _config5_sample(c, n_rows, seed):
+    rng = np.random.default_rng(seed)
+    M = c["M"]
+    pick = np.sort(rng.choice(M, n_rows, replace=False)).astype(np.int32)
+    pick[0], pick[-1] = 0, M - 1
+    pick[1], pick[2] = 127, 128                     # both sides of a tile boundary
+    return np.unique(pick).astype(np.int32)
+
+
+@pytest.fixture(scope="module")
+def cfg5():
+    c = synth.config5(DEV)
+    assert c["hidden"].shape == (16384, 5120) and c["weight"].shape == (5120, 152064)
+    c["hb"], c["wb"] = synth.bf16_bits(c["hidden"]), synth.bf16_bits(c["weight"])
+    c["pick"] = _config5_sample(c, 16, seed=50)
+    c["x_pick"] = oracle.lmhead_logits_rows(c["hb"], c["wb"], c["pick"])
+    lp = oracle.logprob(c["x_pick"], c["targets"][c["pick"]])
+    old = (LOG_V_MODEL + c["old_logp_noise"]).astype(np.float32)
+    old[c["pick"]] = (lp + c["old_logp_noise"][c["pick"]]).astype(np.float32)
+    c["old_logp"] = old
+    yield c
+    del c["hidden"], c["weight"]
+    torch.cuda.empty_cache()
+
+
+def test_config5_full_sampled_rows(cfg5):
+    c = cfg5
+    M, K, V, pick = c["M"], c["K"], c["V"], c["pick"]
+    out = run_lmhead(c["hidden"], c["weight"], c["targets"], c["old_logp"], c["adv"], c["eps_low"],
+                     c["eps_high"])
+    assert out["stats"][0] == M and out["stats"][3] == 0
+    ref = oracle.policy_loss(c["x_pick"], c["targets"][pick], None, None, c["old_logp"][pick],
+                             c["adv"][pick], f32(c["eps_low"]), f32(c["eps_high"]), denom=float(M))
+    np.testing.assert_allclose(out["logp"][pick], ref["logp"], rtol=0, atol=LOGP_ATOL)
+    np.testing.assert_allclose(out["token_loss"][pick], ref["token_loss"], rtol=0, atol=4 * LOGP_ATOL)
+    grad_close(out["dh"][pick], *ref_dhidden(ref["dlogits"], c["wb"]), "dhidden rows")
+    # properties that hold at any size
+    assert np.all(np.isfinite(out["logp"])) and np.all(out["logp"] < 0)
+    assert abs(out["loss"] - float(np.mean(out["token_loss"].astype(np.float64)))) <= 1e-5
+    dw = out["dw_t"].float()
+    assert bool(torch.isfinite(dw).all()) and bool(torch.isfinite(out["dh_t"].float()).all())
+    # every dX row sums to zero, hence every dweight row does
+    row_sum = dw.sum(dim=1).abs()
+    row_abs = dw.abs().sum(dim=1)
+    assert float((row_sum / row_abs).max()) < 1e-3
+    # the run is reproducible bit for bit
+    again = run_lmhead(c["hidden"], c["weight"], c["targets"], c["old_logp"], c["adv"], c["eps_low"],
+                       c["eps_high"])
+    assert again["loss"] == out["loss"] and torch.equal(again["dw_t"], out["dw_t"]) and \
+        torch.equal(again["dh_t"], out["dh_t"])
+
+
+def test_config5_full_dweight_from_sampled_rows(cfg5):
+    c = cfg5
+    M, K, V, pick = c["M"], c["K"], c["V"], c["pick"]
+    adv = np.zeros(M, np.float32)
+    adv[pick] = c["adv"][pick]
+    out = run_lmhead(c["hidden"], c["weight"], c["targets"], c["old_logp"], adv, c["eps_low"],
+                     c["eps_high"])
+    assert out["stats"][3] == 0
+    ref = oracle.policy_loss(c["x_pick"], c["targets"][pick], None, None, c["old_logp"][pick],
+                             adv[pick], f32(c["eps_low"]), f32(c["eps_high"]), denom=float(M))
+    assert np.any(ref["dlogits"] != 0)
+    rng = np.random.default_rng(51)
+    cols = np.concatenate([rng.choice(V, 1500, replace=False), [0, 255, 256, V - 1, V - 8],
+                           c["targets"][pick]]).astype(np.int64)
+    cols = np.unique(cols)
+    got = out["dw_t"][:, torch.from_numpy(cols).to(DEV)].float().cpu().numpy()
+    dx_cols = np.ascontiguousarray(ref["dlogits"][:, cols])
+    hb_pick = np.ascontiguousarray(c["hb"][pick])
+    grad_close(got, *ref_dweight(hb_pick, dx_cols), "dweight columns")
+    # rows without advantage have an exactly zero gradient; the sampled ones match the oracle
+    others = np.setdiff1d(np.arange(M), pick)
+    assert float(out["dh_t"][torch.from_numpy(others).to(DEV)].float().abs().max()) == 0.0
+    grad_close(out["dh"][pick], *ref_dhidden(ref["dlogits"], c["wb"]), "dhidden rows")
