@@ -9,6 +9,11 @@ on 16384 value tokens.  The metric is selected (policy) tokens per second.
 
   python bench.py [--gpus N] [--steps K] [--warmup W]            CUDA path (this repo)
   python bench.py --impl reference ...                           float64 CPU oracle on host cores
+  python bench.py --workload lmhead ...                          the LM-head variant as the bench line
+
+The default line also carries an "lmhead_variant" object: the tensor-core variant that forms the
+logits from hidden states [16384, 5120] and the LM-head weight [5120, 152064] without storing them,
+timed on its own after the main measurement (a few calls) against the bf16 tensor roofline.
 
 Prints one JSON line.  With N > 1 (torchrun) every rank runs the same per-GPU workload (the path
 shards by sequence with no data-path collective); the time is the max over ranks.
@@ -46,6 +51,16 @@ def measured_peaks():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return 6650.0, "fallback"
+
+
+def measured_tensor_peaks():
+    """(burst, sustained) dense bf16 TFLOP/s of this machine's B200s and where the figures come from."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            j = json.load(f)
+            return float(j["bf16_tflops"]), float(j["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return 1590.0, 1400.0, "fallback"
 
 
 class ClockSampler:
@@ -192,6 +207,88 @@ class Step:
     KERNELS_PER_STEP = 6   # egae scan, select, policy prepare + sweep + finish, value loss
 
 
+class LmHeadStep:
+    """Device-resident state of the LM-head workload (config 5) and its one C-ABI call."""
+    KERNELS_FIXED = 4      # prepare, statistics GEMM, row merge, finish
+
+    def __init__(self, dev, M=16384, K=5120, V=synth.V_QWEN):
+        from paper_2506_15050_b200 import binding as b
+        self.b, self.dev = b, dev
+        c = synth.config5(dev, M=M, K=K, V=V)
+        self.c, self.M, self.K, self.V = c, M, K, V
+        t = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).to(dev)
+        self.hidden, self.weight = c["hidden"], c["weight"]
+        self.targets, self.adv = t(c["targets"], torch.int32), t(c["adv"], torch.float32)
+        self.old_logp = torch.zeros(M, device=dev)
+        self.logp, self.tok_loss = torch.zeros(M, device=dev), torch.zeros(M, device=dev)
+        self.loss = torch.zeros(1, device=dev)
+        self.stats = torch.zeros(4, dtype=torch.int32, device=dev)
+        self.dhidden = torch.empty_like(self.hidden)
+        self.dweight = torch.empty_like(self.weight)
+        self.ws = b.workspace(b.OP_LMHEAD, M, K, 0, V, dev)
+        # old-policy log-probs: forward-only call of the same entry point, plus noise
+        self.run(forward_only=True)
+        torch.cuda.synchronize()
+        self.old_logp.copy_(self.logp + t(c["old_logp_noise"], torch.float32))
+
+    def run(self, forward_only=False):
+        c = self.c
+        self.b.tppo_lmhead_logprob_fwd_bwd(
+            self.hidden, self.weight, self.targets, None, self.old_logp, self.adv, c["eps_low"],
+            c["eps_high"], 0.0, self.logp, self.tok_loss, self.loss, self.stats,
+            None if forward_only else self.dhidden, None if forward_only else self.dweight, self.ws)
+
+    def gemm_flops(self):
+        return 2.0 * self.M * self.K * self.V
+
+    def roofline(self, ms):
+        """Tensor roofline: three GEMM-sized contractions are what the result needs (logits, dhidden,
+        dweight); the kernels execute a fourth (the logits are recomputed instead of stored)."""
+        burst, sustained, kind = measured_tensor_peaks()
+        achieved = 3.0 * self.gemm_flops() / (ms * 1e-3) / 1e12
+        return {"bound": "tensor", "achieved": achieved, "peak": sustained, "unit": "TFLOP/s",
+                "frac": achieved / sustained, "peak_kind": kind + ", sustained (calls run back to back)",
+                "frac_of_burst_peak": achieved / burst, "traffic": None,
+                "executed_tflops": 4.0 * self.gemm_flops() / (ms * 1e-3) / 1e12,
+                "executed_frac": 4.0 * self.gemm_flops() / (ms * 1e-3) / 1e12 / sustained,
+                "kernel": "umma_gemm_kernel (statistics, dX, dhidden, dweight epilogues)",
+                "call_ms": ms, "algorithmic_flops_per_call": 3.0 * self.gemm_flops()}
+
+
+def time_lmhead(lm, calls, warmup):
+    for _ in range(warmup):
+        lm.run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(calls):
+        lm.run()
+    e1.record()
+    torch.cuda.synchronize()
+    assert int(lm.stats[3].item()) == 0 and int(lm.stats[0].item()) == lm.M
+    return e0.elapsed_time(e1) / calls
+
+
+def cpu_oracle_lmhead_seconds(lm, sample_rows):
+    """The oracle on `sample_rows` rows of the LM-head workload: float64 logits, Eq. 1, dhidden rows
+    and those rows' share of dweight; scaled by rows to the whole call."""
+    import oracle
+    f32 = lambda x: float(np.float32(x))
+    c = lm.c
+    rows = np.arange(sample_rows, dtype=np.int32)
+    hb = synth.bf16_bits(lm.hidden[:sample_rows])
+    wb = synth.bf16_bits(lm.weight)
+    old = lm.old_logp[:sample_rows].cpu().numpy()
+    t0 = time.perf_counter()
+    x = oracle.lmhead_logits_rows(hb, wb, rows)
+    ref = oracle.policy_loss(x, c["targets"][:sample_rows], None, None, old, c["adv"][:sample_rows],
+                             f32(c["eps_low"]), f32(c["eps_high"]), denom=float(lm.M))
+    oracle.lmhead_dhidden_rows(ref["dlogits"], wb)
+    oracle.lmhead_dweight_cols(hb, ref["dlogits"])
+    t = time.perf_counter() - t0
+    return t * (lm.M / sample_rows), oracle.num_threads()
+
+
 def cpu_oracle_step_seconds(c, n_tokens, sample_rows):
     """Times the oracle, as it stands, on host cores: EGAE and selection on the full batch, policy
     loss forward+backward on `sample_rows` rows of the micro-batch (scaled to n_tokens), value loss."""
@@ -258,6 +355,11 @@ def main():
     ap.add_argument("--hint", type=int, default=0, help="kernel_hint passed to the policy loss")
     ap.add_argument("--rows", type=int, default=16384,
                     help="rows of the loss micro-batch (smaller only for profiler captures)")
+    ap.add_argument("--workload", default="cfg3", choices=["cfg3", "lmhead"])
+    ap.add_argument("--lmhead-calls", type=int, default=5)
+    ap.add_argument("--lm-rows", type=int, default=16384,
+                    help="rows of the LM-head workload (smaller only for profiler captures)")
+    ap.add_argument("--no-lmhead", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -271,6 +373,9 @@ def main():
     warmup = max(args.warmup, 3)
     dev = f"cuda:{local}"
     torch.cuda.set_device(local)
+    if args.workload == "lmhead":
+        run_lmhead_workload(args, rank, world, local, dev, warmup)
+        return
     st = Step(dev, rows=args.rows)
     st.hint = args.hint
 
@@ -357,6 +462,21 @@ def main():
                           f"{args.cpu_rows} of {n_tok} rows scaled to the micro-batch"),
                "seconds": {k: round(v, 4) for k, v in parts.items()}}
 
+    lmhead = None
+    if rank == 0 and not args.no_lmhead:
+        del st.logits, st.dlogits, st.c["logits"]
+        torch.cuda.empty_cache()
+        lm = LmHeadStep(dev, M=args.lm_rows)
+        ms = time_lmhead(lm, args.lmhead_calls, 3)
+        lmhead = {"workload": "cfg5: hidden [%d,%d] x LM-head weight [%d,%d] bf16, loss + dhidden + "
+                              "dweight, logits never stored" % (lm.M, lm.K, lm.K, lm.V),
+                  "value": lm.M / (ms * 1e-3), "unit": UNIT, "ms_per_call": ms,
+                  "calls": args.lmhead_calls, "roofline": lm.roofline(ms)}
+        del lm
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
     if rank == 0:
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -375,7 +495,83 @@ def main():
                          "kernel": "policy_cluster_kernel", "kernel_ms": pol_ms,
                          "algorithmic_bytes_per_launch": n_tok * ALGO_BYTES_PER_TOKEN},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": Step.KERNELS_PER_STEP * args.steps,
-            "clocks": clocks}))
+            "clocks": clocks, "lmhead_variant": lmhead}))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def run_lmhead_workload(args, rank, world, local, dev, warmup):
+    """The LM-head variant as the bench line: one step = one call (loss, dhidden, dweight)."""
+    lm = LmHeadStep(dev, M=args.lm_rows)
+    steps = args.steps if args.steps != 200 else 20
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        lm.run()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        lm.run()
+    t1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms = t0.elapsed_time(t1) / steps
+    if world > 1:
+        import torch.distributed as dist
+        tt = torch.tensor([ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    assert int(lm.stats[3].item()) == 0
+    e2e = None
+    if not args.no_e2e:
+        h_h, h_w = lm.hidden.cpu().pin_memory(), lm.weight.cpu().pin_memory()
+        h_loss = torch.empty(1, dtype=torch.float32).pin_memory()
+
+        def e2e_step():
+            lm.hidden.copy_(h_h, non_blocking=True)
+            lm.weight.copy_(h_w, non_blocking=True)
+            lm.run()
+            h_loss.copy_(lm.loss, non_blocking=True)
+            torch.cuda.synchronize()
+
+        e2e_step()
+        barrier()
+        w0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        barrier()
+        e2e_s = (time.perf_counter() - w0) / args.e2e_steps
+        e2e = {"value": world * lm.M / e2e_s, "unit": UNIT,
+               "h2d_bytes_per_step": int((h_h.numel() + h_w.numel()) * 2), "d2h_bytes_per_step": 4,
+               "ms_per_step": e2e_s * 1e3, "steps": args.e2e_steps}
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        t, cores = cpu_oracle_lmhead_seconds(lm, 8)
+        cpu = {"value": lm.M / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": "8 of %d rows (float64 logits, Eq. 1, dhidden rows, dweight share), scaled by rows" % lm.M}
+    n_chunk_launches = 3 * ((lm.V + 255) // 256 + 61) // 62
+    if rank == 0:
+        print(json.dumps({
+            "metric": "selected tokens/s, LM-head variant: fused hidden x vocab contraction + PPO loss "
+                      "fwd+bwd, V=152064 bf16; % tensor peak",
+            "value": world * lm.M / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
+            "config": {"workload": "cfg5: hidden [%d,%d] x LM-head weight [%d,%d] bf16, loss + dhidden + "
+                                   "dweight, logits never stored" % (lm.M, lm.K, lm.K, lm.V),
+                       "l2": "inputs larger than L2 (%.2f GB of weights per sweep)" % (lm.K * lm.V * 2 / 1e9)},
+            "roofline": lm.roofline(ms), "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": (LmHeadStep.KERNELS_FIXED + n_chunk_launches) * steps, "clocks": clocks}))
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
