@@ -8,6 +8,9 @@
 // left, publishes the composite, and obtains the value entering from its right-hand neighbour by
 // decoupled look-back over the tiles behind it.  A composite whose `a` has become 0 (a segment
 // ended inside the range) ends the look-back early.  State is fp64, rounded once on store.
+// Tiles are staged in shared memory so that every global access is a coalesced 16-byte one.
+#include <cstddef>
+
 #include "common.cuh"
 
 namespace tppo {
@@ -16,6 +19,8 @@ constexpr int kScanThreads = 256;
 constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kScanItems = 8;
 constexpr int kScanTile = kScanThreads * kScanItems;  // 2048 positions
+constexpr int kSegCap = 96;                           // segments of one tile kept in shared memory
+constexpr int kScanCtasPerSm = 3;
 constexpr uint32_t kScanSpinLimit = 1u << 22;
 
 struct Affine2 {  // x -> (aA*xA + bA, aR*xR + bR)
@@ -31,12 +36,31 @@ __device__ __forceinline__ Affine2 shfl_down(const Affine2& f, int d) {
                    __shfl_down_sync(0xffffffffu, f.aR, d), __shfl_down_sync(0xffffffffu, f.bR, d)};
 }
 
-struct TileState {     // one per tile, 64 bytes
-    double agg[4];     // composite of the tile (valid when flag >= 1)
-    double inc[2];     // A and R at the tile's first position (valid when flag == 2)
-    int flag;
-    int pad[3];
+// One per tile, 64 bytes, three self-validating 16-byte pairs.  The array starts out as all-ones
+// bytes; a pair counts as published only when neither of its two words holds that pattern, so a
+// reader needs one load per pair and neither a separate flag nor a fence (each 8-byte word is
+// written whole, and a pair with one word still unset is simply read again).
+struct TileState {
+    double aggA[2];    // (a, b) of the tile's composite for the advantage recurrence
+    double aggR[2];    // (a, b) of the tile's composite for the return recurrence
+    double inc[2];     // A and R at the tile's first position
+    double pad[2];
 };
+static_assert(sizeof(TileState) == 64, "tile state is four 16-byte pairs");
+constexpr unsigned long long kUnset = 0xffffffffffffffffull;
+// NaNs are published with the canonical quiet pattern so that no result can look unset.
+__device__ __forceinline__ double publishable(double x) {
+    return x != x ? __longlong_as_double(0x7ff8000000000000ll) : x;
+}
+__device__ __forceinline__ void st_pair(double* p, double x, double y) {
+    asm volatile("st.relaxed.gpu.global.v2.f64 [%0], {%1, %2};"
+                 ::"l"(p), "d"(publishable(x)), "d"(publishable(y)) : "memory");
+}
+__device__ __forceinline__ bool ld_pair(const double* p, double& x, double& y) {
+    asm volatile("ld.relaxed.gpu.global.v2.f64 {%0, %1}, [%2];" : "=d"(x), "=d"(y) : "l"(p) : "memory");
+    return (unsigned long long)__double_as_longlong(x) != kUnset &&
+           (unsigned long long)__double_as_longlong(y) != kUnset;
+}
 
 struct EgaeArgs {
     const float* rewards;
@@ -48,6 +72,7 @@ struct EgaeArgs {
     int32_t B;
     int32_t N;
     int32_t num_tiles;
+    int32_t vec_ok;   // rewards, values, adv, ret are all 16-byte aligned
     double gamma;
     double gl;  // gamma * lambda
     float* adv;
@@ -57,154 +82,349 @@ struct EgaeArgs {
     uint32_t* ticket;
 };
 
-// number of entries of arr[0..n) that are <= key
-__device__ __forceinline__ int seg_count_le(const int32_t* __restrict__ arr, int n, int32_t key) {
-    int lo = 0, hi = n;
+// Number of entries of the ascending array arr[0..n) that are <= key, found by a whole warp: each
+// round probes 32 evenly spaced entries, so 4096 entries take three rounds of one load each
+// instead of twelve dependent loads.  Every lane returns the same count.  An array that is not
+// ascending still yields an in-range answer.
+__device__ __forceinline__ int warp_count_le(const int32_t* __restrict__ arr, int n, int32_t key,
+                                             int lane) {
+    int lo = 0, hi = n;       // the answer lies in [lo, hi]
     while (lo < hi) {
-        int mid = (lo + hi) >> 1;
-        if (__ldg(arr + mid) <= key) lo = mid + 1; else hi = mid;
+        const int span = hi - lo;
+        const int step = (span + 31) >> 5;
+        const int idx = lo + lane * step;
+        const bool le = idx < hi && __ldg(arr + idx) <= key;
+        const uint32_t m = __ballot_sync(0xffffffffu, le);
+        const int c = __ffs(int(~m)) - 1;          // leading run of probes that are <= key
+        if (c < 0) { lo = min(lo + 31 * step + 1, hi); continue; }   // all 32 probes <= key
+        const int new_hi = min(lo + c * step, hi);
+        if (c > 0) lo = lo + (c - 1) * step + 1;
+        hi = new_hi;
     }
     return lo;
 }
 
-__global__ void __launch_bounds__(kScanThreads) egae_scan_kernel(const EgaeArgs a) {
-    __shared__ uint32_t s_ticket;
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                 ::"r"(uint32_t(__cvta_generic_to_shared(smem_dst))), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.wait_all;" ::: "memory");
+}
+
+// Shared-memory image of one tile: its inputs (later overwritten by its outputs) and the window of
+// segments that can touch it.  Aligned and sized to 16 bytes: r and v are accessed as float4 and by
+// 16-byte cp.async in both halves of a two-element array.
+struct __align__(16) TileBuf {
+    float r[kScanTile];          // rewards in, advantages out
+    float v[kScanTile + 4];      // values in (+1 look-ahead), returns out
+    int32_t seg_b[kSegCap], seg_e[kSegCap];
+    float seg_boot[kSegCap];
+    uint8_t seg_t[kSegCap];
+    int win_lo, win_hi;          // segment indices [win_lo, win_hi) may touch the tile
+};
+static_assert(sizeof(TileBuf) % 16 == 0 && offsetof(TileBuf, v) % 16 == 0, "vector access alignment");
+
+// Starts the copy of a tile's rewards and values into `buf`.  16-byte chunks go through cp.async
+// (the caller waits with cp_async_wait_all and a barrier); a ragged tail or unaligned arrays are
+// read directly.
+__device__ __forceinline__ void egae_stage_inputs(const EgaeArgs& a, TileBuf& buf, int64_t t0,
+                                                  int n_tile) {
+    if (a.vec_ok) {
+        for (int u = threadIdx.x; u < kScanTile / 4; u += kScanThreads) {
+            if (4 * u + 4 <= n_tile) {
+                cp_async16(buf.r + 4 * u, a.rewards + t0 + 4 * u);
+                cp_async16(buf.v + 4 * u, a.values + t0 + 4 * u);
+            } else {
+                for (int k = 4 * u; k < n_tile; ++k) {
+                    buf.r[k] = __ldg(a.rewards + t0 + k);
+                    buf.v[k] = __ldg(a.values + t0 + k);
+                }
+            }
+        }
+    } else {
+        for (int k = threadIdx.x; k < n_tile; k += kScanThreads) {
+            buf.r[k] = __ldg(a.rewards + t0 + k);
+            buf.v[k] = __ldg(a.values + t0 + k);
+        }
+    }
+    if (threadIdx.x == kScanThreads - 1)    // value of the position after the tile, if there is one
+        buf.v[n_tile] = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
+}
+
+// Segments are ascending and disjoint, so seg_begin and seg_end are both ascending: the window of
+// a tile starts after the segments that end at or before its first position and stops before those
+// that begin after its last one.  Called by two whole warps (which = 0: lower end, 1: upper end).
+__device__ __forceinline__ void egae_window_search(const EgaeArgs& a, TileBuf& buf, int64_t t0,
+                                                   int n_tile, int which, int lane) {
+    if (which == 0) {
+        const int lo = warp_count_le(a.seg_end, a.B, int32_t(t0), lane);
+        if (lane == 0) buf.win_lo = lo;
+    } else {
+        const int hi = warp_count_le(a.seg_begin, a.B, int32_t(t0 + n_tile - 1), lane);
+        if (lane == 0) buf.win_hi = hi;
+    }
+}
+// Copies the window's segments into shared memory (when they fit).  Returns true when a segment
+// with bounds outside [0, N] or end < begin was seen; such a segment is treated as empty.
+__device__ __forceinline__ bool egae_window_load(const EgaeArgs& a, TileBuf& buf) {
+    const int win_lo = buf.win_lo, win_n = buf.win_hi - buf.win_lo;
+    bool bad = false;
+    if (win_n <= kSegCap) {
+        for (int j = threadIdx.x; j < win_n; j += kScanThreads) {
+            const int i = win_lo + j;
+            int32_t b = __ldg(a.seg_begin + i), e = __ldg(a.seg_end + i);
+            if (b < 0 || e > a.N || e < b) { bad = true; e = b; }
+            buf.seg_b[j] = b;
+            buf.seg_e[j] = e;
+            buf.seg_t[j] = __ldg(a.truncated + i);
+            buf.seg_boot[j] = a.bootstrap ? __ldg(a.bootstrap + i) : 0.f;
+        }
+    }
+    return bad;
+}
+
+// Persistent CTAs take tiles by ticket, from the END of the arrays backwards, so the tiles a tile
+// looks back at (those to its right) hold earlier tickets and are running or done.  While a tile is
+// being scanned the next ticket is drawn, the next tile's inputs stream into the other buffer
+// (cp.async) and two idle warps find its segment window, so none of those latencies is exposed.
+__global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel(const EgaeArgs a) {
+    __shared__ __align__(16) TileBuf s_buf[2];
+    __shared__ uint32_t s_ticket[2];
     __shared__ Affine2 s_warp[kScanWarps];
+    __shared__ Affine2 s_right[kScanWarps];      // composite of the warps to the right of warp w
     __shared__ double s_carry[kScanWarps][2];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) s_ticket = atomicAdd(a.ticket, 1u);
+    if (threadIdx.x == 0) s_ticket[0] = atomicAdd(a.ticket, 1u);
     __syncthreads();
-    if (s_ticket >= uint32_t(a.num_tiles)) return;
-    // Tickets go to tiles from the END of the arrays backwards, so the tiles this one looks back
-    // at (those to its right) already hold earlier tickets and are running or done.
-    const int tile = a.num_tiles - 1 - int(s_ticket);
-    const int64_t base = int64_t(tile) * kScanTile + int64_t(threadIdx.x) * kScanItems;
+    uint32_t ticket = s_ticket[0];
+    if (ticket >= uint32_t(a.num_tiles)) return;
+    bool bad = false;
+    {   // first tile of this CTA: nothing to overlap with
+        const int tile = a.num_tiles - 1 - int(ticket);
+        const int64_t t0 = int64_t(tile) * kScanTile;
+        const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
+        egae_stage_inputs(a, s_buf[0], t0, n_tile);
+        if (warp < 2) egae_window_search(a, s_buf[0], t0, n_tile, warp, lane);
+        __syncthreads();
+        bad |= egae_window_load(a, s_buf[0]);
+        cp_async_wait_all();
+        __syncthreads();
+    }
 
-    // ---- per-position maps, right to left -------------------------------------------------
-    double delta[kScanItems], rew[kScanItems];
-    uint32_t cont = 0;  // bit k: position k continues into position k+1 (same segment)
-    Affine2 f = identity2();
-    {
-        const int64_t p_last = min(base + kScanItems, int64_t(a.N)) - 1;
-        int i = (p_last >= base) ? seg_count_le(a.seg_begin, a.B, int32_t(p_last)) - 1 : -1;
-        bool bad = false;
+    for (int it = 0;; ++it) {
+        TileBuf& buf = s_buf[it & 1];
+        TileBuf& nbuf = s_buf[(it & 1) ^ 1];
+        const int tile = a.num_tiles - 1 - int(ticket);
+        const int64_t t0 = int64_t(tile) * kScanTile;
+        const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
+        if (threadIdx.x == 0) s_ticket[(it & 1) ^ 1] = atomicAdd(a.ticket, 1u);   // next tile
+
+        // ---- per-position maps, right to left -----------------------------------------------
+        const int win_lo = buf.win_lo;
+        const int win_n = max(buf.win_hi - win_lo, 0);
+        const bool win_smem = win_n <= kSegCap;
+        const int l0 = threadIdx.x * kScanItems;  // first position of this thread inside the tile
+        double delta[kScanItems];
+        float rew[kScanItems];
+        uint32_t cont = 0;  // bit k: position k continues into position k+1 (same segment)
+        Affine2 f = identity2();
+        {
+            // index (inside the window) of the last segment that begins at or before the thread's
+            // last position, or -1
+            const int l_last = min(l0 + kScanItems, n_tile) - 1;
+            int i = -1;
+            if (l_last >= l0) {
+                const int32_t key = int32_t(t0 + l_last);
+                int lo = 0, hi = win_n;
+                if (win_smem) {
+                    while (lo < hi) {
+                        const int mid = (lo + hi) >> 1;
+                        if (buf.seg_b[mid] <= key) lo = mid + 1; else hi = mid;
+                    }
+                } else {
+                    while (lo < hi) {
+                        const int mid = (lo + hi) >> 1;
+                        if (__ldg(a.seg_begin + win_lo + mid) <= key) lo = mid + 1; else hi = mid;
+                    }
+                }
+                i = lo - 1;
+            }
+            float vnext_f = buf.v[min(l0 + kScanItems, n_tile)];
+#pragma unroll
+            for (int k = kScanItems - 1; k >= 0; --k) {
+                const int l = l0 + k;
+                delta[k] = 0.0;
+                rew[k] = 0.f;
+                if (l >= n_tile) continue;   // past the end: the identity map
+                const int32_t p = int32_t(t0 + l);
+                const float vf = buf.v[l];
+                int32_t b = 0, e = 0;
+                bool have = false;
+                while (i >= 0) {
+                    if (win_smem) {
+                        b = buf.seg_b[i];
+                        e = buf.seg_e[i];
+                    } else {
+                        b = __ldg(a.seg_begin + win_lo + i);
+                        e = __ldg(a.seg_end + win_lo + i);
+                        if (b < 0 || e > a.N || e < b) { bad = true; e = b; }
+                    }
+                    if (p >= b) { have = true; break; }
+                    --i;
+                }
+                const bool inside = have && p < e;
+                double aA = 0.0, aR = 0.0;
+                if (inside) {
+                    const float r = buf.r[l];
+                    const double v = double(vf);
+                    double v_next;
+                    if (p + 1 < e) {
+                        v_next = double(vnext_f);
+                        aA = a.gl;
+                        aR = a.gamma;
+                        cont |= 1u << k;
+                    } else {
+                        const bool tr = win_smem ? (buf.seg_t[i] != 0)
+                                                 : (__ldg(a.truncated + win_lo + i) != 0);
+                        if (tr) {
+                            v_next = a.bootstrap ? double(win_smem ? buf.seg_boot[i]
+                                                                   : __ldg(a.bootstrap + win_lo + i))
+                                                 : v;
+                        } else {
+                            v_next = 0.0;
+                        }
+                    }
+                    delta[k] = fma(a.gamma, v_next, double(r)) - v;
+                    rew[k] = r;
+                }
+                vnext_f = vf;
+                f = compose(Affine2{aA, delta[k], aR, double(rew[k])}, f);
+            }
+        }
+
+        // ---- inclusive suffix composition inside the warp: S_l = f_l o f_{l+1} o ... o f_31 ---
+        Affine2 S = f;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const Affine2 o = shfl_down(S, d);
+            if (lane + d < 32) S = compose(S, o);
+        }
+        Affine2 excl = shfl_down(S, 1);   // composite of the lanes to the right
+        if (lane == 31) excl = identity2();
+        if (lane == 0) s_warp[warp] = S;
+        __syncthreads();                                                      // (A)
+
+        // ---- next tile: start its loads and its window search while warp 0 looks back ---------
+        const uint32_t next_ticket = s_ticket[(it & 1) ^ 1];
+        const bool has_next = next_ticket < uint32_t(a.num_tiles);
+        const int ntile = a.num_tiles - 1 - int(next_ticket);
+        const int64_t nt0 = int64_t(ntile) * kScanTile;
+        const int nn_tile = int(min(int64_t(kScanTile), int64_t(a.N) - nt0));
+        if (has_next) {
+            egae_stage_inputs(a, nbuf, nt0, nn_tile);
+            if (warp == 1 || warp == 2) egae_window_search(a, nbuf, nt0, nn_tile, warp - 1, lane);
+        }
+
+        // ---- tile composite, look-back, per-warp carries ------------------------------------
+        if (threadIdx.x == 0) {
+            Affine2 acc = identity2();
+            for (int w = kScanWarps - 1; w >= 0; --w) {
+                s_right[w] = acc;
+                acc = compose(s_warp[w], acc);
+            }
+            const Affine2 tile_f = acc;
+            TileState* st = a.state;
+            if (tile + 1 < a.num_tiles) {
+                st_pair(st[tile].aggA, tile_f.aA, tile_f.bA);
+                st_pair(st[tile].aggR, tile_f.aR, tile_f.bR);
+            }
+            // value entering from the right: look back over tiles tile+1, tile+2, ...
+            Affine2 F = identity2();
+            double xA = 0.0, xR = 0.0;
+            bool timed_out = false;
+            for (int j = tile + 1;; ++j) {
+                if (j >= a.num_tiles) { xA = F.bA; xR = F.bR; break; }   // nothing beyond the end
+                double i0 = 0.0, i1 = 0.0, pa = 0.0, pb = 0.0, qa = 0.0, qb = 0.0;
+                uint32_t spins = 0;
+                bool got_inc = false;
+                for (;;) {
+                    got_inc = ld_pair(st[j].inc, i0, i1);
+                    if (got_inc) break;
+                    const bool ga = ld_pair(st[j].aggA, pa, pb);
+                    const bool gr = ld_pair(st[j].aggR, qa, qb);
+                    if (ga && gr) break;
+                    if (++spins > kScanSpinLimit) { timed_out = true; break; }
+                    __nanosleep(20);
+                }
+                if (timed_out) break;
+                if (got_inc) {
+                    xA = fma(F.aA, i0, F.bA);
+                    xR = fma(F.aR, i1, F.bR);
+                    break;
+                }
+                F = compose(F, Affine2{pa, pb, qa, qb});
+                if (F.aA == 0.0 && F.aR == 0.0) { xA = F.bA; xR = F.bR; break; }  // a segment ended
+            }
+            if (timed_out) { atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
+            st_pair(st[tile].inc, fma(tile_f.aA, xA, tile_f.bA), fma(tile_f.aR, xR, tile_f.bR));
+            for (int w = 0; w < kScanWarps; ++w) {
+                s_carry[w][0] = fma(s_right[w].aA, xA, s_right[w].bA);
+                s_carry[w][1] = fma(s_right[w].aR, xR, s_right[w].bR);
+            }
+        }
+        __syncthreads();                                                      // (B)
+        if (has_next) bad |= egae_window_load(a, nbuf);
+
+        // ---- replay the thread's positions with the true incoming values ----------------------
+        double A = fma(excl.aA, s_carry[warp][0], excl.bA);
+        double G = fma(excl.aR, s_carry[warp][1], excl.bR);
 #pragma unroll
         for (int k = kScanItems - 1; k >= 0; --k) {
-            const int64_t p = base + k;
-            delta[k] = 0.0;
-            rew[k] = 0.0;
-            if (p >= a.N) continue;   // past the end: the identity map
-            while (i >= 0 && int32_t(p) < __ldg(a.seg_begin + i)) --i;
-            bool inside = false;
-            int64_t e = 0;
-            if (i >= 0) {
-                const int64_t b = __ldg(a.seg_begin + i);
-                e = __ldg(a.seg_end + i);
-                if (b < 0 || e > a.N || e < b) { bad = true; e = b; }
-                inside = p < e;
-            }
-            double aA = 0.0, aR = 0.0;
-            if (inside) {
-                const double r = double(__ldg(a.rewards + p));
-                const double v = double(__ldg(a.values + p));
-                double v_next;
-                if (p + 1 < e) {
-                    v_next = double(__ldg(a.values + p + 1));
-                    aA = a.gl;
-                    aR = a.gamma;
-                    cont |= 1u << k;
-                } else if (__ldg(a.truncated + i)) {
-                    v_next = a.bootstrap ? double(__ldg(a.bootstrap + i)) : v;
+            const int l = l0 + k;
+            if (l >= n_tile) continue;
+            const bool c = (cont >> k) & 1u;
+            A = c ? fma(a.gl, A, delta[k]) : delta[k];
+            G = c ? fma(a.gamma, G, double(rew[k])) : double(rew[k]);
+            buf.r[l] = float(A);    // every read of the staged inputs happened before barrier (A)
+            buf.v[l] = float(G);
+        }
+        __syncthreads();                                                      // (C)
+
+        // ---- coalesced stores ---------------------------------------------------------------
+        if (a.vec_ok) {
+            float4* oa = reinterpret_cast<float4*>(a.adv + t0);
+            float4* og = a.ret ? reinterpret_cast<float4*>(a.ret + t0) : nullptr;
+            for (int u = threadIdx.x; u < kScanTile / 4; u += kScanThreads) {
+                if (4 * u + 4 <= n_tile) {
+                    oa[u] = reinterpret_cast<const float4*>(buf.r)[u];
+                    if (og) og[u] = reinterpret_cast<const float4*>(buf.v)[u];
                 } else {
-                    v_next = 0.0;
+                    for (int k = 4 * u; k < n_tile; ++k) {
+                        a.adv[t0 + k] = buf.r[k];
+                        if (a.ret) a.ret[t0 + k] = buf.v[k];
+                    }
                 }
-                delta[k] = fma(a.gamma, v_next, r) - v;
-                rew[k] = r;
             }
-            f = compose(Affine2{aA, delta[k], aR, rew[k]}, f);
-        }
-        if (bad) atomicOr(a.status, TPPO_DEV_BAD_SEGMENT);
-    }
-
-    // ---- inclusive suffix composition inside the warp: S_l = f_l o f_{l+1} o ... o f_31 -------
-    Affine2 S = f;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const Affine2 o = shfl_down(S, d);
-        if (lane + d < 32) S = compose(S, o);
-    }
-    Affine2 excl = shfl_down(S, 1);   // composite of the lanes to the right
-    if (lane == 31) excl = identity2();
-    if (lane == 0) s_warp[warp] = S;
-    __syncthreads();
-
-    // ---- tile composite, look-back, per-warp carries --------------------------------------
-    if (threadIdx.x == 0) {
-        Affine2 right[kScanWarps];      // right[w]: composite of warps w+1 .. last
-        Affine2 acc = identity2();
-        for (int w = kScanWarps - 1; w >= 0; --w) {
-            right[w] = acc;
-            acc = compose(s_warp[w], acc);
-        }
-        const Affine2 tile_f = acc;
-        TileState* st = a.state;
-        if (tile + 1 < a.num_tiles) {
-            st[tile].agg[0] = tile_f.aA; st[tile].agg[1] = tile_f.bA;
-            st[tile].agg[2] = tile_f.aR; st[tile].agg[3] = tile_f.bR;
-            __threadfence();
-            *reinterpret_cast<volatile int*>(&st[tile].flag) = 1;
-        }
-        // value entering from the right: look back over tiles tile+1, tile+2, ...
-        Affine2 F = identity2();
-        double xA = 0.0, xR = 0.0;
-        bool timed_out = false;
-        for (int j = tile + 1;; ++j) {
-            if (j >= a.num_tiles) { xA = F.bA; xR = F.bR; break; }   // nothing beyond the end
-            volatile int* fl = reinterpret_cast<volatile int*>(&st[j].flag);
-            int flag = *fl;
-            uint32_t spins = 0;
-            while (flag == 0) {
-                if (++spins > kScanSpinLimit) { timed_out = true; break; }
-                __nanosleep(20);
-                flag = *fl;
+        } else {
+            for (int k = threadIdx.x; k < n_tile; k += kScanThreads) {
+                a.adv[t0 + k] = buf.r[k];
+                if (a.ret) a.ret[t0 + k] = buf.v[k];
             }
-            if (timed_out) break;
-            __threadfence();
-            const volatile double* pd = reinterpret_cast<const volatile double*>(&st[j]);
-            if (flag == 2) {
-                xA = fma(F.aA, pd[4], F.bA);
-                xR = fma(F.aR, pd[5], F.bR);
-                break;
-            }
-            F = compose(F, Affine2{pd[0], pd[1], pd[2], pd[3]});
-            if (F.aA == 0.0 && F.aR == 0.0) { xA = F.bA; xR = F.bR; break; }  // a segment ended
         }
-        if (timed_out) { atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
-        st[tile].inc[0] = fma(tile_f.aA, xA, tile_f.bA);
-        st[tile].inc[1] = fma(tile_f.aR, xR, tile_f.bR);
-        __threadfence();
-        *reinterpret_cast<volatile int*>(&st[tile].flag) = 2;
-        for (int w = 0; w < kScanWarps; ++w) {
-            s_carry[w][0] = fma(right[w].aA, xA, right[w].bA);
-            s_carry[w][1] = fma(right[w].aR, xR, right[w].bR);
-        }
+        if (!has_next) break;
+        cp_async_wait_all();
+        __syncthreads();                                                      // (D)
+        ticket = next_ticket;
     }
-    __syncthreads();
+    if (bad) atomicOr(a.status, TPPO_DEV_BAD_SEGMENT);
+}
 
-    // ---- replay the thread's positions with the true incoming values ------------------------
-    double A = fma(excl.aA, s_carry[warp][0], excl.bA);
-    double G = fma(excl.aR, s_carry[warp][1], excl.bR);
-#pragma unroll
-    for (int k = kScanItems - 1; k >= 0; --k) {
-        const int64_t p = base + k;
-        if (p >= a.N) continue;
-        const bool c = (cont >> k) & 1u;
-        A = c ? fma(a.gl, A, delta[k]) : delta[k];
-        G = c ? fma(a.gamma, G, rew[k]) : rew[k];
-        a.adv[p] = float(A);
-        if (a.ret) a.ret[p] = float(G);
-    }
+// persistent grid: as many CTAs as can be resident, fewer when there are fewer tiles
+static inline int egae_grid(int num_tiles) {
+    const int resident = kNumSms * kScanCtasPerSm;
+    return num_tiles < resident ? num_tiles : resident;
 }
 
 size_t egae_workspace_bytes(int64_t N) {
@@ -233,7 +453,10 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
     if (N == 0) return TPPO_OK;
-    TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0, need, s));
+    const size_t ticket_bytes = align_up(sizeof(uint32_t), kWsAlign);
+    TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0, ticket_bytes, s));
+    TPPO_CUDA_CHECK(cudaMemsetAsync(static_cast<char*>(workspace) + ticket_bytes, 0xff,
+                                    need - ticket_bytes, s));    // tile states start out unset
     EgaeArgs a;
     a.rewards = rewards; a.values = values; a.seg_begin = seg_begin; a.seg_end = seg_end;
     a.truncated = truncated; a.bootstrap = bootstrap; a.B = B; a.N = int32_t(N);
@@ -241,10 +464,12 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
     a.gamma = double(gamma);
     a.gl = double(gamma) * double(lambda);
     a.adv = advantages; a.ret = returns; a.status = status;
+    a.vec_ok = aligned(rewards, 16) && aligned(values, 16) && aligned(advantages, 16) &&
+               (!returns || aligned(returns, 16));
     a.ticket = static_cast<uint32_t*>(workspace);
     a.state = reinterpret_cast<TileState*>(static_cast<char*>(workspace) +
                                            align_up(sizeof(uint32_t), kWsAlign));
-    egae_scan_kernel<<<a.num_tiles, kScanThreads, 0, s>>>(a);
+    egae_scan_kernel<<<egae_grid(a.num_tiles), kScanThreads, 0, s>>>(a);
     TPPO_CUDA_CHECK(cudaGetLastError());
     return TPPO_OK;
 }
@@ -307,11 +532,16 @@ TPPO_API int tppo_egae_static(const float* rewards, const float* values, const i
     a.gamma = double(gamma);
     a.gl = double(gamma) * double(lambda);
     a.adv = advantages; a.ret = returns; a.status = status;
+    a.vec_ok = aligned(rewards, 16) && aligned(values, 16) && aligned(advantages, 16) &&
+               (!returns || aligned(returns, 16));
     a.ticket = static_cast<uint32_t*>(scratch);
     a.state = reinterpret_cast<TileState*>(static_cast<char*>(scratch) + 256);
-    // the array still holds the previous call's flags and ticket: clear the part this call uses
-    TPPO_CUDA_CHECK(cudaMemsetAsync(scratch, 0, 256 + size_t(a.num_tiles) * sizeof(TileState), s));
-    egae_scan_kernel<<<a.num_tiles, kScanThreads, 0, s>>>(a);
+    // the array still holds the previous call's tile states and ticket: reset the part this call
+    // uses (ticket to zero, tile states to the all-ones "unset" pattern)
+    TPPO_CUDA_CHECK(cudaMemsetAsync(scratch, 0, 256, s));
+    TPPO_CUDA_CHECK(cudaMemsetAsync(static_cast<char*>(scratch) + 256, 0xff,
+                                    size_t(a.num_tiles) * sizeof(TileState), s));
+    egae_scan_kernel<<<egae_grid(a.num_tiles), kScanThreads, 0, s>>>(a);
     TPPO_CUDA_CHECK(cudaGetLastError());
     return TPPO_OK;
 }

@@ -36,17 +36,38 @@ __global__ void __launch_bounds__(kValThreads) value_loss_kernel(const ValueArgs
 
     double acc = 0.0;
     bool bad = false;
-    for (int64_t j = int64_t(blockIdx.x) * kValThreads + threadIdx.x; j < n;
-         j += int64_t(gridDim.x) * kValThreads) {
-        const int64_t p = a.value_idx ? int64_t(__ldg(a.value_idx + j)) : j;
-        if (p < 0 || p >= a.N) { bad = true; continue; }
-        const float v = __ldg(a.values + p), vo = __ldg(a.old_values + p), R = __ldg(a.returns + p);
-        const float vc = fminf(fmaxf(v, vo - a.xi_low), vo + a.xi_high);
-        const float e1 = (v - R) * (v - R), e2 = (vc - R) * (vc - R);
-        float g;
-        if (e1 >= e2) { acc += 0.5 * double(e1); g = v - R; }
-        else { acc += 0.5 * double(e2); g = (vc == v) ? (vc - R) : 0.f; }
-        if (a.dvalues) a.dvalues[p] = g * inv_d;
+    // Four independent tokens per thread and trip, so that the index load and the three gathers of
+    // one token overlap with those of the others.
+    constexpr int kUnroll = 4;
+    const int64_t stride = int64_t(gridDim.x) * kValThreads;
+    for (int64_t j0 = int64_t(blockIdx.x) * kValThreads + threadIdx.x; j0 < n; j0 += stride * kUnroll) {
+        int64_t p[kUnroll];
+        bool ok[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int64_t j = j0 + u * stride;
+            p[u] = j < n ? (a.value_idx ? int64_t(__ldg(a.value_idx + j)) : j) : -1;
+            ok[u] = p[u] >= 0 && p[u] < a.N;
+            if (j < n && !ok[u]) bad = true;
+        }
+        float v[kUnroll], vo[kUnroll], R[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int64_t q = ok[u] ? p[u] : 0;
+            v[u] = ok[u] ? __ldg(a.values + q) : 0.f;
+            vo[u] = ok[u] ? __ldg(a.old_values + q) : 0.f;
+            R[u] = ok[u] ? __ldg(a.returns + q) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            if (!ok[u]) continue;
+            const float vc = fminf(fmaxf(v[u], vo[u] - a.xi_low), vo[u] + a.xi_high);
+            const float e1 = (v[u] - R[u]) * (v[u] - R[u]), e2 = (vc - R[u]) * (vc - R[u]);
+            float g;
+            if (e1 >= e2) { acc += 0.5 * double(e1); g = v[u] - R[u]; }
+            else { acc += 0.5 * double(e2); g = (vc == v[u]) ? (vc - R[u]) : 0.f; }
+            if (a.dvalues) a.dvalues[p[u]] = g * inv_d;
+        }
     }
     if (bad) atomicOr(a.stats + 1, TPPO_DEV_BAD_INDEX);
     acc = warp_sum(acc);
