@@ -112,12 +112,11 @@ __device__ __forceinline__ void cp_async_wait_all() {
     asm volatile("cp.async.wait_all;" ::: "memory");
 }
 
-// Shared-memory image of one tile: its inputs (later overwritten by its outputs) and the window of
-// segments that can touch it.  Aligned and sized to 16 bytes: r and v are accessed as float4 and by
+// Shared-memory image of one tile: its inputs and the window of segments that can touch it.  Aligned and sized to 16 bytes: r and v are accessed as float4 and by
 // 16-byte cp.async in both halves of a two-element array.
 struct __align__(16) TileBuf {
-    float r[kScanTile];          // rewards in, advantages out
-    float v[kScanTile + 4];      // values in (+1 look-ahead), returns out
+    float r[kScanTile];          // rewards
+    float v[kScanTile + 4];      // values (+1 look-ahead)
     int32_t seg_b[kSegCap], seg_e[kSegCap];
     float seg_boot[kSegCap];
     uint8_t seg_t[kSegCap];
@@ -192,7 +191,6 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
     __shared__ __align__(16) TileBuf s_buf[2];
     __shared__ uint32_t s_ticket[2];
     __shared__ Affine2 s_warp[kScanWarps];
-    __shared__ Affine2 s_right[kScanWarps];      // composite of the warps to the right of warp w
     __shared__ double s_carry[kScanWarps][2];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -230,27 +228,55 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
         float rew[kScanItems];
         uint32_t cont = 0;  // bit k: position k continues into position k+1 (same segment)
         Affine2 f = identity2();
-        {
-            // index (inside the window) of the last segment that begins at or before the thread's
-            // last position, or -1
-            const int l_last = min(l0 + kScanItems, n_tile) - 1;
-            int i = -1;
-            if (l_last >= l0) {
-                const int32_t key = int32_t(t0 + l_last);
-                int lo = 0, hi = win_n;
-                if (win_smem) {
-                    while (lo < hi) {
-                        const int mid = (lo + hi) >> 1;
-                        if (buf.seg_b[mid] <= key) lo = mid + 1; else hi = mid;
-                    }
-                } else {
-                    while (lo < hi) {
-                        const int mid = (lo + hi) >> 1;
-                        if (__ldg(a.seg_begin + win_lo + mid) <= key) lo = mid + 1; else hi = mid;
-                    }
+        // index (inside the window) of the last segment that begins at or before the thread's
+        // last position, or -1
+        const int l_last = min(l0 + kScanItems, n_tile) - 1;
+        int i = -1;
+        if (l_last >= l0) {
+            const int32_t key = int32_t(t0 + l_last);
+            int lo = 0, hi = win_n;
+            if (win_smem && win_n <= 4) {
+                while (lo < win_n && buf.seg_b[lo] <= key) ++lo;
+            } else if (win_smem) {
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (buf.seg_b[mid] <= key) lo = mid + 1; else hi = mid;
                 }
-                i = lo - 1;
+            } else {
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (__ldg(a.seg_begin + win_lo + mid) <= key) lo = mid + 1; else hi = mid;
+                }
             }
+            i = lo - 1;
+        }
+        // The common case: all eight positions lie inside one segment and none of them is its last
+        // token.  Then every map has the same multiplier and no per-position segment test is needed.
+        bool fast = false;
+        if (win_smem && i >= 0 && l0 + kScanItems <= n_tile)
+            fast = int64_t(buf.seg_b[i]) <= t0 + l0 && t0 + l0 + kScanItems < int64_t(buf.seg_e[i]);
+        if (fast) {
+            const float4 ra = *reinterpret_cast<const float4*>(buf.r + l0);
+            const float4 rb = *reinterpret_cast<const float4*>(buf.r + l0 + 4);
+            const float4 va = *reinterpret_cast<const float4*>(buf.v + l0);
+            const float4 vb = *reinterpret_cast<const float4*>(buf.v + l0 + 4);
+            const float rr[kScanItems] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+            const float vv[kScanItems] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+            double dn = double(buf.v[l0 + kScanItems]);
+            double bA = 0.0, bR = 0.0;
+#pragma unroll
+            for (int k = kScanItems - 1; k >= 0; --k) {
+                const double dv = double(vv[k]), dr = double(rr[k]);
+                delta[k] = fma(a.gamma, dn, dr) - dv;
+                rew[k] = rr[k];
+                bA = fma(a.gl, bA, delta[k]);
+                bR = fma(a.gamma, bR, dr);
+                dn = dv;
+            }
+            const double gl2 = a.gl * a.gl, gl4 = gl2 * gl2, g2 = a.gamma * a.gamma, g4 = g2 * g2;
+            f = Affine2{gl4 * gl4, bA, g4 * g4, bR};
+            cont = 0xffu;
+        } else {
             float vnext_f = buf.v[min(l0 + kScanItems, n_tile)];
 #pragma unroll
             for (int k = kScanItems - 1; k >= 0; --k) {
@@ -327,90 +353,89 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
             if (warp == 1 || warp == 2) egae_window_search(a, nbuf, nt0, nn_tile, warp - 1, lane);
         }
 
-        // ---- tile composite, look-back, per-warp carries ------------------------------------
-        if (threadIdx.x == 0) {
-            Affine2 acc = identity2();
-            for (int w = kScanWarps - 1; w >= 0; --w) {
-                s_right[w] = acc;
-                acc = compose(s_warp[w], acc);
-            }
-            const Affine2 tile_f = acc;
-            TileState* st = a.state;
-            if (tile + 1 < a.num_tiles) {
-                st_pair(st[tile].aggA, tile_f.aA, tile_f.bA);
-                st_pair(st[tile].aggR, tile_f.aR, tile_f.bR);
-            }
-            // value entering from the right: look back over tiles tile+1, tile+2, ...
-            Affine2 F = identity2();
+        // ---- tile composite, look-back, per-warp carries (warp 0) ------------------------------
+        if (warp == 0) {
+            // lane w < 8 holds warp w's composite; suffix-compose them in three steps, so that
+            // lane w ends with W_w o ... o W_7 and lane 0 with the tile's composite
+            Affine2 W = lane < kScanWarps ? s_warp[lane] : identity2();
+#pragma unroll
+            for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
+            Affine2 right = shfl_down(W, 1);            // composite of the warps to the right
+            if (lane >= kScanWarps - 1) right = identity2();
             double xA = 0.0, xR = 0.0;
-            bool timed_out = false;
-            for (int j = tile + 1;; ++j) {
-                if (j >= a.num_tiles) { xA = F.bA; xR = F.bR; break; }   // nothing beyond the end
-                double i0 = 0.0, i1 = 0.0, pa = 0.0, pb = 0.0, qa = 0.0, qb = 0.0;
-                uint32_t spins = 0;
-                bool got_inc = false;
-                for (;;) {
-                    got_inc = ld_pair(st[j].inc, i0, i1);
-                    if (got_inc) break;
-                    const bool ga = ld_pair(st[j].aggA, pa, pb);
-                    const bool gr = ld_pair(st[j].aggR, qa, qb);
-                    if (ga && gr) break;
-                    if (++spins > kScanSpinLimit) { timed_out = true; break; }
-                    __nanosleep(20);
+            if (lane == 0) {
+                const Affine2 tile_f = W;
+                TileState* st = a.state;
+                if (tile + 1 < a.num_tiles) {
+                    st_pair(st[tile].aggA, tile_f.aA, tile_f.bA);
+                    st_pair(st[tile].aggR, tile_f.aR, tile_f.bR);
                 }
-                if (timed_out) break;
-                if (got_inc) {
-                    xA = fma(F.aA, i0, F.bA);
-                    xR = fma(F.aR, i1, F.bR);
-                    break;
+                // value entering from the right: look back over tiles tile+1, tile+2, ...
+                Affine2 F = identity2();
+                bool timed_out = false;
+                for (int j = tile + 1;; ++j) {
+                    if (j >= a.num_tiles) { xA = F.bA; xR = F.bR; break; }   // nothing beyond the end
+                    double i0, i1, pa, pb, qa, qb;
+                    uint32_t spins = 0;
+                    bool got_inc;
+                    for (;;) {       // the three pairs are requested together: one round trip
+                        got_inc = ld_pair(st[j].inc, i0, i1);
+                        const bool ga = ld_pair(st[j].aggA, pa, pb);
+                        const bool gr = ld_pair(st[j].aggR, qa, qb);
+                        if (got_inc || (ga && gr)) break;
+                        if (++spins > kScanSpinLimit) { timed_out = true; break; }
+                        __nanosleep(20);
+                    }
+                    if (timed_out) break;
+                    if (got_inc) {
+                        xA = fma(F.aA, i0, F.bA);
+                        xR = fma(F.aR, i1, F.bR);
+                        break;
+                    }
+                    F = compose(F, Affine2{pa, pb, qa, qb});
+                    if (F.aA == 0.0 && F.aR == 0.0) { xA = F.bA; xR = F.bR; break; }  // a segment ended
                 }
-                F = compose(F, Affine2{pa, pb, qa, qb});
-                if (F.aA == 0.0 && F.aR == 0.0) { xA = F.bA; xR = F.bR; break; }  // a segment ended
+                if (timed_out) { atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
+                st_pair(st[tile].inc, fma(tile_f.aA, xA, tile_f.bA), fma(tile_f.aR, xR, tile_f.bR));
             }
-            if (timed_out) { atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
-            st_pair(st[tile].inc, fma(tile_f.aA, xA, tile_f.bA), fma(tile_f.aR, xR, tile_f.bR));
-            for (int w = 0; w < kScanWarps; ++w) {
-                s_carry[w][0] = fma(s_right[w].aA, xA, s_right[w].bA);
-                s_carry[w][1] = fma(s_right[w].aR, xR, s_right[w].bR);
+            xA = __shfl_sync(0xffffffffu, xA, 0);
+            xR = __shfl_sync(0xffffffffu, xR, 0);
+            if (lane < kScanWarps) {
+                s_carry[lane][0] = fma(right.aA, xA, right.bA);
+                s_carry[lane][1] = fma(right.aR, xR, right.bR);
             }
         }
         __syncthreads();                                                      // (B)
         if (has_next) bad |= egae_window_load(a, nbuf);
 
-        // ---- replay the thread's positions with the true incoming values ----------------------
+        // ---- replay the thread's positions with the true incoming values, store -----------------
         double A = fma(excl.aA, s_carry[warp][0], excl.bA);
         double G = fma(excl.aR, s_carry[warp][1], excl.bR);
+        float oa[kScanItems], og[kScanItems];
 #pragma unroll
         for (int k = kScanItems - 1; k >= 0; --k) {
-            const int l = l0 + k;
-            if (l >= n_tile) continue;
             const bool c = (cont >> k) & 1u;
             A = c ? fma(a.gl, A, delta[k]) : delta[k];
             G = c ? fma(a.gamma, G, double(rew[k])) : double(rew[k]);
-            buf.r[l] = float(A);    // every read of the staged inputs happened before barrier (A)
-            buf.v[l] = float(G);
+            oa[k] = float(A);
+            og[k] = float(G);
         }
-        __syncthreads();                                                      // (C)
-
-        // ---- coalesced stores ---------------------------------------------------------------
-        if (a.vec_ok) {
-            float4* oa = reinterpret_cast<float4*>(a.adv + t0);
-            float4* og = a.ret ? reinterpret_cast<float4*>(a.ret + t0) : nullptr;
-            for (int u = threadIdx.x; u < kScanTile / 4; u += kScanThreads) {
-                if (4 * u + 4 <= n_tile) {
-                    oa[u] = reinterpret_cast<const float4*>(buf.r)[u];
-                    if (og) og[u] = reinterpret_cast<const float4*>(buf.v)[u];
-                } else {
-                    for (int k = 4 * u; k < n_tile; ++k) {
-                        a.adv[t0 + k] = buf.r[k];
-                        if (a.ret) a.ret[t0 + k] = buf.v[k];
-                    }
-                }
+        if (a.vec_ok && l0 + kScanItems <= n_tile) {
+            float4* pa4 = reinterpret_cast<float4*>(a.adv + t0 + l0);
+            pa4[0] = make_float4(oa[0], oa[1], oa[2], oa[3]);
+            pa4[1] = make_float4(oa[4], oa[5], oa[6], oa[7]);
+            if (a.ret) {
+                float4* pg4 = reinterpret_cast<float4*>(a.ret + t0 + l0);
+                pg4[0] = make_float4(og[0], og[1], og[2], og[3]);
+                pg4[1] = make_float4(og[4], og[5], og[6], og[7]);
             }
         } else {
-            for (int k = threadIdx.x; k < n_tile; k += kScanThreads) {
-                a.adv[t0 + k] = buf.r[k];
-                if (a.ret) a.ret[t0 + k] = buf.v[k];
+#pragma unroll
+            for (int k = 0; k < kScanItems; ++k) {
+                if (l0 + k < n_tile) {
+                    a.adv[t0 + l0 + k] = oa[k];
+                    if (a.ret) a.ret[t0 + l0 + k] = og[k];
+                }
             }
         }
         if (!has_next) break;
