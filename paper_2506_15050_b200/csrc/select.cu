@@ -1,6 +1,7 @@
 // Token filter + stream compaction (Section 3.2 of the paper): one pass over the packed token
-// positions, warp-ballot ranks inside a warp, shared-memory prefix across the warps of a tile,
-// and a decoupled look-back chain across tiles, so that every selected position is written once
+// positions.  A thread turns its 16 consecutive positions into two 16-bit words by interval
+// arithmetic on the sequences that overlap them, ranks come from popcounts and a warp / tile
+// prefix, a decoupled look-back chain links the tiles, and every selected position is written once
 // in ascending order.  Integer work throughout: the result is bit-exact and run-to-run identical.
 #include "common.cuh"
 
@@ -62,38 +63,37 @@ struct SelectArgs {
     uint32_t* ticket;           // [1]
 };
 
-// Position ranges of one sequence: policy tokens [pol_lo, pol_hi), value tokens [val_lo, val_hi),
-// and the first position of the next sequence.
-struct SeqBounds {
-    int64_t next, pol_lo, pol_hi, val_lo, val_hi;
-};
-__device__ __forceinline__ SeqBounds seq_bounds(const SelectArgs& a, int i) {
-    SeqBounds s;
-    if (i < 0 || i >= a.B) {        // before the first or after the last sequence: nothing selected
-        s.next = i < 0 ? int64_t(__ldg(a.seq_begin)) : (int64_t(1) << 40);
-        s.pol_lo = s.pol_hi = s.val_lo = s.val_hi = 0;
-        return s;
-    }
-    const int64_t begin = __ldg(a.seq_begin + i);
-    s.next = __ldg(a.seq_begin + i + 1);
-    const int64_t resp0 = begin + __ldg(a.prompt_len + i);
-    const int64_t new0 = resp0 + __ldg(a.prev_len + i);
-    const int64_t end = new0 + __ldg(a.new_len + i);
-    const bool trunc = __ldg(a.truncated + i) != 0;
-    s.pol_lo = new0;
-    s.pol_hi = end - (trunc ? a.tail_drop : 0);
-    s.val_lo = resp0;
-    s.val_hi = trunc ? resp0 : end;
-    return s;
+constexpr int kSeqCap = 320;   // sequence starts of one tile kept in shared memory
+
+// 16 mask bytes -> 16 bits (bit k set iff byte k is non-zero).
+__device__ __forceinline__ uint32_t nonzero_bytes4(uint32_t w) {
+    // high bit of each byte set iff the byte is non-zero, then the four high bits gathered
+    const uint32_t t = (w | ((w & 0x7f7f7f7fu) + 0x7f7f7f7fu)) & 0x80808080u;
+    return ((t >> 7) * 0x00204081u >> 21) & 0xfu;
+}
+__device__ __forceinline__ uint32_t nonzero_bytes16(uint4 v) {
+    return nonzero_bytes4(v.x) | (nonzero_bytes4(v.y) << 4) | (nonzero_bytes4(v.z) << 8) |
+           (nonzero_bytes4(v.w) << 12);
+}
+// Bits [lo - p0, hi - p0) of a 16-bit word, for the positions of [lo, hi) that fall in [p0, p0+16).
+__device__ __forceinline__ uint32_t range_bits16(int64_t lo, int64_t hi, int64_t p0) {
+    const int64_t a = min(max(lo - p0, int64_t(0)), int64_t(16));
+    const int64_t b = min(max(hi - p0, int64_t(0)), int64_t(16));
+    return b > a ? ((1u << int(b)) - 1u) & ~((1u << int(a)) - 1u) : 0u;
 }
 
+// Each thread owns 16 consecutive positions.  Its policy / value bits come from interval
+// arithmetic on the few sequences that overlap those positions (usually one) and from one 16-byte
+// load per byte mask, not from a test per position; selected positions are first compacted inside
+// the tile in shared memory and then copied out with coalesced stores.
 __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const SelectArgs a) {
-    __shared__ __align__(16) uint8_t s_pm[kSelTile];
-    __shared__ __align__(16) uint8_t s_vm[kSelTile];
+    __shared__ int32_t s_out_pol[kSelTile];
+    __shared__ int32_t s_out_val[kSelTile];
+    __shared__ int32_t s_sb[kSeqCap + 1];
     __shared__ uint32_t s_tile;
-    __shared__ int s_seq0;
-    __shared__ uint32_t s_warp_pol[kSelWarps], s_warp_val[kSelWarps];
-    __shared__ uint32_t s_base_pol, s_base_val;
+    __shared__ int s_seq0, s_seq1;
+    __shared__ uint32_t s_warp_cnt[kSelWarps];      // policy count | value count << 16
+    __shared__ uint32_t s_base_pol, s_base_val, s_tot_pol, s_tot_val;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // Tiles are handed out in launch order, so every tile this one waits for is already running.
@@ -103,64 +103,112 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     if (tile >= uint32_t(a.num_tiles)) return;
     const int64_t t0 = int64_t(tile) * kSelTile;
     const int n_tile = int(min(int64_t(kSelTile), int64_t(a.N) - t0));
+    const int l0 = threadIdx.x * kSelItems;
+    const int64_t p0 = t0 + l0;
+    const int n_mine = max(0, min(kSelItems, n_tile - l0));    // positions this thread really owns
 
-    // ---- stage the optional byte masks (one 16-byte load per thread and mask) ------------------
-    {
-        const int l = threadIdx.x * 16;
-        if (a.mask_vec_ok && l + 16 <= n_tile) {
-            if (a.pol_mask)
-                reinterpret_cast<uint4*>(s_pm)[threadIdx.x] =
-                    __ldg(reinterpret_cast<const uint4*>(a.pol_mask + t0) + threadIdx.x);
-            if (a.val_mask)
-                reinterpret_cast<uint4*>(s_vm)[threadIdx.x] =
-                    __ldg(reinterpret_cast<const uint4*>(a.val_mask + t0) + threadIdx.x);
-        } else {
-            for (int k = l; k < min(l + 16, n_tile); ++k) {
-                if (a.pol_mask) s_pm[k] = __ldg(a.pol_mask + t0 + k);
-                if (a.val_mask) s_vm[k] = __ldg(a.val_mask + t0 + k);
-            }
+    // ---- the byte masks of this thread's positions, as bits (issued first: longest latency) ----
+    uint32_t pm_bits = 0xffffu, vm_bits = 0xffffu;
+    if (n_mine == kSelItems && a.mask_vec_ok) {
+        if (a.pol_mask) pm_bits = nonzero_bytes16(__ldg(reinterpret_cast<const uint4*>(a.pol_mask + p0)));
+        if (a.val_mask) vm_bits = nonzero_bytes16(__ldg(reinterpret_cast<const uint4*>(a.val_mask + p0)));
+    } else {
+        if (a.pol_mask) {
+            pm_bits = 0;
+            for (int k = 0; k < n_mine; ++k) pm_bits |= uint32_t(__ldg(a.pol_mask + p0 + k) != 0) << k;
+        }
+        if (a.val_mask) {
+            vm_bits = 0;
+            for (int k = 0; k < n_mine; ++k) vm_bits |= uint32_t(__ldg(a.val_mask + p0 + k) != 0) << k;
         }
     }
-    // sequence that holds the tile's first position (-1: before the first sequence)
+    const uint32_t own_bits = n_mine >= kSelItems ? 0xffffu : ((1u << n_mine) - 1u);
+
+    // ---- window of sequences that can touch the tile: [seq0, seq1), seq0 may be -1 -------------
     if (warp == 0) {
         const int c = warp_count_le(a.seq_begin, a.B + 1, int32_t(t0), lane);
         if (lane == 0) s_seq0 = c - 1;
+    } else if (warp == 1) {
+        const int c = warp_count_le(a.seq_begin, a.B + 1, int32_t(t0 + n_tile - 1), lane);
+        if (lane == 0) s_seq1 = c;     // sequences with index < c begin at or before the last position
     }
     __syncthreads();
+    const int seq0 = s_seq0, seq1 = s_seq1;
+    const int first = max(seq0, 0);
+    const int n_win = min(seq1, a.B) - first + 1;         // entries first .. min(seq1, B) inclusive
+    const bool win_smem = n_win <= kSeqCap + 1;
+    if (win_smem) {
+        for (int j = threadIdx.x; j < n_win; j += kSelThreads) s_sb[j] = __ldg(a.seq_begin + first + j);
+        __syncthreads();
+    }
 
-    // ---- phase 1: predicates, kept as one bit per item in two 16-bit lane masks ------------
-    const int warp_l0 = warp * (32 * kSelItems);
+    // ---- policy / value bits of this thread's 16 positions --------------------------------------
     uint32_t pol_bits = 0, val_bits = 0;
-    {
-        int i = s_seq0;
-        SeqBounds sb = seq_bounds(a, i);
-#pragma unroll 4
-        for (int j = 0; j < kSelItems; ++j) {
-            const int l = warp_l0 + lane + j * 32;
-            if (l >= n_tile) break;
-            const int64_t p = t0 + l;
-            while (i < a.B && p >= sb.next) sb = seq_bounds(a, ++i);
-            bool is_pol = p >= sb.pol_lo && p < sb.pol_hi;
-            bool is_val = p >= sb.val_lo && p < sb.val_hi;
-            if (is_pol && a.pol_mask) is_pol = s_pm[l] != 0;
-            if (is_val && a.val_mask) is_val = s_vm[l] != 0;
-            pol_bits |= uint32_t(is_pol) << j;
-            val_bits |= uint32_t(is_val) << j;
+    if (n_mine > 0 && seq1 > 0) {
+        // last sequence of the window that begins at or before p0 (-1: none)
+        int lo = 0, hi = min(seq1, a.B + 1) - first;       // entries first .. first+hi-1 are <= t_last
+        const int32_t key = int32_t(p0);
+        if (win_smem) {
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (s_sb[mid] <= key) lo = mid + 1; else hi = mid;
+            }
+        } else {
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (__ldg(a.seq_begin + first + mid) <= key) lo = mid + 1; else hi = mid;
+            }
+        }
+        int i = first + lo - 1;                             // may be first-1 = -1 only when first == 0
+        if (i < 0) i = 0;                                   // positions before sequence 0 select nothing
+        const int64_t p_end = p0 + n_mine;
+        for (; i < a.B; ++i) {
+            const int64_t begin = win_smem ? s_sb[i - first] : __ldg(a.seq_begin + i);
+            if (begin >= p_end) break;
+            const int64_t next = win_smem ? s_sb[i + 1 - first] : __ldg(a.seq_begin + i + 1);
+            if (next <= p0 || next <= begin) continue;      // empty, or entirely before this thread
+            const int64_t resp0 = begin + __ldg(a.prompt_len + i);
+            const int64_t new0 = resp0 + __ldg(a.prev_len + i);
+            const int64_t end = new0 + __ldg(a.new_len + i);
+            const bool trunc = __ldg(a.truncated + i) != 0;
+            // a position belongs to the last sequence that begins at or before it: clip to [begin, next)
+            pol_bits |= range_bits16(max(new0, begin), min(end - (trunc ? a.tail_drop : 0), next), p0);
+            if (!trunc) val_bits |= range_bits16(max(resp0, begin), min(end, next), p0);
         }
     }
-    uint32_t warp_pol = 0, warp_val = 0;
+    pol_bits &= pm_bits & own_bits;
+    val_bits &= vm_bits & own_bits;
+
+    // ---- ranks inside the warp and the tile -----------------------------------------------------
+    const uint32_t mine = uint32_t(__popc(pol_bits)) | (uint32_t(__popc(val_bits)) << 16);
+    uint32_t incl = mine;
 #pragma unroll
-    for (int j = 0; j < kSelItems; ++j) {
-        warp_pol += __popc(__ballot_sync(0xffffffffu, (pol_bits >> j) & 1u));
-        warp_val += __popc(__ballot_sync(0xffffffffu, (val_bits >> j) & 1u));
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += o;
     }
-    if (lane == 0) { s_warp_pol[warp] = warp_pol; s_warp_val[warp] = warp_val; }
+    if (lane == 31) s_warp_cnt[warp] = incl;
     __syncthreads();
+    uint32_t before = incl - mine;                           // selected by lower lanes of this warp
+    uint32_t tile_tot = 0;
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) {
+        const uint32_t c = s_warp_cnt[w];
+        if (w < warp) before += c;
+        tile_tot += c;
+    }
+    // compact inside the tile (needs no global offset, so it overlaps the look-back below)
+    {
+        uint32_t op = before & 0xffffu, ov = before >> 16;
+        uint32_t b = pol_bits;
+        while (b) { s_out_pol[op++] = int32_t(p0) + (__ffs(int(b)) - 1); b &= b - 1; }
+        b = val_bits;
+        while (b) { s_out_val[ov++] = int32_t(p0) + (__ffs(int(b)) - 1); b &= b - 1; }
+    }
 
     // ---- tile total -> publish -> warp-wide look-back over earlier tiles ----------------------
     if (warp == 0) {
-        uint32_t tp = 0, tv = 0;
-        for (int w = 0; w < kSelWarps; ++w) { tp += s_warp_pol[w]; tv += s_warp_val[w]; }
+        const uint32_t tp = tile_tot & 0xffffu, tv = tile_tot >> 16;
         volatile unsigned long long* st = a.state;
         if (lane == 0 && tile > 0) st[tile] = sel_pack(1, tp, tv);
         uint32_t ep = 0, ev = 0;
@@ -189,6 +237,8 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
             st[tile] = sel_pack(2, ep + tp, ev + tv);
             s_base_pol = ep;
             s_base_val = ev;
+            s_tot_pol = tp;
+            s_tot_val = tv;
             if (tile == uint32_t(a.num_tiles) - 1) {
                 a.counts[0] = int32_t(ep + tp);
                 a.counts[1] = int32_t(ev + tv);
@@ -197,19 +247,13 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     }
     __syncthreads();
 
-    // ---- phase 2: scatter --------------------------------------------------------------------
-    uint32_t off_pol = s_base_pol, off_val = s_base_val;
-    for (int w = 0; w < warp; ++w) { off_pol += s_warp_pol[w]; off_val += s_warp_val[w]; }
-    const uint32_t lt = (1u << lane) - 1u;
-#pragma unroll
-    for (int j = 0; j < kSelItems; ++j) {
-        const int32_t p = int32_t(t0 + warp_l0 + lane + j * 32);
-        const uint32_t bp = __ballot_sync(0xffffffffu, (pol_bits >> j) & 1u);
-        const uint32_t bv = __ballot_sync(0xffffffffu, (val_bits >> j) & 1u);
-        if ((pol_bits >> j) & 1u) a.policy_idx[off_pol + __popc(bp & lt)] = p;
-        if ((val_bits >> j) & 1u) a.value_idx[off_val + __popc(bv & lt)] = p;
-        off_pol += __popc(bp);
-        off_val += __popc(bv);
+    // ---- copy the tile's two lists out, coalesced ----------------------------------------------
+    {
+        int32_t* dp = a.policy_idx + s_base_pol;
+        int32_t* dv = a.value_idx + s_base_val;
+        const int np = int(s_tot_pol), nv = int(s_tot_val);
+        for (int k = threadIdx.x; k < np; k += kSelThreads) dp[k] = s_out_pol[k];
+        for (int k = threadIdx.x; k < nv; k += kSelThreads) dv[k] = s_out_val[k];
     }
 }
 
