@@ -159,6 +159,8 @@ class Step:
         self.ws_val = b.workspace(b.OP_VALUE_LOSS, N, 0, N, 0, dev)
         self.ev = None
         self.hint = 0
+        self.denom_pol = 0.0      # > 0: selected-token counts of the whole job (several GPUs)
+        self.denom_val = 0.0
         # old-policy log-probs (Algorithm 1 line 3): forward-only pass of the same kernel, plus noise
         self.egae()
         self.select()
@@ -181,14 +183,14 @@ class Step:
         c, b = self.c, self.b
         b.tppo_policy_loss_fwd_bwd(
             self.logits, self.targets, None, self.counts[0:1], self.n, self.pol, self.old_logp,
-            self.adv, c["eps_low"], c["eps_high"], 0.0, self.logp, self.tok_loss, self.loss,
+            self.adv, c["eps_low"], c["eps_high"], self.denom_pol, self.logp, self.tok_loss, self.loss,
             self.stats, None if forward_only else self.dlogits,
             b.DLOGITS_NONE if forward_only else b.DLOGITS_COMPACT, self.ws_pol, kernel_hint=self.hint)
 
     def value(self):
         c = self.c
         self.b.tppo_value_loss(self.values, self.old_values, self.ret, self.val, self.counts[1:2],
-                               self.N, c["xi_low"], c["xi_high"], 0.0, self.vloss, self.dvalues,
+                               self.N, c["xi_low"], c["xi_high"], self.denom_val, self.vloss, self.dvalues,
                                self.vstats, self.ws_val)
 
     def run(self, events=None):
@@ -376,8 +378,15 @@ def main():
     if args.workload == "lmhead":
         run_lmhead_workload(args, rank, world, local, dev, warmup)
         return
-    st = Step(dev, rows=args.rows)
+    st = Step(dev, seed=2 + rank, rows=args.rows)      # every rank holds its own batch
     st.hint = args.hint
+    if world > 1:
+        # token-level mean over the whole job: each rank divides by the global selected-token counts
+        from paper_2506_15050_b200 import shard
+        torch.cuda.synchronize()
+        n_pol, n_val = shard.global_token_counts(int(st.counts[0].item()), int(st.counts[1].item()),
+                                                 device=dev)
+        st.denom_pol, st.denom_val = float(n_pol), float(n_val)
 
     def barrier():
         if world > 1:
