@@ -184,3 +184,29 @@ def lmhead_dweight_cols(hidden_bits, dx_cols):
     lib().oracle_lmhead_dweight_cols(_p(h), _p(g), C.c_int64(M), C.c_int32(K),
                                      C.c_int64(g.shape[1]), _p(dw))
     return dw
+
+
+def advance_batch(seq_begin, prompt_len, prev_len, new_len, truncated, tokens, queue_begin,
+                  queue_tokens, capacity=None):
+    """Successive batching between two steps.  Returns dict(next_prompt_len, next_prev_len,
+    next_seq_begin, next_tokens[:total], free_slots[:n_free], slot_source, n_free, n_refilled, total)."""
+    sb = _arr(seq_begin, np.int32)
+    pl, pv, nl = _arr(prompt_len, np.int32), _arr(prev_len, np.int32), _arr(new_len, np.int32)
+    tr = _arr(truncated, np.uint8)
+    tk = _arr(tokens, np.int32)
+    qb, qt = _arr(queue_begin, np.int32), _arr(queue_tokens, np.int32)
+    B, M = pl.shape[0], qb.shape[0] - 1
+    if capacity is None:
+        capacity = int(tk.shape[0] + qt.shape[0])
+    npl, npv = np.zeros(B, np.int32), np.zeros(B, np.int32)
+    nsb = np.zeros(B + 1, np.int32)
+    ntk = np.full(max(capacity, 1), -7, np.int32)
+    fs, src = np.full(max(B, 1), -9, np.int32), np.zeros(max(B, 1), np.int32)
+    counts = np.zeros(3, np.int64)
+    lib().oracle_advance_batch(_p(sb), _p(pl), _p(pv), _p(nl), _p(tr), _p(tk), _p(qb), _p(qt),
+                               C.c_int32(B), C.c_int32(M), _p(npl), _p(npv), _p(nsb), _p(ntk),
+                               C.c_int64(capacity), _p(fs), _p(src), _p(counts))
+    n_free, n_ref, total = (int(x) for x in counts)
+    return dict(next_prompt_len=npl, next_prev_len=npv, next_seq_begin=nsb,
+                next_tokens=ntk[:min(total, capacity)], free_slots=fs[:n_free], slot_source=src[:B],
+                n_free=n_free, n_refilled=n_ref, total=total)

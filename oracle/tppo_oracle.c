@@ -322,3 +322,62 @@ void oracle_lmhead_dweight_cols(const uint16_t *hidden, const double *dx_cols,
         }
     }
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Successive batching between two training steps (Section 3.2, the batching figure; Algorithm 1
+ * line 2): the batch keeps its B slots.  A slot whose sequence reached an end condition is
+ * freed and takes the next queued prompt; a slot whose sequence was cut at the window keeps it,
+ * and the tokens generated in this step join those of earlier windows.
+ *
+ * Slots are visited in ascending order; the k-th freed slot takes queued prompt k while the
+ * queue lasts (M prompts), later freed slots stay empty.  The context of the next step (what is
+ * known before generation) is packed slot by slot:
+ *   kept slot      prompt | all generated tokens so far     (copied from `tokens`)
+ *   refilled slot  the queued prompt                        (copied from `queue_tokens`)
+ *   empty slot     nothing
+ * slot_source[i] = -1 kept, k >= 0 refilled with prompt k, -2 empty.
+ * counts: [0] freed slots, [1] refilled slots, [2] context tokens of the next step.
+ * next_tokens has room for `capacity` tokens; tokens beyond it are not written.
+ * ---------------------------------------------------------------------------------------- */
+void oracle_advance_batch(const int32_t *seq_begin, const int32_t *prompt_len,
+                          const int32_t *prev_len, const int32_t *new_len,
+                          const uint8_t *truncated, const int32_t *tokens,
+                          const int32_t *queue_begin, const int32_t *queue_tokens,
+                          int32_t B, int32_t M,
+                          int32_t *next_prompt_len, int32_t *next_prev_len,
+                          int32_t *next_seq_begin, int32_t *next_tokens, int64_t capacity,
+                          int32_t *free_slots, int32_t *slot_source, int64_t *counts)
+{
+    int64_t n_free = 0, n_refilled = 0, pos = 0;
+    for (int32_t i = 0; i < B; ++i) {
+        next_seq_begin[i] = (int32_t)pos;
+        if (truncated[i]) {                       /* unfinished: stays, this window joins the past */
+            next_prompt_len[i] = prompt_len[i];
+            next_prev_len[i] = prev_len[i] + new_len[i];
+            slot_source[i] = -1;
+            const int64_t len = (int64_t)prompt_len[i] + prev_len[i] + new_len[i];
+            for (int64_t o = 0; o < len; ++o, ++pos)
+                if (pos < capacity) next_tokens[pos] = tokens[seq_begin[i] + o];
+        } else {                                  /* finished: the slot is freed */
+            free_slots[n_free] = i;
+            next_prev_len[i] = 0;
+            if (n_free < M) {
+                const int32_t k = (int32_t)n_free;
+                const int32_t len = queue_begin[k + 1] - queue_begin[k];
+                next_prompt_len[i] = len;
+                slot_source[i] = k;
+                for (int32_t o = 0; o < len; ++o, ++pos)
+                    if (pos < capacity) next_tokens[pos] = queue_tokens[queue_begin[k] + o];
+                ++n_refilled;
+            } else {
+                next_prompt_len[i] = 0;
+                slot_source[i] = -2;
+            }
+            ++n_free;
+        }
+    }
+    next_seq_begin[B] = (int32_t)pos;
+    counts[0] = n_free;
+    counts[1] = n_refilled;
+    counts[2] = pos;
+}
