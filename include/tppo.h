@@ -48,7 +48,8 @@ enum {
     TPPO_DEV_BAD_TARGET = 1,  /* targets[row] outside [0, V): that row contributes nothing   */
     TPPO_DEV_WAIT_TIMEOUT = 2,/* a bounded look-back wait gave up: outputs incomplete        */
     TPPO_DEV_BAD_INDEX = 4,   /* a row / token index outside its array: entry skipped        */
-    TPPO_DEV_BAD_SEGMENT = 8  /* segment bounds outside [0, N] or not ascending: skipped     */
+    TPPO_DEV_BAD_SEGMENT = 8, /* segment bounds outside [0, N] or not ascending: skipped     */
+    TPPO_DEV_OVERFLOW = 16    /* an output buffer was too small: the excess was not written  */
 };
 
 typedef enum {
@@ -261,6 +262,42 @@ int tppo_lmhead_logprob_fwd_bwd(const void *hidden, const void *weight,
                                 float *logp, float *token_loss, float *loss, int32_t *stats,
                                 void *dhidden, void *dweight, int32_t chunk_tiles,
                                 void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Successive batching between two training steps (Section 3.2 and its batching figure; Algorithm 1
+ * line 2: "collect K prompts from last step unfinished samples and replace finished samples with
+ * new prompts").  The batch keeps its B slots, visited in ascending order:
+ *   - truncated[i] != 0 (no end condition reached): the sequence stays in slot i; the tokens of this
+ *     window join those of earlier windows: next_prompt_len = prompt_len, next_prev_len = prev_len +
+ *     new_len, slot_source = -1.
+ *   - otherwise the slot is freed and listed in free_slots; the k-th freed slot takes queued prompt
+ *     k while the queue lasts (k < M): next_prompt_len = its length, next_prev_len = 0, slot_source =
+ *     k; later freed slots stay empty (lengths 0, slot_source = -2).
+ * The context of the next step (everything known before generation) is packed slot by slot into
+ * next_tokens with offsets next_seq_begin: a kept slot's prompt and all its generated tokens copied
+ * from `tokens`, a refilled slot's prompt copied from `queue_tokens`.
+ *
+ *   seq_begin [B+1], prompt_len / prev_len / new_len [B] int32, truncated [B] u8: the finished step
+ *   tokens       [N] int32 token ids in that packed layout
+ *   queue_begin  [M+1] int32 offsets of the queued prompts inside queue_tokens [queue_total]
+ *   next_prompt_len, next_prev_len [B]; next_seq_begin [B+1]; next_tokens [capacity] int32 out
+ *   free_slots   [B] int32 out, ascending, first counts[0] entries valid
+ *   slot_source  [B] int32 out
+ *   counts       [4] int32 out: freed slots, refilled slots, context tokens of the next step, device
+ *                status bits (TPPO_DEV_OVERFLOW when the context exceeds `capacity` or 2^31-1: the
+ *                excess is not written; TPPO_DEV_BAD_INDEX for negative lengths or reads outside
+ *                `tokens` / `queue_tokens`, which are skipped)
+ * No workspace.  Bit-exact and run-to-run identical.
+ */
+int tppo_advance_batch(const int32_t *seq_begin, const int32_t *prompt_len,
+                       const int32_t *prev_len, const int32_t *new_len,
+                       const uint8_t *truncated, const int32_t *tokens, int64_t N,
+                       const int32_t *queue_begin, const int32_t *queue_tokens,
+                       int64_t queue_total, int32_t B, int32_t M,
+                       int32_t *next_prompt_len, int32_t *next_prev_len,
+                       int32_t *next_seq_begin, int32_t *next_tokens, int64_t capacity,
+                       int32_t *free_slots, int32_t *slot_source, int32_t *counts,
+                       void *stream);
 
 #ifdef __cplusplus
 }

@@ -24,7 +24,7 @@ OP_EGAE, OP_SELECT_TOKENS, OP_POLICY_LOSS, OP_VALUE_LOSS, OP_LMHEAD = range(5)
 BF16, F32 = 0, 1
 DLOGITS_NONE, DLOGITS_FULL, DLOGITS_COMPACT = 0, 1, 2
 POLICY_AUTO, POLICY_TWO_PASS, POLICY_CLUSTER_SMEM = 0, 1, 2
-DEV_BAD_TARGET, DEV_WAIT_TIMEOUT, DEV_BAD_INDEX, DEV_BAD_SEGMENT = 1, 2, 4, 8
+DEV_BAD_TARGET, DEV_WAIT_TIMEOUT, DEV_BAD_INDEX, DEV_BAD_SEGMENT, DEV_OVERFLOW = 1, 2, 4, 8, 16
 
 _vp, _i32, _i64, _f32, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
 
@@ -52,6 +52,9 @@ _lib.tppo_lmhead_logprob_fwd_bwd.restype = C.c_int
 _lib.tppo_lmhead_logprob_fwd_bwd.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _i64,
                                              _f32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, _i32,
                                              _vp, _sz, _vp]
+_lib.tppo_advance_batch.restype = C.c_int
+_lib.tppo_advance_batch.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _i32, _i32,
+                                    _vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp]
 
 
 class TppoError(RuntimeError):
@@ -178,3 +181,17 @@ def tppo_lmhead_logprob_fwd_bwd(hidden, weight, targets, aux_idx, old_logp, adv,
         _ptr(logp, torch.float32), _ptr(token_loss, torch.float32), _ptr(loss, torch.float32),
         _ptr(stats, torch.int32), _ptr(dhidden, torch.bfloat16), _ptr(dweight, torch.bfloat16),
         chunk_tiles, _ptr(ws), ws.numel(), _stream()))
+
+
+def tppo_advance_batch(seq_begin, prompt_len, prev_len, new_len, truncated, tokens, queue_begin,
+                       queue_tokens, next_prompt_len, next_prev_len, next_seq_begin, next_tokens,
+                       free_slots, slot_source, counts):
+    B, M = prompt_len.numel(), queue_begin.numel() - 1
+    _check(_lib.tppo_advance_batch(
+        _ptr(seq_begin, torch.int32), _ptr(prompt_len, torch.int32), _ptr(prev_len, torch.int32),
+        _ptr(new_len, torch.int32), _ptr(truncated, torch.uint8), _ptr(tokens, torch.int32),
+        tokens.numel(), _ptr(queue_begin, torch.int32), _ptr(queue_tokens, torch.int32),
+        queue_tokens.numel(), B, M, _ptr(next_prompt_len, torch.int32),
+        _ptr(next_prev_len, torch.int32), _ptr(next_seq_begin, torch.int32),
+        _ptr(next_tokens, torch.int32), next_tokens.numel(), _ptr(free_slots, torch.int32),
+        _ptr(slot_source, torch.int32), _ptr(counts, torch.int32), _stream()))

@@ -26,7 +26,7 @@ def declared_symbols():
 def test_every_declared_symbol_is_exported(lib):
     names = declared_symbols()
     assert {"tppo_egae", "tppo_select_tokens", "tppo_policy_loss_fwd_bwd", "tppo_value_loss",
-            "tppo_lmhead_logprob_fwd_bwd", "tppo_workspace_bytes", "tppo_version",
+            "tppo_lmhead_logprob_fwd_bwd", "tppo_advance_batch", "tppo_workspace_bytes", "tppo_version",
             "tppo_status_string"} <= set(names)
     for n in names:
         assert hasattr(lib, n), n
