@@ -10,6 +10,7 @@ on 16384 value tokens.  The metric is selected (policy) tokens per second.
   python bench.py [--gpus N] [--steps K] [--warmup W]            CUDA path (this repo)
   python bench.py --impl reference ...                           float64 CPU oracle on host cores
   python bench.py --workload lmhead ...                          the LM-head variant as the bench line
+  python bench.py --workload cfg4 ...                            EGAE + compaction sweep (config 4)
 
 The default line also carries an "lmhead_variant" object: the tensor-core variant that forms the
 logits from hidden states [16384, 5120] and the LM-head weight [5120, 152064] without storing them,
@@ -357,7 +358,7 @@ def main():
     ap.add_argument("--hint", type=int, default=0, help="kernel_hint passed to the policy loss")
     ap.add_argument("--rows", type=int, default=16384,
                     help="rows of the loss micro-batch (smaller only for profiler captures)")
-    ap.add_argument("--workload", default="cfg3", choices=["cfg3", "lmhead"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg3", "lmhead", "cfg4"])
     ap.add_argument("--lmhead-calls", type=int, default=5)
     ap.add_argument("--lm-rows", type=int, default=16384,
                     help="rows of the LM-head workload (smaller only for profiler captures)")
@@ -377,6 +378,9 @@ def main():
     torch.cuda.set_device(local)
     if args.workload == "lmhead":
         run_lmhead_workload(args, rank, world, local, dev, warmup)
+        return
+    if args.workload == "cfg4":
+        run_cfg4_workload(args, rank, world, local, dev, warmup)
         return
     st = Step(dev, seed=2 + rank, rows=args.rows)      # every rank holds its own batch
     st.hint = args.hint
@@ -584,6 +588,105 @@ def run_lmhead_workload(args, rank, world, local, dev, warmup):
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+
+
+def run_cfg4_workload(args, rank, world, local, dev, warmup):
+    """Config 4, the bandwidth test of the small kernels: EGAE, token selection, value loss and the
+    batch advance over 4096 ragged segments (17.5 M tokens).  One step = the four calls; every call is
+    also timed on its own (CUDA events) against its algorithmic bytes."""
+    from paper_2506_15050_b200 import binding as b
+    c = synth.config4()
+    N, B = c["N"], c["B"]
+    t = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).to(dev)
+    rng = np.random.default_rng(8)
+    rewards, values = t(c["rewards"], torch.float32), t(c["values"], torch.float32)
+    old_values = values + 0.2 * torch.randn(N, device=dev, generator=torch.Generator(dev).manual_seed(3))
+    sb, se, tr = t(c["seg_begin"], torch.int32), t(c["seg_end"], torch.int32), t(c["truncated"], torch.uint8)
+    boot = t(c["bootstrap"], torch.float32)
+    seqb = t(c["seq_begin"], torch.int32)
+    pl, pv, nl = (t(c[k], torch.int32) for k in ("prompt_len", "prev_len", "new_len"))
+    pm, vm = t(c["extra_policy_mask"], torch.uint8), t(c["extra_value_mask"], torch.uint8)
+    tokens = t(rng.integers(0, synth.V_QWEN, N).astype(np.int32), torch.int32)
+    n_fin = int((c["truncated"] == 0).sum())
+    qlens = rng.integers(16, 2048, n_fin)
+    qb = t(np.concatenate([[0], np.cumsum(qlens)]).astype(np.int32), torch.int32)
+    qt = t(rng.integers(0, synth.V_QWEN, int(qlens.sum())).astype(np.int32), torch.int32)
+    adv, ret = torch.empty(N, device=dev), torch.empty(N, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    pol = torch.empty(N, dtype=torch.int32, device=dev)
+    val = torch.empty(N, dtype=torch.int32, device=dev)
+    counts = torch.zeros(4, dtype=torch.int32, device=dev)
+    loss, dv = torch.zeros(1, device=dev), torch.empty(N, device=dev)
+    vst = torch.zeros(2, dtype=torch.int32, device=dev)
+    npl, npv = torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev)
+    nsb = torch.empty(B + 1, dtype=torch.int32, device=dev)
+    ntk = torch.empty(N + qt.numel(), dtype=torch.int32, device=dev)
+    fs, src = torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev)
+    acn = torch.zeros(4, dtype=torch.int32, device=dev)
+    ws1 = b.workspace(b.OP_EGAE, N, B, 0, 0, dev)
+    ws2 = b.workspace(b.OP_SELECT_TOKENS, N, B, 0, 0, dev)
+    ws3 = b.workspace(b.OP_VALUE_LOSS, N, 0, N, 0, dev)
+    calls = {
+        "egae": lambda: b.tppo_egae(rewards, values, sb, se, tr, boot, 1.0, 0.95, adv, ret, status, ws1),
+        "select": lambda: b.tppo_select_tokens(seqb, pl, pv, nl, tr, 0, pm, vm, N, pol, val, counts, ws2),
+        "value": lambda: b.tppo_value_loss(values, old_values, ret, val, counts[1:2], N, 0.5, 0.6, 0.0,
+                                           loss, dv, vst, ws3),
+        "advance": lambda: b.tppo_advance_batch(seqb, pl, pv, nl, tr, tokens, qb, qt, npl, npv, nsb, ntk,
+                                                fs, src, acn),
+    }
+
+    def step(events=None):
+        for name, f in calls.items():
+            if events is None:
+                f()
+            else:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); f(); e1.record()
+                events[name].append((e0, e1))
+
+    steps = args.steps if args.steps != 200 else 50
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    events = {k: [] for k in calls}
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        step(events)
+    t1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = t0.elapsed_time(t1) / steps
+    cn, an = counts.cpu().numpy(), acn.cpu().numpy()
+    assert int(status) == 0 and cn[2] == 0 and an[3] == 0 and int(vst[1]) == 0
+    peak, kind = measured_peaks()
+    algo = {"egae": 16 * N, "select": 2 * N + 4 * (int(cn[0]) + int(cn[1])),
+            "value": 20 * int(cn[1]) + 4 * N, "advance": 8 * int(an[2])}
+    kernels = {}
+    for k, ev in events.items():
+        us = float(np.mean([a.elapsed_time(b_) for a, b_ in ev])) * 1e3
+        gbs = algo[k] / us / 1e3
+        kernels[k] = {"us": us, "algorithmic_bytes": algo[k], "GB/s": gbs, "frac": gbs / peak}
+    if rank == 0:
+        print(json.dumps({
+            "metric": "tokens/s, EGAE + token compaction + value loss + batch advance, config 4",
+            "value": N / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32 in, f64 scan state, int32 indices", "data": "synthetic",
+            "config": {"workload": "cfg4: %d ragged segments, %d tokens, lengths log-uniform in [16, 32768], "
+                                   "half truncated, Bernoulli(0.5) masks" % (B, N),
+                       "l2": "inputs larger than L2 (%.0f MB per array)" % (N * 4 / 1e6),
+                       "selected": {"policy": int(cn[0]), "value": int(cn[1])},
+                       "advance": {"freed": int(an[0]), "context_tokens": int(an[2])}},
+            "roofline": {"bound": "hbm", "achieved": kernels["egae"]["GB/s"], "peak": peak, "unit": "GB/s",
+                         "frac": kernels["egae"]["frac"], "peak_kind": kind, "traffic": None,
+                         "kernel": "egae_scan_kernel", "kernel_ms": kernels["egae"]["us"] / 1e3,
+                         "algorithmic_bytes_per_launch": algo["egae"]},
+            "kernels": kernels, "gpu_launches": 7 * steps, "clocks": clocks}))
 
 
 if __name__ == "__main__":
