@@ -247,8 +247,9 @@ int tppo_value_loss(const float *values, const float *old_values, const float *r
  *   tppo_policy_loss_fwd_bwd (n = M)
  *   dhidden  [M, K] bf16 out or NULL;  dweight [K, V] bf16 out or NULL (both NULL: forward only)
  *   chunk_tiles  0 = choose automatically; otherwise the number of 256-column vocabulary tiles per
- *                chunk, clamped to the automatic choice (which sizes the workspace).  For tuning
- *                and testing; changes the result only by the rounding order of dhidden's sum.
+ *                chunk (low 16 bits), clamped to the automatic choice (which sizes the workspace).
+ *                Adding 65536 selects the CTA-pair (cta_group::2) GEMM kernels instead of the single-CTA ones.  For
+ *                tuning and testing; changes the result only by the rounding order of dhidden's sum.
  *   workspace    tppo_workspace_bytes(TPPO_OP_LMHEAD, M, K, 0, V) bytes
  * K and V must be multiples of 8 (TPPO_ERR_UNSUPPORTED otherwise).  A row with a target outside
  * [0, V) or an aux index outside [0, aux_len) contributes nothing and raises the status bit.

@@ -13,6 +13,7 @@
 // Four GEMM-sized contractions in total; the chunk buffer is the only logits-shaped memory.
 #include "policy_common.cuh"
 #include "umma_gemm.cuh"
+#include "umma_gemm_pair.cuh"
 
 namespace tppo {
 
@@ -243,6 +244,15 @@ lmhead_rows_kernel(const RowRec* rec, const float2* part, const float* xy, int64
     coef[r] = rl.coef;
 }
 
+// Single-CTA kernels by default; the CTA-pair kernels (a third less operand traffic per FLOP, but no
+// faster under the power cap that bounds this path) are selectable for comparison.
+template <int AMAJ, int BMAJ, class Epi>
+int launch_gemm(bool pair, const CUtensorMap& a, const CUtensorMap& b, const GemmShape& g,
+                const Epi& e, int32_t* status, cudaStream_t s) {
+    return pair ? launch_umma_gemm_pair<AMAJ, BMAJ>(a, b, g, e, status, s)
+                : launch_umma_gemm<AMAJ, BMAJ>(a, b, g, e, status, s);
+}
+
 struct LmPlan {
     int32_t n_tiles;       // 256-column tiles of the vocabulary
     int32_t chunk_tiles;   // tiles per vocabulary chunk
@@ -334,6 +344,8 @@ TPPO_API int tppo_lmhead_logprob_fwd_bwd(const void* hidden, const void* weight,
     const LmWorkspace w = lmhead_carve(workspace, M, K, V);
     LmPlan plan = lmhead_plan(M, K, V);
     const int64_t ldx = int64_t(plan.chunk_tiles) * kTileN;     // row stride of the chunk buffer
+    const bool pair = (chunk_tiles & 0x10000) != 0;             // bit 16: CTA-pair kernels
+    chunk_tiles &= 0xffff;
     if (chunk_tiles > 0 && chunk_tiles < plan.chunk_tiles) plan.chunk_tiles = chunk_tiles;
 
     PolicyArgs a{};
@@ -357,14 +369,15 @@ TPPO_API int tppo_lmhead_logprob_fwd_bwd(const void* hidden, const void* weight,
     if (!make_bf16_tensor_map(&map_h128, hidden, uint64_t(M), uint64_t(K), uint64_t(K), 128) ||
         !make_bf16_tensor_map(&map_h64, hidden, uint64_t(M), uint64_t(K), uint64_t(K), 64) ||
         !make_bf16_tensor_map(&map_w64, weight, uint64_t(K), uint64_t(V), uint64_t(V), 64) ||
-        !make_bf16_tensor_map(&map_w256, weight, uint64_t(K), uint64_t(V), uint64_t(V), 256))
+        !make_bf16_tensor_map(&map_w256, weight, uint64_t(K), uint64_t(V), uint64_t(V),
+                              pair ? 128 : 256))     // K-major B box: 128 rows per CTA of a pair
         return TPPO_ERR_CUDA;
 
     // pass 1: statistics over the whole vocabulary
     {
         const GemmShape g{mt, plan.n_tiles, ks_k, 0, 0, 0, 0, 16};
         const EpiStats e{w.rec, w.part, w.xy, M, V};
-        rc = launch_umma_gemm<0, 1>(map_h128, map_w64, g, e, stats + 3, s);
+        rc = launch_gemm<0, 1>(pair, map_h128, map_w64, g, e, stats + 3, s);
         if (rc != TPPO_OK) return rc;
     }
     const float inv_denom = denom > 0.f ? 1.f / denom : 1.f / float(M);
@@ -390,7 +403,7 @@ TPPO_API int tppo_lmhead_logprob_fwd_bwd(const void* hidden, const void* weight,
         {
             const GemmShape g{mt, ct, ks_k, 0, 0, v0, 0, 16};
             const EpiDx e{w.rec, w.lse2, w.coef, w.dxc, ldx, M, V, v0};
-            rc = launch_umma_gemm<0, 1>(map_h128, map_w64, g, e, stats + 3, s);
+            rc = launch_gemm<0, 1>(pair, map_h128, map_w64, g, e, stats + 3, s);
             if (rc != TPPO_OK) return rc;
         }
         if (dhidden) {
@@ -398,13 +411,13 @@ TPPO_API int tppo_lmhead_logprob_fwd_bwd(const void* hidden, const void* weight,
                               0, 0, 0, v0, 16};
             const EpiDh e{w.dhacc, static_cast<uint16_t*>(dhidden), M, K, ci == 0,
                           ci == n_chunks - 1};
-            rc = launch_umma_gemm<0, 0>(map_dx128, map_w256, g, e, stats + 3, s);
+            rc = launch_gemm<0, 0>(pair, map_dx128, map_w256, g, e, stats + 3, s);
             if (rc != TPPO_OK) return rc;
         }
         if (dweight) {
             const GemmShape g{(K + kTileM - 1) / kTileM, ct, ks_m, 0, 0, 0, 0, 16};
             const EpiDw e{static_cast<uint16_t*>(dweight), K, V, v0};
-            rc = launch_umma_gemm<1, 1>(map_h64, map_dx64, g, e, stats + 3, s);
+            rc = launch_gemm<1, 1>(pair, map_h64, map_dx64, g, e, stats + 3, s);
             if (rc != TPPO_OK) return rc;
         }
     }

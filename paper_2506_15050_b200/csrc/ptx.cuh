@@ -113,6 +113,17 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(cta));
     return r;
 }
+// mbarrier arrivals on a barrier given by its shared::cluster address (this CTA's or another's)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes) {
+    // relaxed: the announcement orders nothing itself (the data arrives with complete_tx), and a
+    // cluster-scope release here would wait on the thread's earlier traffic every stage
+    asm volatile("mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%0], %1;"
+                 ::"r"(cluster_bar), "r"(bytes) : "memory");
+}
 // Asynchronous remote shared-memory stores: the data lands in the target CTA and its bytes are
 // counted on that CTA's mbarrier, so the receiver's wait doubles as the data dependency.
 __device__ __forceinline__ void st_async_f32x2(uint32_t cluster_addr, float a, float b, uint32_t cluster_bar) {

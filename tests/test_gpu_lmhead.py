@@ -93,8 +93,13 @@ def old_logp_from_oracle(hb, wb, targets, noise):
     return x, (lp + noise).astype(np.float32)
 
 
+CTA_PAIR = 65536        # added to chunk_tiles: the CTA-pair (cta_group::2) GEMM kernels
+
+
 @pytest.mark.parametrize("M,K,V,chunk", [(300, 320, 2000, 0), (300, 320, 2000, 3),
-                                         (1024, 512, 8200, 5), (128, 64, 256, 0)])
+                                         (1024, 512, 8200, 5), (128, 64, 256, 0),
+                                         (300, 320, 2000, CTA_PAIR + 3),
+                                         (1024, 512, 8200, CTA_PAIR)])
 def test_lmhead_matches_oracle(M, K, V, chunk):
     hidden, weight, targets, adv, noise = make_case(M, K, V, seed=40 + M % 7)
     hb, wb = synth.bf16_bits(hidden), synth.bf16_bits(weight)
@@ -220,11 +225,12 @@ def cfg5():
     torch.cuda.empty_cache()
 
 
-def test_config5_full_sampled_rows(cfg5):
+@pytest.mark.parametrize("variant", [0, CTA_PAIR])
+def test_config5_full_sampled_rows(cfg5, variant):
     c = cfg5
     M, K, V, pick = c["M"], c["K"], c["V"], c["pick"]
     out = run_lmhead(c["hidden"], c["weight"], c["targets"], c["old_logp"], c["adv"], c["eps_low"],
-                     c["eps_high"])
+                     c["eps_high"], chunk_tiles=variant)
     assert out["stats"][0] == M and out["stats"][3] == 0
     ref = oracle.policy_loss(c["x_pick"], c["targets"][pick], None, None, c["old_logp"][pick],
                              c["adv"][pick], f32(c["eps_low"]), f32(c["eps_high"]), denom=float(M))
@@ -242,7 +248,7 @@ def test_config5_full_sampled_rows(cfg5):
     assert float((row_sum / row_abs).max()) < 1e-3
     # the run is reproducible bit for bit
     again = run_lmhead(c["hidden"], c["weight"], c["targets"], c["old_logp"], c["adv"], c["eps_low"],
-                       c["eps_high"])
+                       c["eps_high"], chunk_tiles=variant)
     assert again["loss"] == out["loss"] and torch.equal(again["dw_t"], out["dw_t"]) and \
         torch.equal(again["dh_t"], out["dh_t"])
 
