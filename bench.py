@@ -162,7 +162,7 @@ class Step:
         self.hint = 0
         self.denom_pol = 0.0      # > 0: selected-token counts of the whole job (several GPUs)
         self.denom_val = 0.0
-        # old-policy log-probs (Algorithm 1 line 3): forward-only pass of the same kernel, plus noise
+        # old-policy log-probs (the old-policy snapshot of Algorithm 1): forward-only pass of the same kernel, plus noise
         self.egae()
         self.select()
         self.policy(forward_only=True)

@@ -4,7 +4,7 @@
  * The library computes the part of a Truncated-PPO training step that the paper's method changes:
  * EGAE advantages over possibly truncated responses (Section 3.1, Eq. 6), the policy / value
  * token filter (Section 3.2), and the two losses restricted to the surviving tokens (Eq. 1 and
- * Eq. 4-5, Algorithm 1 lines 6, 8, 9).
+ * Eq. 4-5; the advantage, policy and value steps of Algorithm 1).
  *
  * Conventions that hold for every entry point
  *   - Every array pointer is a DEVICE pointer unless the comment says "host".  The caller owns all
@@ -65,7 +65,7 @@ enum { TPPO_BF16 = 0, TPPO_F32 = 1 };
 
 /* where the gradient with respect to the logits goes */
 enum {
-    TPPO_DLOGITS_NONE = 0,    /* forward only (e.g. old-policy log-probs, Algorithm 1 line 3) */
+    TPPO_DLOGITS_NONE = 0,    /* forward only (e.g. the old-policy log-probs of Algorithm 1)  */
     TPPO_DLOGITS_FULL = 1,    /* [R, ld] like the logits; rows that are not selected are     */
                               /* zero-filled; may be the logits buffer itself (in place)     */
     TPPO_DLOGITS_COMPACT = 2  /* [n_max, V] dense, row j belongs to the j-th selected row    */
@@ -86,7 +86,7 @@ size_t tppo_workspace_bytes(int op, int64_t N, int32_t B, int64_t n_max, int32_t
 
 /*
  * EGAE advantages and Monte-Carlo returns (Section 3.1, Eq. 6 with the TD residual of Eq. 3;
- * R_t as defined after Eq. 5; Algorithm 1 line 6).
+ * R_t as defined after Eq. 5; the advantage step of Algorithm 1).
  *
  * For each response segment [seg_begin[i], seg_end[i]) of the packed arrays, backwards in t:
  *     delta_t = rewards[t] + gamma * V(s_{t+1}) - values[t]
@@ -170,7 +170,7 @@ int tppo_select_tokens(const int32_t *seq_begin, const int32_t *prompt_len,
 /*
  * Fused per-token log-softmax gather + clipped PPO surrogate, forward and backward to the logits
  * (Eq. 1 with decoupled eps_low / eps_high; token-level mean and no KL term per Section 4.1.1;
- * Algorithm 1 line 8).  For the j-th selected row r = rows[j] (j < n), a = aux_idx[j]:
+ * the policy update of Algorithm 1).  For the j-th selected row r = rows[j] (j < n), a = aux_idx[j]:
  *     logp_j = x[r, y] - log sum_v exp(x[r, v]),            y = targets[r]
  *     rho    = exp(logp_j - old_logp[a])
  *     l_j    = -min(rho*adv[a], clip(rho, 1-eps_low, 1+eps_high)*adv[a])
@@ -215,8 +215,8 @@ enum {
 };
 
 /*
- * Clipped value regression on the value tokens, forward and backward (Eq. 4-5; Algorithm 1
- * line 9).  For p = value_idx[j], j < n = min(*n_sel, n_max):
+ * Clipped value regression on the value tokens, forward and backward (Eq. 4-5; the value update
+ * of Algorithm 1).  For p = value_idx[j], j < n = min(*n_sel, n_max):
  *     Vc = clip(values[p], old_values[p] - xi_low, old_values[p] + xi_high)
  *     l  = 1/2 * max((values[p]-returns[p])^2, (Vc-returns[p])^2),   loss = (1/denom) sum l
  *     dvalues[p] = (values[p]-returns[p])/denom  if the unclipped term is the max (ties included),
@@ -265,9 +265,9 @@ int tppo_lmhead_logprob_fwd_bwd(const void *hidden, const void *weight,
                                 void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * Successive batching between two training steps (Section 3.2 and its batching figure; Algorithm 1
- * line 2: "collect K prompts from last step unfinished samples and replace finished samples with
- * new prompts").  The batch keeps its B slots, visited in ascending order:
+ * Successive batching between two training steps (Section 3.2 and its batching figure; the step of
+ * Algorithm 1 that keeps the unfinished samples of the last step and puts new prompts in the place
+ * of the finished ones).  The batch keeps its B slots, visited in ascending order:
  *   - truncated[i] != 0 (no end condition reached): the sequence stays in slot i; the tokens of this
  *     window join those of earlier windows: next_prompt_len = prompt_len, next_prev_len = prev_len +
  *     new_len, slot_source = -1.

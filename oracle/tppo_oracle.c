@@ -324,8 +324,8 @@ void oracle_lmhead_dweight_cols(const uint16_t *hidden, const double *dx_cols,
 }
 
 /* ------------------------------------------------------------------------------------------
- * Successive batching between two training steps (Section 3.2, the batching figure; Algorithm 1
- * line 2): the batch keeps its B slots.  A slot whose sequence reached an end condition is
+ * Successive batching between two training steps (Section 3.2, the batching figure; the batch
+ * collection step of Algorithm 1): the batch keeps its B slots.  A slot whose sequence reached an end condition is
  * freed and takes the next queued prompt; a slot whose sequence was cut at the window keeps it,
  * and the tokens generated in this step join those of earlier windows.
  *

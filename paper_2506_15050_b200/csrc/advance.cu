@@ -1,6 +1,6 @@
 // Successive batching between two training steps (Section 3.2 of the paper, the batching figure;
-// Algorithm 1 line 2): the batch keeps its B slots, a finished sequence frees its slot for the next
-// queued prompt, an unfinished one stays and the tokens of this window join its earlier ones.  Two
+// the batch collection step of Algorithm 1): the batch keeps its B slots, a finished sequence frees
+// its slot for the next queued prompt, an unfinished one stays and the tokens of this window join its earlier ones.  Two
 // kernels: one CTA walks the slots (two block-wide prefix sums per 1024 slots: rank among the freed
 // slots, then the packed offsets of the next step's context), then a bandwidth-bound ragged copy
 // moves the kept sequences and the queued prompts into the new packed token buffer.  Integer work

@@ -194,7 +194,9 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
     __shared__ double s_carry[kScanWarps][2];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) s_ticket[0] = atomicAdd(a.ticket, 1u);
+    // the ticket counter starts at all-ones like the rest of the workspace (one memset): + 1 wraps
+    // the first draw to ticket 0
+    if (threadIdx.x == 0) s_ticket[0] = atomicAdd(a.ticket, 1u) + 1u;
     __syncthreads();
     uint32_t ticket = s_ticket[0];
     if (ticket >= uint32_t(a.num_tiles)) return;
@@ -217,7 +219,7 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
         const int tile = a.num_tiles - 1 - int(ticket);
         const int64_t t0 = int64_t(tile) * kScanTile;
         const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
-        if (threadIdx.x == 0) s_ticket[(it & 1) ^ 1] = atomicAdd(a.ticket, 1u);   // next tile
+        if (threadIdx.x == 0) s_ticket[(it & 1) ^ 1] = atomicAdd(a.ticket, 1u) + 1u;   // next tile
 
         // ---- per-position maps, right to left -----------------------------------------------
         const int win_lo = buf.win_lo;
@@ -478,10 +480,8 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
     if (N == 0) return TPPO_OK;
-    const size_t ticket_bytes = align_up(sizeof(uint32_t), kWsAlign);
-    TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0, ticket_bytes, s));
-    TPPO_CUDA_CHECK(cudaMemsetAsync(static_cast<char*>(workspace) + ticket_bytes, 0xff,
-                                    need - ticket_bytes, s));    // tile states start out unset
+    // one memset: tile states start out unset (all-ones), the ticket counter at all-ones too
+    TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0xff, need, s));
     EgaeArgs a;
     a.rewards = rewards; a.values = values; a.seg_begin = seg_begin; a.seg_end = seg_end;
     a.truncated = truncated; a.bootstrap = bootstrap; a.B = B; a.N = int32_t(N);
@@ -562,10 +562,8 @@ TPPO_API int tppo_egae_static(const float* rewards, const float* values, const i
     a.ticket = static_cast<uint32_t*>(scratch);
     a.state = reinterpret_cast<TileState*>(static_cast<char*>(scratch) + 256);
     // the array still holds the previous call's tile states and ticket: reset the part this call
-    // uses (ticket to zero, tile states to the all-ones "unset" pattern)
-    TPPO_CUDA_CHECK(cudaMemsetAsync(scratch, 0, 256, s));
-    TPPO_CUDA_CHECK(cudaMemsetAsync(static_cast<char*>(scratch) + 256, 0xff,
-                                    size_t(a.num_tiles) * sizeof(TileState), s));
+    // uses to the all-ones pattern (tile states unset, ticket counter one draw before ticket 0)
+    TPPO_CUDA_CHECK(cudaMemsetAsync(scratch, 0xff, 256 + size_t(a.num_tiles) * sizeof(TileState), s));
     egae_scan_kernel<<<egae_grid(a.num_tiles), kScanThreads, 0, s>>>(a);
     TPPO_CUDA_CHECK(cudaGetLastError());
     return TPPO_OK;

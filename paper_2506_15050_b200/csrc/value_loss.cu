@@ -1,5 +1,5 @@
 // Clipped value regression on the value tokens, forward and backward (Eq. 4-5 of the paper;
-// Algorithm 1 line 9).  A gather over value_idx: 3 fp32 reads + 1 index read + 1 gradient write
+// the value update of Algorithm 1).  A gather over value_idx: 3 fp32 reads + 1 index read + 1 gradient write
 // per value token.  The mean is reduced in a fixed order (per-thread strided partials in fp64,
 // fixed shuffle tree, per-block partials summed by one block), so results are run-to-run
 // identical.

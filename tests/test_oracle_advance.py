@@ -1,4 +1,5 @@
-"""Pins for the oracle's successive-batching step (Section 3.2, batching figure; Algorithm 1 line 2):
+"""Pins for the oracle's successive-batching step (Section 3.2, batching figure; the batch
+collection step of Algorithm 1):
 an independent list-based restatement, exhaustive enumeration on tiny batches, and invariants."""
 import itertools
 
