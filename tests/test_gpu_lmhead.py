@@ -98,6 +98,8 @@ CTA_PAIR = 65536        # added to chunk_tiles: the CTA-pair (cta_group::2) GEMM
 
 @pytest.mark.parametrize("M,K,V,chunk", [(300, 320, 2000, 0), (300, 320, 2000, 3),
                                          (1024, 512, 8200, 5), (128, 64, 256, 0),
+                                         (1, 64, 264, 0), (130, 328, 2008, 2),
+                                         (130, 328, 2008, CTA_PAIR + 2),
                                          (300, 320, 2000, CTA_PAIR + 3),
                                          (1024, 512, 8200, CTA_PAIR)])
 def test_lmhead_matches_oracle(M, K, V, chunk):
