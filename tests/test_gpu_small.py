@@ -409,3 +409,29 @@ def test_value_loss_config1():
     rl, rdv = oracle.value_loss(c["values"], c["old_values"], ret.astype(np.float32), val, f32(0.5), f32(0.6))
     assert n == 42 and abs(loss - rl) < 1e-6
     np.testing.assert_allclose(dv, rdv, rtol=1e-5, atol=1e-9)
+
+
+# ------------------------------------------------------------------------------------------------
+# many tiny sequences: more sequence starts per tile than the kernels keep in shared memory, so the
+# paths that search the global arrays run
+# ------------------------------------------------------------------------------------------------
+def test_select_and_egae_many_tiny_sequences():
+    rng = np.random.default_rng(12)
+    B = 6000
+    prompt = rng.integers(0, 3, B)
+    prev = rng.integers(0, 3, B) * rng.integers(0, 2, B)
+    new = rng.integers(0, 6, B)
+    trunc = rng.integers(0, 2, B).astype(np.uint8)
+    sb, seg_b, seg_e = synth.pack(prompt, prev, new)
+    N = int(sb[-1])
+    assert B / max(N // 4096, 1) > 400           # several hundred sequences per 4096-position tile
+    c = dict(seq_begin=sb, prompt_len=prompt, prev_len=prev, new_len=new, truncated=trunc)
+    pm = rng.integers(0, 2, N).astype(np.uint8)
+    vm = rng.integers(0, 2, N).astype(np.uint8)
+    check_select(c, tail_drop=1)
+    check_select(c, 2, pm, vm)
+    r = rng.standard_normal(N).astype(np.float32)
+    v = rng.standard_normal(N).astype(np.float32)
+    boot = rng.standard_normal(B).astype(np.float32)
+    check_egae(B, r, v, seg_b, seg_e, trunc, boot, 0.99, 0.95)
+    check_egae(B, r, v, seg_b, seg_e, trunc, None, 1.0, 1.0)
