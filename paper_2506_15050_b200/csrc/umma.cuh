@@ -1,6 +1,7 @@
 // Inline-PTX wrappers for the sm_100a tensor-core path: tensor memory (TMEM) allocation,
 // tcgen05.mma issue / commit / load, shared-memory matrix descriptors, the instruction descriptor
-// and tiled TMA loads.  Single-CTA (cta_group::1) forms only; no multicast anywhere.
+// and tiled TMA loads, in single-CTA (cta_group::1) and CTA-pair (cta_group::2) forms; no multicast
+// anywhere.
 #pragma once
 
 #include <cuda.h>          // CUtensorMap (type only; the encoder is looked up at run time)
@@ -156,13 +157,6 @@ __device__ __forceinline__ void mma_bf16_pair(uint32_t tmem_d, uint64_t a_desc, 
 __device__ __forceinline__ void mma_commit_pair(uint32_t cluster_bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                  ::"r"(cluster_bar) : "memory");
-}
-// The same arrival delivered by one instruction to the barrier at this shared-memory offset in both
-// CTAs of the pair (commit multicast; this is a barrier signal, not a data copy).
-__device__ __forceinline__ void mma_commit_pair_both(uint32_t bar) {
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-        ::"r"(bar), "h"(uint16_t(3)) : "memory");
 }
 // Tiled TMA load into this CTA's shared memory whose bytes are counted on an mbarrier that may
 // live in the peer CTA (shared::cluster address).  No multicast.

@@ -158,11 +158,13 @@ umma_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
                                             umma::smem_desc_advance(bd, j * b_kstep), idesc,
                                             (ks | j) != 0 ? 1u : 0u);
                     // the stage is reusable in both CTAs once these MMAs have read it
-                    umma::mma_commit_pair_both(empty_bar + 8 * stage);
+                    umma::mma_commit_pair(ptx::map_to_cta(empty_bar + 8 * stage, 0));
+                    umma::mma_commit_pair(ptx::map_to_cta(empty_bar + 8 * stage, 1));
                     if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
                 }
                 if (timed_out) break;
-                umma::mma_commit_pair_both(acc_full_bar + 8 * acc);
+                umma::mma_commit_pair(ptx::map_to_cta(acc_full_bar + 8 * acc, 0));
+                umma::mma_commit_pair(ptx::map_to_cta(acc_full_bar + 8 * acc, 1));
             }
         }
     } else {
