@@ -1,5 +1,5 @@
 // Token filter + stream compaction (Section 3.2 of the paper): one pass over the packed token
-// positions.  A thread turns its 16 consecutive positions into two 16-bit words by interval
+// positions.  A thread turns its 32 consecutive positions into two 32-bit words by interval
 // arithmetic on the sequences that overlap them, ranks come from popcounts and a warp / tile
 // prefix, a decoupled look-back chain links the tiles, and every selected position is written once
 // in ascending order.  Integer work throughout: the result is bit-exact and run-to-run identical.
@@ -9,8 +9,8 @@ namespace tppo {
 
 constexpr int kSelThreads = 256;
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kSelItems = 16;                                  // positions per lane
-constexpr int kSelTile = kSelThreads * kSelItems;              // 4096 positions per tile
+constexpr int kSelItems = 32;                                  // positions per thread
+constexpr int kSelTile = kSelThreads * kSelItems;              // 8192 positions per tile
 constexpr uint32_t kSelSpinLimit = 1u << 22;
 
 // tile state word: [63:62] flag (1 = tile total, 2 = inclusive prefix), [61:31] policy count,
@@ -63,7 +63,7 @@ struct SelectArgs {
     uint32_t* ticket;           // [1]
 };
 
-constexpr int kSeqCap = 320;   // sequence starts of one tile kept in shared memory
+constexpr int kSeqCap = 640;   // sequence starts of one tile kept in shared memory
 
 // 16 mask bytes -> 16 bits (bit k set iff byte k is non-zero).
 __device__ __forceinline__ uint32_t nonzero_bytes4(uint32_t w) {
@@ -75,20 +75,23 @@ __device__ __forceinline__ uint32_t nonzero_bytes16(uint4 v) {
     return nonzero_bytes4(v.x) | (nonzero_bytes4(v.y) << 4) | (nonzero_bytes4(v.z) << 8) |
            (nonzero_bytes4(v.w) << 12);
 }
-// Bits [lo - p0, hi - p0) of a 16-bit word, for the positions of [lo, hi) that fall in [p0, p0+16).
-__device__ __forceinline__ uint32_t range_bits16(int64_t lo, int64_t hi, int64_t p0) {
-    const int64_t a = min(max(lo - p0, int64_t(0)), int64_t(16));
-    const int64_t b = min(max(hi - p0, int64_t(0)), int64_t(16));
-    return b > a ? ((1u << int(b)) - 1u) & ~((1u << int(a)) - 1u) : 0u;
+// Bits [lo - p0, hi - p0) of a 32-bit word, for the positions of [lo, hi) that fall in [p0, p0+32).
+__device__ __forceinline__ uint32_t range_bits32(int64_t lo, int64_t hi, int64_t p0) {
+    const int64_t a = min(max(lo - p0, int64_t(0)), int64_t(32));
+    const int64_t b = min(max(hi - p0, int64_t(0)), int64_t(32));
+    if (b <= a) return 0u;                                       // then a < 32
+    const uint32_t upto_b = b >= 32 ? 0xffffffffu : ((1u << int(b)) - 1u);
+    return upto_b & ~((1u << int(a)) - 1u);
 }
 
-// Each thread owns 16 consecutive positions.  Its policy / value bits come from interval
+// Each thread owns 32 consecutive positions.  Its policy / value bits come from interval
 // arithmetic on the few sequences that overlap those positions (usually one) and from one 16-byte
-// load per byte mask, not from a test per position; selected positions are first compacted inside
+// loads per byte mask, not from a test per position; selected positions are first compacted inside
 // the tile in shared memory and then copied out with coalesced stores.
 __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const SelectArgs a) {
-    __shared__ int32_t s_out_pol[kSelTile];
-    __shared__ int32_t s_out_val[kSelTile];
+    // the tile's two compacted lists, as 16-bit offsets inside the tile (halves the shared memory)
+    __shared__ uint16_t s_out_pol[kSelTile];
+    __shared__ uint16_t s_out_val[kSelTile];
     __shared__ int32_t s_sb[kSeqCap + 1];
     __shared__ uint32_t s_tile;
     __shared__ int s_seq0, s_seq1;
@@ -108,10 +111,16 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     const int n_mine = max(0, min(kSelItems, n_tile - l0));    // positions this thread really owns
 
     // ---- the byte masks of this thread's positions, as bits (issued first: longest latency) ----
-    uint32_t pm_bits = 0xffffu, vm_bits = 0xffffu;
+    uint32_t pm_bits = 0xffffffffu, vm_bits = 0xffffffffu;
     if (n_mine == kSelItems && a.mask_vec_ok) {
-        if (a.pol_mask) pm_bits = nonzero_bytes16(__ldg(reinterpret_cast<const uint4*>(a.pol_mask + p0)));
-        if (a.val_mask) vm_bits = nonzero_bytes16(__ldg(reinterpret_cast<const uint4*>(a.val_mask + p0)));
+        if (a.pol_mask) {
+            const uint4* m = reinterpret_cast<const uint4*>(a.pol_mask + p0);
+            pm_bits = nonzero_bytes16(__ldg(m)) | (nonzero_bytes16(__ldg(m + 1)) << 16);
+        }
+        if (a.val_mask) {
+            const uint4* m = reinterpret_cast<const uint4*>(a.val_mask + p0);
+            vm_bits = nonzero_bytes16(__ldg(m)) | (nonzero_bytes16(__ldg(m + 1)) << 16);
+        }
     } else {
         if (a.pol_mask) {
             pm_bits = 0;
@@ -122,7 +131,7 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
             for (int k = 0; k < n_mine; ++k) vm_bits |= uint32_t(__ldg(a.val_mask + p0 + k) != 0) << k;
         }
     }
-    const uint32_t own_bits = n_mine >= kSelItems ? 0xffffu : ((1u << n_mine) - 1u);
+    const uint32_t own_bits = n_mine >= kSelItems ? 0xffffffffu : ((1u << n_mine) - 1u);
 
     // ---- window of sequences that can touch the tile: [seq0, seq1), seq0 may be -1 -------------
     if (warp == 0) {
@@ -142,7 +151,7 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
         __syncthreads();
     }
 
-    // ---- policy / value bits of this thread's 16 positions --------------------------------------
+    // ---- policy / value bits of this thread's 32 positions --------------------------------------
     uint32_t pol_bits = 0, val_bits = 0;
     if (n_mine > 0 && seq1 > 0) {
         // last sequence of the window that begins at or before p0 (-1: none)
@@ -172,8 +181,8 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
             const int64_t end = new0 + __ldg(a.new_len + i);
             const bool trunc = __ldg(a.truncated + i) != 0;
             // a position belongs to the last sequence that begins at or before it: clip to [begin, next)
-            pol_bits |= range_bits16(max(new0, begin), min(end - (trunc ? a.tail_drop : 0), next), p0);
-            if (!trunc) val_bits |= range_bits16(max(resp0, begin), min(end, next), p0);
+            pol_bits |= range_bits32(max(new0, begin), min(end - (trunc ? a.tail_drop : 0), next), p0);
+            if (!trunc) val_bits |= range_bits32(max(resp0, begin), min(end, next), p0);
         }
     }
     pol_bits &= pm_bits & own_bits;
@@ -197,20 +206,23 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
         if (w < warp) before += c;
         tile_tot += c;
     }
-    // compact inside the tile (needs no global offset, so it overlaps the look-back below)
+    // publish the tile's totals as early as possible: later tiles wait for them in their look-back
+    if (threadIdx.x == 0 && tile > 0)
+        reinterpret_cast<volatile unsigned long long*>(a.state)[tile] =
+            sel_pack(1, tile_tot & 0xffffu, tile_tot >> 16);
+    // compact inside the tile (needs no global offset; earlier tiles finish meanwhile)
     {
         uint32_t op = before & 0xffffu, ov = before >> 16;
         uint32_t b = pol_bits;
-        while (b) { s_out_pol[op++] = int32_t(p0) + (__ffs(int(b)) - 1); b &= b - 1; }
+        while (b) { s_out_pol[op++] = uint16_t(l0 + __ffs(int(b)) - 1); b &= b - 1; }
         b = val_bits;
-        while (b) { s_out_val[ov++] = int32_t(p0) + (__ffs(int(b)) - 1); b &= b - 1; }
+        while (b) { s_out_val[ov++] = uint16_t(l0 + __ffs(int(b)) - 1); b &= b - 1; }
     }
 
     // ---- tile total -> publish -> warp-wide look-back over earlier tiles ----------------------
     if (warp == 0) {
         const uint32_t tp = tile_tot & 0xffffu, tv = tile_tot >> 16;
         volatile unsigned long long* st = a.state;
-        if (lane == 0 && tile > 0) st[tile] = sel_pack(1, tp, tv);
         uint32_t ep = 0, ev = 0;
         bool timed_out = false;
         // 32 predecessors per round: lane l looks at tile j0 - l; positions before tile 0 count as
@@ -252,8 +264,9 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
         int32_t* dp = a.policy_idx + s_base_pol;
         int32_t* dv = a.value_idx + s_base_val;
         const int np = int(s_tot_pol), nv = int(s_tot_val);
-        for (int k = threadIdx.x; k < np; k += kSelThreads) dp[k] = s_out_pol[k];
-        for (int k = threadIdx.x; k < nv; k += kSelThreads) dv[k] = s_out_val[k];
+        const int32_t base = int32_t(t0);
+        for (int k = threadIdx.x; k < np; k += kSelThreads) dp[k] = base + int32_t(s_out_pol[k]);
+        for (int k = threadIdx.x; k < nv; k += kSelThreads) dv[k] = base + int32_t(s_out_val[k]);
     }
 }
 
