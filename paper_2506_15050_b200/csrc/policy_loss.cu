@@ -55,11 +55,23 @@ __global__ void __launch_bounds__(1024) policy_finish_kernel(const PolicyArgs a)
     const int64_t n = policy_n(a);
     double acc = 0.0;
     int lo = 0, hi = 0;
-    for (int64_t j = threadIdx.x; j < n; j += blockDim.x) {
-        acc += double(a.row_loss[j]);
-        const uint8_t c = a.row_clip[j];
-        lo += c == 1;
-        hi += c == 2;
+    // four rows per trip, loads first, so that their latencies overlap; the order of the adds is fixed
+    const int64_t step = blockDim.x;
+    for (int64_t j = threadIdx.x; j < n; j += 4 * step) {
+        float l[4];
+        uint8_t c[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t q = j + u * step;
+            l[u] = q < n ? a.row_loss[q] : 0.f;
+            c[u] = q < n ? a.row_clip[q] : uint8_t(0);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            acc += double(l[u]);
+            lo += c[u] == 1;
+            hi += c[u] == 2;
+        }
     }
     acc = warp_sum(acc);
     lo = __reduce_add_sync(0xffffffffu, lo);

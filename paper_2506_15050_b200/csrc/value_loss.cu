@@ -81,12 +81,20 @@ __global__ void __launch_bounds__(kValThreads) value_loss_kernel(const ValueArgs
         s_last = atomicAdd(a.done, 1u) == gridDim.x - 1;
     }
     __syncthreads();
-    if (s_last && threadIdx.x == 0) {   // the last block to finish adds the partials in order
+    if (s_last) {   // the last block to finish adds the partials: strided per thread, then a fixed tree
         __threadfence();
         double t = 0.0;
-        for (unsigned b = 0; b < gridDim.x; ++b) t += reinterpret_cast<volatile double*>(a.partial)[b];
-        *a.loss = n > 0 ? float(t / d) : 0.f;
-        a.stats[0] = int32_t(n);
+        for (unsigned b = threadIdx.x; b < gridDim.x; b += kValThreads)
+            t += reinterpret_cast<volatile double*>(a.partial)[b];
+        t = warp_sum(t);
+        if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = t;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double tot = 0.0;
+            for (int w = 0; w < kValThreads / 32; ++w) tot += s_red[w];
+            *a.loss = n > 0 ? float(tot / d) : 0.f;
+            a.stats[0] = int32_t(n);
+        }
     }
 }
 
