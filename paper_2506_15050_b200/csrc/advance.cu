@@ -1,7 +1,7 @@
 // Successive batching between two training steps (Section 3.2 of the paper, the batching figure;
 // the batch collection step of Algorithm 1): the batch keeps its B slots, a finished sequence frees
 // its slot for the next queued prompt, an unfinished one stays and the tokens of this window join its earlier ones.  Two
-// kernels: one CTA walks the slots (two block-wide prefix sums per 1024 slots: rank among the freed
+// kernels: one CTA walks the slots (two block-wide prefix sums per 4096 slots: rank among the freed
 // slots, then the packed offsets of the next step's context), then a bandwidth-bound ragged copy
 // moves the kept sequences and the queued prompts into the new packed token buffer.  Integer work
 // throughout: bit-exact and run-to-run identical.
@@ -11,8 +11,8 @@ namespace tppo {
 
 constexpr int kAdvSlotThreads = 1024;
 constexpr int kAdvCopyThreads = 256;
-constexpr int kAdvCopyItems = 16;
-constexpr int kAdvCopyTile = kAdvCopyThreads * kAdvCopyItems;     // 4096 tokens per CTA
+constexpr int kAdvCopyItems = 32;
+constexpr int kAdvCopyTile = kAdvCopyThreads * kAdvCopyItems;     // 8192 tokens per CTA
 
 struct AdvanceArgs {
     const int32_t* seq_begin;
@@ -62,46 +62,68 @@ __device__ __forceinline__ T block_exclusive_sum(T v, T* s_warp, T& total) {
     return before + incl - v;
 }
 
+constexpr int kAdvSlotItems = 4;                               // consecutive slots per thread
+
 __global__ void __launch_bounds__(kAdvSlotThreads) advance_slots_kernel(const AdvanceArgs a) {
     __shared__ long long s_scan[32];
     long long free_base = 0, pos_base = 0;
     int bad = 0;
-    for (int c0 = 0; c0 < a.B; c0 += kAdvSlotThreads) {
-        const int i = c0 + int(threadIdx.x);
-        const bool valid = i < a.B;
-        const bool fin = valid && __ldg(a.truncated + i) == 0;
+    for (int c0 = 0; c0 < a.B; c0 += kAdvSlotThreads * kAdvSlotItems) {
+        const int i0 = c0 + int(threadIdx.x) * kAdvSlotItems;
+        bool valid[kAdvSlotItems], fin[kAdvSlotItems];
+        long long p[kAdvSlotItems], q[kAdvSlotItems], n[kAdvSlotItems];
+        int my_fin = 0;
+#pragma unroll
+        for (int u = 0; u < kAdvSlotItems; ++u) {
+            const int i = i0 + u;
+            valid[u] = i < a.B;
+            fin[u] = valid[u] && __ldg(a.truncated + i) == 0;
+            p[u] = valid[u] ? __ldg(a.prompt_len + i) : 0;
+            q[u] = valid[u] ? __ldg(a.prev_len + i) : 0;
+            n[u] = valid[u] ? __ldg(a.new_len + i) : 0;
+            my_fin += fin[u];
+        }
         long long n_fin;
-        const long long rank = free_base + block_exclusive_sum<long long>(fin ? 1 : 0, s_scan, n_fin);
-        long long len = 0;
-        int32_t pl = 0, pv = 0, src = -2;
-        if (valid) {
-            if (!fin) {                                   // unfinished: stays in its slot
-                const long long p = __ldg(a.prompt_len + i), q = __ldg(a.prev_len + i),
-                                n = __ldg(a.new_len + i);
-                if (p < 0 || q < 0 || n < 0 || q + n > 0x7fffffffll) bad |= TPPO_DEV_BAD_INDEX;
-                pl = int32_t(p);
-                pv = int32_t(q + n);
-                src = -1;
-                len = p + q + n;
-            } else {                                      // finished: freed, refilled while the queue lasts
-                a.free_slots[rank] = i;
+        long long rank = free_base + block_exclusive_sum<long long>(my_fin, s_scan, n_fin);
+        long long len[kAdvSlotItems];
+        int32_t pl[kAdvSlotItems], pv[kAdvSlotItems], src[kAdvSlotItems];
+        long long my_len = 0;
+#pragma unroll
+        for (int u = 0; u < kAdvSlotItems; ++u) {
+            len[u] = 0; pl[u] = 0; pv[u] = 0; src[u] = -2;
+            if (!valid[u]) continue;
+            if (!fin[u]) {                                    // unfinished: stays in its slot
+                if (p[u] < 0 || q[u] < 0 || n[u] < 0 || q[u] + n[u] > 0x7fffffffll) bad |= TPPO_DEV_BAD_INDEX;
+                pl[u] = int32_t(p[u]);
+                pv[u] = int32_t(q[u] + n[u]);
+                src[u] = -1;
+                len[u] = p[u] + q[u] + n[u];
+            } else {                                          // finished: freed, refilled while the queue lasts
+                a.free_slots[rank] = i0 + u;
                 if (rank < a.M) {
                     const int32_t k = int32_t(rank);
-                    len = (long long)__ldg(a.queue_begin + k + 1) - __ldg(a.queue_begin + k);
-                    if (len < 0) { bad |= TPPO_DEV_BAD_INDEX; len = 0; }
-                    pl = int32_t(len);
-                    src = k;
+                    len[u] = (long long)__ldg(a.queue_begin + k + 1) - __ldg(a.queue_begin + k);
+                    if (len[u] < 0) { bad |= TPPO_DEV_BAD_INDEX; len[u] = 0; }
+                    pl[u] = int32_t(len[u]);
+                    src[u] = k;
                 }
+                ++rank;
             }
-            if (len < 0) len = 0;
+            if (len[u] < 0) len[u] = 0;
+            my_len += len[u];
         }
         long long n_tok;
-        const long long begin = pos_base + block_exclusive_sum<long long>(len, s_scan, n_tok);
-        if (valid) {
-            a.next_prompt_len[i] = pl;
-            a.next_prev_len[i] = pv;
-            a.slot_source[i] = src;
-            a.next_seq_begin[i] = int32_t(begin < 0x7fffffffll ? begin : 0x7fffffffll);
+        long long begin = pos_base + block_exclusive_sum<long long>(my_len, s_scan, n_tok);
+#pragma unroll
+        for (int u = 0; u < kAdvSlotItems; ++u) {
+            if (valid[u]) {
+                const int i = i0 + u;
+                a.next_prompt_len[i] = pl[u];
+                a.next_prev_len[i] = pv[u];
+                a.slot_source[i] = src[u];
+                a.next_seq_begin[i] = int32_t(begin < 0x7fffffffll ? begin : 0x7fffffffll);
+                begin += len[u];
+            }
         }
         free_base += n_fin;
         pos_base += n_tok;
@@ -152,23 +174,34 @@ __global__ void __launch_bounds__(kAdvCopyThreads) advance_copy_kernel(const Adv
     int32_t src = a.slot_source[i];
     int64_t src_base = src == -1 ? int64_t(a.seq_begin[i]) : (src >= 0 ? int64_t(a.queue_begin[src]) : 0);
     int bad = 0;
-#pragma unroll 4
-    for (int j = 0; j < kAdvCopyItems; ++j) {
-        const int64_t p = t0 + threadIdx.x + int64_t(j) * kAdvCopyThreads;
-        if (p >= total) break;
-        while (p >= next && i + 1 < a.B) {
-            ++i;
-            begin = next;
-            next = a.next_seq_begin[i + 1];
-            src = a.slot_source[i];
-            src_base = src == -1 ? int64_t(a.seq_begin[i]) : (src >= 0 ? int64_t(a.queue_begin[src]) : 0);
+    // batches of eight positions: resolve the sources, issue the eight loads, then store
+    for (int j0 = 0; j0 < kAdvCopyItems; j0 += 8) {
+        const int32_t* srcp[8];
+        int64_t pos[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int64_t p = t0 + threadIdx.x + int64_t(j0 + u) * kAdvCopyThreads;
+            pos[u] = p;
+            srcp[u] = nullptr;
+            if (p >= total) continue;
+            while (p >= next && i + 1 < a.B) {
+                ++i;
+                begin = next;
+                next = a.next_seq_begin[i + 1];
+                src = a.slot_source[i];
+                src_base = src == -1 ? int64_t(a.seq_begin[i]) : (src >= 0 ? int64_t(a.queue_begin[src]) : 0);
+            }
+            const int64_t q = src_base + (p - begin);
+            if (src == -1 && q >= 0 && q < a.N) srcp[u] = a.tokens + q;
+            else if (src >= 0 && q >= 0 && q < a.queue_total) srcp[u] = a.queue_tokens + q;
+            else bad = TPPO_DEV_BAD_INDEX;
         }
-        const int64_t q = src_base + (p - begin);
-        int32_t v = 0;
-        if (src == -1 && q >= 0 && q < a.N) v = __ldg(a.tokens + q);
-        else if (src >= 0 && q >= 0 && q < a.queue_total) v = __ldg(a.queue_tokens + q);
-        else bad = TPPO_DEV_BAD_INDEX;
-        a.next_tokens[p] = v;
+        int32_t v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = srcp[u] ? __ldg(srcp[u]) : 0;
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (pos[u] < total) a.next_tokens[pos[u]] = v[u];
     }
     if (bad) atomicOr(a.counts + 3, bad);
 }
