@@ -205,3 +205,19 @@ def test_lmhead_rows_equal_matmul():
     cols = [7, 1, 39]
     np.testing.assert_allclose(oracle.lmhead_dweight_cols(hb, dx[:, cols]),
                                (H.double().numpy().T @ dx)[:, cols], rtol=1e-12, atol=1e-13)
+
+
+def test_float64_logits_give_the_float32_results_on_representable_values():
+    """The LM-head tests hand the loss routine float64 logits; on values that float32 holds exactly
+    the two input types must agree to the last bit."""
+    rng = np.random.default_rng(9)
+    n, V = 7, 33
+    x32 = rng.standard_normal((n, V)).astype(np.float32)
+    t = rng.integers(0, V, n).astype(np.int32)
+    old = (-3.0 + 0.1 * rng.standard_normal(n)).astype(np.float32)
+    adv = rng.standard_normal(n).astype(np.float32)
+    a = oracle.policy_loss(x32, t, None, None, old, adv, 0.2, 0.28)
+    b = oracle.policy_loss(x32.astype(np.float64), t, None, None, old, adv, 0.2, 0.28)
+    assert a["loss"] == b["loss"] and np.array_equal(a["logp"], b["logp"])
+    assert np.array_equal(a["dlogits"], b["dlogits"])
+    assert np.array_equal(oracle.logprob(x32, t), oracle.logprob(x32.astype(np.float64), t))
