@@ -265,6 +265,53 @@ int tppo_lmhead_logprob_fwd_bwd(const void *hidden, const void *weight,
                                 void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same operation with the vocabulary split across devices (the LM-head weight held as column
+ * shards, one per rank; the rows, targets and per-token scalars replicated).  Eq. 1 needs, per row,
+ * the maximum logit, the sum of exponentials and the target's logit over the WHOLE vocabulary, so
+ * the work is two calls with one exchange between them that the caller performs (the library
+ * issues no collective):
+ *
+ *   1. tppo_lmhead_shard_stats on each rank: over the V_shard columns of its shard (vocabulary ids
+ *      v_offset .. v_offset + V_shard - 1), per row r
+ *          row_max[r] = max_v x[r,v],  row_sumexp[r] = sum_v exp(x[r,v] - row_max[r]),
+ *          row_target_logit[r] = x[r, targets[r]] if the target lies in the shard, else 0.
+ *      Rows with a target outside [0, V_total) get (0, 0, 0) and raise the status bit.
+ *   2. the merge across ranks, m = max_r m_r;  S = sum_r s_r * exp(m_r - m);  xy = sum_r xy_r:
+ *      the caller all-reduces (max) a copy of row_max into row_max_all, calls
+ *      tppo_lmhead_shard_rescale, which multiplies row_sumexp[r] by exp(row_max[r] - row_max_all[r])
+ *      in place (a skipped row keeps 0), and all-reduces (sum) row_sumexp and row_target_logit.
+ *   3. tppo_lmhead_shard_fwd_bwd on each rank with the merged vectors: evaluates Eq. 1 (loss, logp,
+ *      token_loss and stats come out identical on every rank), then forms the gradient for its
+ *      columns only: dweight_shard [K, V_shard] is complete; dhidden_partial [M, K] holds this
+ *      shard's term of dX * weight^T and the caller sums it over the ranks.
+ *
+ * All arrays live on the device.  row_max, row_sumexp, row_target_logit: [M] fp32.
+ *   stats of tppo_lmhead_shard_stats: [4] int32, only the status bits (stats[3]) are written.
+ *   workspace for either call: tppo_workspace_bytes(TPPO_OP_LMHEAD, M, K, 0, V_shard) bytes.
+ * Every other argument, the limits on K and V_shard (multiples of 8) and the errors are those of
+ * tppo_lmhead_logprob_fwd_bwd; 0 <= v_offset <= V_total - V_shard or TPPO_ERR_INVALID_ARG.  With one
+ * shard (v_offset = 0, V_shard = V_total) the two calls compute exactly what the unsharded call does.
+ */
+int tppo_lmhead_shard_stats(const void *hidden, const void *weight_shard,
+                            int64_t M, int32_t K, int32_t V_shard, int32_t v_offset, int32_t V_total,
+                            const int32_t *targets,
+                            float *row_max, float *row_sumexp, float *row_target_logit,
+                            int32_t *stats, int32_t chunk_tiles,
+                            void *workspace, size_t workspace_bytes, void *stream);
+int tppo_lmhead_shard_rescale(const float *row_max, const float *row_max_all, float *row_sumexp,
+                              int64_t M, void *stream);
+int tppo_lmhead_shard_fwd_bwd(const void *hidden, const void *weight_shard,
+                              int64_t M, int32_t K, int32_t V_shard, int32_t v_offset, int32_t V_total,
+                              const int32_t *targets, const int32_t *aux_idx,
+                              const float *old_logp, const float *adv, int64_t aux_len,
+                              float eps_low, float eps_high, float denom,
+                              const float *row_max, const float *row_sumexp,
+                              const float *row_target_logit,
+                              float *logp, float *token_loss, float *loss, int32_t *stats,
+                              void *dhidden_partial, void *dweight_shard, int32_t chunk_tiles,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Successive batching between two training steps (Section 3.2 and its batching figure; the step of
  * Algorithm 1 that keeps the unfinished samples of the last step and puts new prompts in the place
  * of the finished ones).  The batch keeps its B slots, visited in ascending order:

@@ -52,6 +52,15 @@ _lib.tppo_lmhead_logprob_fwd_bwd.restype = C.c_int
 _lib.tppo_lmhead_logprob_fwd_bwd.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _i64,
                                              _f32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, _i32,
                                              _vp, _sz, _vp]
+_lib.tppo_lmhead_shard_stats.restype = C.c_int
+_lib.tppo_lmhead_shard_stats.argtypes = [_vp, _vp, _i64, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp,
+                                         _vp, _i32, _vp, _sz, _vp]
+_lib.tppo_lmhead_shard_rescale.restype = C.c_int
+_lib.tppo_lmhead_shard_rescale.argtypes = [_vp, _vp, _vp, _i64, _vp]
+_lib.tppo_lmhead_shard_fwd_bwd.restype = C.c_int
+_lib.tppo_lmhead_shard_fwd_bwd.argtypes = [_vp, _vp, _i64, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp,
+                                           _i64, _f32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                           _vp, _vp, _i32, _vp, _sz, _vp]
 _lib.tppo_advance_batch.restype = C.c_int
 _lib.tppo_advance_batch.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _i32, _i32,
                                     _vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp]
@@ -181,6 +190,41 @@ def tppo_lmhead_logprob_fwd_bwd(hidden, weight, targets, aux_idx, old_logp, adv,
         _ptr(logp, torch.float32), _ptr(token_loss, torch.float32), _ptr(loss, torch.float32),
         _ptr(stats, torch.int32), _ptr(dhidden, torch.bfloat16), _ptr(dweight, torch.bfloat16),
         chunk_tiles, _ptr(ws), ws.numel(), _stream()))
+
+
+def tppo_lmhead_shard_stats(hidden, weight_shard, v_offset, V_total, targets, row_max, row_sumexp,
+                            row_target_logit, stats, ws, chunk_tiles=0):
+    M, K = hidden.shape
+    assert weight_shard.shape[0] == K
+    _check(_lib.tppo_lmhead_shard_stats(
+        _ptr(hidden, torch.bfloat16), _ptr(weight_shard, torch.bfloat16), M, K,
+        weight_shard.shape[1], v_offset, V_total, _ptr(targets, torch.int32),
+        _ptr(row_max, torch.float32), _ptr(row_sumexp, torch.float32),
+        _ptr(row_target_logit, torch.float32), _ptr(stats, torch.int32), chunk_tiles,
+        _ptr(ws), ws.numel(), _stream()))
+
+
+def tppo_lmhead_shard_rescale(row_max, row_max_all, row_sumexp):
+    _check(_lib.tppo_lmhead_shard_rescale(
+        _ptr(row_max, torch.float32), _ptr(row_max_all, torch.float32),
+        _ptr(row_sumexp, torch.float32), row_max.numel(), _stream()))
+
+
+def tppo_lmhead_shard_fwd_bwd(hidden, weight_shard, v_offset, V_total, targets, aux_idx, old_logp,
+                              adv, eps_low, eps_high, denom, row_max, row_sumexp, row_target_logit,
+                              logp, token_loss, loss, stats, dhidden_partial, dweight_shard, ws,
+                              chunk_tiles=0):
+    M, K = hidden.shape
+    assert weight_shard.shape[0] == K
+    _check(_lib.tppo_lmhead_shard_fwd_bwd(
+        _ptr(hidden, torch.bfloat16), _ptr(weight_shard, torch.bfloat16), M, K,
+        weight_shard.shape[1], v_offset, V_total, _ptr(targets, torch.int32),
+        _ptr(aux_idx, torch.int32), _ptr(old_logp, torch.float32), _ptr(adv, torch.float32),
+        old_logp.numel(), eps_low, eps_high, denom, _ptr(row_max, torch.float32),
+        _ptr(row_sumexp, torch.float32), _ptr(row_target_logit, torch.float32),
+        _ptr(logp, torch.float32), _ptr(token_loss, torch.float32), _ptr(loss, torch.float32),
+        _ptr(stats, torch.int32), _ptr(dhidden_partial, torch.bfloat16),
+        _ptr(dweight_shard, torch.bfloat16), chunk_tiles, _ptr(ws), ws.numel(), _stream()))
 
 
 def tppo_advance_batch(seq_begin, prompt_len, prev_len, new_len, truncated, tokens, queue_begin,

@@ -31,11 +31,14 @@ struct EpiStats {
     float2* part;      // [n_tiles][M]: (max, sum exp(x - max)) of the tile's valid columns
     float* xy;         // [M]: logit of the target token
     int64_t M;
-    int32_t V;
+    int32_t V;         // columns of this weight matrix (a vocabulary shard when v_off / V differ from the whole)
+    int32_t v_off;     // vocabulary id of column 0
     __device__ __forceinline__ void operator()(int mt, int nt, int row, uint32_t taddr) const {
         const int64_t r = int64_t(mt) * kTileM + row;
         const int n0 = nt * kTileN;
-        const int y = r < M ? load_rec(rec + r).y : -1;
+        const int yg = r < M ? load_rec(rec + r).y : -1;
+        // column of the target; far off when the row is skipped or the target lies in another shard
+        const int y = (yg >= v_off && yg - v_off < V) ? yg - v_off : -1 - kTileN;
         float m = -kInf, s = 0.f, xv = 0.f;
         bool found = false;
 #pragma unroll 1
@@ -92,12 +95,14 @@ struct EpiDx {
     int64_t ldx;
     int64_t M;
     int32_t V, v0;
+    int32_t v_off;         // vocabulary id of column 0 of the weight matrix
     __device__ __forceinline__ void operator()(int mt, int nt, int row, uint32_t taddr) const {
         const int64_t r = int64_t(mt) * kTileM + row;
         const bool live = r < M;
         const float l2 = live ? __ldg(lse2 + r) : kInf;
         const float cf = live ? __ldg(coef + r) : 0.f;
-        const int y = live ? load_rec(rec + r).y : -1;
+        const int yg = live ? load_rec(rec + r).y : -1;
+        const int y = (yg >= v_off && yg - v_off < V) ? yg - v_off : -1 - kTileN;
         uint16_t* out = dx + (live ? r : 0) * ldx + nt * kTileN;
 #pragma unroll 1
         for (int c = 0; c < kTileN; c += 32) {
@@ -214,7 +219,8 @@ struct EpiDw {
 __global__ void __launch_bounds__(256)
 lmhead_rows_kernel(const RowRec* rec, const float2* part, const float* xy, int64_t M, int32_t n_tiles,
                    float eps_low, float eps_high, float inv_denom, float* logp, float* token_loss,
-                   float* row_loss, uint8_t* row_clip, float* lse2, float* coef) {
+                   float* row_loss, uint8_t* row_clip, float* lse2, float* coef,
+                   const float* ext_max, const float* ext_sum, const float* ext_xy) {
     const int64_t r = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     if (r >= M) return;
     const RowRec rr = load_rec(rec + r);
@@ -227,15 +233,21 @@ lmhead_rows_kernel(const RowRec* rec, const float2* part, const float* xy, int64
         coef[r] = 0.f;
         return;
     }
-    float m = -kInf;
-    for (int t = 0; t < n_tiles; ++t) m = fmaxf(m, part[int64_t(t) * M + r].x);
-    float s = 0.f;
-    for (int t = 0; t < n_tiles; ++t) {
-        const float2 p = part[int64_t(t) * M + r];
-        s += p.y * expf(p.x - m);
+    float m = -kInf, s = 0.f, x_y;
+    if (ext_max) {               // whole-vocabulary statistics supplied by the caller (vocabulary shards)
+        m = ext_max[r];
+        s = ext_sum[r];
+        x_y = ext_xy[r];
+    } else {
+        for (int t = 0; t < n_tiles; ++t) m = fmaxf(m, part[int64_t(t) * M + r].x);
+        for (int t = 0; t < n_tiles; ++t) {
+            const float2 p = part[int64_t(t) * M + r];
+            s += p.y * expf(p.x - m);
+        }
+        x_y = xy[r];
     }
     const float log_sum = logf(s);
-    const RowLoss rl = ppo_row(xy[r] - m, log_sum, rr.old_logp, rr.adv, eps_low, eps_high, inv_denom);
+    const RowLoss rl = ppo_row(x_y - m, log_sum, rr.old_logp, rr.adv, eps_low, eps_high, inv_denom);
     if (logp) logp[r] = rl.logp;
     if (token_loss) token_loss[r] = rl.loss;
     row_loss[r] = rl.loss;
@@ -251,6 +263,38 @@ int launch_gemm(bool pair, const CUtensorMap& a, const CUtensorMap& b, const Gem
                 const Epi& e, int32_t* status, cudaStream_t s) {
     return pair ? launch_umma_gemm_pair<AMAJ, BMAJ>(a, b, g, e, status, s)
                 : launch_umma_gemm<AMAJ, BMAJ>(a, b, g, e, status, s);
+}
+
+// Vocabulary shards: the statistics of this shard's columns for every row, to be merged by the caller
+// across shards (m = max m_r, S = sum s_r exp(m_r - m), target logit = sum over shards).
+__global__ void __launch_bounds__(256)
+lmhead_merge_kernel(const RowRec* rec, const float2* part, const float* xy, int64_t M, int32_t n_tiles,
+                    float* row_max, float* row_sum, float* row_xy) {
+    const int64_t r = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (r >= M) return;
+    if (load_rec(rec + r).y < 0) {       // skipped row: neutral statistics
+        row_max[r] = 0.f; row_sum[r] = 0.f; row_xy[r] = 0.f;
+        return;
+    }
+    float m = -kInf, s = 0.f;
+    for (int t = 0; t < n_tiles; ++t) m = fmaxf(m, part[int64_t(t) * M + r].x);
+    for (int t = 0; t < n_tiles; ++t) {
+        const float2 p = part[int64_t(t) * M + r];
+        s += p.y * expf(p.x - m);
+    }
+    row_max[r] = m;
+    row_sum[r] = s;
+    row_xy[r] = xy[r];
+}
+
+// Step between the two all-reduces of the vocabulary-parallel merge: bring a shard's sum of
+// exponentials from its own maximum to the maximum over all shards.
+__global__ void __launch_bounds__(256)
+lmhead_rescale_kernel(const float* row_max, const float* row_max_all, float* row_sum, int64_t M) {
+    const int64_t r = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (r >= M) return;
+    const float s = row_sum[r];
+    row_sum[r] = s > 0.f ? s * expf(row_max[r] - row_max_all[r]) : 0.f;
 }
 
 struct LmPlan {
@@ -319,46 +363,68 @@ size_t lmhead_workspace_bytes(int64_t M, int32_t K, int32_t V) {
 
 using namespace tppo;
 
-TPPO_API int tppo_lmhead_logprob_fwd_bwd(const void* hidden, const void* weight, int64_t M, int32_t K,
-                                         int32_t V, const int32_t* targets, const int32_t* aux_idx,
-                                         const float* old_logp, const float* adv, int64_t aux_len,
-                                         float eps_low, float eps_high, float denom, float* logp,
-                                         float* token_loss, float* loss, int32_t* stats,
-                                         void* dhidden, void* dweight, int32_t chunk_tiles,
-                                         void* workspace, size_t workspace_bytes, void* stream) {
-    if (M < 0 || K <= 0 || V <= 0 || aux_len < 0 || M >= (int64_t(1) << 31) - kTileM)
+namespace {
+
+enum LmMode { kLmFull = 0, kLmShardStats = 1, kLmShardGrads = 2 };
+
+struct LmCall {
+    LmMode mode;
+    const void* hidden; const void* weight;
+    int64_t M; int32_t K; int32_t V;          // V: columns of `weight` (the shard width)
+    int32_t v_off; int32_t V_total;           // vocabulary id of column 0, size of the whole vocabulary
+    const int32_t* targets; const int32_t* aux_idx; const float* old_logp; const float* adv;
+    int64_t aux_len; float eps_low, eps_high, denom;
+    const float* in_max; const float* in_sum; const float* in_xy;    // kLmShardGrads: whole-vocabulary statistics
+    float* out_max; float* out_sum; float* out_xy;                   // kLmShardStats: this shard's statistics
+    float* logp; float* token_loss; float* loss; int32_t* stats;
+    void* dhidden; void* dweight; int32_t chunk_tiles;
+    void* workspace; size_t workspace_bytes; void* stream;
+};
+
+int lmhead_run(const LmCall& c) {
+    const int64_t M = c.M;
+    const int32_t K = c.K, V = c.V;
+    if (M < 0 || K <= 0 || V <= 0 || c.aux_len < 0 || M >= (int64_t(1) << 31) - kTileM)
         return TPPO_ERR_INVALID_ARG;
-    if (!loss || !stats) return TPPO_ERR_INVALID_ARG;
-    if (M > 0 && (!hidden || !weight || !targets || !old_logp || !adv)) return TPPO_ERR_INVALID_ARG;
-    if (!(eps_low >= 0.f) || !(eps_high >= 0.f) || chunk_tiles < 0) return TPPO_ERR_INVALID_ARG;
+    if (c.v_off < 0 || c.V_total < V || c.v_off > c.V_total - V) return TPPO_ERR_INVALID_ARG;
+    if (!c.stats) return TPPO_ERR_INVALID_ARG;
+    if (c.mode != kLmShardStats && !c.loss) return TPPO_ERR_INVALID_ARG;
+    if (M > 0 && (!c.hidden || !c.weight || !c.targets)) return TPPO_ERR_INVALID_ARG;
+    if (M > 0 && c.mode != kLmShardStats && (!c.old_logp || !c.adv)) return TPPO_ERR_INVALID_ARG;
+    if (M > 0 && c.mode == kLmShardStats && (!c.out_max || !c.out_sum || !c.out_xy))
+        return TPPO_ERR_INVALID_ARG;
+    if (M > 0 && c.mode == kLmShardGrads && (!c.in_max || !c.in_sum || !c.in_xy))
+        return TPPO_ERR_INVALID_ARG;
+    if (!(c.eps_low >= 0.f) || !(c.eps_high >= 0.f) || c.chunk_tiles < 0) return TPPO_ERR_INVALID_ARG;
     // TMA row strides and the 16-byte vector stores need K and V to be multiples of 8 bf16.
     if (K % 8 != 0 || V % 8 != 0) return TPPO_ERR_UNSUPPORTED;
-    if (!aligned(hidden, 16) || !aligned(weight, 16) || (dhidden && !aligned(dhidden, 16)) ||
-        (dweight && !aligned(dweight, 16)))
+    if (!aligned(c.hidden, 16) || !aligned(c.weight, 16) || (c.dhidden && !aligned(c.dhidden, 16)) ||
+        (c.dweight && !aligned(c.dweight, 16)))
         return TPPO_ERR_INVALID_ARG;
-    if (!workspace || !aligned(workspace, kWsAlign) ||
-        workspace_bytes < lmhead_workspace_bytes(M, K, V))
+    if (!c.workspace || !aligned(c.workspace, kWsAlign) ||
+        c.workspace_bytes < lmhead_workspace_bytes(M, K, V))
         return TPPO_ERR_WORKSPACE;
 
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const LmWorkspace w = lmhead_carve(workspace, M, K, V);
+    cudaStream_t s = static_cast<cudaStream_t>(c.stream);
+    const LmWorkspace w = lmhead_carve(c.workspace, M, K, V);
     LmPlan plan = lmhead_plan(M, K, V);
     const int64_t ldx = int64_t(plan.chunk_tiles) * kTileN;     // row stride of the chunk buffer
-    const bool pair = (chunk_tiles & 0x10000) != 0;             // bit 16: CTA-pair kernels
-    chunk_tiles &= 0xffff;
+    const bool pair = (c.chunk_tiles & 0x10000) != 0;           // bit 16: CTA-pair kernels
+    const int32_t chunk_tiles = c.chunk_tiles & 0xffff;
     if (chunk_tiles > 0 && chunk_tiles < plan.chunk_tiles) plan.chunk_tiles = chunk_tiles;
+    int32_t* stats = c.stats;
 
+    // Targets are validated against the whole vocabulary; columns are local to the shard.
     PolicyArgs a{};
-    a.logits = nullptr; a.R = M; a.V = V; a.ld = V; a.targets = targets; a.rows = nullptr;
-    a.n_sel = nullptr; a.n_max = M; a.aux_idx = aux_idx; a.old_logp = old_logp; a.adv = adv;
-    a.aux_len = aux_len; a.eps_low = eps_low; a.eps_high = eps_high; a.denom = denom;
-    a.logp = logp; a.token_loss = token_loss; a.loss = loss; a.stats = stats;
-    a.dlogits = nullptr; a.mode = TPPO_DLOGITS_NONE;
+    a.logits = nullptr; a.R = M; a.V = c.V_total; a.ld = c.V_total; a.targets = c.targets;
+    a.rows = nullptr; a.n_sel = nullptr; a.n_max = M; a.aux_idx = c.aux_idx;
+    a.old_logp = c.old_logp; a.adv = c.adv; a.aux_len = c.aux_len; a.eps_low = c.eps_low;
+    a.eps_high = c.eps_high; a.denom = c.denom; a.logp = c.logp; a.token_loss = c.token_loss;
+    a.loss = c.loss; a.stats = stats; a.dlogits = nullptr; a.mode = TPPO_DLOGITS_NONE;
     a.row_loss = w.row_loss; a.row_clip = w.row_clip; a.row_flag = nullptr; a.rec = w.rec;
 
     TPPO_CUDA_CHECK(cudaMemsetAsync(stats, 0, 4 * sizeof(int32_t), s));
-    if (M == 0) return launch_policy_finish(a, s);
-    TPPO_CUDA_CHECK(cudaMemsetAsync(w.xy, 0, size_t(M) * 4, s));
+    if (M == 0) return c.mode == kLmShardStats ? TPPO_OK : launch_policy_finish(a, s);
     int rc = launch_policy_prepare(a, s);
     if (rc != TPPO_OK) return rc;
 
@@ -366,28 +432,35 @@ TPPO_API int tppo_lmhead_logprob_fwd_bwd(const void* hidden, const void* weight,
     const int32_t ks_k = (K + kTileK - 1) / kTileK;
     const int32_t ks_m = int32_t((M + kTileK - 1) / kTileK);
     CUtensorMap map_h128, map_h64, map_w64, map_w256;
-    if (!make_bf16_tensor_map(&map_h128, hidden, uint64_t(M), uint64_t(K), uint64_t(K), 128) ||
-        !make_bf16_tensor_map(&map_h64, hidden, uint64_t(M), uint64_t(K), uint64_t(K), 64) ||
-        !make_bf16_tensor_map(&map_w64, weight, uint64_t(K), uint64_t(V), uint64_t(V), 64) ||
-        !make_bf16_tensor_map(&map_w256, weight, uint64_t(K), uint64_t(V), uint64_t(V),
+    if (!make_bf16_tensor_map(&map_h128, c.hidden, uint64_t(M), uint64_t(K), uint64_t(K), 128) ||
+        !make_bf16_tensor_map(&map_h64, c.hidden, uint64_t(M), uint64_t(K), uint64_t(K), 64) ||
+        !make_bf16_tensor_map(&map_w64, c.weight, uint64_t(K), uint64_t(V), uint64_t(V), 64) ||
+        !make_bf16_tensor_map(&map_w256, c.weight, uint64_t(K), uint64_t(V), uint64_t(V),
                               pair ? 128 : 256))     // K-major B box: 128 rows per CTA of a pair
         return TPPO_ERR_CUDA;
 
-    // pass 1: statistics over the whole vocabulary
-    {
+    // pass 1: statistics over the columns of this weight matrix
+    if (c.mode != kLmShardGrads) {
+        TPPO_CUDA_CHECK(cudaMemsetAsync(w.xy, 0, size_t(M) * 4, s));
         const GemmShape g{mt, plan.n_tiles, ks_k, 0, 0, 0, 0, 16};
-        const EpiStats e{w.rec, w.part, w.xy, M, V};
+        const EpiStats e{w.rec, w.part, w.xy, M, V, c.v_off};
         rc = launch_gemm<0, 1>(pair, map_h128, map_w64, g, e, stats + 3, s);
         if (rc != TPPO_OK) return rc;
     }
-    const float inv_denom = denom > 0.f ? 1.f / denom : 1.f / float(M);
+    if (c.mode == kLmShardStats) {
+        lmhead_merge_kernel<<<unsigned((M + 255) / 256), 256, 0, s>>>(
+            w.rec, w.part, w.xy, M, plan.n_tiles, c.out_max, c.out_sum, c.out_xy);
+        TPPO_CUDA_CHECK(cudaGetLastError());
+        return TPPO_OK;
+    }
+    const float inv_denom = c.denom > 0.f ? 1.f / c.denom : 1.f / float(M);
     lmhead_rows_kernel<<<unsigned((M + 255) / 256), 256, 0, s>>>(
-        w.rec, w.part, w.xy, M, plan.n_tiles, eps_low, eps_high, inv_denom, logp, token_loss,
-        w.row_loss, w.row_clip, w.lse2, w.coef);
+        w.rec, w.part, w.xy, M, plan.n_tiles, c.eps_low, c.eps_high, inv_denom, c.logp, c.token_loss,
+        w.row_loss, w.row_clip, w.lse2, w.coef, c.in_max, c.in_sum, c.in_xy);
     TPPO_CUDA_CHECK(cudaGetLastError());
     rc = launch_policy_finish(a, s);
     if (rc != TPPO_OK) return rc;
-    if (!dhidden && !dweight) return TPPO_OK;
+    if (!c.dhidden && !c.dweight) return TPPO_OK;
 
     // pass 2: gradients, one vocabulary chunk at a time
     const int32_t chunk_cols = plan.chunk_tiles * kTileN;
@@ -402,24 +475,91 @@ TPPO_API int tppo_lmhead_logprob_fwd_bwd(const void* hidden, const void* weight,
             return TPPO_ERR_CUDA;
         {
             const GemmShape g{mt, ct, ks_k, 0, 0, v0, 0, 16};
-            const EpiDx e{w.rec, w.lse2, w.coef, w.dxc, ldx, M, V, v0};
+            const EpiDx e{w.rec, w.lse2, w.coef, w.dxc, ldx, M, V, v0, c.v_off};
             rc = launch_gemm<0, 1>(pair, map_h128, map_w64, g, e, stats + 3, s);
             if (rc != TPPO_OK) return rc;
         }
-        if (dhidden) {
+        if (c.dhidden) {
             const GemmShape g{mt, (K + kTileN - 1) / kTileN, (width + kTileK - 1) / kTileK,
                               0, 0, 0, v0, 16};
-            const EpiDh e{w.dhacc, static_cast<uint16_t*>(dhidden), M, K, ci == 0,
+            const EpiDh e{w.dhacc, static_cast<uint16_t*>(c.dhidden), M, K, ci == 0,
                           ci == n_chunks - 1};
             rc = launch_gemm<0, 0>(pair, map_dx128, map_w256, g, e, stats + 3, s);
             if (rc != TPPO_OK) return rc;
         }
-        if (dweight) {
+        if (c.dweight) {
             const GemmShape g{(K + kTileM - 1) / kTileM, ct, ks_m, 0, 0, 0, 0, 16};
-            const EpiDw e{static_cast<uint16_t*>(dweight), K, V, v0};
+            const EpiDw e{static_cast<uint16_t*>(c.dweight), K, V, v0};
             rc = launch_gemm<1, 1>(pair, map_h64, map_dx64, g, e, stats + 3, s);
             if (rc != TPPO_OK) return rc;
         }
     }
+    return TPPO_OK;
+}
+
+}  // namespace
+
+TPPO_API int tppo_lmhead_logprob_fwd_bwd(const void* hidden, const void* weight, int64_t M, int32_t K,
+                                         int32_t V, const int32_t* targets, const int32_t* aux_idx,
+                                         const float* old_logp, const float* adv, int64_t aux_len,
+                                         float eps_low, float eps_high, float denom, float* logp,
+                                         float* token_loss, float* loss, int32_t* stats,
+                                         void* dhidden, void* dweight, int32_t chunk_tiles,
+                                         void* workspace, size_t workspace_bytes, void* stream) {
+    LmCall c{};
+    c.mode = kLmFull; c.hidden = hidden; c.weight = weight; c.M = M; c.K = K; c.V = V;
+    c.v_off = 0; c.V_total = V; c.targets = targets; c.aux_idx = aux_idx; c.old_logp = old_logp;
+    c.adv = adv; c.aux_len = aux_len; c.eps_low = eps_low; c.eps_high = eps_high; c.denom = denom;
+    c.logp = logp; c.token_loss = token_loss; c.loss = loss; c.stats = stats; c.dhidden = dhidden;
+    c.dweight = dweight; c.chunk_tiles = chunk_tiles; c.workspace = workspace;
+    c.workspace_bytes = workspace_bytes; c.stream = stream;
+    return lmhead_run(c);
+}
+
+TPPO_API int tppo_lmhead_shard_stats(const void* hidden, const void* weight_shard, int64_t M, int32_t K,
+                                     int32_t V_shard, int32_t v_offset, int32_t V_total,
+                                     const int32_t* targets, float* row_max, float* row_sumexp,
+                                     float* row_target_logit, int32_t* stats, int32_t chunk_tiles,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
+    LmCall c{};
+    c.mode = kLmShardStats; c.hidden = hidden; c.weight = weight_shard; c.M = M; c.K = K;
+    c.V = V_shard; c.v_off = v_offset; c.V_total = V_total; c.targets = targets;
+    c.aux_len = M;      // no per-token scalars are read here: every row with a valid target counts
+    c.out_max = row_max; c.out_sum = row_sumexp; c.out_xy = row_target_logit; c.stats = stats;
+    c.chunk_tiles = chunk_tiles; c.workspace = workspace; c.workspace_bytes = workspace_bytes;
+    c.stream = stream;
+    return lmhead_run(c);
+}
+
+TPPO_API int tppo_lmhead_shard_fwd_bwd(const void* hidden, const void* weight_shard, int64_t M,
+                                       int32_t K, int32_t V_shard, int32_t v_offset, int32_t V_total,
+                                       const int32_t* targets, const int32_t* aux_idx,
+                                       const float* old_logp, const float* adv, int64_t aux_len,
+                                       float eps_low, float eps_high, float denom,
+                                       const float* row_max, const float* row_sumexp,
+                                       const float* row_target_logit, float* logp, float* token_loss,
+                                       float* loss, int32_t* stats, void* dhidden_partial,
+                                       void* dweight_shard, int32_t chunk_tiles, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+    LmCall c{};
+    c.mode = kLmShardGrads; c.hidden = hidden; c.weight = weight_shard; c.M = M; c.K = K;
+    c.V = V_shard; c.v_off = v_offset; c.V_total = V_total; c.targets = targets; c.aux_idx = aux_idx;
+    c.old_logp = old_logp; c.adv = adv; c.aux_len = aux_len; c.eps_low = eps_low;
+    c.eps_high = eps_high; c.denom = denom; c.in_max = row_max; c.in_sum = row_sumexp;
+    c.in_xy = row_target_logit; c.logp = logp; c.token_loss = token_loss; c.loss = loss;
+    c.stats = stats; c.dhidden = dhidden_partial; c.dweight = dweight_shard;
+    c.chunk_tiles = chunk_tiles; c.workspace = workspace; c.workspace_bytes = workspace_bytes;
+    c.stream = stream;
+    return lmhead_run(c);
+}
+
+TPPO_API int tppo_lmhead_shard_rescale(const float* row_max, const float* row_max_all,
+                                       float* row_sumexp, int64_t M, void* stream) {
+    if (M < 0) return TPPO_ERR_INVALID_ARG;
+    if (M == 0) return TPPO_OK;
+    if (!row_max || !row_max_all || !row_sumexp) return TPPO_ERR_INVALID_ARG;
+    lmhead_rescale_kernel<<<unsigned((M + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        row_max, row_max_all, row_sumexp, M);
+    TPPO_CUDA_CHECK(cudaGetLastError());
     return TPPO_OK;
 }

@@ -16,8 +16,8 @@ __global__ void policy_prepare_kernel(const PolicyArgs a) {
         RowRec r;
         r.row = m.row_ok ? int32_t(m.row) : -1;
         r.y = m.ok ? m.y : -1;
-        r.adv = m.ok ? __ldg(a.adv + m.aux) : 0.f;
-        r.old_logp = m.ok ? __ldg(a.old_logp + m.aux) : 0.f;
+        r.adv = (m.ok && a.adv) ? __ldg(a.adv + m.aux) : 0.f;              // absent when only the
+        r.old_logp = (m.ok && a.old_logp) ? __ldg(a.old_logp + m.aux) : 0.f; // row statistics are wanted
         a.rec[j] = r;
         if (!m.ok) bad |= policy_bad_bits(m, a);
         if (m.row_ok && a.rows && a.mode == TPPO_DLOGITS_FULL) a.row_flag[m.row] = 1;

@@ -6,7 +6,11 @@ coupling is the token-level mean of Eq. 1 and of the value loss (Section 4.1.1 o
 on a token-level loss): every rank must divide by the number of selected tokens of the WHOLE batch.
 That takes one all-reduce of two integers before the loss calls (the result is passed as `denom`)
 and one all-reduce of the scalar losses after them; the gradients need no exchange here because
-they are per token.  No arithmetic of the method lives in this file.
+they are per token.
+
+The LM-head variant can instead be split by vocabulary (every rank holds a column shard of the
+weight and all rows): `combine_row_stats` is the exchange between its two calls.  No arithmetic of
+the method lives in this file; the one arithmetic step of that exchange is passed in as a callable.
 """
 from __future__ import annotations
 
@@ -74,3 +78,27 @@ def reduce_losses(policy_loss: float, value_loss: float, group=None, device="cpu
     if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
         dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
     return float(t[0]), float(t[1])
+
+
+def combine_row_stats(row_max, row_sumexp, row_target_logit, rescale, group=None):
+    """Whole-vocabulary row statistics from each rank's shard statistics, in place.
+
+    row_max, row_sumexp, row_target_logit: this rank's [M] float32 tensors (maximum logit, sum of
+    exponentials relative to it, target logit or 0) over its vocabulary shard.  `rescale(row_max,
+    row_max_all, row_sumexp)` multiplies row_sumexp by exp(row_max - row_max_all) in place (on a GPU:
+    `binding.tppo_lmhead_shard_rescale`).  Afterwards all three hold the whole-vocabulary values on
+    every rank.  Two all-reduces' worth of traffic: 4 bytes x M for the maximum, 8 bytes x M for the sums.
+    """
+    import torch.distributed as dist
+    multi = dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1
+    if not multi:
+        return row_max, row_sumexp, row_target_logit
+    row_max_all = row_max.clone()
+    dist.all_reduce(row_max_all, op=dist.ReduceOp.MAX, group=group)
+    rescale(row_max, row_max_all, row_sumexp)
+    sums = torch.stack([row_sumexp, row_target_logit])
+    dist.all_reduce(sums, op=dist.ReduceOp.SUM, group=group)
+    row_max.copy_(row_max_all)
+    row_sumexp.copy_(sums[0])
+    row_target_logit.copy_(sums[1])
+    return row_max, row_sumexp, row_target_logit

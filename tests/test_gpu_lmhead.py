@@ -278,3 +278,123 @@ def test_config5_full_dweight_from_sampled_rows(cfg5):
     others = np.setdiff1d(np.arange(M), pick)
     assert float(out["dh_t"][torch.from_numpy(others).to(DEV)].float().abs().max()) == 0.0
     grad_close(out["dh"][pick], *ref_dhidden(ref["dlogits"], c["wb"]), "dhidden rows")
+
+
+# ---- vocabulary shards (weight split by columns; the ranks are emulated one after another) --------
+def run_lmhead_sharded(hidden, weight, bounds, targets, old_logp, adv, eps_low, eps_high, denom=0.0,
+                       aux=None, chunk_tiles=0):
+    """Both shard calls for every shard [bounds[i], bounds[i+1]) with the merge a caller performs
+    between them (max, rescale, sum) done by torch reductions over the emulated ranks."""
+    M, K = hidden.shape
+    V = weight.shape[1]
+    tg, ax = t(targets, torch.int32), t(aux, torch.int32)
+    olp, ad = t(old_logp, torch.float32), t(adv, torch.float32)
+    shards = [weight[:, lo:hi].contiguous() for lo, hi in zip(bounds[:-1], bounds[1:])]
+    rm, rs, rxy, bits = [], [], [], 0
+    for lo, wsd in zip(bounds[:-1], shards):
+        m_, s_, xy_ = (torch.full((M,), float("nan"), device=DEV) for _ in range(3))
+        st = torch.full((4,), -1, dtype=torch.int32, device=DEV)
+        ws = b.workspace(b.OP_LMHEAD, M, K, 0, wsd.shape[1], DEV)
+        b.tppo_lmhead_shard_stats(hidden, wsd, lo, V, tg, m_, s_, xy_, st, ws, chunk_tiles=chunk_tiles)
+        bits |= int(st[3])
+        rm.append(m_); rs.append(s_); rxy.append(xy_)
+    m_all = torch.stack(rm).max(dim=0).values
+    for m_, s_ in zip(rm, rs):
+        b.tppo_lmhead_shard_rescale(m_, m_all, s_)
+    s_all, xy_all = torch.stack(rs).sum(dim=0), torch.stack(rxy).sum(dim=0)
+    outs = []
+    for lo, wsd in zip(bounds[:-1], shards):
+        Vs = wsd.shape[1]
+        logp = torch.full((M,), float("nan"), device=DEV)
+        tl = torch.full((M,), float("nan"), device=DEV)
+        loss = torch.full((1,), float("nan"), device=DEV)
+        st = torch.full((4,), -1, dtype=torch.int32, device=DEV)
+        dh = torch.full((M, K), float("nan"), dtype=torch.bfloat16, device=DEV)
+        dw = torch.full((K, Vs), float("nan"), dtype=torch.bfloat16, device=DEV)
+        ws = b.workspace(b.OP_LMHEAD, M, K, 0, Vs, DEV)
+        b.tppo_lmhead_shard_fwd_bwd(hidden, wsd, lo, V, tg, ax, olp, ad, eps_low, eps_high, denom,
+                                    m_all, s_all, xy_all, logp, tl, loss, st, dh, dw, ws,
+                                    chunk_tiles=chunk_tiles)
+        outs.append(dict(logp=logp, tl=tl, loss=loss, st=st, dh=dh, dw=dw))
+    torch.cuda.synchronize()
+    for o in outs[1:]:           # the replicated outputs agree bit for bit across the shards
+        for k in ("logp", "tl", "loss", "st"):
+            assert torch.equal(o[k], outs[0][k]), k
+    return dict(logp=outs[0]["logp"].cpu().numpy(), token_loss=outs[0]["tl"].cpu().numpy(),
+                loss=float(outs[0]["loss"]), stats=outs[0]["st"].cpu().numpy(), stats_bits=bits,
+                dh=torch.stack([o["dh"].float() for o in outs]).sum(dim=0).cpu().numpy(),
+                dw=torch.cat([o["dw"].float() for o in outs], dim=1).cpu().numpy(),
+                dh_parts=[o["dh"] for o in outs], dw_parts=[o["dw"] for o in outs])
+
+
+@pytest.mark.parametrize("M,K,V,bounds,chunk", [(300, 320, 2000, (0, 840, 2000), 0),
+                                                (130, 328, 2008, (0, 8, 1000, 2008), 2),
+                                                (1024, 512, 8200, (0, 4096, 8200), CTA_PAIR)])
+def test_lmhead_vocabulary_shards_match_oracle(M, K, V, bounds, chunk):
+    hidden, weight, targets, adv, noise = make_case(M, K, V, seed=90 + M % 7)
+    targets[:4] = [0, bounds[1] - 1, bounds[1], V - 1]           # shard edges
+    hb, wb = synth.bf16_bits(hidden), synth.bf16_bits(weight)
+    x, old_logp = old_logp_from_oracle(hb, wb, targets, noise)
+    eps_low, eps_high = 0.2, 0.28
+    ref = oracle.policy_loss(x, targets, None, None, old_logp, adv, f32(eps_low), f32(eps_high))
+    out = run_lmhead_sharded(hidden, weight, bounds, targets, old_logp, adv, eps_low, eps_high,
+                             chunk_tiles=chunk)
+    assert out["stats_bits"] == 0 and out["stats"][3] == 0 and out["stats"][0] == M
+    assert np.max(np.abs(out["logp"] - ref["logp"])) <= LOGP_ATOL
+    rho = np.exp(ref["logp"] - old_logp)
+    edge = (np.abs(rho - (1 - eps_low)) < 1e-3) | (np.abs(rho - (1 + eps_high)) < 1e-3)
+    assert np.max(np.abs(out["token_loss"] - ref["token_loss"])[~edge]) <= LOGP_ATOL
+    assert abs(out["loss"] - ref["loss"]) <= LOGP_ATOL
+    dx = ref["dlogits"]
+    dx[edge] = 0.0
+    keep = ~edge
+    ref_dh, abs_dh = ref_dhidden(dx, wb)
+    # every shard's partial dhidden is rounded to bf16 before the sum: |p_i| <= its sum of |a||b|
+    grad_close(out["dh"][keep], ref_dh[keep], 2.0 * abs_dh[keep], "dhidden")
+    if not edge.any():
+        grad_close(out["dw"], *ref_dweight(hb, dx), "dweight")
+
+
+def test_lmhead_one_shard_equals_the_unsharded_call():
+    M, K, V = 200, 128, 1032
+    hidden, weight, targets, adv, noise = make_case(M, K, V, seed=5)
+    hb, wb = synth.bf16_bits(hidden), synth.bf16_bits(weight)
+    _, old_logp = old_logp_from_oracle(hb, wb, targets, noise)
+    whole = run_lmhead(hidden, weight, targets, old_logp, adv, 0.2, 0.28)
+    one = run_lmhead_sharded(hidden, weight, (0, V), targets, old_logp, adv, 0.2, 0.28)
+    for k in ("logp", "token_loss", "stats"):
+        assert np.array_equal(whole[k], one[k]), k
+    assert whole["loss"] == one["loss"]
+    assert torch.equal(whole["dh_t"], one["dh_parts"][0])
+    assert torch.equal(whole["dw_t"], one["dw_parts"][0])
+
+
+def test_lmhead_shards_bad_target_aux_and_host_errors():
+    M, K, V = 64, 64, 512
+    hidden, weight, targets, adv, noise = make_case(M, K, V, seed=11)
+    hb, wb = synth.bf16_bits(hidden), synth.bf16_bits(weight)
+    _, old_logp = old_logp_from_oracle(hb, wb, targets, noise)
+    bad = targets.copy()
+    bad[3], bad[9] = V, -1                                   # outside the whole vocabulary
+    aux = np.random.default_rng(2).permutation(M).astype(np.int32)
+    olp_a, adv_a = np.empty_like(old_logp), np.empty_like(adv)
+    olp_a[aux], adv_a[aux] = old_logp, adv                   # row r reads entry aux[r]
+    out = run_lmhead_sharded(hidden, weight, (0, 256, 512), bad, olp_a, adv_a, 0.2, 0.28, aux=aux)
+    assert out["stats_bits"] & b.DEV_BAD_TARGET and out["stats"][3] & b.DEV_BAD_TARGET
+    good = np.ones(M, bool)
+    good[[3, 9]] = False
+    x = oracle.lmhead_logits_rows(hb, wb, np.arange(M, dtype=np.int32))
+    ref = oracle.policy_loss(x[good], bad[good], None, None, old_logp[good], adv[good], f32(0.2),
+                             f32(0.28), denom=float(M))
+    assert np.max(np.abs(out["logp"][good] - ref["logp"])) <= LOGP_ATOL
+    assert np.all(out["logp"][~good] == 0) and np.all(out["dh"][~good] == 0)
+    assert abs(out["loss"] - ref["loss"]) <= LOGP_ATOL
+    # host-detectable errors: offset outside the vocabulary, shard wider than the vocabulary
+    wsd = weight[:, :256].contiguous()
+    m_, s_, xy_ = (torch.zeros(M, device=DEV) for _ in range(3))
+    st = torch.zeros(4, dtype=torch.int32, device=DEV)
+    ws = b.workspace(b.OP_LMHEAD, M, K, 0, 256, DEV)
+    for off, vt in ((-1, V), (300, V), (0, 128)):
+        with pytest.raises(b.TppoError) as e:
+            b.tppo_lmhead_shard_stats(hidden, wsd, off, vt, t(bad, torch.int32), m_, s_, xy_, st, ws)
+        assert e.value.status == 1

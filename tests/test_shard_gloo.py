@@ -107,3 +107,50 @@ def test_shard_batch_rebases_offsets():
     assert np.array_equal(s["values"], c["values"][off:off + s["N"]])
     assert np.array_equal(s["seg_end"] + off, c["seg_end"][1:3])
     assert np.array_equal(s["truncated"], c["truncated"][1:3])
+
+
+# ---- vocabulary-parallel LM-head: the exchange between the two shard calls -----------------------
+def _vocab_worker(rank, world, port, out_path):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        c = _batch()
+        x = c["logits"].astype(np.float64)
+        V = x.shape[1]
+        lo, hi = (0, 40) if rank == 0 else (40, V)          # unequal shards
+        xs = x[:, lo:hi]
+        m = xs.max(axis=1)
+        s = np.exp(xs - m[:, None]).sum(axis=1)
+        y = c["targets"].astype(np.int64)
+        inside = (y >= lo) & (y < hi)
+        xy = np.where(inside, x[np.arange(len(y)), np.clip(y, lo, hi - 1)], 0.0)
+
+        def rescale(row_max, row_max_all, row_sumexp):
+            row_sumexp.mul_(torch.exp(row_max - row_max_all))
+
+        tm, ts, txy = (torch.from_numpy(a.copy()) for a in (m, s, xy))
+        shard.combine_row_stats(tm, ts, txy, rescale)
+        logp = txy - tm - torch.log(ts)
+        gathered = [None] * world
+        dist.all_gather_object(gathered, logp.numpy())
+        if rank == 0:
+            np.savez(out_path, a=gathered[0], b=gathered[1])
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.timeout(180)
+def test_two_vocabulary_shards_merge_to_the_whole_log_softmax(tmp_path):
+    out = str(tmp_path / "vocab.npz")
+    mp.spawn(_vocab_worker, args=(2, _free_port(), out), nprocs=2, join=True)
+    got = np.load(out)
+    c = _batch()
+    ref = oracle.logprob(c["logits"], c["targets"])
+    np.testing.assert_array_equal(got["a"], got["b"])        # every rank ends with the same values
+    np.testing.assert_allclose(got["a"], ref, rtol=0, atol=1e-12)
+
+
+def test_combine_row_stats_is_the_identity_on_one_rank():
+    m, s, xy = torch.tensor([1.0, 2.0]), torch.tensor([3.0, 4.0]), torch.tensor([0.5, 0.0])
+    out = shard.combine_row_stats(m, s, xy, rescale=None)
+    assert out[0] is m and out[1] is s and out[2] is xy
