@@ -15,12 +15,12 @@
 
 namespace tppo {
 
-constexpr int kScanThreads = 256;
+constexpr int kScanThreads = 128;
 constexpr int kScanWarps = kScanThreads / 32;
-constexpr int kScanItems = 8;
+constexpr int kScanItems = 16;
 constexpr int kScanTile = kScanThreads * kScanItems;  // 2048 positions
-constexpr int kSegCap = 96;                           // segments of one tile kept in shared memory
-constexpr int kScanCtasPerSm = 3;
+constexpr int kSegCap = 64;                           // segments of one tile kept in shared memory
+constexpr int kScanCtasPerSm = 6;
 constexpr uint32_t kScanSpinLimit = 1u << 22;
 
 struct Affine2 {  // x -> (aA*xA + bA, aR*xR + bR)
@@ -75,6 +75,7 @@ struct EgaeArgs {
     int32_t vec_ok;   // rewards, values, adv, ret are all 16-byte aligned
     double gamma;
     double gl;  // gamma * lambda
+    double gamma_run, gl_run;   // gamma and gamma*lambda to the power kScanItems
     float* adv;
     float* ret;
     int32_t* status;
@@ -112,8 +113,11 @@ __device__ __forceinline__ void cp_async_wait_all() {
     asm volatile("cp.async.wait_all;" ::: "memory");
 }
 
-// Shared-memory image of one tile: its inputs and the window of segments that can touch it.  Aligned and sized to 16 bytes: r and v are accessed as float4 and by
-// 16-byte cp.async in both halves of a two-element array.
+// Shared-memory image of one tile: its inputs and the window of segments that can touch it.
+// r and v are stored in 16-byte chunks (four positions); a thread owns four consecutive chunks,
+// so chunk c sits at slot c ^ ((c >> 3) & 3): the eight lanes of a quarter warp then read eight
+// different bank groups instead of two.  Aligned and sized to 16 bytes: float4 and cp.async access
+// in both halves of a two-element array.
 struct __align__(16) TileBuf {
     float r[kScanTile];          // rewards
     float v[kScanTile + 4];      // values (+1 look-ahead)
@@ -123,32 +127,35 @@ struct __align__(16) TileBuf {
     int win_lo, win_hi;          // segment indices [win_lo, win_hi) may touch the tile
 };
 static_assert(sizeof(TileBuf) % 16 == 0 && offsetof(TileBuf, v) % 16 == 0, "vector access alignment");
+__device__ __forceinline__ int chunk_slot(int c) { return c ^ ((c >> 3) & 3); }
+__device__ __forceinline__ int pos_slot(int l) { return (chunk_slot(l >> 2) << 2) | (l & 3); }
 
-// Starts the copy of a tile's rewards and values into `buf`.  16-byte chunks go through cp.async
-// (the caller waits with cp_async_wait_all and a barrier); a ragged tail or unaligned arrays are
-// read directly.
+// Starts the copy of a tile's rewards and values into `buf`, by threads first, first + step, ...
+// 16-byte chunks go through cp.async (the caller waits with cp_async_wait_all and a barrier); a
+// ragged tail or unaligned arrays are read directly.
 __device__ __forceinline__ void egae_stage_inputs(const EgaeArgs& a, TileBuf& buf, int64_t t0,
-                                                  int n_tile) {
+                                                  int n_tile, int first, int step) {
     if (a.vec_ok) {
-        for (int u = threadIdx.x; u < kScanTile / 4; u += kScanThreads) {
+        for (int u = first; u < kScanTile / 4; u += step) {
             if (4 * u + 4 <= n_tile) {
-                cp_async16(buf.r + 4 * u, a.rewards + t0 + 4 * u);
-                cp_async16(buf.v + 4 * u, a.values + t0 + 4 * u);
+                const int s = 4 * chunk_slot(u);
+                cp_async16(buf.r + s, a.rewards + t0 + 4 * u);
+                cp_async16(buf.v + s, a.values + t0 + 4 * u);
             } else {
                 for (int k = 4 * u; k < n_tile; ++k) {
-                    buf.r[k] = __ldg(a.rewards + t0 + k);
-                    buf.v[k] = __ldg(a.values + t0 + k);
+                    buf.r[pos_slot(k)] = __ldg(a.rewards + t0 + k);
+                    buf.v[pos_slot(k)] = __ldg(a.values + t0 + k);
                 }
             }
         }
     } else {
-        for (int k = threadIdx.x; k < n_tile; k += kScanThreads) {
-            buf.r[k] = __ldg(a.rewards + t0 + k);
-            buf.v[k] = __ldg(a.values + t0 + k);
+        for (int k = first; k < n_tile; k += step) {
+            buf.r[pos_slot(k)] = __ldg(a.rewards + t0 + k);
+            buf.v[pos_slot(k)] = __ldg(a.values + t0 + k);
         }
     }
-    if (threadIdx.x == kScanThreads - 1)    // value of the position after the tile, if there is one
-        buf.v[n_tile] = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
+    if (first == 0)    // value of the position after the tile, if there is one
+        buf.v[pos_slot(n_tile)] = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
 }
 
 // Segments are ascending and disjoint, so seg_begin and seg_end are both ascending: the window of
@@ -183,10 +190,68 @@ __device__ __forceinline__ bool egae_window_load(const EgaeArgs& a, TileBuf& buf
     return bad;
 }
 
+// Value entering a tile from its right-hand side, by a whole warp: lane i inspects tile first + i.
+// A tile that has published its first-position values (or lies beyond the end, or whose composite
+// has multiplier 0 because a segment ended inside it) terminates the search; the composites of the
+// tiles before it are folded in order.  One round of loads usually suffices, where a single lane
+// walking tile by tile would pay one L2 round trip per tile.  Returns false when the bounded wait
+// ran out.  The result is valid in lane 0.
+__device__ __forceinline__ bool egae_look_back(const EgaeArgs& a, int first, int lane, double& xA,
+                                               double& xR) {
+    Affine2 F = identity2();      // composite of the tiles folded so far (meaningful in lane 0)
+    for (int base = first;; base += 32) {
+        const int j = base + lane;
+        const bool beyond = j >= a.num_tiles;
+        const TileState* st = a.state + (beyond ? 0 : j);
+        double i0 = 0.0, i1 = 0.0, pa = 1.0, pb = 0.0, qa = 1.0, qb = 0.0;
+        bool got_inc = beyond, got_agg = false;
+        int p = 32;
+        uint32_t spins = 0;
+        for (;;) {
+            if (!beyond) {     // the three pairs are requested together: one round trip
+                if (!got_inc) got_inc = ld_pair(st->inc, i0, i1);
+                if (!got_agg) {
+                    double ta, tb, ua, ub;
+                    const bool ga = ld_pair(st->aggA, ta, tb);
+                    const bool gr = ld_pair(st->aggR, ua, ub);
+                    if (ga && gr) { got_agg = true; pa = ta; pb = tb; qa = ua; qb = ub; }
+                }
+            }
+            const bool term = got_inc || (got_agg && pa == 0.0 && qa == 0.0);
+            const uint32_t tmask = __ballot_sync(0xffffffffu, term);
+            const uint32_t rmask = __ballot_sync(0xffffffffu, got_inc || got_agg);
+            p = tmask ? __ffs(int(tmask)) - 1 : 32;
+            const uint32_t need = p < 32 ? ((1u << p) - 1u) : 0xffffffffu;
+            if ((rmask & need) == need) break;
+            if (++spins > kScanSpinLimit) return false;     // uniform: decided from the ballots
+            __nanosleep(20);
+        }
+        // lane < p: the tile's composite; lane p: the constant map to its value; beyond p: identity
+        Affine2 m = identity2();
+        if (lane < p) m = Affine2{pa, pb, qa, qb};
+        else if (lane == p) m = got_inc ? Affine2{0.0, i0, 0.0, i1} : Affine2{0.0, pb, 0.0, qb};
+        if (p > 0) {
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const Affine2 o = shfl_down(m, d);
+                if (lane + d < 32) m = compose(m, o);
+            }
+        }
+        if (p < 32) {       // m is constant in lane 0: its b is the value entering the first folded tile
+            xA = fma(F.aA, m.bA, F.bA);
+            xR = fma(F.aR, m.bR, F.bR);
+            return true;
+        }
+        F = compose(F, m);
+    }
+}
+
 // Persistent CTAs take tiles by ticket, from the END of the arrays backwards, so the tiles a tile
 // looks back at (those to its right) hold earlier tickets and are running or done.  While a tile is
 // being scanned the next ticket is drawn, the next tile's inputs stream into the other buffer
-// (cp.async) and two idle warps find its segment window, so none of those latencies is exposed.
+// (cp.async, issued by the warps that do not look back) and two of them find its segment window, so
+// none of those latencies is exposed.  A thread owns sixteen consecutive positions: the warp scan
+// and the barriers are paid once per 512 positions of a warp.
 __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel(const EgaeArgs a) {
     __shared__ __align__(16) TileBuf s_buf[2];
     __shared__ uint32_t s_ticket[2];
@@ -205,7 +270,7 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
         const int tile = a.num_tiles - 1 - int(ticket);
         const int64_t t0 = int64_t(tile) * kScanTile;
         const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
-        egae_stage_inputs(a, s_buf[0], t0, n_tile);
+        egae_stage_inputs(a, s_buf[0], t0, n_tile, threadIdx.x, kScanThreads);
         if (warp < 2) egae_window_search(a, s_buf[0], t0, n_tile, warp, lane);
         __syncthreads();
         bad |= egae_window_load(a, s_buf[0]);
@@ -226,9 +291,10 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
         const int win_n = max(buf.win_hi - win_lo, 0);
         const bool win_smem = win_n <= kSegCap;
         const int l0 = threadIdx.x * kScanItems;  // first position of this thread inside the tile
+        const int swz = (threadIdx.x >> 1) & 3;   // the thread's chunks 4*tid + q sit at slot (4*tid + q) ^ swz
         double delta[kScanItems];
-        float rew[kScanItems];
-        uint32_t cont = 0;  // bit k: position k continues into position k+1 (same segment)
+        uint32_t cont = 0;    // bit k: position k continues into position k+1 (same segment)
+        uint32_t inside = 0;  // bit k: position k lies inside a segment
         Affine2 f = identity2();
         // index (inside the window) of the last segment that begins at or before the thread's
         // last position, or -1
@@ -252,42 +318,43 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
             }
             i = lo - 1;
         }
-        // The common case: all eight positions lie inside one segment and none of them is its last
-        // token.  Then every map has the same multiplier and no per-position segment test is needed.
+        // The common case: all sixteen positions lie inside one segment and none of them is its
+        // last token.  Then every map has the same multiplier and no per-position test is needed.
         bool fast = false;
         if (win_smem && i >= 0 && l0 + kScanItems <= n_tile)
             fast = int64_t(buf.seg_b[i]) <= t0 + l0 && t0 + l0 + kScanItems < int64_t(buf.seg_e[i]);
         if (fast) {
-            const float4 ra = *reinterpret_cast<const float4*>(buf.r + l0);
-            const float4 rb = *reinterpret_cast<const float4*>(buf.r + l0 + 4);
-            const float4 va = *reinterpret_cast<const float4*>(buf.v + l0);
-            const float4 vb = *reinterpret_cast<const float4*>(buf.v + l0 + 4);
-            const float rr[kScanItems] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
-            const float vv[kScanItems] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
-            double dn = double(buf.v[l0 + kScanItems]);
+            double dn = double(buf.v[pos_slot(l0 + kScanItems)]);
             double bA = 0.0, bR = 0.0;
 #pragma unroll
-            for (int k = kScanItems - 1; k >= 0; --k) {
-                const double dv = double(vv[k]), dr = double(rr[k]);
-                delta[k] = fma(a.gamma, dn, dr) - dv;
-                rew[k] = rr[k];
-                bA = fma(a.gl, bA, delta[k]);
-                bR = fma(a.gamma, bR, dr);
-                dn = dv;
+            for (int q = kScanItems / 4 - 1; q >= 0; --q) {
+                const int s = 4 * ((4 * threadIdx.x + q) ^ swz);
+                const float4 r4 = *reinterpret_cast<const float4*>(buf.r + s);
+                const float4 v4 = *reinterpret_cast<const float4*>(buf.v + s);
+                const float rr[4] = {r4.x, r4.y, r4.z, r4.w};
+                const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+                for (int e = 3; e >= 0; --e) {
+                    const double dv = double(vv[e]), dr = double(rr[e]);
+                    const double d = fma(a.gamma, dn, dr) - dv;
+                    delta[4 * q + e] = d;
+                    bA = fma(a.gl, bA, d);
+                    bR = fma(a.gamma, bR, dr);
+                    dn = dv;
+                }
             }
-            const double gl2 = a.gl * a.gl, gl4 = gl2 * gl2, g2 = a.gamma * a.gamma, g4 = g2 * g2;
-            f = Affine2{gl4 * gl4, bA, g4 * g4, bR};
-            cont = 0xffu;
+            f = Affine2{a.gl_run, bA, a.gamma_run, bR};
+            cont = 0xffffu;
+            inside = 0xffffu;
         } else {
-            float vnext_f = buf.v[min(l0 + kScanItems, n_tile)];
+            float vnext_f = buf.v[pos_slot(min(l0 + kScanItems, n_tile))];
 #pragma unroll
             for (int k = kScanItems - 1; k >= 0; --k) {
                 const int l = l0 + k;
                 delta[k] = 0.0;
-                rew[k] = 0.f;
                 if (l >= n_tile) continue;   // past the end: the identity map
                 const int32_t p = int32_t(t0 + l);
-                const float vf = buf.v[l];
+                const float vf = buf.v[pos_slot(l)];
                 int32_t b = 0, e = 0;
                 bool have = false;
                 while (i >= 0) {
@@ -302,10 +369,9 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
                     if (p >= b) { have = true; break; }
                     --i;
                 }
-                const bool inside = have && p < e;
-                double aA = 0.0, aR = 0.0;
-                if (inside) {
-                    const float r = buf.r[l];
+                double aA = 0.0, aR = 0.0, dr = 0.0;
+                if (have && p < e) {
+                    dr = double(buf.r[pos_slot(l)]);
                     const double v = double(vf);
                     double v_next;
                     if (p + 1 < e) {
@@ -324,11 +390,11 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
                             v_next = 0.0;
                         }
                     }
-                    delta[k] = fma(a.gamma, v_next, double(r)) - v;
-                    rew[k] = r;
+                    delta[k] = fma(a.gamma, v_next, dr) - v;
+                    inside |= 1u << k;
                 }
                 vnext_f = vf;
-                f = compose(Affine2{aA, delta[k], aR, double(rew[k])}, f);
+                f = compose(Affine2{aA, delta[k], aR, dr}, f);
             }
         }
 
@@ -344,61 +410,36 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
         if (lane == 0) s_warp[warp] = S;
         __syncthreads();                                                      // (A)
 
-        // ---- next tile: start its loads and its window search while warp 0 looks back ---------
         const uint32_t next_ticket = s_ticket[(it & 1) ^ 1];
         const bool has_next = next_ticket < uint32_t(a.num_tiles);
-        const int ntile = a.num_tiles - 1 - int(next_ticket);
-        const int64_t nt0 = int64_t(ntile) * kScanTile;
-        const int nn_tile = int(min(int64_t(kScanTile), int64_t(a.N) - nt0));
-        if (has_next) {
-            egae_stage_inputs(a, nbuf, nt0, nn_tile);
-            if (warp == 1 || warp == 2) egae_window_search(a, nbuf, nt0, nn_tile, warp - 1, lane);
-        }
-
-        // ---- tile composite, look-back, per-warp carries (warp 0) ------------------------------
-        if (warp == 0) {
-            // lane w < 8 holds warp w's composite; suffix-compose them in three steps, so that
-            // lane w ends with W_w o ... o W_7 and lane 0 with the tile's composite
+        if (warp != 0) {
+            // ---- next tile: start its loads and its window search while warp 0 looks back -----
+            if (has_next) {
+                const int ntile = a.num_tiles - 1 - int(next_ticket);
+                const int64_t nt0 = int64_t(ntile) * kScanTile;
+                const int nn_tile = int(min(int64_t(kScanTile), int64_t(a.N) - nt0));
+                egae_stage_inputs(a, nbuf, nt0, nn_tile, threadIdx.x - 32, kScanThreads - 32);
+                if (warp <= 2) egae_window_search(a, nbuf, nt0, nn_tile, warp - 1, lane);
+            }
+        } else {
+            // ---- tile composite, look-back, per-warp carries (warp 0) --------------------------
+            // lane w < 4 holds warp w's composite; suffix-compose them, so that lane w ends with
+            // W_w o ... o W_3 and lane 0 with the tile's composite
             Affine2 W = lane < kScanWarps ? s_warp[lane] : identity2();
 #pragma unroll
             for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
             Affine2 right = shfl_down(W, 1);            // composite of the warps to the right
             if (lane >= kScanWarps - 1) right = identity2();
+            TileState* st = a.state;
+            if (lane == 0 && tile + 1 < a.num_tiles) {
+                st_pair(st[tile].aggA, W.aA, W.bA);
+                st_pair(st[tile].aggR, W.aR, W.bR);
+            }
             double xA = 0.0, xR = 0.0;
+            const bool ok = egae_look_back(a, tile + 1, lane, xA, xR);
             if (lane == 0) {
-                const Affine2 tile_f = W;
-                TileState* st = a.state;
-                if (tile + 1 < a.num_tiles) {
-                    st_pair(st[tile].aggA, tile_f.aA, tile_f.bA);
-                    st_pair(st[tile].aggR, tile_f.aR, tile_f.bR);
-                }
-                // value entering from the right: look back over tiles tile+1, tile+2, ...
-                Affine2 F = identity2();
-                bool timed_out = false;
-                for (int j = tile + 1;; ++j) {
-                    if (j >= a.num_tiles) { xA = F.bA; xR = F.bR; break; }   // nothing beyond the end
-                    double i0, i1, pa, pb, qa, qb;
-                    uint32_t spins = 0;
-                    bool got_inc;
-                    for (;;) {       // the three pairs are requested together: one round trip
-                        got_inc = ld_pair(st[j].inc, i0, i1);
-                        const bool ga = ld_pair(st[j].aggA, pa, pb);
-                        const bool gr = ld_pair(st[j].aggR, qa, qb);
-                        if (got_inc || (ga && gr)) break;
-                        if (++spins > kScanSpinLimit) { timed_out = true; break; }
-                        __nanosleep(20);
-                    }
-                    if (timed_out) break;
-                    if (got_inc) {
-                        xA = fma(F.aA, i0, F.bA);
-                        xR = fma(F.aR, i1, F.bR);
-                        break;
-                    }
-                    F = compose(F, Affine2{pa, pb, qa, qb});
-                    if (F.aA == 0.0 && F.aR == 0.0) { xA = F.bA; xR = F.bR; break; }  // a segment ended
-                }
-                if (timed_out) { atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
-                st_pair(st[tile].inc, fma(tile_f.aA, xA, tile_f.bA), fma(tile_f.aR, xR, tile_f.bR));
+                if (!ok) { atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
+                st_pair(st[tile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
             }
             xA = __shfl_sync(0xffffffffu, xA, 0);
             xR = __shfl_sync(0xffffffffu, xR, 0);
@@ -413,30 +454,36 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
         // ---- replay the thread's positions with the true incoming values, store -----------------
         double A = fma(excl.aA, s_carry[warp][0], excl.bA);
         double G = fma(excl.aR, s_carry[warp][1], excl.bR);
-        float oa[kScanItems], og[kScanItems];
+        const bool full = a.vec_ok && l0 + kScanItems <= n_tile;
 #pragma unroll
-        for (int k = kScanItems - 1; k >= 0; --k) {
-            const bool c = (cont >> k) & 1u;
-            A = c ? fma(a.gl, A, delta[k]) : delta[k];
-            G = c ? fma(a.gamma, G, double(rew[k])) : double(rew[k]);
-            oa[k] = float(A);
-            og[k] = float(G);
-        }
-        if (a.vec_ok && l0 + kScanItems <= n_tile) {
-            float4* pa4 = reinterpret_cast<float4*>(a.adv + t0 + l0);
-            pa4[0] = make_float4(oa[0], oa[1], oa[2], oa[3]);
-            pa4[1] = make_float4(oa[4], oa[5], oa[6], oa[7]);
-            if (a.ret) {
-                float4* pg4 = reinterpret_cast<float4*>(a.ret + t0 + l0);
-                pg4[0] = make_float4(og[0], og[1], og[2], og[3]);
-                pg4[1] = make_float4(og[4], og[5], og[6], og[7]);
+        for (int q = kScanItems / 4 - 1; q >= 0; --q) {
+            float rr[4] = {0.f, 0.f, 0.f, 0.f};
+            if (l0 + 4 * q < n_tile) {       // the chunk was staged (a ragged one only in part: masked below)
+                const float4 r4 = *reinterpret_cast<const float4*>(buf.r + 4 * ((4 * threadIdx.x + q) ^ swz));
+                rr[0] = r4.x; rr[1] = r4.y; rr[2] = r4.z; rr[3] = r4.w;
             }
-        } else {
+            float oa[4], og[4];
 #pragma unroll
-            for (int k = 0; k < kScanItems; ++k) {
-                if (l0 + k < n_tile) {
-                    a.adv[t0 + l0 + k] = oa[k];
-                    if (a.ret) a.ret[t0 + l0 + k] = og[k];
+            for (int e = 3; e >= 0; --e) {
+                const int k = 4 * q + e;
+                const bool c = (cont >> k) & 1u;
+                const double dr = ((inside >> k) & 1u) ? double(rr[e]) : 0.0;
+                A = c ? fma(a.gl, A, delta[k]) : delta[k];
+                G = c ? fma(a.gamma, G, dr) : dr;
+                oa[e] = float(A);
+                og[e] = float(G);
+            }
+            if (full) {
+                *reinterpret_cast<float4*>(a.adv + t0 + l0 + 4 * q) = make_float4(oa[0], oa[1], oa[2], oa[3]);
+                if (a.ret)
+                    *reinterpret_cast<float4*>(a.ret + t0 + l0 + 4 * q) = make_float4(og[0], og[1], og[2], og[3]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (l0 + 4 * q + e < n_tile) {
+                        a.adv[t0 + l0 + 4 * q + e] = oa[e];
+                        if (a.ret) a.ret[t0 + l0 + 4 * q + e] = og[e];
+                    }
                 }
             }
         }
@@ -488,6 +535,8 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
     a.num_tiles = int32_t((N + kScanTile - 1) / kScanTile);
     a.gamma = double(gamma);
     a.gl = double(gamma) * double(lambda);
+    a.gamma_run = 1.0; a.gl_run = 1.0;
+    for (int k = 0; k < kScanItems; ++k) { a.gamma_run *= a.gamma; a.gl_run *= a.gl; }
     a.adv = advantages; a.ret = returns; a.status = status;
     a.vec_ok = aligned(rewards, 16) && aligned(values, 16) && aligned(advantages, 16) &&
                (!returns || aligned(returns, 16));
@@ -556,6 +605,8 @@ TPPO_API int tppo_egae_static(const float* rewards, const float* values, const i
     a.num_tiles = int32_t((N + kScanTile - 1) / kScanTile);
     a.gamma = double(gamma);
     a.gl = double(gamma) * double(lambda);
+    a.gamma_run = 1.0; a.gl_run = 1.0;
+    for (int k = 0; k < kScanItems; ++k) { a.gamma_run *= a.gamma; a.gl_run *= a.gl; }
     a.adv = advantages; a.ret = returns; a.status = status;
     a.vec_ok = aligned(rewards, 16) && aligned(values, 16) && aligned(advantages, 16) &&
                (!returns || aligned(returns, 16));
