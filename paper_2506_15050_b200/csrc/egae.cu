@@ -1,17 +1,37 @@
 // EGAE advantages and Monte-Carlo returns (Section 3.1, Eq. 6 with the TD residual of Eq. 3; R_t
 // after Eq. 5) as ONE segmented reverse scan over the packed token arrays.
 //
-// Both recurrences are affine in the value at the next position,
-//     A_t = delta_t + (gamma*lambda) * A_{t+1},      R_t = r_t + gamma * R_{t+1},
-// so every position carries a map x -> a*x + b, with a = 0 on the last token of a segment and
-// outside every segment.  Maps compose associatively; a tile composes its positions right to
-// left, publishes the composite, and obtains the value entering from its right-hand neighbour by
-// decoupled look-back over the tiles behind it.  A composite whose `a` has become 0 (a segment
-// ended inside the range) ends the look-back early.  State is fp64, rounded once on store.
-// Tiles are staged in shared memory so that every global access is a coalesced 16-byte one.
+// The advantage recurrence A_t = delta_t + (gamma*lambda) A_{t+1} is carried as G_t = A_t + V_t,
+//     G_t = r_t + gamma (1 - lambda) V_{t+1} + (gamma*lambda) G_{t+1},    R_t = r_t + gamma R_{t+1},
+// (on the last token of a segment G_t = r_t + gamma V_next, with V_next the boundary value), so the
+// values enter additively and successive values never cancel against each other.  Both recurrences
+// are affine in the value at the next position: every position carries a map x -> a*x + b, with
+// a = 0 on the last token of a segment and outside every segment.  Maps compose associatively.
+//
+// Precision.  A thread owns sixteen consecutive positions and runs them sequentially in fp32 (the
+// multiplier gamma*lambda, the only factor that is raised to high powers, is split into two floats
+// so that it is exact to 2^-48); everything that crosses threads -- the thread composites, the warp
+// scan, the tile composites and the look-back -- is fp64, and the value entering a thread's run is
+// rounded to fp32 once.  The rounding error of a result is a few units of 2^-24 of the largest
+// |G| or |R| in its run; nothing accumulates over the length of a segment.
+//
+// One CTA per tile of 2048 positions, tiles taken by ticket from the END of the arrays backwards,
+// so the tiles a tile looks back at (those to its right) hold earlier tickets and are running or
+// done.  A tile composes its positions right to left, publishes the composite, and obtains the
+// value entering from its right-hand neighbour by decoupled look-back over the tiles behind it.  A
+// composite whose `a` has become 0 (a segment ended inside the range) ends the look-back early.
+// The inputs of a whole tile arrive by two tiled TMA copies (rows of 32 positions, 128-byte
+// swizzle: the four 16-byte chunks a thread owns then sit in different bank groups from its
+// neighbours'); there is no per-thread staging code.  Latencies (ticket, copy, window search,
+// look-back) are covered by the other CTAs resident on the SM rather than by software pipelining.
 #include <cstddef>
+#include <cstring>
+
+#include <cuda.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
+#include "umma.cuh"
 
 namespace tppo {
 
@@ -19,8 +39,8 @@ constexpr int kScanThreads = 128;
 constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kScanItems = 16;
 constexpr int kScanTile = kScanThreads * kScanItems;  // 2048 positions
-constexpr int kSegCap = 64;                           // segments of one tile kept in shared memory
-constexpr int kScanCtasPerSm = 6;
+constexpr int kSegCap = 32;                           // segments of one tile kept in shared memory
+constexpr int kScanCtasPerSm = 8;
 constexpr uint32_t kScanSpinLimit = 1u << 22;
 
 struct Affine2 {  // x -> (aA*xA + bA, aR*xR + bR)
@@ -56,11 +76,22 @@ __device__ __forceinline__ void st_pair(double* p, double x, double y) {
     asm volatile("st.relaxed.gpu.global.v2.f64 [%0], {%1, %2};"
                  ::"l"(p), "d"(publishable(x)), "d"(publishable(y)) : "memory");
 }
-__device__ __forceinline__ bool ld_pair(const double* p, double& x, double& y) {
-    asm volatile("ld.relaxed.gpu.global.v2.f64 {%0, %1}, [%2];" : "=d"(x), "=d"(y) : "l"(p) : "memory");
+__device__ __forceinline__ bool pair_set(double x, double y) {
     return (unsigned long long)__double_as_longlong(x) != kUnset &&
            (unsigned long long)__double_as_longlong(y) != kUnset;
 }
+// The three pairs of a tile state in one go: the loads are issued back to back (one round trip to
+// L2 instead of three).
+__device__ __forceinline__ void ld_state(const TileState* st, double& pa, double& pb, double& qa,
+                                         double& qb, double& i0, double& i1) {
+    asm volatile(
+        "ld.relaxed.gpu.global.v2.f64 {%0, %1}, [%6];\n\t"
+        "ld.relaxed.gpu.global.v2.f64 {%2, %3}, [%6+16];\n\t"
+        "ld.relaxed.gpu.global.v2.f64 {%4, %5}, [%6+32];"
+        : "=d"(pa), "=d"(pb), "=d"(qa), "=d"(qb), "=d"(i0), "=d"(i1) : "l"(st) : "memory");
+}
+static_assert(offsetof(TileState, aggA) == 0 && offsetof(TileState, aggR) == 16 &&
+              offsetof(TileState, inc) == 32, "ld_state reads the pairs by offset");
 
 struct EgaeArgs {
     const float* rewards;
@@ -73,9 +104,13 @@ struct EgaeArgs {
     int32_t N;
     int32_t num_tiles;
     int32_t vec_ok;   // rewards, values, adv, ret are all 16-byte aligned
+    int32_t tma_ok;   // the two tensor maps are valid: whole tiles arrive by TMA
     double gamma;
     double gl;  // gamma * lambda
     double gamma_run, gl_run;   // gamma and gamma*lambda to the power kScanItems
+    float gamma_f;              // gamma (an fp32 input: exact)
+    float gl_hi, gl_lo;         // gamma*lambda = gl_hi + gl_lo up to 2^-48
+    float c1;                   // gamma * (1 - lambda)
     float* adv;
     float* ret;
     int32_t* status;
@@ -84,13 +119,14 @@ struct EgaeArgs {
 };
 
 // Number of entries of the ascending array arr[0..n) that are <= key, found by a whole warp: each
-// round probes 32 evenly spaced entries, so 4096 entries take three rounds of one load each
-// instead of twelve dependent loads.  Every lane returns the same count.  An array that is not
-// ascending still yields an in-range answer.
+// round probes 32 evenly spaced entries until at most 128 remain, which are then read in one go
+// (four independent loads per lane), so 4096 entries take two dependent rounds instead of twelve
+// dependent loads.  Every lane returns the same count.  An array that is not ascending still
+// yields an in-range answer.
 __device__ __forceinline__ int warp_count_le(const int32_t* __restrict__ arr, int n, int32_t key,
                                              int lane) {
     int lo = 0, hi = n;       // the answer lies in [lo, hi]
-    while (lo < hi) {
+    while (hi - lo > 128) {
         const int span = hi - lo;
         const int step = (span + 31) >> 5;
         const int idx = lo + lane * step;
@@ -102,60 +138,36 @@ __device__ __forceinline__ int warp_count_le(const int32_t* __restrict__ arr, in
         if (c > 0) lo = lo + (c - 1) * step + 1;
         hi = new_hi;
     }
-    return lo;
+    bool le[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int idx = lo + 32 * j + lane;
+        le[j] = idx < hi && __ldg(arr + idx) <= key;
+    }
+    int count = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) count += __popc(__ballot_sync(0xffffffffu, le[j]));
+    return lo + count;
 }
 
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
-                 ::"r"(uint32_t(__cvta_generic_to_shared(smem_dst))), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() {
-    asm volatile("cp.async.wait_all;" ::: "memory");
-}
-
-// Shared-memory image of one tile: its inputs and the window of segments that can touch it.
-// r and v are stored in 16-byte chunks (four positions); a thread owns four consecutive chunks,
-// so chunk c sits at slot c ^ ((c >> 3) & 3): the eight lanes of a quarter warp then read eight
-// different bank groups instead of two.  Aligned and sized to 16 bytes: float4 and cp.async access
-// in both halves of a two-element array.
-struct __align__(16) TileBuf {
+// Shared-memory image of one tile.  r and v are 64 rows of 32 positions (128 bytes) in the layout
+// the TMA's 128-byte swizzle writes: 16-byte chunk c of row y sits at chunk c ^ (y & 7) of that row
+// (the arrays are 1024-byte aligned, eight rows).  A thread owns half a row; the eight lanes of a
+// quarter warp then read eight different bank groups.
+constexpr int kRowPos = 32;
+struct __align__(1024) TileBuf {
     float r[kScanTile];          // rewards
-    float v[kScanTile + 4];      // values (+1 look-ahead)
+    float v[kScanTile];          // values
     int32_t seg_b[kSegCap], seg_e[kSegCap];
     float seg_boot[kSegCap];
     uint8_t seg_t[kSegCap];
+    float v_after;               // value of the position after the tile (0 beyond the arrays)
     int win_lo, win_hi;          // segment indices [win_lo, win_hi) may touch the tile
 };
-static_assert(sizeof(TileBuf) % 16 == 0 && offsetof(TileBuf, v) % 16 == 0, "vector access alignment");
-__device__ __forceinline__ int chunk_slot(int c) { return c ^ ((c >> 3) & 3); }
-__device__ __forceinline__ int pos_slot(int l) { return (chunk_slot(l >> 2) << 2) | (l & 3); }
-
-// Starts the copy of a tile's rewards and values into `buf`, by threads first, first + step, ...
-// 16-byte chunks go through cp.async (the caller waits with cp_async_wait_all and a barrier); a
-// ragged tail or unaligned arrays are read directly.
-__device__ __forceinline__ void egae_stage_inputs(const EgaeArgs& a, TileBuf& buf, int64_t t0,
-                                                  int n_tile, int first, int step) {
-    if (a.vec_ok) {
-        for (int u = first; u < kScanTile / 4; u += step) {
-            if (4 * u + 4 <= n_tile) {
-                const int s = 4 * chunk_slot(u);
-                cp_async16(buf.r + s, a.rewards + t0 + 4 * u);
-                cp_async16(buf.v + s, a.values + t0 + 4 * u);
-            } else {
-                for (int k = 4 * u; k < n_tile; ++k) {
-                    buf.r[pos_slot(k)] = __ldg(a.rewards + t0 + k);
-                    buf.v[pos_slot(k)] = __ldg(a.values + t0 + k);
-                }
-            }
-        }
-    } else {
-        for (int k = first; k < n_tile; k += step) {
-            buf.r[pos_slot(k)] = __ldg(a.rewards + t0 + k);
-            buf.v[pos_slot(k)] = __ldg(a.values + t0 + k);
-        }
-    }
-    if (first == 0)    // value of the position after the tile, if there is one
-        buf.v[pos_slot(n_tile)] = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
+static_assert(offsetof(TileBuf, v) % 1024 == 0, "swizzle atom alignment");
+__device__ __forceinline__ int pos_slot(int l) {      // float index of position l
+    const int y = l >> 5;
+    return (y << 5) | (((((l >> 2) & 7) ^ (y & 7)) << 2)) | (l & 3);
 }
 
 // Segments are ascending and disjoint, so seg_begin and seg_end are both ascending: the window of
@@ -190,6 +202,52 @@ __device__ __forceinline__ bool egae_window_load(const EgaeArgs& a, TileBuf& buf
     return bad;
 }
 
+// What one position contributes, for threads that touch a segment boundary or lie outside every
+// segment (the others never call this).  `i` is the index, inside the window, of the last segment
+// that begins at or before the positions still to come; the caller walks l downwards and `i`
+// follows.  x is the additive term of the G recurrence, r the reward; cont says that the position
+// continues into position l + 1 of the same segment (otherwise its map is constant).
+struct PosTerm {
+    float x, r, v;
+    bool cont, inside;
+};
+__device__ __forceinline__ PosTerm egae_position(const EgaeArgs& a, const TileBuf& buf, int64_t t0,
+                                                 int n_tile, int win_lo, bool win_smem, int l, int& i,
+                                                 bool& bad) {
+    PosTerm o{0.f, 0.f, 0.f, false, false};
+    if (l >= n_tile) return o;
+    const int32_t p = int32_t(t0 + l);
+    int32_t b = 0, e = 0;
+    bool have = false;
+    while (i >= 0) {
+        if (win_smem) {
+            b = buf.seg_b[i];
+            e = buf.seg_e[i];
+        } else {
+            b = __ldg(a.seg_begin + win_lo + i);
+            e = __ldg(a.seg_end + win_lo + i);
+            if (b < 0 || e > a.N || e < b) { bad = true; e = b; }
+        }
+        if (p >= b) { have = true; break; }
+        --i;
+    }
+    if (!have || p >= e) return o;
+    o.inside = true;
+    o.r = buf.r[pos_slot(l)];
+    o.v = buf.v[pos_slot(l)];
+    if (p + 1 < e) {
+        const float v_next = l + 1 < kScanTile ? buf.v[pos_slot(l + 1)] : buf.v_after;
+        o.x = fmaf(a.c1, v_next, o.r);
+        o.cont = true;
+    } else {      // last token: G = r + gamma * (0 | bootstrap value | its own value)
+        const bool tr = win_smem ? (buf.seg_t[i] != 0) : (__ldg(a.truncated + win_lo + i) != 0);
+        float v_next = 0.f;
+        if (tr) v_next = a.bootstrap ? (win_smem ? buf.seg_boot[i] : __ldg(a.bootstrap + win_lo + i)) : o.v;
+        o.x = fmaf(a.gamma_f, v_next, o.r);
+    }
+    return o;
+}
+
 // Value entering a tile from its right-hand side, by a whole warp: lane i inspects tile first + i.
 // A tile that has published its first-position values (or lies beyond the end, or whose composite
 // has multiplier 0 because a segment ended inside it) terminates the search; the composites of the
@@ -208,13 +266,12 @@ __device__ __forceinline__ bool egae_look_back(const EgaeArgs& a, int first, int
         int p = 32;
         uint32_t spins = 0;
         for (;;) {
-            if (!beyond) {     // the three pairs are requested together: one round trip
-                if (!got_inc) got_inc = ld_pair(st->inc, i0, i1);
-                if (!got_agg) {
-                    double ta, tb, ua, ub;
-                    const bool ga = ld_pair(st->aggA, ta, tb);
-                    const bool gr = ld_pair(st->aggR, ua, ub);
-                    if (ga && gr) { got_agg = true; pa = ta; pb = tb; qa = ua; qb = ub; }
+            if (!beyond && !got_inc) {
+                double ta, tb, ua, ub, j0, j1;
+                ld_state(st, ta, tb, ua, ub, j0, j1);
+                if (pair_set(j0, j1)) { got_inc = true; i0 = j0; i1 = j1; }
+                if (!got_agg && pair_set(ta, tb) && pair_set(ua, ub)) {
+                    got_agg = true; pa = ta; pb = tb; qa = ua; qb = ub;
                 }
             }
             const bool term = got_inc || (got_agg && pa == 0.0 && qa == 0.0);
@@ -246,232 +303,195 @@ __device__ __forceinline__ bool egae_look_back(const EgaeArgs& a, int first, int
     }
 }
 
-// Persistent CTAs take tiles by ticket, from the END of the arrays backwards, so the tiles a tile
-// looks back at (those to its right) hold earlier tickets and are running or done.  While a tile is
-// being scanned the next ticket is drawn, the next tile's inputs stream into the other buffer
-// (cp.async, issued by the warps that do not look back) and two of them find its segment window, so
-// none of those latencies is exposed.  A thread owns sixteen consecutive positions: the warp scan
-// and the barriers are paid once per 512 positions of a warp.
-__global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel(const EgaeArgs a) {
-    __shared__ __align__(16) TileBuf s_buf[2];
-    __shared__ uint32_t s_ticket[2];
+__global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm)
+egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
+                 const __grid_constant__ CUtensorMap map_v) {
+    __shared__ TileBuf buf;
+    __shared__ __align__(8) uint64_t s_bar;      // the tile's inputs have arrived
+    __shared__ uint32_t s_ticket;
     __shared__ Affine2 s_warp[kScanWarps];
     __shared__ double s_carry[kScanWarps][2];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // the ticket counter starts at all-ones like the rest of the workspace (one memset): + 1 wraps
-    // the first draw to ticket 0
-    if (threadIdx.x == 0) s_ticket[0] = atomicAdd(a.ticket, 1u) + 1u;
-    __syncthreads();
-    uint32_t ticket = s_ticket[0];
-    if (ticket >= uint32_t(a.num_tiles)) return;
-    bool bad = false;
-    {   // first tile of this CTA: nothing to overlap with
-        const int tile = a.num_tiles - 1 - int(ticket);
-        const int64_t t0 = int64_t(tile) * kScanTile;
-        const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
-        egae_stage_inputs(a, s_buf[0], t0, n_tile, threadIdx.x, kScanThreads);
-        if (warp < 2) egae_window_search(a, s_buf[0], t0, n_tile, warp, lane);
-        __syncthreads();
-        bad |= egae_window_load(a, s_buf[0]);
-        cp_async_wait_all();
-        __syncthreads();
+    const uint32_t bar = ptx::smem_addr(&s_bar);
+    if (threadIdx.x == 0) {
+        // the ticket counter starts at all-ones like the rest of the workspace (one memset): + 1
+        // wraps the first draw to ticket 0
+        s_ticket = atomicAdd(a.ticket, 1u) + 1u;
+        ptx::mbar_init(bar, 1);
+        ptx::fence_mbar_init_cluster();
     }
+    __syncthreads();
+    const uint32_t ticket = s_ticket;
+    if (ticket >= uint32_t(a.num_tiles)) return;       // (the grid has exactly num_tiles CTAs)
+    const int tile = a.num_tiles - 1 - int(ticket);
+    const int64_t t0 = int64_t(tile) * kScanTile;
+    const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
+    const bool by_tma = a.tma_ok && n_tile == kScanTile;
 
-    for (int it = 0;; ++it) {
-        TileBuf& buf = s_buf[it & 1];
-        TileBuf& nbuf = s_buf[(it & 1) ^ 1];
-        const int tile = a.num_tiles - 1 - int(ticket);
-        const int64_t t0 = int64_t(tile) * kScanTile;
-        const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
-        if (threadIdx.x == 0) s_ticket[(it & 1) ^ 1] = atomicAdd(a.ticket, 1u) + 1u;   // next tile
-
-        // ---- per-position maps, right to left -----------------------------------------------
-        const int win_lo = buf.win_lo;
-        const int win_n = max(buf.win_hi - win_lo, 0);
-        const bool win_smem = win_n <= kSegCap;
-        const int l0 = threadIdx.x * kScanItems;  // first position of this thread inside the tile
-        const int swz = (threadIdx.x >> 1) & 3;   // the thread's chunks 4*tid + q sit at slot (4*tid + q) ^ swz
-        double delta[kScanItems];
-        uint32_t cont = 0;    // bit k: position k continues into position k+1 (same segment)
-        uint32_t inside = 0;  // bit k: position k lies inside a segment
-        Affine2 f = identity2();
-        // index (inside the window) of the last segment that begins at or before the thread's
-        // last position, or -1
-        const int l_last = min(l0 + kScanItems, n_tile) - 1;
-        int i = -1;
-        if (l_last >= l0) {
-            const int32_t key = int32_t(t0 + l_last);
-            int lo = 0, hi = win_n;
-            if (win_smem && win_n <= 4) {
-                while (lo < win_n && buf.seg_b[lo] <= key) ++lo;
-            } else if (win_smem) {
-                while (lo < hi) {
-                    const int mid = (lo + hi) >> 1;
-                    if (buf.seg_b[mid] <= key) lo = mid + 1; else hi = mid;
-                }
-            } else {
-                while (lo < hi) {
-                    const int mid = (lo + hi) >> 1;
-                    if (__ldg(a.seg_begin + win_lo + mid) <= key) lo = mid + 1; else hi = mid;
-                }
-            }
-            i = lo - 1;
+    // ---- inputs: two TMA copies for a whole tile, plain loads for a ragged or unaligned one ------
+    if (by_tma) {
+        if (threadIdx.x == 0) {
+            ptx::mbar_arrive_expect_tx(bar, 2 * kScanTile * uint32_t(sizeof(float)));
+            umma::tma_load_2d(ptx::smem_addr(buf.r), &map_r, bar, 0, int32_t(t0 / kRowPos));
+            umma::tma_load_2d(ptx::smem_addr(buf.v), &map_v, bar, 0, int32_t(t0 / kRowPos));
         }
-        // The common case: all sixteen positions lie inside one segment and none of them is its
-        // last token.  Then every map has the same multiplier and no per-position test is needed.
-        bool fast = false;
-        if (win_smem && i >= 0 && l0 + kScanItems <= n_tile)
-            fast = int64_t(buf.seg_b[i]) <= t0 + l0 && t0 + l0 + kScanItems < int64_t(buf.seg_e[i]);
-        if (fast) {
-            double dn = double(buf.v[pos_slot(l0 + kScanItems)]);
-            double bA = 0.0, bR = 0.0;
-#pragma unroll
-            for (int q = kScanItems / 4 - 1; q >= 0; --q) {
-                const int s = 4 * ((4 * threadIdx.x + q) ^ swz);
-                const float4 r4 = *reinterpret_cast<const float4*>(buf.r + s);
-                const float4 v4 = *reinterpret_cast<const float4*>(buf.v + s);
-                const float rr[4] = {r4.x, r4.y, r4.z, r4.w};
-                const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
-#pragma unroll
-                for (int e = 3; e >= 0; --e) {
-                    const double dv = double(vv[e]), dr = double(rr[e]);
-                    const double d = fma(a.gamma, dn, dr) - dv;
-                    delta[4 * q + e] = d;
-                    bA = fma(a.gl, bA, d);
-                    bR = fma(a.gamma, bR, dr);
-                    dn = dv;
-                }
-            }
-            f = Affine2{a.gl_run, bA, a.gamma_run, bR};
-            cont = 0xffffu;
-            inside = 0xffffu;
-        } else {
-            float vnext_f = buf.v[pos_slot(min(l0 + kScanItems, n_tile))];
-#pragma unroll
-            for (int k = kScanItems - 1; k >= 0; --k) {
-                const int l = l0 + k;
-                delta[k] = 0.0;
-                if (l >= n_tile) continue;   // past the end: the identity map
-                const int32_t p = int32_t(t0 + l);
-                const float vf = buf.v[pos_slot(l)];
-                int32_t b = 0, e = 0;
-                bool have = false;
-                while (i >= 0) {
-                    if (win_smem) {
-                        b = buf.seg_b[i];
-                        e = buf.seg_e[i];
-                    } else {
-                        b = __ldg(a.seg_begin + win_lo + i);
-                        e = __ldg(a.seg_end + win_lo + i);
-                        if (b < 0 || e > a.N || e < b) { bad = true; e = b; }
-                    }
-                    if (p >= b) { have = true; break; }
-                    --i;
-                }
-                double aA = 0.0, aR = 0.0, dr = 0.0;
-                if (have && p < e) {
-                    dr = double(buf.r[pos_slot(l)]);
-                    const double v = double(vf);
-                    double v_next;
-                    if (p + 1 < e) {
-                        v_next = double(vnext_f);
-                        aA = a.gl;
-                        aR = a.gamma;
-                        cont |= 1u << k;
-                    } else {
-                        const bool tr = win_smem ? (buf.seg_t[i] != 0)
-                                                 : (__ldg(a.truncated + win_lo + i) != 0);
-                        if (tr) {
-                            v_next = a.bootstrap ? double(win_smem ? buf.seg_boot[i]
-                                                                   : __ldg(a.bootstrap + win_lo + i))
-                                                 : v;
-                        } else {
-                            v_next = 0.0;
-                        }
-                    }
-                    delta[k] = fma(a.gamma, v_next, dr) - v;
-                    inside |= 1u << k;
-                }
-                vnext_f = vf;
-                f = compose(Affine2{aA, delta[k], aR, dr}, f);
-            }
+    } else {
+        for (int k = threadIdx.x; k < n_tile; k += kScanThreads) {
+            buf.r[pos_slot(k)] = __ldg(a.rewards + t0 + k);
+            buf.v[pos_slot(k)] = __ldg(a.values + t0 + k);
         }
+    }
+    if (threadIdx.x == kScanThreads - 1)
+        buf.v_after = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
+    if (warp < 2) egae_window_search(a, buf, t0, n_tile, warp, lane);
+    __syncthreads();
+    bool bad = egae_window_load(a, buf);
+    if (by_tma && !ptx::mbar_wait<false>(bar, 0)) atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT);
+    __syncthreads();
 
-        // ---- inclusive suffix composition inside the warp: S_l = f_l o f_{l+1} o ... o f_31 ---
-        Affine2 S = f;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const Affine2 o = shfl_down(S, d);
-            if (lane + d < 32) S = compose(S, o);
-        }
-        Affine2 excl = shfl_down(S, 1);   // composite of the lanes to the right
-        if (lane == 31) excl = identity2();
-        if (lane == 0) s_warp[warp] = S;
-        __syncthreads();                                                      // (A)
-
-        const uint32_t next_ticket = s_ticket[(it & 1) ^ 1];
-        const bool has_next = next_ticket < uint32_t(a.num_tiles);
-        if (warp != 0) {
-            // ---- next tile: start its loads and its window search while warp 0 looks back -----
-            if (has_next) {
-                const int ntile = a.num_tiles - 1 - int(next_ticket);
-                const int64_t nt0 = int64_t(ntile) * kScanTile;
-                const int nn_tile = int(min(int64_t(kScanTile), int64_t(a.N) - nt0));
-                egae_stage_inputs(a, nbuf, nt0, nn_tile, threadIdx.x - 32, kScanThreads - 32);
-                if (warp <= 2) egae_window_search(a, nbuf, nt0, nn_tile, warp - 1, lane);
+    // ---- the thread's sixteen positions, right to left: its composite map -------------------------
+    const int win_lo = buf.win_lo;
+    const int win_n = max(buf.win_hi - win_lo, 0);
+    const bool win_smem = win_n <= kSegCap;
+    const int l0 = threadIdx.x * kScanItems;        // first position of this thread inside the tile
+    // its four chunks: row tid/2, chunks 4*(tid&1) + q, stored at chunk ^ (row & 7)
+    const int row_base = (threadIdx.x >> 1) << 5;
+    const int chunk0 = (threadIdx.x & 1) << 2, swz = (threadIdx.x >> 1) & 7;
+    // index (inside the window) of the last segment that begins at or before the thread's last
+    // position, or -1
+    const int l_last = min(l0 + kScanItems, n_tile) - 1;
+    int i_start = -1;
+    if (l_last >= l0) {
+        const int32_t key = int32_t(t0 + l_last);
+        int lo = 0, hi = win_n;
+        if (win_smem && win_n <= 4) {
+            while (lo < win_n && buf.seg_b[lo] <= key) ++lo;
+        } else if (win_smem) {
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (buf.seg_b[mid] <= key) lo = mid + 1; else hi = mid;
             }
         } else {
-            // ---- tile composite, look-back, per-warp carries (warp 0) --------------------------
-            // lane w < 4 holds warp w's composite; suffix-compose them, so that lane w ends with
-            // W_w o ... o W_3 and lane 0 with the tile's composite
-            Affine2 W = lane < kScanWarps ? s_warp[lane] : identity2();
-#pragma unroll
-            for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
-            Affine2 right = shfl_down(W, 1);            // composite of the warps to the right
-            if (lane >= kScanWarps - 1) right = identity2();
-            TileState* st = a.state;
-            if (lane == 0 && tile + 1 < a.num_tiles) {
-                st_pair(st[tile].aggA, W.aA, W.bA);
-                st_pair(st[tile].aggR, W.aR, W.bR);
-            }
-            double xA = 0.0, xR = 0.0;
-            const bool ok = egae_look_back(a, tile + 1, lane, xA, xR);
-            if (lane == 0) {
-                if (!ok) { atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
-                st_pair(st[tile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
-            }
-            xA = __shfl_sync(0xffffffffu, xA, 0);
-            xR = __shfl_sync(0xffffffffu, xR, 0);
-            if (lane < kScanWarps) {
-                s_carry[lane][0] = fma(right.aA, xA, right.bA);
-                s_carry[lane][1] = fma(right.aR, xR, right.bR);
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (__ldg(a.seg_begin + win_lo + mid) <= key) lo = mid + 1; else hi = mid;
             }
         }
-        __syncthreads();                                                      // (B)
-        if (has_next) bad |= egae_window_load(a, nbuf);
-
-        // ---- replay the thread's positions with the true incoming values, store -----------------
-        double A = fma(excl.aA, s_carry[warp][0], excl.bA);
-        double G = fma(excl.aR, s_carry[warp][1], excl.bR);
-        const bool full = a.vec_ok && l0 + kScanItems <= n_tile;
+        i_start = lo - 1;
+    }
+    // The common case: all sixteen positions lie inside one segment and none of them is its last
+    // token.  Then every map has the same multiplier and no per-position test is needed.
+    bool fast = false;
+    if (win_smem && i_start >= 0 && l0 + kScanItems <= n_tile)
+        fast = int64_t(buf.seg_b[i_start]) <= t0 + l0 &&
+               t0 + l0 + kScanItems < int64_t(buf.seg_e[i_start]);
+    // value of the position after the thread's run (only the fast path uses it: the run then
+    // continues into that position)
+    const float v_right = l0 + kScanItems < kScanTile ? buf.v[pos_slot(l0 + kScanItems)] : buf.v_after;
+    Affine2 f;
+    if (fast) {
+        float bG = 0.f, bR = 0.f, vn = v_right;
 #pragma unroll
         for (int q = kScanItems / 4 - 1; q >= 0; --q) {
-            float rr[4] = {0.f, 0.f, 0.f, 0.f};
-            if (l0 + 4 * q < n_tile) {       // the chunk was staged (a ragged one only in part: masked below)
-                const float4 r4 = *reinterpret_cast<const float4*>(buf.r + 4 * ((4 * threadIdx.x + q) ^ swz));
-                rr[0] = r4.x; rr[1] = r4.y; rr[2] = r4.z; rr[3] = r4.w;
+            const int s = row_base + (((chunk0 + q) ^ swz) << 2);
+            const float4 r4 = *reinterpret_cast<const float4*>(buf.r + s);
+            const float4 v4 = *reinterpret_cast<const float4*>(buf.v + s);
+            const float rr[4] = {r4.x, r4.y, r4.z, r4.w};
+            const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+            for (int e = 3; e >= 0; --e) {
+                const float x = fmaf(a.c1, vn, rr[e]);
+                bG = fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, x));
+                bR = fmaf(a.gamma_f, bR, rr[e]);
+                vn = vv[e];
             }
+        }
+        f = Affine2{a.gl_run, double(bG), a.gamma_run, double(bR)};
+    } else {
+        float bG = 0.f, bR = 0.f;
+        double aG = 1.0, aR = 1.0;
+        int i = i_start;
+        for (int k = kScanItems - 1; k >= 0; --k) {
+            const PosTerm t = egae_position(a, buf, t0, n_tile, win_lo, win_smem, l0 + k, i, bad);
+            if (t.cont) {
+                bG = fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, t.x));
+                bR = fmaf(a.gamma_f, bR, t.r);
+                aG *= a.gl;
+                aR *= a.gamma;
+            } else {
+                bG = t.x;
+                bR = t.r;
+                aG = 0.0;
+                aR = 0.0;
+            }
+        }
+        f = Affine2{aG, double(bG), aR, double(bR)};
+    }
+
+    // ---- inclusive suffix composition inside the warp: S_l = f_l o f_{l+1} o ... o f_31 ----------
+    Affine2 S = f;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const Affine2 o = shfl_down(S, d);
+        if (lane + d < 32) S = compose(S, o);
+    }
+    Affine2 excl = shfl_down(S, 1);   // composite of the lanes to the right
+    if (lane == 31) excl = identity2();
+    if (lane == 0) s_warp[warp] = S;
+    __syncthreads();                                                      // (A)
+
+    // ---- tile composite, look-back, per-warp carries (warp 0) ------------------------------------
+    if (warp == 0) {
+        // lane w < 4 holds warp w's composite; suffix-compose them, so that lane w ends with
+        // W_w o ... o W_3 and lane 0 with the tile's composite
+        Affine2 W = lane < kScanWarps ? s_warp[lane] : identity2();
+#pragma unroll
+        for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
+        Affine2 right = shfl_down(W, 1);            // composite of the warps to the right
+        if (lane >= kScanWarps - 1) right = identity2();
+        TileState* st = a.state;
+        if (lane == 0 && tile + 1 < a.num_tiles) {
+            st_pair(st[tile].aggA, W.aA, W.bA);
+            st_pair(st[tile].aggR, W.aR, W.bR);
+        }
+        double xA = 0.0, xR = 0.0;
+        const bool ok = egae_look_back(a, tile + 1, lane, xA, xR);
+        if (lane == 0) {
+            if (!ok) { atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
+            st_pair(st[tile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
+        }
+        xA = __shfl_sync(0xffffffffu, xA, 0);
+        xR = __shfl_sync(0xffffffffu, xR, 0);
+        if (lane < kScanWarps) {
+            s_carry[lane][0] = fma(right.aA, xA, right.bA);
+            s_carry[lane][1] = fma(right.aR, xR, right.bR);
+        }
+    }
+    __syncthreads();                                                      // (B)
+
+    // ---- replay the thread's positions from the true incoming values, store -----------------------
+    float G = float(fma(excl.aA, s_carry[warp][0], excl.bA));
+    float R = float(fma(excl.aR, s_carry[warp][1], excl.bR));
+    const bool full = a.vec_ok && l0 + kScanItems <= n_tile;
+    if (fast) {
+        float vn = v_right;
+#pragma unroll
+        for (int q = kScanItems / 4 - 1; q >= 0; --q) {
+            const int s = row_base + (((chunk0 + q) ^ swz) << 2);
+            const float4 r4 = *reinterpret_cast<const float4*>(buf.r + s);
+            const float4 v4 = *reinterpret_cast<const float4*>(buf.v + s);
+            const float rr[4] = {r4.x, r4.y, r4.z, r4.w};
+            const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
             float oa[4], og[4];
 #pragma unroll
             for (int e = 3; e >= 0; --e) {
-                const int k = 4 * q + e;
-                const bool c = (cont >> k) & 1u;
-                const double dr = ((inside >> k) & 1u) ? double(rr[e]) : 0.0;
-                A = c ? fma(a.gl, A, delta[k]) : delta[k];
-                G = c ? fma(a.gamma, G, dr) : dr;
-                oa[e] = float(A);
-                og[e] = float(G);
+                const float x = fmaf(a.c1, vn, rr[e]);
+                G = fmaf(a.gl_hi, G, fmaf(a.gl_lo, G, x));
+                R = fmaf(a.gamma_f, R, rr[e]);
+                vn = vv[e];
+                oa[e] = G - vn;
+                og[e] = R;
             }
             if (full) {
                 *reinterpret_cast<float4*>(a.adv + t0 + l0 + 4 * q) = make_float4(oa[0], oa[1], oa[2], oa[3]);
@@ -480,25 +500,54 @@ __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm) egae_scan_kernel
             } else {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    if (l0 + 4 * q + e < n_tile) {
-                        a.adv[t0 + l0 + 4 * q + e] = oa[e];
-                        if (a.ret) a.ret[t0 + l0 + 4 * q + e] = og[e];
-                    }
+                    a.adv[t0 + l0 + 4 * q + e] = oa[e];
+                    if (a.ret) a.ret[t0 + l0 + 4 * q + e] = og[e];
                 }
             }
         }
-        if (!has_next) break;
-        cp_async_wait_all();
-        __syncthreads();                                                      // (D)
-        ticket = next_ticket;
+    } else {
+        int i = i_start;
+        for (int k = kScanItems - 1; k >= 0; --k) {
+            const int l = l0 + k;
+            const PosTerm t = egae_position(a, buf, t0, n_tile, win_lo, win_smem, l, i, bad);
+            G = t.cont ? fmaf(a.gl_hi, G, fmaf(a.gl_lo, G, t.x)) : t.x;
+            R = t.cont ? fmaf(a.gamma_f, R, t.r) : t.r;
+            if (l < n_tile) {
+                a.adv[t0 + l] = t.inside ? G - t.v : 0.f;
+                if (a.ret) a.ret[t0 + l] = R;
+            }
+        }
     }
     if (bad) atomicOr(a.status, TPPO_DEV_BAD_SEGMENT);
 }
 
-// persistent grid: as many CTAs as can be resident, fewer when there are fewer tiles
-static inline int egae_grid(int num_tiles) {
-    const int resident = kNumSms * kScanCtasPerSm;
-    return num_tiles < resident ? num_tiles : resident;
+bool make_f32_rows_tensor_map(CUtensorMap* map, const void* base, uint64_t rows);
+
+// Fills the constants derived from gamma and lambda and the tensor maps, then launches one CTA per
+// tile.  The caller has set the pointers, sizes, state and ticket.
+static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
+    a.num_tiles = int32_t((int64_t(a.N) + kScanTile - 1) / kScanTile);
+    a.gamma = double(gamma);
+    a.gl = double(gamma) * double(lambda);
+    a.gamma_run = 1.0; a.gl_run = 1.0;
+    for (int k = 0; k < kScanItems; ++k) { a.gamma_run *= a.gamma; a.gl_run *= a.gl; }
+    a.gamma_f = gamma;
+    a.gl_hi = float(a.gl);
+    a.gl_lo = float(a.gl - double(a.gl_hi));
+    a.c1 = float(double(gamma) * (1.0 - double(lambda)));
+    a.vec_ok = aligned(a.rewards, 16) && aligned(a.values, 16) && aligned(a.adv, 16) &&
+               (!a.ret || aligned(a.ret, 16));
+    CUtensorMap map_r, map_v;
+    memset(&map_r, 0, sizeof(map_r));
+    memset(&map_v, 0, sizeof(map_v));
+    // whole tiles exist only from 2048 positions on; without the driver's encoder (or with
+    // unaligned arrays) every tile takes the plain-load path
+    a.tma_ok = a.vec_ok && a.N >= kScanTile &&
+               make_f32_rows_tensor_map(&map_r, a.rewards, uint64_t(a.N) / kRowPos) &&
+               make_f32_rows_tensor_map(&map_v, a.values, uint64_t(a.N) / kRowPos);
+    egae_scan_kernel<<<a.num_tiles, kScanThreads, 0, s>>>(a, map_r, map_v);
+    TPPO_CUDA_CHECK(cudaGetLastError());
+    return TPPO_OK;
 }
 
 size_t egae_workspace_bytes(int64_t N) {
@@ -529,23 +578,14 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
     if (N == 0) return TPPO_OK;
     // one memset: tile states start out unset (all-ones), the ticket counter at all-ones too
     TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0xff, need, s));
-    EgaeArgs a;
+    EgaeArgs a{};
     a.rewards = rewards; a.values = values; a.seg_begin = seg_begin; a.seg_end = seg_end;
     a.truncated = truncated; a.bootstrap = bootstrap; a.B = B; a.N = int32_t(N);
-    a.num_tiles = int32_t((N + kScanTile - 1) / kScanTile);
-    a.gamma = double(gamma);
-    a.gl = double(gamma) * double(lambda);
-    a.gamma_run = 1.0; a.gl_run = 1.0;
-    for (int k = 0; k < kScanItems; ++k) { a.gamma_run *= a.gamma; a.gl_run *= a.gl; }
     a.adv = advantages; a.ret = returns; a.status = status;
-    a.vec_ok = aligned(rewards, 16) && aligned(values, 16) && aligned(advantages, 16) &&
-               (!returns || aligned(returns, 16));
     a.ticket = static_cast<uint32_t*>(workspace);
     a.state = reinterpret_cast<TileState*>(static_cast<char*>(workspace) +
                                            align_up(sizeof(uint32_t), kWsAlign));
-    egae_scan_kernel<<<egae_grid(a.num_tiles), kScanThreads, 0, s>>>(a);
-    TPPO_CUDA_CHECK(cudaGetLastError());
-    return TPPO_OK;
+    return egae_launch(a, gamma, lambda, s);
 }
 
 // ---- allocation-free variant ------------------------------------------------------------------
@@ -599,23 +639,15 @@ TPPO_API int tppo_egae_static(const float* rewards, const float* values, const i
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
     if (N == 0) return TPPO_OK;
-    EgaeArgs a;
+    EgaeArgs a{};
     a.rewards = rewards; a.values = values; a.seg_begin = seg_begin; a.seg_end = seg_end;
     a.truncated = truncated; a.bootstrap = bootstrap; a.B = B; a.N = int32_t(N);
-    a.num_tiles = int32_t((N + kScanTile - 1) / kScanTile);
-    a.gamma = double(gamma);
-    a.gl = double(gamma) * double(lambda);
-    a.gamma_run = 1.0; a.gl_run = 1.0;
-    for (int k = 0; k < kScanItems; ++k) { a.gamma_run *= a.gamma; a.gl_run *= a.gl; }
     a.adv = advantages; a.ret = returns; a.status = status;
-    a.vec_ok = aligned(rewards, 16) && aligned(values, 16) && aligned(advantages, 16) &&
-               (!returns || aligned(returns, 16));
     a.ticket = static_cast<uint32_t*>(scratch);
     a.state = reinterpret_cast<TileState*>(static_cast<char*>(scratch) + 256);
     // the array still holds the previous call's tile states and ticket: reset the part this call
     // uses to the all-ones pattern (tile states unset, ticket counter one draw before ticket 0)
-    TPPO_CUDA_CHECK(cudaMemsetAsync(scratch, 0xff, 256 + size_t(a.num_tiles) * sizeof(TileState), s));
-    egae_scan_kernel<<<egae_grid(a.num_tiles), kScanThreads, 0, s>>>(a);
-    TPPO_CUDA_CHECK(cudaGetLastError());
-    return TPPO_OK;
+    const size_t tiles = size_t((N + kScanTile - 1) / kScanTile);
+    TPPO_CUDA_CHECK(cudaMemsetAsync(scratch, 0xff, 256 + tiles * sizeof(TileState), s));
+    return egae_launch(a, gamma, lambda, s);
 }

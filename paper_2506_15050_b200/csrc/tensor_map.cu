@@ -38,4 +38,18 @@ bool make_bf16_tensor_map(CUtensorMap* map, const void* base, uint64_t rows, uin
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 array viewed as rows of 32 elements (128 bytes); a box is 64 rows, written with the 128-byte
+// swizzle.  `rows` counts whole rows only.
+bool make_f32_rows_tensor_map(CUtensorMap* map, const void* base, uint64_t rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || rows < 64) return false;
+    const cuuint64_t dims[2] = {32, rows};
+    const cuuint64_t strides[1] = {128};
+    const cuuint32_t box[2] = {32, 64};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace tppo
