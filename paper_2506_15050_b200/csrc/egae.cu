@@ -15,15 +15,14 @@
 // rounded to fp32 once.  The rounding error of a result is a few units of 2^-24 of the largest
 // |G| or |R| in its run; nothing accumulates over the length of a segment.
 //
-// One CTA per tile of 2048 positions, tiles taken by ticket from the END of the arrays backwards,
-// so the tiles a tile looks back at (those to its right) hold earlier tickets and are running or
-// done.  A tile composes its positions right to left, publishes the composite, and obtains the
-// value entering from its right-hand neighbour by decoupled look-back over the tiles behind it.  A
-// composite whose `a` has become 0 (a segment ended inside the range) ends the look-back early.
-// The inputs of a whole tile arrive by two tiled TMA copies (rows of 32 positions, 128-byte
-// swizzle: the four 16-byte chunks a thread owns then sit in different bank groups from its
-// neighbours'); there is no per-thread staging code.  Latencies (ticket, copy, window search,
-// look-back) are covered by the other CTAs resident on the SM rather than by software pipelining.
+// Tiles of 2048 positions are taken by ticket from the END of the arrays backwards, so the tiles a
+// tile looks back at (those to its right) hold earlier tickets and are running or done.  A tile
+// composes its positions right to left, publishes the composite, and obtains the value entering
+// from its right-hand neighbour by decoupled look-back over the tiles behind it.  A composite whose
+// `a` has become 0 (a segment ended inside the range) ends the look-back early.  The inputs of a
+// whole tile arrive by two tiled TMA copies (rows of 32 positions, 128-byte swizzle: the four
+// 16-byte chunks a thread owns then sit in different bank groups from its neighbours'); there is no
+// per-thread staging code.
 #include <cstddef>
 #include <cstring>
 
@@ -40,7 +39,7 @@ constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kScanItems = 16;
 constexpr int kScanTile = kScanThreads * kScanItems;  // 2048 positions
 constexpr int kSegCap = 32;                           // segments of one tile kept in shared memory
-constexpr int kScanCtasPerSm = 8;
+constexpr int kScanCtasPerSm = 6;
 constexpr uint32_t kScanSpinLimit = 1u << 22;
 
 struct Affine2 {  // x -> (aA*xA + bA, aR*xR + bR)
@@ -118,38 +117,6 @@ struct EgaeArgs {
     uint32_t* ticket;
 };
 
-// Number of entries of the ascending array arr[0..n) that are <= key, found by a whole warp: each
-// round probes 32 evenly spaced entries until at most 128 remain, which are then read in one go
-// (four independent loads per lane), so 4096 entries take two dependent rounds instead of twelve
-// dependent loads.  Every lane returns the same count.  An array that is not ascending still
-// yields an in-range answer.
-__device__ __forceinline__ int warp_count_le(const int32_t* __restrict__ arr, int n, int32_t key,
-                                             int lane) {
-    int lo = 0, hi = n;       // the answer lies in [lo, hi]
-    while (hi - lo > 128) {
-        const int span = hi - lo;
-        const int step = (span + 31) >> 5;
-        const int idx = lo + lane * step;
-        const bool le = idx < hi && __ldg(arr + idx) <= key;
-        const uint32_t m = __ballot_sync(0xffffffffu, le);
-        const int c = __ffs(int(~m)) - 1;          // leading run of probes that are <= key
-        if (c < 0) { lo = min(lo + 31 * step + 1, hi); continue; }   // all 32 probes <= key
-        const int new_hi = min(lo + c * step, hi);
-        if (c > 0) lo = lo + (c - 1) * step + 1;
-        hi = new_hi;
-    }
-    bool le[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int idx = lo + 32 * j + lane;
-        le[j] = idx < hi && __ldg(arr + idx) <= key;
-    }
-    int count = 0;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) count += __popc(__ballot_sync(0xffffffffu, le[j]));
-    return lo + count;
-}
-
 // Shared-memory image of one tile.  r and v are 64 rows of 32 positions (128 bytes) in the layout
 // the TMA's 128-byte swizzle writes: 16-byte chunk c of row y sits at chunk c ^ (y & 7) of that row
 // (the arrays are 1024-byte aligned, eight rows).  A thread owns half a row; the eight lanes of a
@@ -158,48 +125,20 @@ constexpr int kRowPos = 32;
 struct __align__(1024) TileBuf {
     float r[kScanTile];          // rewards
     float v[kScanTile];          // values
+    float v_after;               // value of the position after the tile (0 beyond the arrays)
+};
+// The segments that can touch a tile (its window), copied next to it when they are few.
+struct TileWin {
     int32_t seg_b[kSegCap], seg_e[kSegCap];
     float seg_boot[kSegCap];
     uint8_t seg_t[kSegCap];
-    float v_after;               // value of the position after the tile (0 beyond the arrays)
     int win_lo, win_hi;          // segment indices [win_lo, win_hi) may touch the tile
+    int tile;                    // the tile itself, -1: there are no more tiles
 };
 static_assert(offsetof(TileBuf, v) % 1024 == 0, "swizzle atom alignment");
 __device__ __forceinline__ int pos_slot(int l) {      // float index of position l
     const int y = l >> 5;
     return (y << 5) | (((((l >> 2) & 7) ^ (y & 7)) << 2)) | (l & 3);
-}
-
-// Segments are ascending and disjoint, so seg_begin and seg_end are both ascending: the window of
-// a tile starts after the segments that end at or before its first position and stops before those
-// that begin after its last one.  Called by two whole warps (which = 0: lower end, 1: upper end).
-__device__ __forceinline__ void egae_window_search(const EgaeArgs& a, TileBuf& buf, int64_t t0,
-                                                   int n_tile, int which, int lane) {
-    if (which == 0) {
-        const int lo = warp_count_le(a.seg_end, a.B, int32_t(t0), lane);
-        if (lane == 0) buf.win_lo = lo;
-    } else {
-        const int hi = warp_count_le(a.seg_begin, a.B, int32_t(t0 + n_tile - 1), lane);
-        if (lane == 0) buf.win_hi = hi;
-    }
-}
-// Copies the window's segments into shared memory (when they fit).  Returns true when a segment
-// with bounds outside [0, N] or end < begin was seen; such a segment is treated as empty.
-__device__ __forceinline__ bool egae_window_load(const EgaeArgs& a, TileBuf& buf) {
-    const int win_lo = buf.win_lo, win_n = buf.win_hi - buf.win_lo;
-    bool bad = false;
-    if (win_n <= kSegCap) {
-        for (int j = threadIdx.x; j < win_n; j += kScanThreads) {
-            const int i = win_lo + j;
-            int32_t b = __ldg(a.seg_begin + i), e = __ldg(a.seg_end + i);
-            if (b < 0 || e > a.N || e < b) { bad = true; e = b; }
-            buf.seg_b[j] = b;
-            buf.seg_e[j] = e;
-            buf.seg_t[j] = __ldg(a.truncated + i);
-            buf.seg_boot[j] = a.bootstrap ? __ldg(a.bootstrap + i) : 0.f;
-        }
-    }
-    return bad;
 }
 
 // What one position contributes, for threads that touch a segment boundary or lie outside every
@@ -211,7 +150,8 @@ struct PosTerm {
     float x, r, v;
     bool cont, inside;
 };
-__device__ __forceinline__ PosTerm egae_position(const EgaeArgs& a, const TileBuf& buf, int64_t t0,
+__device__ __forceinline__ PosTerm egae_position(const EgaeArgs& a, const TileBuf& buf,
+                                                 const TileWin& win, int64_t t0,
                                                  int n_tile, int win_lo, bool win_smem, int l, int& i,
                                                  bool& bad) {
     PosTerm o{0.f, 0.f, 0.f, false, false};
@@ -221,8 +161,8 @@ __device__ __forceinline__ PosTerm egae_position(const EgaeArgs& a, const TileBu
     bool have = false;
     while (i >= 0) {
         if (win_smem) {
-            b = buf.seg_b[i];
-            e = buf.seg_e[i];
+            b = win.seg_b[i];
+            e = win.seg_e[i];
         } else {
             b = __ldg(a.seg_begin + win_lo + i);
             e = __ldg(a.seg_end + win_lo + i);
@@ -240,9 +180,9 @@ __device__ __forceinline__ PosTerm egae_position(const EgaeArgs& a, const TileBu
         o.x = fmaf(a.c1, v_next, o.r);
         o.cont = true;
     } else {      // last token: G = r + gamma * (0 | bootstrap value | its own value)
-        const bool tr = win_smem ? (buf.seg_t[i] != 0) : (__ldg(a.truncated + win_lo + i) != 0);
+        const bool tr = win_smem ? (win.seg_t[i] != 0) : (__ldg(a.truncated + win_lo + i) != 0);
         float v_next = 0.f;
-        if (tr) v_next = a.bootstrap ? (win_smem ? buf.seg_boot[i] : __ldg(a.bootstrap + win_lo + i)) : o.v;
+        if (tr) v_next = a.bootstrap ? (win_smem ? win.seg_boot[i] : __ldg(a.bootstrap + win_lo + i)) : o.v;
         o.x = fmaf(a.gamma_f, v_next, o.r);
     }
     return o;
@@ -303,74 +243,122 @@ __device__ __forceinline__ bool egae_look_back(const EgaeArgs& a, int first, int
     }
 }
 
-__global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm)
-egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
-                 const __grid_constant__ CUtensorMap map_v) {
-    __shared__ TileBuf buf;
-    __shared__ __align__(8) uint64_t s_bar;      // the tile's inputs have arrived
-    __shared__ uint32_t s_ticket;
-    __shared__ Affine2 s_warp[kScanWarps];
-    __shared__ double s_carry[kScanWarps][2];
-
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t bar = ptx::smem_addr(&s_bar);
-    if (threadIdx.x == 0) {
-        // the ticket counter starts at all-ones like the rest of the workspace (one memset): + 1
-        // wraps the first draw to ticket 0
-        s_ticket = atomicAdd(a.ticket, 1u) + 1u;
-        ptx::mbar_init(bar, 1);
-        ptx::fence_mbar_init_cluster();
-    }
-    __syncthreads();
-    const uint32_t ticket = s_ticket;
-    if (ticket >= uint32_t(a.num_tiles)) return;       // (the grid has exactly num_tiles CTAs)
-    const int tile = a.num_tiles - 1 - int(ticket);
-    const int64_t t0 = int64_t(tile) * kScanTile;
-    const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
-    const bool by_tma = a.tma_ok && n_tile == kScanTile;
-
-    // ---- inputs: two TMA copies for a whole tile, plain loads for a ragged or unaligned one ------
-    if (by_tma) {
-        if (threadIdx.x == 0) {
-            ptx::mbar_arrive_expect_tx(bar, 2 * kScanTile * uint32_t(sizeof(float)));
-            umma::tma_load_2d(ptx::smem_addr(buf.r), &map_r, bar, 0, int32_t(t0 / kRowPos));
-            umma::tma_load_2d(ptx::smem_addr(buf.v), &map_v, bar, 0, int32_t(t0 / kRowPos));
+// Number of entries of an ascending array arr[0..n) that are <= key, found by a whole warp: each
+// round probes 32 evenly spaced entries until at most 128 remain, which are then read in one go
+// (four independent loads per lane), so 4096 entries take two dependent rounds instead of twelve
+// dependent loads.  Every lane returns the same count; an array that is not ascending still yields
+// an in-range answer.  Two counts at once (the two ends of a tile's segment window), the rounds of
+// both searches overlapped so that their loads are in flight together.
+__device__ __forceinline__ void warp_count_le2(const int32_t* __restrict__ arr1, int32_t key1,
+                                               const int32_t* __restrict__ arr2, int32_t key2, int n,
+                                               int lane, int& c1, int& c2) {
+    int lo1 = 0, hi1 = n, lo2 = 0, hi2 = n;
+    while (hi1 - lo1 > 128 || hi2 - lo2 > 128) {
+        const bool go1 = hi1 - lo1 > 128, go2 = hi2 - lo2 > 128;
+        const int step1 = (hi1 - lo1 + 31) >> 5, step2 = (hi2 - lo2 + 31) >> 5;
+        const int idx1 = lo1 + lane * step1, idx2 = lo2 + lane * step2;
+        const int32_t x1 = go1 && idx1 < hi1 ? __ldg(arr1 + idx1) : INT32_MAX;
+        const int32_t x2 = go2 && idx2 < hi2 ? __ldg(arr2 + idx2) : INT32_MAX;
+        const uint32_t m1 = __ballot_sync(0xffffffffu, go1 && idx1 < hi1 && x1 <= key1);
+        const uint32_t m2 = __ballot_sync(0xffffffffu, go2 && idx2 < hi2 && x2 <= key2);
+        if (go1) {
+            const int c = __ffs(int(~m1)) - 1;      // leading run of probes that are <= key
+            if (c < 0) {
+                lo1 = min(lo1 + 31 * step1 + 1, hi1);
+            } else {
+                const int new_hi = min(lo1 + c * step1, hi1);
+                if (c > 0) lo1 = lo1 + (c - 1) * step1 + 1;
+                hi1 = new_hi;
+            }
         }
-    } else {
-        for (int k = threadIdx.x; k < n_tile; k += kScanThreads) {
-            buf.r[pos_slot(k)] = __ldg(a.rewards + t0 + k);
-            buf.v[pos_slot(k)] = __ldg(a.values + t0 + k);
+        if (go2) {
+            const int c = __ffs(int(~m2)) - 1;
+            if (c < 0) {
+                lo2 = min(lo2 + 31 * step2 + 1, hi2);
+            } else {
+                const int new_hi = min(lo2 + c * step2, hi2);
+                if (c > 0) lo2 = lo2 + (c - 1) * step2 + 1;
+                hi2 = new_hi;
+            }
         }
     }
-    if (threadIdx.x == kScanThreads - 1)
-        buf.v_after = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
-    if (warp < 2) egae_window_search(a, buf, t0, n_tile, warp, lane);
-    __syncthreads();
-    bool bad = egae_window_load(a, buf);
-    if (by_tma && !ptx::mbar_wait<false>(bar, 0)) atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT);
-    __syncthreads();
+    bool le1[4], le2[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int i1 = lo1 + 32 * j + lane, i2 = lo2 + 32 * j + lane;
+        le1[j] = i1 < hi1 && __ldg(arr1 + i1) <= key1;
+        le2[j] = i2 < hi2 && __ldg(arr2 + i2) <= key2;
+    }
+    c1 = lo1;
+    c2 = lo2;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        c1 += __popc(__ballot_sync(0xffffffffu, le1[j]));
+        c2 += __popc(__ballot_sync(0xffffffffu, le2[j]));
+    }
+}
 
-    // ---- the thread's sixteen positions, right to left: its composite map -------------------------
-    const int win_lo = buf.win_lo;
-    const int win_n = max(buf.win_hi - win_lo, 0);
+// The segment window of a tile, found and copied into shared memory by one warp.  Returns true when
+// a segment with bounds outside [0, N] or end < begin was seen; such a segment is treated as empty.
+static_assert(kSegCap == 32, "one lane per window segment");
+__device__ __forceinline__ bool egae_window(const EgaeArgs& a, TileWin& win, int64_t t0, int n_tile,
+                                            int lane) {
+    // segments are ascending and disjoint, so seg_begin and seg_end are both ascending: the window
+    // starts after the segments that end at or before the tile's first position and stops before
+    // those that begin after its last one
+    int lo, hi;
+    warp_count_le2(a.seg_end, int32_t(t0), a.seg_begin, int32_t(t0 + n_tile - 1), a.B, lane, lo, hi);
+    if (lane == 0) { win.win_lo = lo; win.win_hi = hi; }
+    bool bad = false;
+    if (hi - lo <= kSegCap && lane < hi - lo) {
+        const int i = lo + lane;
+        int32_t b = __ldg(a.seg_begin + i), e = __ldg(a.seg_end + i);
+        if (b < 0 || e > a.N || e < b) { bad = true; e = b; }
+        win.seg_b[lane] = b;
+        win.seg_e[lane] = e;
+        win.seg_t[lane] = __ldg(a.truncated + i);
+        win.seg_boot[lane] = a.bootstrap ? __ldg(a.bootstrap + i) : 0.f;
+    }
+    return bad;
+}
+
+// What a compute thread keeps of a tile between composing its maps and replaying them.
+struct RunState {
+    Affine2 excl;     // composite of the lanes to its right inside the warp
+    int i_start;      // window index of the last segment that begins at or before its last position
+    bool fast;        // its sixteen positions lie inside one segment, none of them the last token
+    // Otherwise, when at most one segment ends inside the run (`masked`): which positions lie inside
+    // a segment (bits 0-15), which of them continue into the next position (bits 16-31), and for the
+    // one last token, its position (or -1) and the value its TD residual bootstraps from
+    bool masked;
+    uint32_t bits;
+    int k_last;
+    float v_boundary;
+    bool boundary_own;   // the boundary value is the last token's own value (no bootstrap array)
+};
+
+// The thread's sixteen positions, right to left: its composite map.
+__device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, const TileBuf& buf,
+                                                const TileWin& win, int64_t t0,
+                                                int n_tile, int tid, RunState& rs, bool& bad) {
+    const int win_lo = win.win_lo;
+    const int win_n = max(win.win_hi - win_lo, 0);
     const bool win_smem = win_n <= kSegCap;
-    const int l0 = threadIdx.x * kScanItems;        // first position of this thread inside the tile
+    const int l0 = tid * kScanItems;        // first position of this thread inside the tile
     // its four chunks: row tid/2, chunks 4*(tid&1) + q, stored at chunk ^ (row & 7)
-    const int row_base = (threadIdx.x >> 1) << 5;
-    const int chunk0 = (threadIdx.x & 1) << 2, swz = (threadIdx.x >> 1) & 7;
-    // index (inside the window) of the last segment that begins at or before the thread's last
-    // position, or -1
+    const int row_base = (tid >> 1) << 5;
+    const int chunk0 = (tid & 1) << 2, swz = (tid >> 1) & 7;
     const int l_last = min(l0 + kScanItems, n_tile) - 1;
     int i_start = -1;
     if (l_last >= l0) {
         const int32_t key = int32_t(t0 + l_last);
         int lo = 0, hi = win_n;
         if (win_smem && win_n <= 4) {
-            while (lo < win_n && buf.seg_b[lo] <= key) ++lo;
+            while (lo < win_n && win.seg_b[lo] <= key) ++lo;
         } else if (win_smem) {
             while (lo < hi) {
                 const int mid = (lo + hi) >> 1;
-                if (buf.seg_b[mid] <= key) lo = mid + 1; else hi = mid;
+                if (win.seg_b[mid] <= key) lo = mid + 1; else hi = mid;
             }
         } else {
             while (lo < hi) {
@@ -380,18 +368,78 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
         }
         i_start = lo - 1;
     }
-    // The common case: all sixteen positions lie inside one segment and none of them is its last
-    // token.  Then every map has the same multiplier and no per-position test is needed.
     bool fast = false;
     if (win_smem && i_start >= 0 && l0 + kScanItems <= n_tile)
-        fast = int64_t(buf.seg_b[i_start]) <= t0 + l0 &&
-               t0 + l0 + kScanItems < int64_t(buf.seg_e[i_start]);
-    // value of the position after the thread's run (only the fast path uses it: the run then
-    // continues into that position)
+        fast = int64_t(win.seg_b[i_start]) <= t0 + l0 &&
+               t0 + l0 + kScanItems < int64_t(win.seg_e[i_start]);
+    rs.i_start = i_start;
+    rs.fast = fast;
+    rs.masked = false;
     const float v_right = l0 + kScanItems < kScanTile ? buf.v[pos_slot(l0 + kScanItems)] : buf.v_after;
-    Affine2 f;
-    if (fast) {
+    if (!fast && win_smem) {
+        // The segments that overlap the run, from the right: usually one or two.  With at most one
+        // segment end inside the run the per-position work stays branch-free (two bit masks and one
+        // special position); runs that hold several tiny segments take the general loop below.
+        const int64_t p0 = t0 + l0;
+        uint32_t inside = 0, cont = 0;
+        int n_last = 0;
+        rs.k_last = -1;
+        rs.v_boundary = 0.f;
+        rs.boundary_own = false;
+        for (int i = i_start; i >= 0; --i) {
+            const int64_t b = win.seg_b[i], e = win.seg_e[i];
+            if (e <= p0 && e > b) break;      // ascending and disjoint: the earlier ones end earlier still
+            const int lo = int(max(b, p0) - p0), hi = int(min(e, p0 + kScanItems) - p0);
+            if (hi <= lo) continue;
+            const uint32_t m = ((1u << hi) - 1u) & ~((1u << lo) - 1u);
+            inside |= m;
+            cont |= m;
+            if (e <= p0 + kScanItems) {       // the segment's last token lies in the run
+                const int k = int(e - 1 - p0);
+                cont &= ~(1u << k);
+                ++n_last;
+                rs.k_last = k;
+                rs.v_boundary = 0.f;
+                rs.boundary_own = false;
+                if (win.seg_t[i]) {
+                    if (a.bootstrap) rs.v_boundary = win.seg_boot[i];
+                    else rs.boundary_own = true;
+                }
+            }
+        }
+        rs.bits = inside | (cont << 16);
+        rs.masked = n_last <= 1;
+    }
+    if (rs.masked) {
+        const uint32_t inside = rs.bits & 0xffffu, cont = rs.bits >> 16;
         float bG = 0.f, bR = 0.f, vn = v_right;
+#pragma unroll
+        for (int q = kScanItems / 4 - 1; q >= 0; --q) {
+            const int s = row_base + (((chunk0 + q) ^ swz) << 2);
+            const float4 r4 = *reinterpret_cast<const float4*>(buf.r + s);
+            const float4 v4 = *reinterpret_cast<const float4*>(buf.v + s);
+            const float rr[4] = {r4.x, r4.y, r4.z, r4.w};
+            const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+            for (int e = 3; e >= 0; --e) {
+                const int k = 4 * q + e;
+                const bool in = (inside >> k) & 1u, c = (cont >> k) & 1u;
+                float x = fmaf(a.c1, vn, rr[e]);
+                if (k == rs.k_last) x = fmaf(a.gamma_f, rs.boundary_own ? vv[e] : rs.v_boundary, rr[e]);
+                x = in ? x : 0.f;
+                const float re = in ? rr[e] : 0.f;
+                bG = c ? fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, x)) : x;
+                bR = c ? fmaf(a.gamma_f, bR, re) : re;
+                vn = vv[e];
+            }
+        }
+        const bool whole = cont == 0xffffu;
+        return Affine2{whole ? a.gl_run : 0.0, double(bG), whole ? a.gamma_run : 0.0, double(bR)};
+    }
+    if (fast) {
+        // every map has the same multiplier and no per-position test is needed
+        float bG = 0.f, bR = 0.f;
+        float vn = v_right;
 #pragma unroll
         for (int q = kScanItems / 4 - 1; q >= 0; --q) {
             const int s = row_base + (((chunk0 + q) ^ swz) << 2);
@@ -407,75 +455,38 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
                 vn = vv[e];
             }
         }
-        f = Affine2{a.gl_run, double(bG), a.gamma_run, double(bR)};
-    } else {
-        float bG = 0.f, bR = 0.f;
-        double aG = 1.0, aR = 1.0;
-        int i = i_start;
-        for (int k = kScanItems - 1; k >= 0; --k) {
-            const PosTerm t = egae_position(a, buf, t0, n_tile, win_lo, win_smem, l0 + k, i, bad);
-            if (t.cont) {
-                bG = fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, t.x));
-                bR = fmaf(a.gamma_f, bR, t.r);
-                aG *= a.gl;
-                aR *= a.gamma;
-            } else {
-                bG = t.x;
-                bR = t.r;
-                aG = 0.0;
-                aR = 0.0;
-            }
-        }
-        f = Affine2{aG, double(bG), aR, double(bR)};
+        return Affine2{a.gl_run, double(bG), a.gamma_run, double(bR)};
     }
-
-    // ---- inclusive suffix composition inside the warp: S_l = f_l o f_{l+1} o ... o f_31 ----------
-    Affine2 S = f;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const Affine2 o = shfl_down(S, d);
-        if (lane + d < 32) S = compose(S, o);
-    }
-    Affine2 excl = shfl_down(S, 1);   // composite of the lanes to the right
-    if (lane == 31) excl = identity2();
-    if (lane == 0) s_warp[warp] = S;
-    __syncthreads();                                                      // (A)
-
-    // ---- tile composite, look-back, per-warp carries (warp 0) ------------------------------------
-    if (warp == 0) {
-        // lane w < 4 holds warp w's composite; suffix-compose them, so that lane w ends with
-        // W_w o ... o W_3 and lane 0 with the tile's composite
-        Affine2 W = lane < kScanWarps ? s_warp[lane] : identity2();
-#pragma unroll
-        for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
-        Affine2 right = shfl_down(W, 1);            // composite of the warps to the right
-        if (lane >= kScanWarps - 1) right = identity2();
-        TileState* st = a.state;
-        if (lane == 0 && tile + 1 < a.num_tiles) {
-            st_pair(st[tile].aggA, W.aA, W.bA);
-            st_pair(st[tile].aggR, W.aR, W.bR);
-        }
-        double xA = 0.0, xR = 0.0;
-        const bool ok = egae_look_back(a, tile + 1, lane, xA, xR);
-        if (lane == 0) {
-            if (!ok) { atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
-            st_pair(st[tile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
-        }
-        xA = __shfl_sync(0xffffffffu, xA, 0);
-        xR = __shfl_sync(0xffffffffu, xR, 0);
-        if (lane < kScanWarps) {
-            s_carry[lane][0] = fma(right.aA, xA, right.bA);
-            s_carry[lane][1] = fma(right.aR, xR, right.bR);
+    float bG = 0.f, bR = 0.f;
+    double aG = 1.0, aR = 1.0;
+    int i = i_start;
+    for (int k = kScanItems - 1; k >= 0; --k) {
+        const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l0 + k, i, bad);
+        if (t.cont) {
+            bG = fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, t.x));
+            bR = fmaf(a.gamma_f, bR, t.r);
+            aG *= a.gl;
+            aR *= a.gamma;
+        } else {
+            bG = t.x;
+            bR = t.r;
+            aG = 0.0;
+            aR = 0.0;
         }
     }
-    __syncthreads();                                                      // (B)
+    return Affine2{aG, double(bG), aR, double(bR)};
+}
 
-    // ---- replay the thread's positions from the true incoming values, store -----------------------
-    float G = float(fma(excl.aA, s_carry[warp][0], excl.bA));
-    float R = float(fma(excl.aR, s_carry[warp][1], excl.bR));
-    const bool full = a.vec_ok && l0 + kScanItems <= n_tile;
-    if (fast) {
-        float vn = v_right;
+// Replays the thread's positions from the values entering its run and stores the results.
+__device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, const TileBuf& buf,
+                                                const TileWin& win, int64_t t0,
+                                                int n_tile, int tid, const RunState& rs, float G,
+                                                float R, bool& bad) {
+    const int l0 = tid * kScanItems;
+    if (rs.fast) {
+        const int row_base = (tid >> 1) << 5;
+        const int chunk0 = (tid & 1) << 2, swz = (tid >> 1) & 7;
+        float vn = l0 + kScanItems < kScanTile ? buf.v[pos_slot(l0 + kScanItems)] : buf.v_after;
 #pragma unroll
         for (int q = kScanItems / 4 - 1; q >= 0; --q) {
             const int s = row_base + (((chunk0 + q) ^ swz) << 2);
@@ -493,7 +504,7 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
                 oa[e] = G - vn;
                 og[e] = R;
             }
-            if (full) {
+            if (a.vec_ok) {
                 *reinterpret_cast<float4*>(a.adv + t0 + l0 + 4 * q) = make_float4(oa[0], oa[1], oa[2], oa[3]);
                 if (a.ret)
                     *reinterpret_cast<float4*>(a.ret + t0 + l0 + 4 * q) = make_float4(og[0], og[1], og[2], og[3]);
@@ -505,20 +516,259 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
                 }
             }
         }
-    } else {
-        int i = i_start;
-        for (int k = kScanItems - 1; k >= 0; --k) {
-            const int l = l0 + k;
-            const PosTerm t = egae_position(a, buf, t0, n_tile, win_lo, win_smem, l, i, bad);
-            G = t.cont ? fmaf(a.gl_hi, G, fmaf(a.gl_lo, G, t.x)) : t.x;
-            R = t.cont ? fmaf(a.gamma_f, R, t.r) : t.r;
-            if (l < n_tile) {
-                a.adv[t0 + l] = t.inside ? G - t.v : 0.f;
-                if (a.ret) a.ret[t0 + l] = R;
+        return;
+    }
+    if (rs.masked) {
+        const int row_base = (tid >> 1) << 5;
+        const int chunk0 = (tid & 1) << 2, swz = (tid >> 1) & 7;
+        const uint32_t inside = rs.bits & 0xffffu, cont = rs.bits >> 16;
+        const bool full = a.vec_ok && l0 + kScanItems <= n_tile;
+        float vn = l0 + kScanItems < kScanTile ? buf.v[pos_slot(l0 + kScanItems)] : buf.v_after;
+#pragma unroll
+        for (int q = kScanItems / 4 - 1; q >= 0; --q) {
+            const int s = row_base + (((chunk0 + q) ^ swz) << 2);
+            const float4 r4 = *reinterpret_cast<const float4*>(buf.r + s);
+            const float4 v4 = *reinterpret_cast<const float4*>(buf.v + s);
+            const float rr[4] = {r4.x, r4.y, r4.z, r4.w};
+            const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+            float oa[4], og[4];
+#pragma unroll
+            for (int e = 3; e >= 0; --e) {
+                const int k = 4 * q + e;
+                const bool in = (inside >> k) & 1u, c = (cont >> k) & 1u;
+                float x = fmaf(a.c1, vn, rr[e]);
+                if (k == rs.k_last) x = fmaf(a.gamma_f, rs.boundary_own ? vv[e] : rs.v_boundary, rr[e]);
+                x = in ? x : 0.f;
+                const float re = in ? rr[e] : 0.f;
+                G = c ? fmaf(a.gl_hi, G, fmaf(a.gl_lo, G, x)) : x;
+                R = c ? fmaf(a.gamma_f, R, re) : re;
+                vn = vv[e];
+                oa[e] = in ? G - vn : 0.f;
+                og[e] = R;
             }
+            if (full) {
+                *reinterpret_cast<float4*>(a.adv + t0 + l0 + 4 * q) = make_float4(oa[0], oa[1], oa[2], oa[3]);
+                if (a.ret)
+                    *reinterpret_cast<float4*>(a.ret + t0 + l0 + 4 * q) = make_float4(og[0], og[1], og[2], og[3]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (l0 + 4 * q + e < n_tile) {
+                        a.adv[t0 + l0 + 4 * q + e] = oa[e];
+                        if (a.ret) a.ret[t0 + l0 + 4 * q + e] = og[e];
+                    }
+                }
+            }
+        }
+        return;
+    }
+    const int win_lo = win.win_lo;
+    const bool win_smem = max(win.win_hi - win_lo, 0) <= kSegCap;
+    int i = rs.i_start;
+    for (int k = kScanItems - 1; k >= 0; --k) {
+        const int l = l0 + k;
+        const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l, i, bad);
+        G = t.cont ? fmaf(a.gl_hi, G, fmaf(a.gl_lo, G, t.x)) : t.x;
+        R = t.cont ? fmaf(a.gamma_f, R, t.r) : t.r;
+        if (l < n_tile) {
+            a.adv[t0 + l] = t.inside ? G - t.v : 0.f;
+            if (a.ret) a.ret[t0 + l] = R;
+        }
+    }
+}
+
+// Persistent CTAs of six warps; tiles are taken by ticket, from the END of the arrays backwards, so
+// the tiles a tile looks back at (those to its right) hold earlier tickets and are running or done.
+// Three roles run as independent loops and meet only at mbarriers:
+//   stager (warp 5):     ticket and segment window of tile m (a ring of four windows, so that the
+//                        search runs ahead of the buffers), then, once the replay of tile m-2 has
+//                        freed the buffer, the two TMA copies of tile m;
+//   compute (warps 0-3): step n = maps + warp scan of tile n, composite published at once (so no
+//                        other CTA waits for this CTA's look-back), then replay + stores of tile n-1;
+//   look-back (warp 4):  value entering tile n from the right, the tile's first-position values
+//                        published, the values entering each warp handed to the replay.
+// The look-back of tile n (L2 round trips, and a wait for the right-hand neighbours) thus runs while
+// the compute warps are on tile n+1.  Two input buffers; four mbarriers per buffer hand it from
+// stage to stage (inputs ready, scan done, carries ready, buffer free).  Every wait is bounded.
+constexpr int kLookWarp = kScanWarps, kStageWarp = kScanWarps + 1;
+constexpr int kCtaThreads = kScanThreads + 64;
+constexpr int kWinRing = 4;
+struct Pipe {
+    uint64_t full[2];     // inputs (and window) of the tile are there                 (stager -> compute)
+    uint64_t scan[2];     // the tile's composites are in s_right / s_tile_f            (compute -> look-back)
+    uint64_t carry[2];    // the values entering each warp are in s_carry              (look-back -> compute)
+    uint64_t free_[2];    // the replay has finished reading the buffer                (compute -> stager)
+};
+__device__ __forceinline__ void compute_warps_sync() {     // named barrier 1: the four compute warps
+    asm volatile("bar.sync 1, %0;" ::"n"(kScanThreads) : "memory");
+}
+
+__global__ void __launch_bounds__(kCtaThreads, kScanCtasPerSm)
+egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
+                 const __grid_constant__ CUtensorMap map_v) {
+    __shared__ TileBuf s_buf[2];
+    __shared__ TileWin s_win[kWinRing];
+    __shared__ __align__(8) Pipe s_pipe;
+    __shared__ Affine2 s_warp[2][kScanWarps];    // warp composites (compute warps only)
+    __shared__ Affine2 s_right[2][kScanWarps];   // composite of the warps to the right of each warp
+    __shared__ Affine2 s_tile_f[2];              // composite of the whole tile
+    __shared__ double s_carry[2][kScanWarps][2];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(ptx::smem_addr(&s_pipe.full[b]), 1);
+            ptx::mbar_init(ptx::smem_addr(&s_pipe.scan[b]), 1);
+            ptx::mbar_init(ptx::smem_addr(&s_pipe.carry[b]), 1);
+            ptx::mbar_init(ptx::smem_addr(&s_pipe.free_[b]), kScanWarps);
+        }
+        ptx::fence_mbar_init_cluster();
+    }
+    __syncthreads();
+    bool bad = false, late = false;      // a bad segment was seen; a bounded wait ran out
+
+    if (warp == kStageWarp) {
+        // =========================== stager ==========================================================
+        // the ticket counter starts at all-ones like the rest of the workspace (one memset): + 1
+        // wraps the first draw to ticket 0
+        uint32_t ticket = 0;
+        if (lane == 0) ticket = atomicAdd(a.ticket, 1u) + 1u;
+        for (int m = 0;; ++m) {
+            const int b = m & 1;
+            const uint32_t t = __shfl_sync(0xffffffffu, ticket, 0);
+            const int tile = t < uint32_t(a.num_tiles) ? a.num_tiles - 1 - int(t) : -1;
+            // draw the next ticket now: its round trip hides behind the window search
+            if (tile >= 0 && lane == 0) ticket = atomicAdd(a.ticket, 1u) + 1u;
+            // window slot m & 3 was last read by the replay of tile m-4, which finished before the
+            // replay of tile m-3 that the previous step waited for
+            TileWin& win = s_win[m & (kWinRing - 1)];
+            const int64_t t0 = int64_t(tile < 0 ? 0 : tile) * kScanTile;
+            const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
+            if (lane == 0) win.tile = tile;
+            if (tile >= 0) bad |= egae_window(a, win, t0, n_tile, lane);
+            const uint32_t full = ptx::smem_addr(&s_pipe.full[b]);
+            if (tile < 0) {
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(full);
+                break;
+            }
+            // the buffer was last used by tile m - 2: its replay must have finished
+            if (m >= 2) late |= !ptx::mbar_wait<false>(ptx::smem_addr(&s_pipe.free_[b]), uint32_t((m >> 1) - 1) & 1u);
+            TileBuf& buf = s_buf[b];
+            const bool by_tma = a.tma_ok && n_tile == kScanTile;
+            if (by_tma) {
+                if (lane == 0) {
+                    ptx::mbar_expect_tx(full, 2 * kScanTile * uint32_t(sizeof(float)));
+                    umma::tma_load_2d(ptx::smem_addr(buf.r), &map_r, full, 0, int32_t(t0 / kRowPos));
+                    umma::tma_load_2d(ptx::smem_addr(buf.v), &map_v, full, 0, int32_t(t0 / kRowPos));
+                }
+            } else {      // a ragged or unaligned tile: plain loads
+                for (int k = lane; k < n_tile; k += 32) {
+                    buf.r[pos_slot(k)] = __ldg(a.rewards + t0 + k);
+                    buf.v[pos_slot(k)] = __ldg(a.values + t0 + k);
+                }
+                ptx::fence_proxy_async_smem();    // a later TMA copy lands on the same bytes
+            }
+            if (lane == 0) buf.v_after = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(full);
+        }
+    } else if (warp == kLookWarp) {
+        // =========================== look-back =======================================================
+        for (int n = 0;; ++n) {
+            const int b = n & 1;
+            late |= !ptx::mbar_wait<false>(ptx::smem_addr(&s_pipe.scan[b]), uint32_t(n >> 1) & 1u);
+            const int tile = s_win[n & (kWinRing - 1)].tile;
+            if (tile < 0) break;
+            double xA = 0.0, xR = 0.0;
+            const bool ok = egae_look_back(a, tile + 1, lane, xA, xR);
+            if (lane == 0) {
+                if (!ok) { late = true; xA = 0.0; xR = 0.0; }
+                const Affine2 W = s_tile_f[b];
+                st_pair(a.state[tile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
+            }
+            xA = __shfl_sync(0xffffffffu, xA, 0);
+            xR = __shfl_sync(0xffffffffu, xR, 0);
+            if (lane < kScanWarps) {
+                const Affine2 right = s_right[b][lane];
+                s_carry[b][lane][0] = fma(right.aA, xA, right.bA);
+                s_carry[b][lane][1] = fma(right.aR, xR, right.bR);
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&s_pipe.carry[b]));
+        }
+    } else {
+        // =========================== compute warps ==================================================
+        RunState prev{};
+        int prev_tile = -1;
+        for (int n = 0;; ++n) {
+            const int b = n & 1;
+            late |= !ptx::mbar_wait<false>(ptx::smem_addr(&s_pipe.full[b]), uint32_t(n >> 1) & 1u);
+            const TileWin& win = s_win[n & (kWinRing - 1)];
+            const int tile = win.tile;
+            RunState cur{};
+            if (tile >= 0) {
+                const int64_t t0 = int64_t(tile) * kScanTile;
+                const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
+                const Affine2 f = egae_run_map(a, s_buf[b], win, t0, n_tile, threadIdx.x, cur, bad);
+                // inclusive suffix composition inside the warp: S_l = f_l o f_{l+1} o ... o f_31
+                Affine2 S = f;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const Affine2 o = shfl_down(S, d);
+                    if (lane + d < 32) S = compose(S, o);
+                }
+                cur.excl = shfl_down(S, 1);   // composite of the lanes to the right
+                if (lane == 31) cur.excl = identity2();
+                if (lane == 0) s_warp[b][warp] = S;
+                compute_warps_sync();
+                if (warp == 0) {
+                    // lane w < 4 holds warp w's composite; suffix-compose them, so that lane w ends
+                    // with W_w o ... o W_3 and lane 0 with the tile's composite
+                    Affine2 W = lane < kScanWarps ? s_warp[b][lane] : identity2();
+#pragma unroll
+                    for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
+                    Affine2 right = shfl_down(W, 1);            // composite of the warps to the right
+                    if (lane >= kScanWarps - 1) right = identity2();
+                    if (lane < kScanWarps) s_right[b][lane] = right;
+                    if (lane == 0) {
+                        s_tile_f[b] = W;
+                        if (tile + 1 < a.num_tiles) {
+                            st_pair(a.state[tile].aggA, W.aA, W.bA);
+                            st_pair(a.state[tile].aggR, W.aR, W.bR);
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&s_pipe.scan[b]));
+                }
+            } else if (warp == 0 && lane == 0) {
+                ptx::mbar_arrive(ptx::smem_addr(&s_pipe.scan[b]));     // lets the look-back warp see the end
+            }
+            if (prev_tile >= 0) {
+                const int pb = b ^ 1;
+                late |= !ptx::mbar_wait<false>(ptx::smem_addr(&s_pipe.carry[pb]), uint32_t((n - 1) >> 1) & 1u);
+                const int64_t t0 = int64_t(prev_tile) * kScanTile;
+                const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
+                const float G = float(fma(prev.excl.aA, s_carry[pb][warp][0], prev.excl.bA));
+                const float R = float(fma(prev.excl.aR, s_carry[pb][warp][1], prev.excl.bR));
+                egae_run_replay(a, s_buf[pb], s_win[(n - 1) & (kWinRing - 1)], t0, n_tile, threadIdx.x,
+                                prev, G, R, bad);
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&s_pipe.free_[pb]));
+            }
+            if (tile < 0) break;
+            prev = cur;
+            prev_tile = tile;
         }
     }
     if (bad) atomicOr(a.status, TPPO_DEV_BAD_SEGMENT);
+    if (late) atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT);
+}
+
+// persistent grid: as many CTAs as can be resident, fewer when there are fewer tiles
+static inline int egae_grid(int num_tiles) {
+    const int resident = kNumSms * kScanCtasPerSm;
+    return num_tiles < resident ? num_tiles : resident;
 }
 
 bool make_f32_rows_tensor_map(CUtensorMap* map, const void* base, uint64_t rows);
@@ -545,7 +795,7 @@ static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
     a.tma_ok = a.vec_ok && a.N >= kScanTile &&
                make_f32_rows_tensor_map(&map_r, a.rewards, uint64_t(a.N) / kRowPos) &&
                make_f32_rows_tensor_map(&map_v, a.values, uint64_t(a.N) / kRowPos);
-    egae_scan_kernel<<<a.num_tiles, kScanThreads, 0, s>>>(a, map_r, map_v);
+    egae_scan_kernel<<<egae_grid(a.num_tiles), kCtaThreads, 0, s>>>(a, map_r, map_v);
     TPPO_CUDA_CHECK(cudaGetLastError());
     return TPPO_OK;
 }
