@@ -145,15 +145,16 @@ __device__ __forceinline__ int pos_slot(int l) {      // float index of position
 // segment (the others never call this).  `i` is the index, inside the window, of the last segment
 // that begins at or before the positions still to come; the caller walks l downwards and `i`
 // follows.  x is the additive term of the G recurrence, r the reward; cont says that the position
-// continues into position l + 1 of the same segment (otherwise its map is constant).
+// continues into position l + 1 of the same segment (otherwise its map is constant).  The value of
+// position l + 1 is passed in: by the time of the replay its slot may hold a result already.
 struct PosTerm {
     float x, r, v;
     bool cont, inside;
 };
 __device__ __forceinline__ PosTerm egae_position(const EgaeArgs& a, const TileBuf& buf,
                                                  const TileWin& win, int64_t t0,
-                                                 int n_tile, int win_lo, bool win_smem, int l, int& i,
-                                                 bool& bad) {
+                                                 int n_tile, int win_lo, bool win_smem, int l,
+                                                 float v_next_pos, int& i, bool& bad) {
     PosTerm o{0.f, 0.f, 0.f, false, false};
     if (l >= n_tile) return o;
     const int32_t p = int32_t(t0 + l);
@@ -176,8 +177,7 @@ __device__ __forceinline__ PosTerm egae_position(const EgaeArgs& a, const TileBu
     o.r = buf.r[pos_slot(l)];
     o.v = buf.v[pos_slot(l)];
     if (p + 1 < e) {
-        const float v_next = l + 1 < kScanTile ? buf.v[pos_slot(l + 1)] : buf.v_after;
-        o.x = fmaf(a.c1, v_next, o.r);
+        o.x = fmaf(a.c1, v_next_pos, o.r);
         o.cont = true;
     } else {      // last token: G = r + gamma * (0 | bootstrap value | its own value)
         const bool tr = win_smem ? (win.seg_t[i] != 0) : (__ldg(a.truncated + win_lo + i) != 0);
@@ -335,6 +335,7 @@ struct RunState {
     int k_last;
     float v_boundary;
     bool boundary_own;   // the boundary value is the last token's own value (no bootstrap array)
+    float v_right;       // value of the position after the run (its slot is overwritten by the replay)
 };
 
 // The thread's sixteen positions, right to left: its composite map.
@@ -376,6 +377,7 @@ __device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, const TileBuf
     rs.fast = fast;
     rs.masked = false;
     const float v_right = l0 + kScanItems < kScanTile ? buf.v[pos_slot(l0 + kScanItems)] : buf.v_after;
+    rs.v_right = v_right;
     if (!fast && win_smem) {
         // The segments that overlap the run, from the right: usually one or two.  With at most one
         // segment end inside the run the per-position work stays branch-free (two bit masks and one
@@ -460,8 +462,10 @@ __device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, const TileBuf
     float bG = 0.f, bR = 0.f;
     double aG = 1.0, aR = 1.0;
     int i = i_start;
+    float v_next = v_right;
     for (int k = kScanItems - 1; k >= 0; --k) {
-        const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l0 + k, i, bad);
+        const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l0 + k, v_next, i, bad);
+        v_next = buf.v[pos_slot(l0 + k)];
         if (t.cont) {
             bG = fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, t.x));
             bR = fmaf(a.gamma_f, bR, t.r);
@@ -477,16 +481,38 @@ __device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, const TileBuf
     return Affine2{aG, double(bG), aR, double(bR)};
 }
 
+// Four results of one chunk: into the tile image itself (advantages over the values, returns over
+// the rewards; a TMA store takes them to global memory) or straight to global memory.
+__device__ __forceinline__ void egae_put4(const EgaeArgs& a, TileBuf& buf, bool in_place, int s,
+                                          int64_t pos, int n_left, bool vec, const float (&oa)[4],
+                                          const float (&og)[4]) {
+    if (in_place) {
+        *reinterpret_cast<float4*>(buf.v + s) = make_float4(oa[0], oa[1], oa[2], oa[3]);
+        if (a.ret) *reinterpret_cast<float4*>(buf.r + s) = make_float4(og[0], og[1], og[2], og[3]);
+    } else if (vec && n_left >= 4) {
+        *reinterpret_cast<float4*>(a.adv + pos) = make_float4(oa[0], oa[1], oa[2], oa[3]);
+        if (a.ret) *reinterpret_cast<float4*>(a.ret + pos) = make_float4(og[0], og[1], og[2], og[3]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (e < n_left) {
+                a.adv[pos + e] = oa[e];
+                if (a.ret) a.ret[pos + e] = og[e];
+            }
+        }
+    }
+}
+
 // Replays the thread's positions from the values entering its run and stores the results.
-__device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, const TileBuf& buf,
+__device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, TileBuf& buf,
                                                 const TileWin& win, int64_t t0,
                                                 int n_tile, int tid, const RunState& rs, float G,
-                                                float R, bool& bad) {
+                                                float R, bool in_place, bool& bad) {
     const int l0 = tid * kScanItems;
     if (rs.fast) {
         const int row_base = (tid >> 1) << 5;
         const int chunk0 = (tid & 1) << 2, swz = (tid >> 1) & 7;
-        float vn = l0 + kScanItems < kScanTile ? buf.v[pos_slot(l0 + kScanItems)] : buf.v_after;
+        float vn = rs.v_right;
 #pragma unroll
         for (int q = kScanItems / 4 - 1; q >= 0; --q) {
             const int s = row_base + (((chunk0 + q) ^ swz) << 2);
@@ -504,17 +530,7 @@ __device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, const TileBuf
                 oa[e] = G - vn;
                 og[e] = R;
             }
-            if (a.vec_ok) {
-                *reinterpret_cast<float4*>(a.adv + t0 + l0 + 4 * q) = make_float4(oa[0], oa[1], oa[2], oa[3]);
-                if (a.ret)
-                    *reinterpret_cast<float4*>(a.ret + t0 + l0 + 4 * q) = make_float4(og[0], og[1], og[2], og[3]);
-            } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    a.adv[t0 + l0 + 4 * q + e] = oa[e];
-                    if (a.ret) a.ret[t0 + l0 + 4 * q + e] = og[e];
-                }
-            }
+            egae_put4(a, buf, in_place, s, t0 + l0 + 4 * q, 4, a.vec_ok != 0, oa, og);
         }
         return;
     }
@@ -522,8 +538,7 @@ __device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, const TileBuf
         const int row_base = (tid >> 1) << 5;
         const int chunk0 = (tid & 1) << 2, swz = (tid >> 1) & 7;
         const uint32_t inside = rs.bits & 0xffffu, cont = rs.bits >> 16;
-        const bool full = a.vec_ok && l0 + kScanItems <= n_tile;
-        float vn = l0 + kScanItems < kScanTile ? buf.v[pos_slot(l0 + kScanItems)] : buf.v_after;
+        float vn = rs.v_right;
 #pragma unroll
         for (int q = kScanItems / 4 - 1; q >= 0; --q) {
             const int s = row_base + (((chunk0 + q) ^ swz) << 2);
@@ -546,32 +561,26 @@ __device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, const TileBuf
                 oa[e] = in ? G - vn : 0.f;
                 og[e] = R;
             }
-            if (full) {
-                *reinterpret_cast<float4*>(a.adv + t0 + l0 + 4 * q) = make_float4(oa[0], oa[1], oa[2], oa[3]);
-                if (a.ret)
-                    *reinterpret_cast<float4*>(a.ret + t0 + l0 + 4 * q) = make_float4(og[0], og[1], og[2], og[3]);
-            } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if (l0 + 4 * q + e < n_tile) {
-                        a.adv[t0 + l0 + 4 * q + e] = oa[e];
-                        if (a.ret) a.ret[t0 + l0 + 4 * q + e] = og[e];
-                    }
-                }
-            }
+            egae_put4(a, buf, in_place, s, t0 + l0 + 4 * q, n_tile - (l0 + 4 * q), a.vec_ok != 0, oa, og);
         }
         return;
     }
     const int win_lo = win.win_lo;
     const bool win_smem = max(win.win_hi - win_lo, 0) <= kSegCap;
     int i = rs.i_start;
+    float v_next = rs.v_right;
     for (int k = kScanItems - 1; k >= 0; --k) {
         const int l = l0 + k;
-        const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l, i, bad);
+        const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l, v_next, i, bad);
+        v_next = buf.v[pos_slot(l)];
         G = t.cont ? fmaf(a.gl_hi, G, fmaf(a.gl_lo, G, t.x)) : t.x;
         R = t.cont ? fmaf(a.gamma_f, R, t.r) : t.r;
-        if (l < n_tile) {
-            a.adv[t0 + l] = t.inside ? G - t.v : 0.f;
+        const float adv = t.inside ? G - t.v : 0.f;
+        if (in_place) {
+            buf.v[pos_slot(l)] = adv;
+            if (a.ret) buf.r[pos_slot(l)] = R;
+        } else if (l < n_tile) {
+            a.adv[t0 + l] = adv;
             if (a.ret) a.ret[t0 + l] = R;
         }
     }
@@ -605,7 +614,8 @@ __device__ __forceinline__ void compute_warps_sync() {     // named barrier 1: t
 
 __global__ void __launch_bounds__(kCtaThreads, kScanCtasPerSm)
 egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
-                 const __grid_constant__ CUtensorMap map_v) {
+                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_adv,
+                 const __grid_constant__ CUtensorMap map_ret) {
     __shared__ TileBuf s_buf[2];
     __shared__ TileWin s_win[kWinRing];
     __shared__ __align__(8) Pipe s_pipe;
@@ -633,7 +643,22 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
         // wraps the first draw to ticket 0
         uint32_t ticket = 0;
         if (lane == 0) ticket = atomicAdd(a.ticket, 1u) + 1u;
-        for (int m = 0;; ++m) {
+        int held[2] = {-1, -1};          // tile whose results sit in each buffer, waiting to be stored
+        // The results of a whole tile were written over its inputs; two TMA stores take them to
+        // global memory.  The buffer may be refilled once they have been read out of it.
+        auto store_results = [&](int b) {
+            if (held[b] >= 0 && lane == 0) {
+                const int32_t y = held[b] * (kScanTile / kRowPos);
+                umma::tma_store_2d(&map_adv, ptx::smem_addr(s_buf[b].v), 0, y);
+                if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(s_buf[b].r), 0, y);
+                ptx::bulk_commit();
+                ptx::bulk_wait_read<0>();
+            }
+            held[b] = -1;
+            __syncwarp();
+        };
+        int m = 0;
+        for (;; ++m) {
             const int b = m & 1;
             const uint32_t t = __shfl_sync(0xffffffffu, ticket, 0);
             const int tile = t < uint32_t(a.num_tiles) ? a.num_tiles - 1 - int(t) : -1;
@@ -654,8 +679,10 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
             }
             // the buffer was last used by tile m - 2: its replay must have finished
             if (m >= 2) late |= !ptx::mbar_wait<false>(ptx::smem_addr(&s_pipe.free_[b]), uint32_t((m >> 1) - 1) & 1u);
+            store_results(b);
             TileBuf& buf = s_buf[b];
             const bool by_tma = a.tma_ok && n_tile == kScanTile;
+            if (by_tma) held[b] = tile;
             if (by_tma) {
                 if (lane == 0) {
                     ptx::mbar_expect_tx(full, 2 * kScanTile * uint32_t(sizeof(float)));
@@ -673,6 +700,14 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(full);
         }
+        // the last two tiles: their results leave once their replays are done
+        for (int d = m; d < m + 2; ++d) {
+            const int b = d & 1;
+            if (held[b] < 0) continue;
+            late |= !ptx::mbar_wait<false>(ptx::smem_addr(&s_pipe.free_[b]), uint32_t((d >> 1) - 1) & 1u);
+            store_results(b);
+        }
+        if (lane == 0) ptx::bulk_wait<0>();
     } else if (warp == kLookWarp) {
         // =========================== look-back =======================================================
         for (int n = 0;; ++n) {
@@ -751,8 +786,10 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
                 const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
                 const float G = float(fma(prev.excl.aA, s_carry[pb][warp][0], prev.excl.bA));
                 const float R = float(fma(prev.excl.aR, s_carry[pb][warp][1], prev.excl.bR));
+                const bool in_place = a.tma_ok && n_tile == kScanTile;
                 egae_run_replay(a, s_buf[pb], s_win[(n - 1) & (kWinRing - 1)], t0, n_tile, threadIdx.x,
-                                prev, G, R, bad);
+                                prev, G, R, in_place, bad);
+                if (in_place) ptx::fence_proxy_async_smem();   // the TMA store reads what was just written
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&s_pipe.free_[pb]));
             }
@@ -787,15 +824,19 @@ static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
     a.c1 = float(double(gamma) * (1.0 - double(lambda)));
     a.vec_ok = aligned(a.rewards, 16) && aligned(a.values, 16) && aligned(a.adv, 16) &&
                (!a.ret || aligned(a.ret, 16));
-    CUtensorMap map_r, map_v;
+    CUtensorMap map_r, map_v, map_adv, map_ret;
     memset(&map_r, 0, sizeof(map_r));
     memset(&map_v, 0, sizeof(map_v));
+    memset(&map_adv, 0, sizeof(map_adv));
+    memset(&map_ret, 0, sizeof(map_ret));
     // whole tiles exist only from 2048 positions on; without the driver's encoder (or with
     // unaligned arrays) every tile takes the plain-load path
     a.tma_ok = a.vec_ok && a.N >= kScanTile &&
                make_f32_rows_tensor_map(&map_r, a.rewards, uint64_t(a.N) / kRowPos) &&
-               make_f32_rows_tensor_map(&map_v, a.values, uint64_t(a.N) / kRowPos);
-    egae_scan_kernel<<<egae_grid(a.num_tiles), kCtaThreads, 0, s>>>(a, map_r, map_v);
+               make_f32_rows_tensor_map(&map_v, a.values, uint64_t(a.N) / kRowPos) &&
+               make_f32_rows_tensor_map(&map_adv, a.adv, uint64_t(a.N) / kRowPos) &&
+               (!a.ret || make_f32_rows_tensor_map(&map_ret, a.ret, uint64_t(a.N) / kRowPos));
+    egae_scan_kernel<<<egae_grid(a.num_tiles), kCtaThreads, 0, s>>>(a, map_r, map_v, map_adv, map_ret);
     TPPO_CUDA_CHECK(cudaGetLastError());
     return TPPO_OK;
 }
