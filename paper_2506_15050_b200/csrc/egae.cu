@@ -39,7 +39,7 @@ constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kScanItems = 16;
 constexpr int kScanTile = kScanThreads * kScanItems;  // 2048 positions
 constexpr int kSegCap = 32;                           // segments of one tile kept in shared memory
-constexpr int kScanCtasPerSm = 6;
+constexpr int kScanCtasPerSm = 8;
 constexpr uint32_t kScanSpinLimit = 1u << 22;
 
 struct Affine2 {  // x -> (aA*xA + bA, aR*xR + bR)
@@ -133,7 +133,6 @@ struct TileWin {
     float seg_boot[kSegCap];
     uint8_t seg_t[kSegCap];
     int win_lo, win_hi;          // segment indices [win_lo, win_hi) may touch the tile
-    int tile;                    // the tile itself, -1: there are no more tiles
 };
 static_assert(offsetof(TileBuf, v) % 1024 == 0, "swizzle atom alignment");
 __device__ __forceinline__ int pos_slot(int l) {      // float index of position l
@@ -322,7 +321,7 @@ __device__ __forceinline__ bool egae_window(const EgaeArgs& a, TileWin& win, int
     return bad;
 }
 
-// What a compute thread keeps of a tile between composing its maps and replaying them.
+// What a thread keeps of its run between composing its maps and replaying them.
 struct RunState {
     Affine2 excl;     // composite of the lanes to its right inside the warp
     int i_start;      // window index of the last segment that begins at or before its last position
@@ -463,6 +462,7 @@ __device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, const TileBuf
     double aG = 1.0, aR = 1.0;
     int i = i_start;
     float v_next = v_right;
+#pragma unroll 1
     for (int k = kScanItems - 1; k >= 0; --k) {
         const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l0 + k, v_next, i, bad);
         v_next = buf.v[pos_slot(l0 + k)];
@@ -569,6 +569,7 @@ __device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, TileBuf& buf,
     const bool win_smem = max(win.win_hi - win_lo, 0) <= kSegCap;
     int i = rs.i_start;
     float v_next = rs.v_right;
+#pragma unroll 1
     for (int k = kScanItems - 1; k >= 0; --k) {
         const int l = l0 + k;
         const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l, v_next, i, bad);
@@ -586,226 +587,119 @@ __device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, TileBuf& buf,
     }
 }
 
-// Persistent CTAs of six warps; tiles are taken by ticket, from the END of the arrays backwards, so
-// the tiles a tile looks back at (those to its right) hold earlier tickets and are running or done.
-// Three roles run as independent loops and meet only at mbarriers:
-//   stager (warp 5):     ticket and segment window of tile m (a ring of four windows, so that the
-//                        search runs ahead of the buffers), then, once the replay of tile m-2 has
-//                        freed the buffer, the two TMA copies of tile m;
-//   compute (warps 0-3): step n = maps + warp scan of tile n, composite published at once (so no
-//                        other CTA waits for this CTA's look-back), then replay + stores of tile n-1;
-//   look-back (warp 4):  value entering tile n from the right, the tile's first-position values
-//                        published, the values entering each warp handed to the replay.
-// The look-back of tile n (L2 round trips, and a wait for the right-hand neighbours) thus runs while
-// the compute warps are on tile n+1.  Two input buffers; four mbarriers per buffer hand it from
-// stage to stage (inputs ready, scan done, carries ready, buffer free).  Every wait is bounded.
-constexpr int kLookWarp = kScanWarps, kStageWarp = kScanWarps + 1;
-constexpr int kCtaThreads = kScanThreads + 64;
-constexpr int kWinRing = 4;
-struct Pipe {
-    uint64_t full[2];     // inputs (and window) of the tile are there                 (stager -> compute)
-    uint64_t scan[2];     // the tile's composites are in s_right / s_tile_f            (compute -> look-back)
-    uint64_t carry[2];    // the values entering each warp are in s_carry              (look-back -> compute)
-    uint64_t free_[2];    // the replay has finished reading the buffer                (compute -> stager)
-};
-__device__ __forceinline__ void compute_warps_sync() {     // named barrier 1: the four compute warps
-    asm volatile("bar.sync 1, %0;" ::"n"(kScanThreads) : "memory");
-}
-
-__global__ void __launch_bounds__(kCtaThreads, kScanCtasPerSm)
+// One CTA per tile of 2048 positions; tiles are taken by ticket, from the END of the arrays
+// backwards, so the tiles a tile looks back at (those to its right) hold earlier tickets and are
+// running or done.  The latencies of a tile (ticket, copy, window search, look-back) are covered by
+// the other CTAs resident on the SM.  A whole tile's results are written over its inputs in shared
+// memory and leave by two TMA stores.
+__global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm)
 egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
                  const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_adv,
                  const __grid_constant__ CUtensorMap map_ret) {
-    __shared__ TileBuf s_buf[2];
-    __shared__ TileWin s_win[kWinRing];
-    __shared__ __align__(8) Pipe s_pipe;
-    __shared__ Affine2 s_warp[2][kScanWarps];    // warp composites (compute warps only)
-    __shared__ Affine2 s_right[2][kScanWarps];   // composite of the warps to the right of each warp
-    __shared__ Affine2 s_tile_f[2];              // composite of the whole tile
-    __shared__ double s_carry[2][kScanWarps][2];
+    __shared__ TileBuf buf;
+    __shared__ TileWin win;
+    __shared__ __align__(8) uint64_t s_bar;      // the tile's inputs have arrived
+    __shared__ uint32_t s_ticket;
+    __shared__ Affine2 s_warp[kScanWarps];
+    __shared__ double s_carry[kScanWarps][2];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t bar = ptx::smem_addr(&s_bar);
     if (threadIdx.x == 0) {
-        for (int b = 0; b < 2; ++b) {
-            ptx::mbar_init(ptx::smem_addr(&s_pipe.full[b]), 1);
-            ptx::mbar_init(ptx::smem_addr(&s_pipe.scan[b]), 1);
-            ptx::mbar_init(ptx::smem_addr(&s_pipe.carry[b]), 1);
-            ptx::mbar_init(ptx::smem_addr(&s_pipe.free_[b]), kScanWarps);
-        }
+        // the ticket counter starts at all-ones like the rest of the workspace (one memset): + 1
+        // wraps the first draw to ticket 0
+        s_ticket = atomicAdd(a.ticket, 1u) + 1u;
+        ptx::mbar_init(bar, 1);
         ptx::fence_mbar_init_cluster();
     }
     __syncthreads();
-    bool bad = false, late = false;      // a bad segment was seen; a bounded wait ran out
+    const uint32_t ticket = s_ticket;
+    if (ticket >= uint32_t(a.num_tiles)) return;       // (the grid has exactly num_tiles CTAs)
+    const int tile = a.num_tiles - 1 - int(ticket);
+    const int64_t t0 = int64_t(tile) * kScanTile;
+    const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
+    const bool by_tma = a.tma_ok && n_tile == kScanTile;
+    bool bad = false;
 
-    if (warp == kStageWarp) {
-        // =========================== stager ==========================================================
-        // the ticket counter starts at all-ones like the rest of the workspace (one memset): + 1
-        // wraps the first draw to ticket 0
-        uint32_t ticket = 0;
-        if (lane == 0) ticket = atomicAdd(a.ticket, 1u) + 1u;
-        int held[2] = {-1, -1};          // tile whose results sit in each buffer, waiting to be stored
-        // The results of a whole tile were written over its inputs; two TMA stores take them to
-        // global memory.  The buffer may be refilled once they have been read out of it.
-        auto store_results = [&](int b) {
-            if (held[b] >= 0 && lane == 0) {
-                const int32_t y = held[b] * (kScanTile / kRowPos);
-                umma::tma_store_2d(&map_adv, ptx::smem_addr(s_buf[b].v), 0, y);
-                if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(s_buf[b].r), 0, y);
-                ptx::bulk_commit();
-                ptx::bulk_wait_read<0>();
-            }
-            held[b] = -1;
-            __syncwarp();
-        };
-        int m = 0;
-        for (;; ++m) {
-            const int b = m & 1;
-            const uint32_t t = __shfl_sync(0xffffffffu, ticket, 0);
-            const int tile = t < uint32_t(a.num_tiles) ? a.num_tiles - 1 - int(t) : -1;
-            // draw the next ticket now: its round trip hides behind the window search
-            if (tile >= 0 && lane == 0) ticket = atomicAdd(a.ticket, 1u) + 1u;
-            // window slot m & 3 was last read by the replay of tile m-4, which finished before the
-            // replay of tile m-3 that the previous step waited for
-            TileWin& win = s_win[m & (kWinRing - 1)];
-            const int64_t t0 = int64_t(tile < 0 ? 0 : tile) * kScanTile;
-            const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
-            if (lane == 0) win.tile = tile;
-            if (tile >= 0) bad |= egae_window(a, win, t0, n_tile, lane);
-            const uint32_t full = ptx::smem_addr(&s_pipe.full[b]);
-            if (tile < 0) {
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(full);
-                break;
-            }
-            // the buffer was last used by tile m - 2: its replay must have finished
-            if (m >= 2) late |= !ptx::mbar_wait<false>(ptx::smem_addr(&s_pipe.free_[b]), uint32_t((m >> 1) - 1) & 1u);
-            store_results(b);
-            TileBuf& buf = s_buf[b];
-            const bool by_tma = a.tma_ok && n_tile == kScanTile;
-            if (by_tma) held[b] = tile;
-            if (by_tma) {
-                if (lane == 0) {
-                    ptx::mbar_expect_tx(full, 2 * kScanTile * uint32_t(sizeof(float)));
-                    umma::tma_load_2d(ptx::smem_addr(buf.r), &map_r, full, 0, int32_t(t0 / kRowPos));
-                    umma::tma_load_2d(ptx::smem_addr(buf.v), &map_v, full, 0, int32_t(t0 / kRowPos));
-                }
-            } else {      // a ragged or unaligned tile: plain loads
-                for (int k = lane; k < n_tile; k += 32) {
-                    buf.r[pos_slot(k)] = __ldg(a.rewards + t0 + k);
-                    buf.v[pos_slot(k)] = __ldg(a.values + t0 + k);
-                }
-                ptx::fence_proxy_async_smem();    // a later TMA copy lands on the same bytes
-            }
-            if (lane == 0) buf.v_after = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(full);
-        }
-        // the last two tiles: their results leave once their replays are done
-        for (int d = m; d < m + 2; ++d) {
-            const int b = d & 1;
-            if (held[b] < 0) continue;
-            late |= !ptx::mbar_wait<false>(ptx::smem_addr(&s_pipe.free_[b]), uint32_t((d >> 1) - 1) & 1u);
-            store_results(b);
-        }
-        if (lane == 0) ptx::bulk_wait<0>();
-    } else if (warp == kLookWarp) {
-        // =========================== look-back =======================================================
-        for (int n = 0;; ++n) {
-            const int b = n & 1;
-            late |= !ptx::mbar_wait<false>(ptx::smem_addr(&s_pipe.scan[b]), uint32_t(n >> 1) & 1u);
-            const int tile = s_win[n & (kWinRing - 1)].tile;
-            if (tile < 0) break;
-            double xA = 0.0, xR = 0.0;
-            const bool ok = egae_look_back(a, tile + 1, lane, xA, xR);
-            if (lane == 0) {
-                if (!ok) { late = true; xA = 0.0; xR = 0.0; }
-                const Affine2 W = s_tile_f[b];
-                st_pair(a.state[tile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
-            }
-            xA = __shfl_sync(0xffffffffu, xA, 0);
-            xR = __shfl_sync(0xffffffffu, xR, 0);
-            if (lane < kScanWarps) {
-                const Affine2 right = s_right[b][lane];
-                s_carry[b][lane][0] = fma(right.aA, xA, right.bA);
-                s_carry[b][lane][1] = fma(right.aR, xR, right.bR);
-            }
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&s_pipe.carry[b]));
+    // ---- inputs: two TMA copies for a whole tile, plain loads for a ragged or unaligned one ------
+    if (by_tma) {
+        if (threadIdx.x == 0) {
+            ptx::mbar_arrive_expect_tx(bar, 2 * kScanTile * uint32_t(sizeof(float)));
+            umma::tma_load_2d(ptx::smem_addr(buf.r), &map_r, bar, 0, int32_t(t0 / kRowPos));
+            umma::tma_load_2d(ptx::smem_addr(buf.v), &map_v, bar, 0, int32_t(t0 / kRowPos));
         }
     } else {
-        // =========================== compute warps ==================================================
-        RunState prev{};
-        int prev_tile = -1;
-        for (int n = 0;; ++n) {
-            const int b = n & 1;
-            late |= !ptx::mbar_wait<false>(ptx::smem_addr(&s_pipe.full[b]), uint32_t(n >> 1) & 1u);
-            const TileWin& win = s_win[n & (kWinRing - 1)];
-            const int tile = win.tile;
-            RunState cur{};
-            if (tile >= 0) {
-                const int64_t t0 = int64_t(tile) * kScanTile;
-                const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
-                const Affine2 f = egae_run_map(a, s_buf[b], win, t0, n_tile, threadIdx.x, cur, bad);
-                // inclusive suffix composition inside the warp: S_l = f_l o f_{l+1} o ... o f_31
-                Affine2 S = f;
+        for (int k = threadIdx.x; k < n_tile; k += kScanThreads) {
+            buf.r[pos_slot(k)] = __ldg(a.rewards + t0 + k);
+            buf.v[pos_slot(k)] = __ldg(a.values + t0 + k);
+        }
+    }
+    if (threadIdx.x == kScanThreads - 1)
+        buf.v_after = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
+    if (warp == 0) bad |= egae_window(a, win, t0, n_tile, lane);
+    if (by_tma && !ptx::mbar_wait<false>(bar, 0)) atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT);
+    __syncthreads();
+
+    // ---- the thread's sixteen positions, right to left: its composite map; the warp's scan --------
+    RunState rs{};
+    const Affine2 f = egae_run_map(a, buf, win, t0, n_tile, threadIdx.x, rs, bad);
+    // inclusive suffix composition inside the warp: S_l = f_l o f_{l+1} o ... o f_31
+    Affine2 S = f;
 #pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const Affine2 o = shfl_down(S, d);
-                    if (lane + d < 32) S = compose(S, o);
-                }
-                cur.excl = shfl_down(S, 1);   // composite of the lanes to the right
-                if (lane == 31) cur.excl = identity2();
-                if (lane == 0) s_warp[b][warp] = S;
-                compute_warps_sync();
-                if (warp == 0) {
-                    // lane w < 4 holds warp w's composite; suffix-compose them, so that lane w ends
-                    // with W_w o ... o W_3 and lane 0 with the tile's composite
-                    Affine2 W = lane < kScanWarps ? s_warp[b][lane] : identity2();
+    for (int d = 1; d < 32; d <<= 1) {
+        const Affine2 o = shfl_down(S, d);
+        if (lane + d < 32) S = compose(S, o);
+    }
+    rs.excl = shfl_down(S, 1);   // composite of the lanes to the right
+    if (lane == 31) rs.excl = identity2();
+    if (lane == 0) s_warp[warp] = S;
+    __syncthreads();                                                      // (A)
+
+    // ---- tile composite, look-back, per-warp carries (warp 0) ------------------------------------
+    if (warp == 0) {
+        // lane w < 4 holds warp w's composite; suffix-compose them, so that lane w ends with
+        // W_w o ... o W_3 and lane 0 with the tile's composite
+        Affine2 W = lane < kScanWarps ? s_warp[lane] : identity2();
 #pragma unroll
-                    for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
-                    Affine2 right = shfl_down(W, 1);            // composite of the warps to the right
-                    if (lane >= kScanWarps - 1) right = identity2();
-                    if (lane < kScanWarps) s_right[b][lane] = right;
-                    if (lane == 0) {
-                        s_tile_f[b] = W;
-                        if (tile + 1 < a.num_tiles) {
-                            st_pair(a.state[tile].aggA, W.aA, W.bA);
-                            st_pair(a.state[tile].aggR, W.aR, W.bR);
-                        }
-                    }
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&s_pipe.scan[b]));
-                }
-            } else if (warp == 0 && lane == 0) {
-                ptx::mbar_arrive(ptx::smem_addr(&s_pipe.scan[b]));     // lets the look-back warp see the end
-            }
-            if (prev_tile >= 0) {
-                const int pb = b ^ 1;
-                late |= !ptx::mbar_wait<false>(ptx::smem_addr(&s_pipe.carry[pb]), uint32_t((n - 1) >> 1) & 1u);
-                const int64_t t0 = int64_t(prev_tile) * kScanTile;
-                const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
-                const float G = float(fma(prev.excl.aA, s_carry[pb][warp][0], prev.excl.bA));
-                const float R = float(fma(prev.excl.aR, s_carry[pb][warp][1], prev.excl.bR));
-                const bool in_place = a.tma_ok && n_tile == kScanTile;
-                egae_run_replay(a, s_buf[pb], s_win[(n - 1) & (kWinRing - 1)], t0, n_tile, threadIdx.x,
-                                prev, G, R, in_place, bad);
-                if (in_place) ptx::fence_proxy_async_smem();   // the TMA store reads what was just written
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&s_pipe.free_[pb]));
-            }
-            if (tile < 0) break;
-            prev = cur;
-            prev_tile = tile;
+        for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
+        Affine2 right = shfl_down(W, 1);            // composite of the warps to the right
+        if (lane >= kScanWarps - 1) right = identity2();
+        TileState* st = a.state;
+        if (lane == 0 && tile + 1 < a.num_tiles) {
+            st_pair(st[tile].aggA, W.aA, W.bA);
+            st_pair(st[tile].aggR, W.aR, W.bR);
+        }
+        double xA = 0.0, xR = 0.0;
+        const bool ok = egae_look_back(a, tile + 1, lane, xA, xR);
+        if (lane == 0) {
+            if (!ok) { atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
+            st_pair(st[tile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
+        }
+        xA = __shfl_sync(0xffffffffu, xA, 0);
+        xR = __shfl_sync(0xffffffffu, xR, 0);
+        if (lane < kScanWarps) {
+            s_carry[lane][0] = fma(right.aA, xA, right.bA);
+            s_carry[lane][1] = fma(right.aR, xR, right.bR);
+        }
+    }
+    __syncthreads();                                                      // (B)
+
+    // ---- replay the thread's positions from the true incoming values, store -----------------------
+    const float G = float(fma(rs.excl.aA, s_carry[warp][0], rs.excl.bA));
+    const float R = float(fma(rs.excl.aR, s_carry[warp][1], rs.excl.bR));
+    egae_run_replay(a, buf, win, t0, n_tile, threadIdx.x, rs, G, R, by_tma, bad);
+    if (by_tma) {
+        ptx::fence_proxy_async_smem();       // the TMA stores read what was just written
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int32_t y = tile * (kScanTile / kRowPos);
+            umma::tma_store_2d(&map_adv, ptx::smem_addr(buf.v), 0, y);
+            if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(buf.r), 0, y);
+            ptx::bulk_commit();
+            ptx::bulk_wait<0>();             // shared memory must outlive the stores
         }
     }
     if (bad) atomicOr(a.status, TPPO_DEV_BAD_SEGMENT);
-    if (late) atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT);
-}
-
-// persistent grid: as many CTAs as can be resident, fewer when there are fewer tiles
-static inline int egae_grid(int num_tiles) {
-    const int resident = kNumSms * kScanCtasPerSm;
-    return num_tiles < resident ? num_tiles : resident;
 }
 
 bool make_f32_rows_tensor_map(CUtensorMap* map, const void* base, uint64_t rows);
@@ -836,7 +730,7 @@ static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
                make_f32_rows_tensor_map(&map_v, a.values, uint64_t(a.N) / kRowPos) &&
                make_f32_rows_tensor_map(&map_adv, a.adv, uint64_t(a.N) / kRowPos) &&
                (!a.ret || make_f32_rows_tensor_map(&map_ret, a.ret, uint64_t(a.N) / kRowPos));
-    egae_scan_kernel<<<egae_grid(a.num_tiles), kCtaThreads, 0, s>>>(a, map_r, map_v, map_adv, map_ret);
+    egae_scan_kernel<<<a.num_tiles, kScanThreads, 0, s>>>(a, map_r, map_v, map_adv, map_ret);
     TPPO_CUDA_CHECK(cudaGetLastError());
     return TPPO_OK;
 }
