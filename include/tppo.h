@@ -102,7 +102,14 @@ size_t tppo_workspace_bytes(int op, int64_t N, int32_t B, int64_t n_max, int32_t
  *   advantages       [N] fp32 out; returns [N] fp32 out or NULL.  Positions outside every
  *                    segment are written 0.
  *   status           [1] int32 out: device status bits (0 = clean).
- * Sums are carried in fp64 and rounded once to fp32 on store.  N < 2^31.
+ * Precision: the advantage is carried as G_t = A_t + values[t] (G_t = rewards[t] + gamma*(1-lambda)*
+ * V(s_{t+1}) + gamma*lambda*G_{t+1}, so successive values never cancel); runs of 16 consecutive
+ * positions are evaluated in fp32 (gamma*lambda split into two floats, exact to 2^-48), everything
+ * carried across runs, warps and tiles is fp64.  The error of a result is a few units of 2^-24 of
+ * the largest |G| or |R| of its run and does not grow with the length of a response.  N < 2^31.
+ * Arrays that are 16-byte aligned take the fast path (TMA copies); others are still handled.
+ * The first call in a process looks up the driver's tensor-map encoder (without it every tile takes
+ * the slower plain-load path; no error).
  */
 int tppo_egae(const float *rewards, const float *values,
               const int32_t *seg_begin, const int32_t *seg_end,

@@ -63,26 +63,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
 }
 
-// The same wait for warps that expect to wait long (a stage of a software pipeline): each attempt
-// lets the hardware suspend the warp for up to `hint_ns` (it wakes when the phase completes).
-__device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_suspended(uint32_t bar, uint32_t parity) {
-    if (mbar_try_wait_suspend(bar, parity, 20000u)) return true;
-    const uint64_t t0 = globaltimer_ns();
-    for (;;) {
-        if (mbar_try_wait_suspend(bar, parity, 20000u)) return true;
-        if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
-    }
-}
-
 // ---- bulk (TMA, untiled) copies: 16-byte aligned addresses, size a multiple of 16 ------------
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src_gmem, uint32_t bytes,
                                           uint32_t bar) {

@@ -135,6 +135,67 @@ def test_egae_edge_cases():
     assert st == 8      # segment end beyond N is reported, not followed
 
 
+def test_egae_segment_ends_at_every_offset_of_a_run():
+    """A thread evaluates sixteen consecutive positions; the end of one segment and the start of the
+    next are placed at every offset inside such a run and across the tile edge (2048), with the
+    three kinds of boundary value (finished, truncated with and without a bootstrap array)."""
+    rng = np.random.default_rng(8)
+    N = 3 * 2048 + 77
+    r = rng.standard_normal(N).astype(np.float32)
+    v = rng.standard_normal(N).astype(np.float32)
+    for e1 in list(range(2030, 2067)) + [4095, 4096, 4097]:
+        for gap in (0, 1, 5):
+            sb = np.array([3, e1 + gap], np.int32)
+            se = np.array([e1, N - 2], np.int32)
+            boot = rng.standard_normal(2).astype(np.float32)
+            for tr in ((0, 1), (1, 0)):
+                check_egae(2, r, v, sb, se, np.array(tr, np.uint8), boot, 0.99, 0.95)
+            check_egae(2, r, v, sb, se, np.array([1, 1], np.uint8), None, 1.0, 0.95)
+
+
+def test_egae_long_response_dense_rewards_keeps_the_tolerance():
+    """One response of 131072 tokens with a reward on every token and no decay (gamma = lambda = 1,
+    and gamma just below 1): sums over the whole response, where single-precision accumulation
+    over the length would lose the tolerance."""
+    rng = np.random.default_rng(9)
+    N = 131072 + 50
+    r = (0.5 + rng.standard_normal(N)).astype(np.float32)
+    v = rng.standard_normal(N).astype(np.float32)
+    sb, se = np.array([20], np.int32), np.array([N - 30], np.int32)
+    for gamma, lam in ((1.0, 1.0), (0.9999, 1.0), (1.0, 0.999)):
+        check_egae(1, r, v, sb, se, np.array([1], np.uint8), None, gamma, lam)
+
+
+def test_egae_unaligned_arrays_and_no_returns():
+    """Arrays that start off a 16-byte boundary take the plain-load path; returns may be omitted."""
+    from paper_2506_15050_b200 import binding as b
+    rng = np.random.default_rng(10)
+    N, B = 3 * 2048 + 500, 3
+    r = rng.standard_normal(N).astype(np.float32)
+    v = rng.standard_normal(N).astype(np.float32)
+    sb, se = np.array([0, 2500, 5000], np.int32), np.array([2400, 4999, N], np.int32)
+    tr = np.array([1, 0, 1], np.uint8)
+    ra, rr = oracle.egae(r, v, sb, se, tr, None, f32(1.0), f32(0.95))
+    adv, ret, st = run_egae(B, r, v, sb, se, tr, None, 1.0, 0.95, want_returns=False)
+    assert st == 0 and ret is None and adv_close(adv, ra, sb, se, ADV_RTOL) <= 1.0
+    for off_in, off_out in ((1, 0), (0, 1), (3, 2)):
+        rbuf, vbuf = torch.zeros(N + 4, device=DEV), torch.zeros(N + 4, device=DEV)
+        rbuf[off_in:off_in + N] = dev(r, torch.float32)
+        vbuf[off_in:off_in + N] = dev(v, torch.float32)
+        abuf = torch.full((N + 4,), float("nan"), device=DEV)
+        gbuf = torch.full((N + 4,), float("nan"), device=DEV)
+        status = torch.full((1,), -1, dtype=torch.int32, device=DEV)
+        ws = b.workspace(b.OP_EGAE, N, B, 0, 0, DEV)
+        b.tppo_egae(rbuf[off_in:off_in + N], vbuf[off_in:off_in + N], dev(sb, torch.int32),
+                    dev(se, torch.int32), dev(tr, torch.uint8), None, 1.0, 0.95,
+                    abuf[off_out:off_out + N], gbuf[off_out:off_out + N], status, ws)
+        torch.cuda.synchronize()
+        assert int(status) == 0
+        assert adv_close(abuf[off_out:off_out + N].cpu().numpy(), ra, sb, se, ADV_RTOL) <= 1.0
+        assert adv_close(gbuf[off_out:off_out + N].cpu().numpy(), rr, sb, se, ADV_RTOL) <= 1.0
+        assert torch.isnan(abuf[:off_out]).all() and torch.isnan(abuf[off_out + N:]).all()
+
+
 @pytest.mark.parametrize("lam", [0.9, 0.95, 1.0])
 def test_egae_config4_reduced(lam):
     c = synth.config4(B=400)
