@@ -676,7 +676,7 @@ def run_cfg4_workload(args, rank, world, local, dev, warmup):
             "metric": "tokens/s, EGAE + token compaction + value loss + batch advance, config 4",
             "value": N / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": steps, "warmup": warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32 in, f64 scan state, int32 indices", "data": "synthetic",
+            "dtype": "f32 (f64 scan carries), int32 indices", "data": "synthetic",
             "config": {"workload": "cfg4: %d ragged segments, %d tokens, lengths log-uniform in [16, 32768], "
                                    "half truncated, Bernoulli(0.5) masks" % (B, N),
                        "l2": "inputs larger than L2 (%.0f MB per array)" % (N * 4 / 1e6),
