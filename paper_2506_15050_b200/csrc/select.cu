@@ -23,12 +23,14 @@ __device__ __forceinline__ uint32_t sel_pol(uint64_t s) { return uint32_t(s >> 3
 __device__ __forceinline__ uint32_t sel_val(uint64_t s) { return uint32_t(s) & 0x7fffffffu; }
 
 // Number of entries of the ascending array arr[0..n) that are <= key, found by a whole warp: each
-// round probes 32 evenly spaced entries (one load per lane) and narrows the range 32-fold.  Every
-// lane returns the same count; an array that is not ascending still yields an in-range answer.
+// round probes 32 evenly spaced entries (one load per lane) and narrows the range 32-fold until at
+// most 128 entries remain, which are read in one go (four independent loads per lane): 4097
+// entries take two dependent rounds.  Every lane returns the same count; an array that is not
+// ascending still yields an in-range answer.
 __device__ __forceinline__ int warp_count_le(const int32_t* __restrict__ arr, int n, int32_t key,
                                              int lane) {
     int lo = 0, hi = n;       // the answer lies in [lo, hi]
-    while (lo < hi) {
+    while (hi - lo > 128) {
         const int span = hi - lo;
         const int step = (span + 31) >> 5;
         const int idx = lo + lane * step;
@@ -40,7 +42,16 @@ __device__ __forceinline__ int warp_count_le(const int32_t* __restrict__ arr, in
         if (c > 0) lo = lo + (c - 1) * step + 1;
         hi = new_hi;
     }
-    return lo;
+    bool le[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int idx = lo + 32 * j + lane;
+        le[j] = idx < hi && __ldg(arr + idx) <= key;
+    }
+    int count = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) count += __popc(__ballot_sync(0xffffffffu, le[j]));
+    return lo + count;
 }
 
 struct SelectArgs {
