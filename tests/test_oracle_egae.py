@@ -158,3 +158,27 @@ def test_empty_and_length_one_segments():
     assert adv[0] == pytest.approx(0.5 - np.float32(0.1))
     assert adv[1] == 0.0 and ret[1] == 0.0  # the empty segment selects nothing
     assert adv[2] == pytest.approx(0.25)
+
+
+@pytest.mark.parametrize("gamma,lam", [(1.0, 0.95), (0.99, 0.9), (1.0, 1.0), (0.9, 0.0)])
+def test_advantage_is_lambda_return_minus_value(gamma, lam):
+    """A_t + V_t is the lambda-return: G_t = r_t + gamma ((1 - lambda) V_{t+1} + lambda G_{t+1}), with
+    G = r + gamma V_next on the last token (V_next = 0, the bootstrap value, or the token's own
+    value).  A second, textbook form of the same estimator, evaluated here token by token."""
+    rng = np.random.default_rng(11)
+    r, v, sb, se, tr, N = random_case(rng, 7, 40)
+    boots = rng.standard_normal(7).astype(np.float32)
+    for boot in (None, boots):
+        adv, _ = oracle.egae(r, v, sb, se, tr, boot, gamma, lam)
+        ref = np.zeros(N)
+        for i in range(7):
+            b, e = int(sb[i]), int(se[i])
+            G = 0.0
+            for t in range(e - 1, b - 1, -1):
+                if t == e - 1:
+                    vn = (float(v[t]) if boot is None else float(boot[i])) if tr[i] else 0.0
+                    G = float(r[t]) + gamma * vn
+                else:
+                    G = float(r[t]) + gamma * ((1.0 - lam) * float(v[t + 1]) + lam * G)
+                ref[t] = G - float(v[t])
+        np.testing.assert_allclose(adv, ref, rtol=1e-11, atol=1e-11)
