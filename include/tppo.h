@@ -38,7 +38,7 @@ typedef enum {
     TPPO_OK = 0,
     TPPO_ERR_INVALID_ARG = 1, /* null / negative / inconsistent argument, bad alignment      */
     TPPO_ERR_WORKSPACE = 2,   /* workspace pointer null, misaligned or smaller than required */
-    TPPO_ERR_UNSUPPORTED = 3, /* valid request this build cannot serve                       */
+    TPPO_ERR_UNSUPPORTED = 3, /* valid request this library cannot serve                     */
     TPPO_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch error, wrong device)     */
     TPPO_ERR_TOO_LARGE = 5    /* problem exceeds a fixed built-in capacity (see *_static)    */
 } tppo_status;
