@@ -167,3 +167,30 @@ def test_config3_full(inplace):
     # every gradient row sums to ~0 and is finite (property that holds at any size)
     sums = dl.float().sum(dim=1)
     assert bool(torch.isfinite(sums).all()) and float(sums.abs().max()) < 1e-3
+
+
+def test_step_sequence_back_to_back_matches_single_calls():
+    """The four calls of a training step issued back to back, several steps in a row, in the launch
+    configuration the benchmark times (config 3's batch, the cluster-resident policy kernel directly
+    followed by the next step's EGAE scan): every step must reproduce the results of the first one
+    and the advantages must match the oracle."""
+    import os
+    import sys
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+    st = bench.Step(torch.device(DEV), rows=2048)
+    st.run()
+    torch.cuda.synchronize()
+    first = (st.adv.clone(), st.ret.clone(), st.pol.clone(), float(st.loss), float(st.vloss))
+    for _ in range(4):
+        st.run()
+        st.egae()                      # and once more straight after the value loss
+    torch.cuda.synchronize()
+    assert int(st.status) == 0 and int(st.stats[3]) == 0
+    assert torch.equal(st.adv, first[0]) and torch.equal(st.ret, first[1]) and torch.equal(st.pol, first[2])
+    assert float(st.loss) == first[3] and float(st.vloss) == first[4]
+    c = st.c
+    ra, rr = oracle.egae(c["rewards"], c["values"], c["seg_begin"], c["seg_end"], c["truncated"], None,
+                         np.float32(c["gamma"]), np.float32(c["lam"]))
+    assert adv_close(st.adv.cpu().numpy(), ra, c["seg_begin"], c["seg_end"], 1e-5) <= 1.0
+    assert adv_close(st.ret.cpu().numpy(), rr, c["seg_begin"], c["seg_end"], 1e-5) <= 1.0
