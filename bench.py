@@ -272,6 +272,58 @@ def time_lmhead(lm, calls, warmup):
     return e0.elapsed_time(e1) / calls
 
 
+def time_lmhead_rank_of_shards(lm, shards, calls, warmup):
+    """What ONE rank of a vocabulary-parallel LM-head executes per step (its statistics call, the
+    rescale between the two all-reduces, its loss + gradient call), with the other ranks' statistics
+    produced beforehand on the same GPU.  The collectives themselves are not part of the number."""
+    b, dev, M, K, V = lm.b, lm.dev, lm.M, lm.K, lm.V
+    width = (V // shards + 7) // 8 * 8
+    bounds = [min(i * width, V) for i in range(shards)] + [V]
+    stats = []
+    for lo, hi in zip(bounds[:-1], bounds[1:]):
+        w = lm.weight[:, lo:hi].contiguous()
+        m_, s_, xy_ = (torch.empty(M, device=dev) for _ in range(3))
+        st = torch.zeros(4, dtype=torch.int32, device=dev)
+        ws = b.workspace(b.OP_LMHEAD, M, K, 0, hi - lo, dev)
+        b.tppo_lmhead_shard_stats(lm.hidden, w, lo, V, lm.targets, m_, s_, xy_, st, ws)
+        stats.append((m_, s_, xy_))
+        del w, ws
+    m_all = torch.stack([x[0] for x in stats]).max(dim=0).values
+    for m_, s_, _ in stats:
+        b.tppo_lmhead_shard_rescale(m_, m_all, s_)
+    s_all = torch.stack([x[1] for x in stats]).sum(dim=0)
+    xy_all = torch.stack([x[2] for x in stats]).sum(dim=0)
+    w0 = lm.weight[:, bounds[0]:bounds[1]].contiguous()
+    dw0 = torch.empty_like(w0)
+    ws = b.workspace(b.OP_LMHEAD, M, K, 0, bounds[1] - bounds[0], dev)
+    m0, s0, xy0 = (torch.empty(M, device=dev) for _ in range(3))
+    st = torch.zeros(4, dtype=torch.int32, device=dev)
+    c = lm.c
+
+    def rank_step():
+        b.tppo_lmhead_shard_stats(lm.hidden, w0, 0, V, lm.targets, m0, s0, xy0, st, ws)
+        b.tppo_lmhead_shard_rescale(m0, m_all, s0)
+        b.tppo_lmhead_shard_fwd_bwd(lm.hidden, w0, 0, V, lm.targets, None, lm.old_logp, lm.adv,
+                                    c["eps_low"], c["eps_high"], 0.0, m_all, s_all, xy_all, lm.logp,
+                                    lm.tok_loss, lm.loss, lm.stats, lm.dhidden, dw0, ws)
+
+    for _ in range(warmup):
+        rank_step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(calls):
+        rank_step()
+    e1.record()
+    torch.cuda.synchronize()
+    assert int(lm.stats[3].item()) == 0
+    return {"shards": shards, "per_rank_ms": e0.elapsed_time(e1) / calls,
+            "exchange_bytes_per_rank": {"row_statistics_allreduce": 12 * M, "dhidden_allreduce": 2 * M * K},
+            "note": "one rank's three calls timed on one GPU; the other ranks' statistics were "
+                    "produced beforehand; the two small all-reduces and the dhidden all-reduce are "
+                    "not timed"}
+
+
 def cpu_oracle_lmhead_seconds(lm, sample_rows):
     """The oracle on `sample_rows` rows of the LM-head workload: float64 logits, Eq. 1, dhidden rows
     and those rows' share of dweight; scaled by rows to the whole call."""
@@ -360,6 +412,8 @@ def main():
                     help="rows of the loss micro-batch (smaller only for profiler captures)")
     ap.add_argument("--workload", default="cfg3", choices=["cfg3", "lmhead", "cfg4"])
     ap.add_argument("--lmhead-calls", type=int, default=5)
+    ap.add_argument("--lm-shards", type=int, default=1,
+                    help="with --workload lmhead: also time one rank of this many vocabulary shards")
     ap.add_argument("--lm-rows", type=int, default=16384,
                     help="rows of the LM-head workload (smaller only for profiler captures)")
     ap.add_argument("--no-lmhead", action="store_true")
@@ -573,8 +627,13 @@ def run_lmhead_workload(args, rank, world, local, dev, warmup):
         cpu = {"value": lm.M / t, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": "8 of %d rows (float64 logits, Eq. 1, dhidden rows, dweight share), scaled by rows" % lm.M}
     n_chunk_launches = 3 * ((lm.V + 255) // 256 + 61) // 62
+    shard_info = None
+    if args.lm_shards > 1 and world == 1:
+        shard_info = time_lmhead_rank_of_shards(lm, args.lm_shards, max(3, steps // 4), warmup)
+        shard_info["unsharded_ms"] = ms
     if rank == 0:
         print(json.dumps({
+            "vocab_shards": shard_info,
             "metric": "selected tokens/s, LM-head variant: fused hidden x vocab contraction + PPO loss "
                       "fwd+bwd, V=152064 bf16; % tensor peak",
             "value": world * lm.M / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
