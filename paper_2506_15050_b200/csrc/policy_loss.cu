@@ -55,19 +55,21 @@ __global__ void __launch_bounds__(1024) policy_finish_kernel(const PolicyArgs a)
     const int64_t n = policy_n(a);
     double acc = 0.0;
     int lo = 0, hi = 0;
-    // four rows per trip, loads first, so that their latencies overlap; the order of the adds is fixed
+    // sixteen rows per trip (a whole 16384-row micro-batch in one), loads first, so that their
+    // latencies overlap; the order of the adds is fixed
+    constexpr int kPerTrip = 16;
     const int64_t step = blockDim.x;
-    for (int64_t j = threadIdx.x; j < n; j += 4 * step) {
-        float l[4];
-        uint8_t c[4];
+    for (int64_t j = threadIdx.x; j < n; j += kPerTrip * step) {
+        float l[kPerTrip];
+        uint8_t c[kPerTrip];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kPerTrip; ++u) {
             const int64_t q = j + u * step;
             l[u] = q < n ? a.row_loss[q] : 0.f;
             c[u] = q < n ? a.row_clip[q] : uint8_t(0);
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kPerTrip; ++u) {
             acc += double(l[u]);
             lo += c[u] == 1;
             hi += c[u] == 2;
