@@ -83,7 +83,7 @@ def egae(rewards, values, seg_begin, seg_end, truncated, bootstrap, gamma, lam,
 
 
 def select_tokens(seq_begin, prompt_len, prev_len, new_len, truncated, tail_drop=0,
-                  extra_policy_mask=None, extra_value_mask=None, N=None):
+                  extra_policy_mask=None, extra_value_mask=None, N=None, tail_drop_seq=None):
     sb = _arr(seq_begin, np.int32)
     pl = _arr(prompt_len, np.int32)
     pv = _arr(prev_len, np.int32)
@@ -97,8 +97,10 @@ def select_tokens(seq_begin, prompt_len, prev_len, new_len, truncated, tail_drop
     pol = np.empty(max(N, 1), np.int32)
     val = np.empty(max(N, 1), np.int32)
     counts = np.zeros(2, np.int64)
+    tds = _arr(tail_drop_seq, np.int32)
+    assert tds is None or tds.shape[0] == B
     lib().oracle_select_tokens(_p(sb), _p(pl), _p(pv), _p(nl), _p(tr), C.c_int32(tail_drop),
-                               _p(em), _p(ev), C.c_int32(B), C.c_int64(N),
+                               _p(tds), _p(em), _p(ev), C.c_int32(B), C.c_int64(N),
                                _p(pol), _p(val), _p(counts))
     return pol[:counts[0]].copy(), val[:counts[1]].copy()
 

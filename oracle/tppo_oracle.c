@@ -103,13 +103,16 @@ void oracle_egae(const float *rewards, const float *values,
  * Token filtering (Section 3.2).  Sequence i occupies packed positions
  * [seq_begin[i], seq_begin[i+1]) laid out  prompt | earlier-window response | this-window
  * response.  Policy tokens: the response tokens generated in the current step, finished or
- * not, minus the last tail_drop tokens of an unfinished sequence.  Value tokens: every
- * generated token of a finished sequence.  Prompt tokens enter neither set.  Optional byte
- * masks AND with the predicates.  Lists are in ascending position order.
+ * not, minus the latest tokens of an unfinished sequence (Section 3.2 allows leaving some of
+ * them out; how many is a parameter: tail_drop for every unfinished sequence, or
+ * tail_drop_seq[i] for sequence i when that array is given; a negative count means none).
+ * Value tokens: every generated token of a finished sequence.  Prompt tokens enter neither
+ * set.  Optional byte masks AND with the predicates.  Lists are in ascending position order.
  * ---------------------------------------------------------------------------------------- */
 void oracle_select_tokens(const int32_t *seq_begin, const int32_t *prompt_len,
                           const int32_t *prev_len, const int32_t *new_len,
                           const uint8_t *truncated, int32_t tail_drop,
+                          const int32_t *tail_drop_seq /* [B] or NULL */,
                           const uint8_t *extra_policy_mask, const uint8_t *extra_value_mask,
                           int32_t B, int64_t N,
                           int32_t *policy_idx, int32_t *value_idx, int64_t *counts)
@@ -124,7 +127,9 @@ void oracle_select_tokens(const int32_t *seq_begin, const int32_t *prompt_len,
         const int64_t resp0 = prompt_len[i];
         const int64_t new0 = (int64_t)prompt_len[i] + prev_len[i];
         const int64_t end = new0 + new_len[i];
-        int64_t pol_end = end - (truncated[i] ? tail_drop : 0);
+        int64_t drop = tail_drop_seq ? tail_drop_seq[i] : tail_drop;
+        if (drop < 0) drop = 0;
+        int64_t pol_end = end - (truncated[i] ? drop : 0);
         int is_pol = off >= new0 && off < pol_end;
         int is_val = !truncated[i] && off >= resp0 && off < end;
         if (extra_policy_mask) is_pol = is_pol && extra_policy_mask[p] != 0;
