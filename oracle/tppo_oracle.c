@@ -143,9 +143,13 @@ void oracle_select_tokens(const int32_t *seq_begin, const int32_t *prompt_len,
 
 /* ------------------------------------------------------------------------------------------
  * log pi(a|s) of Eq. 1 from a row of logits: x_y - log sum_v exp(x_v), with the usual shift
- * by the row maximum, summed in index order.
+ * by the row maximum m, summed in index order:
+ *     log pi(y) = (x_y - m) - log S,    softmax_v = exp((x_v - m) - log S),    S = sum_v exp(x_v - m).
+ * The maximum and log S are kept apart (never added), so that the result is also exact for
+ * logits of the largest representable magnitude, where m + log S would round log S away.
  * ---------------------------------------------------------------------------------------- */
-static double row_logsumexp(const void *logits, int dtype, int64_t ld, int64_t row, int32_t V)
+static void row_max_and_logsum(const void *logits, int dtype, int64_t ld, int64_t row, int32_t V,
+                               double *row_max, double *log_sum)
 {
     double m = -INFINITY;
     for (int32_t v = 0; v < V; ++v) {
@@ -154,7 +158,8 @@ static double row_logsumexp(const void *logits, int dtype, int64_t ld, int64_t r
     }
     double S = 0.0;
     for (int32_t v = 0; v < V; ++v) S += exp(logit_at(logits, dtype, ld, row, v) - m);
-    return m + log(S);
+    *row_max = m;
+    *log_sum = log(S);
 }
 
 void oracle_logprob(const void *logits, int dtype, int32_t V, int64_t ld,
@@ -164,8 +169,9 @@ void oracle_logprob(const void *logits, int dtype, int32_t V, int64_t ld,
 #pragma omp parallel for schedule(dynamic, 1)
     for (int64_t j = 0; j < n; ++j) {
         const int64_t row = rows ? rows[j] : j;
-        const double lse = row_logsumexp(logits, dtype, ld, row, V);
-        logp[j] = logit_at(logits, dtype, ld, row, targets[row]) - lse;
+        double m, log_sum;
+        row_max_and_logsum(logits, dtype, ld, row, V, &m, &log_sum);
+        logp[j] = (logit_at(logits, dtype, ld, row, targets[row]) - m) - log_sum;
     }
 }
 
@@ -197,8 +203,9 @@ void oracle_policy_loss(const void *logits, int dtype, int32_t V, int64_t ld,
         const int64_t row = rows ? rows[j] : j;
         const int64_t a = aux_idx ? aux_idx[j] : row;
         const int32_t y = targets[row];
-        const double lse = row_logsumexp(logits, dtype, ld, row, V);
-        const double lp = logit_at(logits, dtype, ld, row, y) - lse;
+        double m, log_sum;
+        row_max_and_logsum(logits, dtype, ld, row, V, &m, &log_sum);
+        const double lp = (logit_at(logits, dtype, ld, row, y) - m) - log_sum;
         const double A = (double)adv[a];
         const double rho = exp(lp - (double)old_logp[a]);
         double rc = rho;
@@ -216,7 +223,7 @@ void oracle_policy_loss(const void *logits, int dtype, int32_t V, int64_t ld,
             const double g = active ? -(A * rho) / d : 0.0; /* dL/dlogp */
             double *out = dlogits + j * (int64_t)V;
             for (int32_t v = 0; v < V; ++v) {
-                const double p = exp(logit_at(logits, dtype, ld, row, v) - lse);
+                const double p = exp((logit_at(logits, dtype, ld, row, v) - m) - log_sum);
                 out[v] = g * ((v == y ? 1.0 : 0.0) - p);
             }
         }

@@ -49,6 +49,31 @@ def test_logprob_bf16_and_extremes():
     assert oracle.logprob(x, np.array([4], np.int32))[0] == pytest.approx(-2e4)
 
 
+def test_logprob_and_gradient_at_the_largest_magnitudes():
+    """Closed forms at the largest finite bf16 / fp32 values, where adding log S to the maximum
+    would lose it: a constant row is uniform (log-prob -log V, gradient factor*(1/V - onehot)) and one
+    +max among -max is one-hot (log-prob 0, gradient 0)."""
+    V = 40
+    big = np.float32(3.3895313892515355e38)            # largest finite bf16
+    x = np.zeros((3, V), np.float32)
+    x[0, :] = big
+    x[1, :] = -big
+    x[1, 5] = big
+    x[2, :] = -big
+    y = np.array([7, 5, 0], np.int32)
+    lp = oracle.logprob(x, y)
+    np.testing.assert_allclose(lp, [-np.log(V), 0.0, -np.log(V)], rtol=0, atol=1e-12)
+    adv = np.array([1.0, -1.0, 0.5], np.float32)
+    out = oracle.policy_loss(x, y, None, None, lp.astype(np.float32), adv, 0.2, 0.2)
+    onehot = np.zeros((3, V))
+    onehot[np.arange(3), y] = 1.0
+    p = np.stack([np.full(V, 1.0 / V), onehot[1], np.full(V, 1.0 / V)])
+    rho = np.exp(lp - lp.astype(np.float32))
+    np.testing.assert_allclose(out["dlogits"], (adv * rho / 3)[:, None] * (p - onehot), rtol=1e-12, atol=1e-18)
+    # a constant row of float64 logits at 2^100: uniform as well
+    np.testing.assert_allclose(oracle.logprob(np.full((1, V), 2.0 ** 100), y[:1]), [-np.log(V)], atol=1e-12)
+
+
 def torch_policy_loss(x, y, old, adv, el, eh, denom):
     """Eq. 1 restated with autograd as an independent comparator (float64)."""
     xt = torch.tensor(x, dtype=torch.float64, requires_grad=True)
