@@ -108,15 +108,47 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def dist_setup(n_gpus: int):
+def spawn_ranks(n_gpus: int) -> int:
+    """`python bench.py --gpus N` outside torchrun: start the N ranks of one node ourselves (the same
+    launcher and rendezvous a torchrun command line would use) and return their exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def dist_setup(n_gpus: int, need_cuda: bool = True):
+    """Rank, world size and local rank from the launcher's environment; NCCL between GPUs (gloo when
+    there is no GPU, which only the launcher's own test uses).  The world that came up must be the
+    one that was asked for."""
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != n_gpus:
+        raise SystemExit(f"bench.py: --gpus {n_gpus} but the launcher started {world} rank(s)")
     if world > 1:
         import torch.distributed as dist
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        if need_cuda and torch.cuda.is_available():
+            if torch.cuda.device_count() < world:
+                raise SystemExit(f"bench.py: {world} ranks but {torch.cuda.device_count()} GPU(s)")
+            os.environ.setdefault("NCCL_DEBUG", "INFO")          # the init log shows the ranks of the communicator
+            os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+            torch.cuda.set_device(local)
+            dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        else:
+            dist.init_process_group("gloo")
+        if dist.get_world_size() != n_gpus:
+            raise SystemExit(f"bench.py: process group has {dist.get_world_size()} ranks, wanted {n_gpus}")
     return rank, world, local
+
+
+def time_stats(ms_list):
+    """mean / median / min of per-step device times (ms)."""
+    a = np.asarray(ms_list, np.float64)
+    return {"mean": float(a.mean()), "median": float(np.median(a)), "min": float(a.min())}
 
 
 class Step:
@@ -372,30 +404,65 @@ def cpu_oracle_step_seconds(c, n_tokens, sample_rows):
         {"egae_s": t1 - t0, "select_s": t2 - t1, "policy_sample_s": t3 - t2, "value_s": t4 - t3}
 
 
+def workload_config(N, n_tok, n_val, hint=0):
+    """The `config` object of the bench line: the same for this repo's arm and the reference arm."""
+    return {"workload": "cfg3: EGAE over 512 ragged responses (N=%d tokens), selection, [%d,152064] bf16 "
+                        "fused log-prob+PPO loss fwd+bwd, value loss on %d tokens" % (N, n_tok, n_val),
+            "l2": "inputs larger than L2 (%.2f GB logits per step)" % (n_tok * synth.V_QWEN * 2 / 1e9),
+            "dlogits": "compact, separate buffer", "kernel_hint": hint}
+
+
 def run_reference(args, rank):
-    """The oracle on the host cores: same metric, bounded sample per step."""
+    """The oracle on the host cores, as it stands: same metric, a bounded sample per step.  A step is
+    EGAE, selection and the value loss on the full batch plus the policy loss forward+backward on
+    `--ref-rows` rows of the micro-batch; the reported time is the measured time of that step and the
+    value counts the rows that went through the policy loss in it."""
     if rank != 0:
         return
     c = synth.config3("cpu", with_logits=False)
     sample_rows = args.ref_rows
     c["logits_sample"] = synth.bf16_bits(synth.randn_bf16((sample_rows, synth.V_QWEN), 2.0, 2, "cpu"))
     times = []
+    cores = 1
     for i in range(args.warmup + args.steps):
-        t, cores, parts = cpu_oracle_step_seconds(c, c["n_tokens"], sample_rows)
+        w0 = time.perf_counter()
+        _, cores, parts = cpu_oracle_step_seconds(c, c["n_tokens"], sample_rows)
         if i >= args.warmup:
-            times.append(t)
+            times.append(time.perf_counter() - w0)
     t = float(np.mean(times))
-    value = c["n_tokens"] / t
-    sample = (f"EGAE+selection+value loss on the full batch, policy loss fwd+bwd on {sample_rows} of "
-              f"{c['n_tokens']} rows (V=152064) scaled to the full micro-batch")
+    value = sample_rows / t
+    sample = (f"per step: EGAE+selection+value loss on the full batch, policy loss fwd+bwd on {sample_rows} "
+              f"of {c['n_tokens']} rows (V=152064); value = those {sample_rows} rows / measured step time")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "cfg3: 512-response EGAE batch + [16384,152064] bf16 loss micro-batch"},
+        "config": workload_config(c["N"], c["n_tokens"], int(c["extra_value_mask"].sum()), args.hint),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
+
+
+def run_stub(args, rank, world):
+    """A step that needs no GPU, for the launcher's own test: every rank does a fixed piece of host
+    work, the ranks meet at a barrier, and rank 0 prints the line with the world size that came up."""
+    import torch.distributed as dist
+    x = torch.arange(1 << 16, dtype=torch.float64)
+    w0 = time.perf_counter()
+    for _ in range(args.warmup + args.steps):
+        x = (x * 1.0000001).cumsum(0) % 7.0
+    t = torch.tensor([time.perf_counter() - w0], dtype=torch.float64)
+    if world > 1:
+        dist.barrier()
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    if rank == 0:
+        print(json.dumps({"metric": "stub steps/s (launcher test)", "value": world * args.steps / float(t),
+                          "unit": "steps/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                          "ms_per_step": float(t) * 1e3 / max(args.steps, 1), "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                          "config": {"workload": "stub"}, "gpu_launches": 0}))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 def main():
@@ -410,20 +477,30 @@ def main():
     ap.add_argument("--hint", type=int, default=0, help="kernel_hint passed to the policy loss")
     ap.add_argument("--rows", type=int, default=16384,
                     help="rows of the loss micro-batch (smaller only for profiler captures)")
-    ap.add_argument("--workload", default="cfg3", choices=["cfg3", "lmhead", "cfg4"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg3", "lmhead", "cfg4", "stub"])
     ap.add_argument("--lmhead-calls", type=int, default=5)
     ap.add_argument("--lm-shards", type=int, default=1,
                     help="with --workload lmhead: also time one rank of this many vocabulary shards")
     ap.add_argument("--lm-rows", type=int, default=16384,
                     help="rows of the LM-head workload (smaller only for profiler captures)")
+    ap.add_argument("--cfg4-steps", type=int, default=30, help="steps of the small-kernel measurement")
     ap.add_argument("--no-lmhead", action="store_true")
+    ap.add_argument("--no-small", action="store_true", help="skip the config-4 small-kernel measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
 
-    rank, world, local = dist_setup(args.gpus)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus))           # one process per GPU, started here
+    rank, world, local = dist_setup(args.gpus, need_cuda=args.workload != "stub" and args.impl == "ours")
+    if args.workload == "stub":
+        run_stub(args, rank, world)
+        return
     if args.impl == "reference":
         run_reference(args, rank)
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the CUDA path has no CPU fallback")
@@ -458,27 +535,32 @@ def main():
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    events = []
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record()
+    events, marks = [], [torch.cuda.Event(enable_timing=True)]
+    marks[0].record()
     for _ in range(args.steps):
         st.run(events)
-    t1.record()
+        marks.append(torch.cuda.Event(enable_timing=True))
+        marks[-1].record()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    ms_total = t0.elapsed_time(t1)
+    ms_total = marks[0].elapsed_time(marks[-1])
     if world > 1:
         import torch.distributed as dist
         tt = torch.tensor([ms_total], device=dev)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         ms_total = float(tt.item())
     ms_step = ms_total / args.steps
+    step_ms = time_stats([a.elapsed_time(b) for a, b in zip(marks[:-1], marks[1:])])
     n_tok = int(st.counts[0].item())
+    n_val = int(st.counts[1].item())
     assert n_tok == st.n and int(st.stats[3].item()) == 0 and int(st.status.item()) == 0
     value = world * n_tok / (ms_step * 1e-3)
-    pol_ms = float(np.mean([a.elapsed_time(b) for a, b in events]))
+    pol = time_stats([a.elapsed_time(b) for a, b in events])
+    pol_ms = pol["mean"]
     peak, peak_kind = measured_peaks()
-    achieved = n_tok * ALGO_BYTES_PER_TOKEN / (pol_ms * 1e-3) / 1e9
+    algo_bytes = n_tok * ALGO_BYTES_PER_TOKEN
+    achieved = algo_bytes / (pol_ms * 1e-3) / 1e9
+    traffic = n_tok * NCU_TRAFFIC_BYTES_PER_TOKEN if (st.V == synth.V_QWEN and NCU_TRAFFIC_BYTES_PER_TOKEN) else None
 
     # ---- end to end: host buffers in, losses out, copies inside the timed region ---------------
     e2e = None
@@ -529,10 +611,17 @@ def main():
                           f"{args.cpu_rows} of {n_tok} rows scaled to the micro-batch"),
                "seconds": {k: round(v, 4) for k, v in parts.items()}}
 
+    small_kernels = None
     lmhead = None
-    if rank == 0 and not args.no_lmhead:
+    if rank == 0 and not (args.no_small and args.no_lmhead):
         del st.logits, st.dlogits, st.c["logits"]
         torch.cuda.empty_cache()
+    if rank == 0 and not args.no_small:
+        # the four small calls, against their own algorithmic bytes, on the bandwidth-sized config 4
+        small_kernels = measure_cfg4(dev, args.cfg4_steps, 3)
+        small_kernels.pop("clocks", None)
+        torch.cuda.empty_cache()
+    if rank == 0 and not args.no_lmhead:
         lm = LmHeadStep(dev, M=args.lm_rows)
         ms = time_lmhead(lm, args.lmhead_calls, 3)
         lmhead = {"workload": "cfg5: hidden [%d,%d] x LM-head weight [%d,%d] bf16, loss + dhidden + "
@@ -545,31 +634,143 @@ def main():
         dist.barrier()
 
     if rank == 0:
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_kind": peak_kind,
+                    "frac_of_nominal_8TBs": achieved / 8000.0,
+                    "traffic": traffic,
+                    "traffic_note": "ncu dram__bytes_read.sum + dram__bytes_write.sum of a 2048-row capture "
+                                    "of the same kernel, scaled by rows",
+                    # the same launch time against the bytes ncu saw cross the DRAM interface (less than the
+                    # algorithmic bytes: the last gradient rows are still in L2 when the kernel ends)
+                    "achieved_measured_traffic": None if traffic is None else traffic / (pol_ms * 1e-3) / 1e9,
+                    "frac_measured_traffic": None if traffic is None else traffic / (pol_ms * 1e-3) / 1e9 / peak,
+                    "kernel": "policy_cluster_kernel (+ policy_prepare / policy_finish)",
+                    "kernel_ms": pol_ms, "kernel_ms_median": pol["median"], "kernel_ms_min": pol["min"],
+                    "algorithmic_bytes_per_launch": algo_bytes,
+                    "small_kernels": None if small_kernels is None else small_kernels["kernels"],
+                    "lmhead_variant": None if lmhead is None else lmhead["roofline"]}
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": warmup, "ms_per_step": ms_step, "ms_per_step_median": step_ms["median"],
+            "ms_per_step_min": step_ms["min"],
+            "value_at_median_step": world * n_tok / (step_ms["median"] * 1e-3),
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
-            "config": {"workload": "cfg3: EGAE over 512 ragged responses (N=%d tokens), selection, "
-                                   "[%d,152064] bf16 fused log-prob+PPO loss fwd+bwd, value loss "
-                                   "on %d tokens" % (st.N, st.n, int(st.counts[1].item())),
-                       "l2": "inputs larger than L2 (%.2f GB logits per step)" % (st.n * st.V * 2 / 1e9),
-                       "dlogits": "compact, separate buffer", "kernel_hint": args.hint},
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "peak_kind": peak_kind,
-                         "frac_of_nominal_8TBs": achieved / 8000.0,
-                         "traffic": n_tok * NCU_TRAFFIC_BYTES_PER_TOKEN if st.V == synth.V_QWEN else None,
-                         "traffic_note": "ncu DRAM bytes of a 2048-row capture scaled by rows",
-                         "kernel": "policy_cluster_kernel", "kernel_ms": pol_ms,
-                         "algorithmic_bytes_per_launch": n_tok * ALGO_BYTES_PER_TOKEN},
+            "config": workload_config(st.N, st.n, n_val, args.hint),
+            "roofline": roofline,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": Step.KERNELS_PER_STEP * args.steps,
-            "clocks": clocks, "lmhead_variant": lmhead}))
+            "clocks": clocks, "small_kernels": small_kernels, "lmhead_variant": lmhead}))
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
 
 
+class LmHeadShardStep:
+    """One rank of the vocabulary-parallel LM-head (the weight split by columns over the ranks, rows and
+    per-token scalars replicated): its two shard calls with the exchange between them and the dhidden
+    all-reduce after them, all through `shard.vocab_parallel_step` (NCCL collectives; no rank reads
+    another rank's memory)."""
+
+    def __init__(self, dev, rank, world, M=16384, K=5120, V=synth.V_QWEN):
+        from paper_2506_15050_b200 import binding as b
+        from paper_2506_15050_b200 import shard
+        self.b, self.shard, self.dev, self.M, self.K, self.V = b, shard, dev, M, K, V
+        c = synth.config5(dev, M=M, K=K, V=V)                 # same seed on every rank: replicated inputs
+        self.c = c
+        self.lo, self.hi = shard.vocab_shard_bounds(V, world)[rank]
+        self.weight = c["weight"][:, self.lo:self.hi].contiguous()
+        del c["weight"]
+        torch.cuda.empty_cache()
+        t = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).to(dev)
+        self.hidden = c["hidden"]
+        self.targets, self.adv = t(c["targets"], torch.int32), t(c["adv"], torch.float32)
+        self.old_logp = torch.full((M,), -12.0, device=dev)
+        self.m_, self.s_, self.xy_ = (torch.empty(M, device=dev) for _ in range(3))
+        self.logp, self.tok_loss = torch.zeros(M, device=dev), torch.zeros(M, device=dev)
+        self.loss = torch.zeros(1, device=dev)
+        self.stats = torch.zeros(4, dtype=torch.int32, device=dev)
+        self.sstats = torch.zeros(4, dtype=torch.int32, device=dev)
+        self.dhidden = torch.empty_like(self.hidden)
+        self.dweight = torch.empty_like(self.weight)
+        self.ws = b.workspace(b.OP_LMHEAD, M, K, 0, self.hi - self.lo, dev)
+        # old-policy log-probs: the merged statistics of a first pass give the current ones; add the noise
+        self.run(grads=False)
+        torch.cuda.synchronize()
+        self.old_logp.copy_(self.logp + t(c["old_logp_noise"], torch.float32))
+
+    def run(self, grads=True):
+        b, c = self.b, self.c
+
+        def stats_fn():
+            b.tppo_lmhead_shard_stats(self.hidden, self.weight, self.lo, self.V, self.targets, self.m_,
+                                      self.s_, self.xy_, self.sstats, self.ws)
+            return self.m_, self.s_, self.xy_
+
+        def grads_fn(m, s_, xy):
+            b.tppo_lmhead_shard_fwd_bwd(self.hidden, self.weight, self.lo, self.V, self.targets, None,
+                                        self.old_logp, self.adv, c["eps_low"], c["eps_high"], 0.0, m, s_, xy,
+                                        self.logp, self.tok_loss, self.loss, self.stats,
+                                        self.dhidden if grads else None, self.dweight if grads else None,
+                                        self.ws)
+            return self.dhidden if grads else None
+
+        self.shard.vocab_parallel_step(stats_fn, b.tppo_lmhead_shard_rescale, grads_fn)
+
+
+def run_lmhead_vocab_parallel(args, rank, world, local, dev, warmup):
+    """`--workload lmhead --gpus N`: config 5 with the vocabulary split over N ranks.  One step = the
+    whole exchange (statistics GEMM, two small all-reduces, gradient GEMMs, dhidden all-reduce), timed on
+    the device with the collectives inside; total work is fixed as N grows ("strong")."""
+    import torch.distributed as dist
+    lm = LmHeadShardStep(dev, rank, world, M=args.lm_rows)
+    steps = args.steps if args.steps != 200 else 20
+    for _ in range(warmup):
+        lm.run()
+    dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        lm.run()
+    t1.record()
+    dist.barrier()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    tt = torch.tensor([t0.elapsed_time(t1) / steps], device=dev)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    ms = float(tt.item())
+    bits = torch.tensor([int(lm.stats[3].item()) | int(lm.sstats[3].item())], device=dev)
+    dist.all_reduce(bits, op=dist.ReduceOp.MAX)
+    assert int(bits.item()) == 0
+    burst, sustained, kind = measured_tensor_peaks()
+    flops = 2.0 * lm.M * lm.K * lm.V
+    achieved = 3.0 * flops / (ms * 1e-3) / 1e12 / world           # per GPU
+    if rank == 0:
+        print(json.dumps({
+            "metric": "selected tokens/s, LM-head variant, vocabulary split over the ranks; % tensor peak",
+            "value": lm.M / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
+            "config": {"workload": "cfg5 vocabulary-parallel: hidden [%d,%d] replicated, LM-head weight "
+                                   "[%d,%d] bf16 in %d column shards" % (lm.M, lm.K, lm.K, lm.V, world),
+                       "exchange_bytes_per_rank": {"row_statistics": 12 * lm.M, "dhidden_allreduce": 2 * lm.M * lm.K}},
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": sustained, "unit": "TFLOP/s per GPU",
+                         "frac": achieved / sustained, "peak_kind": kind + ", sustained", "traffic": None,
+                         "kernel": "umma_gemm_kernel, one column shard per rank, collectives inside the step"},
+            "cpu_baseline": None, "e2e": None, "clocks": clocks,
+            "gpu_launches": (6 + 3 * (((lm.hi - lm.lo + 255) // 256 + 61) // 62)) * steps}))
+    dist.destroy_process_group()
+
+
 def run_lmhead_workload(args, rank, world, local, dev, warmup):
-    """The LM-head variant as the bench line: one step = one call (loss, dhidden, dweight)."""
+    """The LM-head variant as the bench line: one step = one call (loss, dhidden, dweight).  With
+    several ranks the vocabulary is split over them (see run_lmhead_vocab_parallel)."""
+    if world > 1:
+        run_lmhead_vocab_parallel(args, rank, world, local, dev, warmup)
+        return
     lm = LmHeadStep(dev, M=args.lm_rows)
     steps = args.steps if args.steps != 200 else 20
 
@@ -651,17 +852,26 @@ def run_lmhead_workload(args, rank, world, local, dev, warmup):
 
 
 
-def run_cfg4_workload(args, rank, world, local, dev, warmup):
+# dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of each small kernel on config 4
+# (profiles/egae_select_value_advance_cfg4.md gives the command); None once a kernel has changed
+# since its counters were taken.
+NCU_CFG4_TRAFFIC = {"egae": None, "select": None, "value": None, "advance": None}
+
+
+def measure_cfg4(dev, steps, warmup):
     """Config 4, the bandwidth test of the small kernels: EGAE, token selection, value loss and the
-    batch advance over 4096 ragged segments (17.5 M tokens).  One step = the four calls; every call is
-    also timed on its own (CUDA events) against its algorithmic bytes."""
+    batch advance over 4096 ragged segments (17.5 M tokens).  One step = the four calls back to back;
+    every call is also timed on its own (CUDA events around the C-ABI call, memsets included) against
+    its algorithmic bytes.  Also times the scan on dense (process) rewards with gamma < 1."""
     from paper_2506_15050_b200 import binding as b
     c = synth.config4()
     N, B = c["N"], c["B"]
     t = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).to(dev)
     rng = np.random.default_rng(8)
     rewards, values = t(c["rewards"], torch.float32), t(c["values"], torch.float32)
-    old_values = values + 0.2 * torch.randn(N, device=dev, generator=torch.Generator(dev).manual_seed(3))
+    gen = torch.Generator(dev).manual_seed(3)
+    old_values = values + 0.2 * torch.randn(N, device=dev, generator=gen)
+    dense_rewards = torch.randn(N, device=dev, generator=gen)
     sb, se, tr = t(c["seg_begin"], torch.int32), t(c["seg_end"], torch.int32), t(c["truncated"], torch.uint8)
     boot = t(c["bootstrap"], torch.float32)
     seqb = t(c["seq_begin"], torch.int32)
@@ -696,20 +906,22 @@ def run_cfg4_workload(args, rank, world, local, dev, warmup):
                                                 fs, src, acn),
     }
 
+    def timed(f, events):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); f(); e1.record()
+        events.append((e0, e1))
+
     def step(events=None):
         for name, f in calls.items():
             if events is None:
                 f()
             else:
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(); f(); e1.record()
-                events[name].append((e0, e1))
+                timed(f, events[name])
 
-    steps = args.steps if args.steps != 200 else 50
     for _ in range(warmup):
         step()
     torch.cuda.synchronize()
-    sampler = ClockSampler(local)
+    sampler = ClockSampler(torch.cuda.current_device())
     sampler.start()
     events = {k: [] for k in calls}
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -722,33 +934,60 @@ def run_cfg4_workload(args, rank, world, local, dev, warmup):
     ms = t0.elapsed_time(t1) / steps
     cn, an = counts.cpu().numpy(), acn.cpu().numpy()
     assert int(status) == 0 and cn[2] == 0 and an[3] == 0 and int(vst[1]) == 0
+    # the scan on dense rewards with discounting (process rewards; the paper trains on gamma = 1)
+    dense = {}
+    for gamma in (0.99, 0.999):
+        ev = []
+        for i in range(3 + max(steps // 3, 5)):
+            timed(lambda: b.tppo_egae(dense_rewards, values, sb, se, tr, boot, gamma, 0.95, adv, ret, status, ws1), ev)
+        torch.cuda.synchronize()
+        assert int(status) == 0
+        dense["gamma_%g" % gamma] = time_stats([a.elapsed_time(b_) * 1e3 for a, b_ in ev[3:]])
     peak, kind = measured_peaks()
     algo = {"egae": 16 * N, "select": 2 * N + 4 * (int(cn[0]) + int(cn[1])),
             "value": 20 * int(cn[1]) + 4 * N, "advance": 8 * int(an[2])}
+    per_unit = {"egae": "16 B/token (rewards, values in; advantages, returns out)",
+                "select": "1 B/token per byte mask read (two masks) + 4 B per selected index written",
+                "value": "20 B/value token (index, value, old value, return, gradient) + 4 B/token of dvalues written",
+                "advance": "8 B/context token (read + write)"}
     kernels = {}
     for k, ev in events.items():
-        us = float(np.mean([a.elapsed_time(b_) for a, b_ in ev])) * 1e3
-        gbs = algo[k] / us / 1e3
-        kernels[k] = {"us": us, "algorithmic_bytes": algo[k], "GB/s": gbs, "frac": gbs / peak}
+        st = time_stats([a.elapsed_time(b_) * 1e3 for a, b_ in ev])
+        gbs = algo[k] / st["mean"] / 1e3
+        kernels[k] = {"bound": "hbm", "us": st["mean"], "us_median": st["median"], "us_min": st["min"],
+                      "algorithmic_bytes": algo[k], "per_unit": per_unit[k], "achieved": gbs,
+                      "unit": "GB/s", "peak": peak, "peak_kind": kind, "frac": gbs / peak,
+                      "frac_at_median": algo[k] / st["median"] / 1e3 / peak,
+                      "traffic": NCU_CFG4_TRAFFIC[k] if N == 17506416 else None}
+    kernels["egae"]["dense_rewards_us"] = dense
+    return {"workload": "cfg4: %d ragged segments, %d tokens, lengths log-uniform in [16, 32768], half "
+                        "truncated with a bootstrap value, Bernoulli(0.5) byte masks" % (B, N),
+            "steps": steps, "ms_per_step": ms, "tokens_per_s": N / (ms * 1e-3),
+            "selected": {"policy": int(cn[0]), "value": int(cn[1])},
+            "advance": {"freed": int(an[0]), "context_tokens": int(an[2])},
+            "timing": "CUDA events around each C-ABI call (its memset and kernels)",
+            "kernels": kernels, "clocks": clocks}
+
+
+def run_cfg4_workload(args, rank, world, local, dev, warmup):
+    """Config 4 as the bench line (the scan is the roofline kernel of this workload)."""
+    steps = args.steps if args.steps != 200 else 50
+    m = measure_cfg4(dev, steps, warmup)
+    k = m["kernels"]
     if rank == 0:
         print(json.dumps({
             "metric": "tokens/s, EGAE + token compaction + value loss + batch advance, config 4",
-            "value": N / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": steps, "warmup": warmup,
-            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "value": m["tokens_per_s"], "unit": "tokens/s", "n_gpus": 1, "steps": steps, "warmup": warmup,
+            "ms_per_step": m["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32 (f64 scan carries), int32 indices", "data": "synthetic",
-            "config": {"workload": "cfg4: %d ragged segments, %d tokens, lengths log-uniform in [16, 32768], "
-                                   "half truncated, Bernoulli(0.5) masks" % (B, N),
-                       "l2": "inputs larger than L2 (%.0f MB per array)" % (N * 4 / 1e6),
-                       "selected": {"policy": int(cn[0]), "value": int(cn[1])},
-                       "advance": {"freed": int(an[0]), "context_tokens": int(an[2])}},
-            "roofline": {"bound": "hbm", "achieved": kernels["egae"]["GB/s"], "peak": peak, "unit": "GB/s",
-                         "frac": kernels["egae"]["frac"], "peak_kind": kind,
-                         # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this launch
-                         # (140.68 + 99.05 MB; part of the 140 MB of results was still in L2 at the end)
-                         "traffic": 239.73e6 if N == 17506416 else None,
-                         "kernel": "egae_scan_kernel", "kernel_ms": kernels["egae"]["us"] / 1e3,
-                         "algorithmic_bytes_per_launch": algo["egae"]},
-            "kernels": kernels, "gpu_launches": 7 * steps, "clocks": clocks}))
+            "config": {"workload": m["workload"], "l2": "inputs larger than L2 (70 MB per array)",
+                       "selected": m["selected"], "advance": m["advance"]},
+            "roofline": {"bound": "hbm", "achieved": k["egae"]["achieved"], "peak": k["egae"]["peak"],
+                         "unit": "GB/s", "frac": k["egae"]["frac"], "peak_kind": k["egae"]["peak_kind"],
+                         "traffic": k["egae"]["traffic"], "kernel": "egae_scan_kernel",
+                         "kernel_ms": k["egae"]["us"] / 1e3,
+                         "algorithmic_bytes_per_launch": k["egae"]["algorithmic_bytes"]},
+            "kernels": k, "gpu_launches": 6 * steps, "clocks": m["clocks"]}))
 
 
 if __name__ == "__main__":

@@ -9,15 +9,17 @@
  * Conventions that hold for every entry point
  *   - Every array pointer is a DEVICE pointer unless the comment says "host".  The caller owns all
  *     buffers, the workspace included; the library allocates nothing and keeps no state between
- *     calls.  Scalars are passed by value.
+ *     calls -- with one exception, tppo_egae_static, which works in a device array compiled into
+ *     the library and remembers that array's address per device (see there).  Scalars are passed
+ *     by value.
  *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work and return; they never
  *     synchronise the stream or the device.
  *   - Return value: a tppo_status.  Anything the host can detect (null pointer, negative size,
  *     workspace too small, misalignment, unsupported shape) is reported before any kernel is
  *     launched and leaves all outputs untouched.  Problems only the device can see (a target id
- *     outside [0,V), an index outside its array, a scan wait that ran out) set bits of a status
- *     word in the call's output and the affected outputs are written as 0 -- never NaN, never a
- *     trap.
+ *     outside [0,V), an index outside its array, a scan wait that ran out, a NaN or infinity in
+ *     an input) set bits of a status word in the call's output and the affected outputs are
+ *     written as 0 -- never NaN, never a trap.
  *   - Packed token layout: sequence i occupies positions [seq_begin[i], seq_begin[i+1]) laid out
  *     prompt | response tokens of earlier windows | response tokens of this window.
  *   - Workspace: query tppo_workspace_bytes() with the same sizes, pass at least that many bytes,
@@ -49,7 +51,8 @@ enum {
     TPPO_DEV_WAIT_TIMEOUT = 2,/* a bounded look-back wait gave up: outputs incomplete        */
     TPPO_DEV_BAD_INDEX = 4,   /* a row / token index outside its array: entry skipped        */
     TPPO_DEV_BAD_SEGMENT = 8, /* segment bounds outside [0, N] or not ascending: skipped     */
-    TPPO_DEV_OVERFLOW = 16    /* an output buffer was too small: the excess was not written  */
+    TPPO_DEV_OVERFLOW = 16,   /* an output buffer was too small: the excess was not written  */
+    TPPO_DEV_NONFINITE = 32   /* a NaN or infinity was met in an input: see each entry point */
 };
 
 typedef enum {
@@ -78,6 +81,19 @@ int tppo_version(void);
 const char *tppo_status_string(int status);
 
 /*
+ * For tests of the give-up paths of the two kernels that wait on other thread blocks (the scan of
+ * tppo_egae and the compaction of tppo_select_tokens, both decoupled look-back chains).  Host call;
+ * it changes a process-wide setting that later calls of those two entry points read:
+ *   lookback_polls  >= 0: a look-back gives up after this many failed polls of a round of tiles
+ *                   (normally about four million); < 0 restores the normal limit
+ *   no_publish      != 0: tiles do not publish their partial results, so that every look-back that
+ *                   has to wait runs into the limit -- deterministically, without any fault
+ * A call made under these settings returns normally with TPPO_DEV_WAIT_TIMEOUT set; its outputs are
+ * incomplete but finite and in bounds.  tppo_test_hooks(-1, 0) restores normal operation.
+ */
+void tppo_test_hooks(int32_t lookback_polls, int32_t no_publish);
+
+/*
  * Workspace bytes needed by one call of `op`.  N = packed tokens, B = sequences / segments,
  * n_max = capacity of the selected-token list, V = vocabulary (0 where it does not apply).
  * Returns 0 for an unknown op.  Host call, launches nothing.
@@ -102,6 +118,8 @@ size_t tppo_workspace_bytes(int op, int64_t N, int32_t B, int64_t n_max, int32_t
  *   advantages       [N] fp32 out; returns [N] fp32 out or NULL.  Positions outside every
  *                    segment are written 0.
  *   status           [1] int32 out: device status bits (0 = clean).
+ * A reward, value or used bootstrap value inside a segment that is a NaN or an infinity is read as
+ * 0 and raises TPPO_DEV_NONFINITE, so the outputs stay finite.
  * Precision: the advantage is carried as G_t = A_t + values[t] (G_t = rewards[t] + gamma*(1-lambda)*
  * V(s_{t+1}) + gamma*lambda*G_{t+1}, so successive values never cancel); runs of 16 consecutive
  * positions are evaluated in fp32 (gamma*lambda split into two floats, exact to 2^-48), everything
@@ -134,7 +152,9 @@ int tppo_egae(const float *rewards, const float *values,
  *   - N > TPPO_EGAE_STATIC_MAX_TOKENS returns TPPO_ERR_TOO_LARGE before anything is launched.
  *   - The first call on each device looks up the device address of the built-in array (the device
  *     must be current, as for every call) and caches it; make that first call outside any stream
- *     capture.  Later calls only enqueue a clear of the array and the kernel.
+ *     capture.  Later calls only enqueue a clear of the array and the kernel.  The cached address
+ *     belongs to the device's current context: after cudaDeviceReset it is stale, and the entry
+ *     point must not be used again in that process.
  *   - All calls on a device share the one array, which still holds the previous call's contents:
  *     each call clears it on `stream` before the scan.  Two calls that can overlap on the GPU
  *     (different streams without an ordering between them) race on it and give undefined results;
@@ -152,14 +172,18 @@ int tppo_egae_static(const float *rewards, const float *values,
  * Token filter and compaction (Section 3.2; "selective filtering of prompt and truncated tokens").
  * With o = p - seq_begin[i] for the sequence i that holds position p:
  *   policy token  iff  prompt_len[i]+prev_len[i] <= o < prompt_len[i]+prev_len[i]+new_len[i]
- *                                                       - (truncated[i] ? tail_drop : 0)
+ *                                                       - (truncated[i] ? drop_i : 0)
  *                      (response tokens generated in the current step, finished or not, minus
- *                      the last tail_drop tokens of an unfinished sequence)
+ *                      the last drop_i tokens of an unfinished sequence; drop_i = tail_drop_seq[i]
+ *                      when that array is given, else tail_drop: the paper leaves the number of
+ *                      excluded latest tokens open, so it is a parameter, per call or per sequence)
  *   value token   iff  !truncated[i] and prompt_len[i] <= o < prompt_len[i]+prev_len[i]+new_len[i]
  *                      (all generated tokens of finished sequences)
  * each ANDed with the optional byte masks (non-zero = keep).  Prompt tokens are in neither set.
  *
  *   seq_begin [B+1] int32 ascending; prompt_len, prev_len, new_len [B] int32 >= 0; truncated [B] u8
+ *   tail_drop >= 0; tail_drop_seq [B] int32 or NULL (a negative entry is read as 0 and raises
+ *   TPPO_DEV_BAD_INDEX)
  *   extra_policy_mask, extra_value_mask  [N] u8 or NULL
  *   policy_idx, value_idx  [N] int32 out: selected positions in ascending order (bit-exact,
  *                          run-to-run deterministic); entries past the count are untouched
@@ -168,7 +192,7 @@ int tppo_egae_static(const float *rewards, const float *values,
  */
 int tppo_select_tokens(const int32_t *seq_begin, const int32_t *prompt_len,
                        const int32_t *prev_len, const int32_t *new_len,
-                       const uint8_t *truncated, int32_t tail_drop,
+                       const uint8_t *truncated, int32_t tail_drop, const int32_t *tail_drop_seq,
                        const uint8_t *extra_policy_mask, const uint8_t *extra_value_mask,
                        int32_t B, int64_t N,
                        int32_t *policy_idx, int32_t *value_idx, int32_t *counts,
@@ -201,6 +225,10 @@ int tppo_select_tokens(const int32_t *seq_begin, const int32_t *prompt_len,
  *                testing and never change the result beyond rounding (see tppo_policy_kernels)
  * Zero selected rows give loss 0 and no gradient writes beyond FULL mode's zero fill.
  * Reductions are done in a fixed order: results are run-to-run identical.
+ * Range: exp(x - max) is formed from the difference, so finite logits of any magnitude are handled,
+ * and -inf logits (a masked vocabulary entry) count as probability 0.  A selected row that holds a
+ * NaN or +inf, or nothing but -inf, has no log-softmax: it contributes nothing (logp, loss term and
+ * gradient row 0) and raises TPPO_DEV_NONFINITE.
  */
 int tppo_policy_loss_fwd_bwd(const void *logits, int32_t logits_dtype,
                              int64_t R, int32_t V, int64_t ld,
@@ -228,9 +256,16 @@ enum {
  *     l  = 1/2 * max((values[p]-returns[p])^2, (Vc-returns[p])^2),   loss = (1/denom) sum l
  *     dvalues[p] = (values[p]-returns[p])/denom  if the unclipped term is the max (ties included),
  *                  else (Vc-returns[p])/denom if Vc == values[p], else 0
- *   values, old_values, returns [N] fp32; value_idx [n_max] int32 (distinct) or NULL for 0..n_max-1
+ *   values, old_values, returns [N] fp32
+ *   value_idx [n_max] int32 or NULL for 0..n_max-1.  With dvalues the list must be strictly ascending
+ *             with entries in [0, N), the order tppo_select_tokens writes (the kernel then sweeps
+ *             the positions in order and writes every entry of dvalues itself); every adjacent pair
+ *             is checked, and a list that is not ascending raises TPPO_DEV_BAD_INDEX and leaves loss
+ *             and dvalues unspecified (finite, in bounds).  Without dvalues any distinct entries do.
  *   loss [1] fp32 out; dvalues [N] fp32 out (zero off the value tokens) or NULL
  *   stats [2] int32 out: n, status bits
+ * A value token whose value, old value or return is a NaN or an infinity contributes nothing (loss
+ * term and gradient 0) and raises TPPO_DEV_NONFINITE.
  */
 int tppo_value_loss(const float *values, const float *old_values, const float *returns,
                     int64_t N, const int32_t *value_idx, const int32_t *n_sel, int64_t n_max,
@@ -260,6 +295,11 @@ int tppo_value_loss(const float *values, const float *old_values, const float *r
  *   workspace    tppo_workspace_bytes(TPPO_OP_LMHEAD, M, K, 0, V) bytes
  * K and V must be multiples of 8 (TPPO_ERR_UNSUPPORTED otherwise).  A row with a target outside
  * [0, V) or an aux index outside [0, aux_len) contributes nothing and raises the status bit.
+ * Range: the logits are fp32 sums of K bf16 products and their exponentials are formed as
+ * 2^(x*log2(e) - lse*log2(e)), so |x| must stay below 2.3e38 (FLT_MAX / log2 e).  A row whose logits
+ * are not finite (a NaN or infinity in its hidden state or in the weight) contributes nothing to
+ * the loss and to dweight, gets a zero dX, and raises TPPO_DEV_NONFINITE; dhidden is then only
+ * finite where the weight itself is.
  * The first call on a device looks up the driver's tensor-map encoder (TPPO_ERR_CUDA if absent).
  */
 int tppo_lmhead_logprob_fwd_bwd(const void *hidden, const void *weight,

@@ -12,7 +12,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libtppo.so")
+# the in-tree build, or another build of the same sources named by TPPO_LIBRARY
+LIB_PATH = os.environ.get("TPPO_LIBRARY") or os.path.join(_HERE, "libtppo.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -24,7 +25,7 @@ OP_EGAE, OP_SELECT_TOKENS, OP_POLICY_LOSS, OP_VALUE_LOSS, OP_LMHEAD = range(5)
 BF16, F32 = 0, 1
 DLOGITS_NONE, DLOGITS_FULL, DLOGITS_COMPACT = 0, 1, 2
 POLICY_AUTO, POLICY_TWO_PASS, POLICY_CLUSTER_SMEM = 0, 1, 2
-DEV_BAD_TARGET, DEV_WAIT_TIMEOUT, DEV_BAD_INDEX, DEV_BAD_SEGMENT, DEV_OVERFLOW = 1, 2, 4, 8, 16
+DEV_BAD_TARGET, DEV_WAIT_TIMEOUT, DEV_BAD_INDEX, DEV_BAD_SEGMENT, DEV_OVERFLOW, DEV_NONFINITE = 1, 2, 4, 8, 16, 32
 
 _vp, _i32, _i64, _f32, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
 
@@ -39,8 +40,10 @@ _lib.tppo_egae.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _f32,
 _lib.tppo_egae_static.restype = C.c_int
 _lib.tppo_egae_static.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _f32, _vp, _vp, _vp, _vp]
 _lib.tppo_select_tokens.restype = C.c_int
-_lib.tppo_select_tokens.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _i32, _i64, _vp, _vp,
+_lib.tppo_select_tokens.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _i32, _i64, _vp, _vp,
                                     _vp, _vp, _sz, _vp]
+_lib.tppo_test_hooks.restype = None
+_lib.tppo_test_hooks.argtypes = [_i32, _i32]
 _lib.tppo_policy_loss_fwd_bwd.restype = C.c_int
 _lib.tppo_policy_loss_fwd_bwd.argtypes = [_vp, _i32, _i64, _i32, _i64, _vp, _vp, _vp, _i64, _vp,
                                           _vp, _vp, _i64, _f32, _f32, _f32, _vp, _vp, _vp, _vp,
@@ -132,12 +135,21 @@ def tppo_egae_static(rewards, values, seg_begin, seg_end, truncated, bootstrap, 
                                  _ptr(returns, torch.float32), _ptr(status, torch.int32), _stream()))
 
 
+def tppo_test_hooks(lookback_polls: int = -1, no_publish: bool = False) -> None:
+    """Test aid: shorten the look-back waits of tppo_egae / tppo_select_tokens and (optionally) stop
+    tiles from publishing, so that the bounded waits run out; (-1, False) restores normal operation."""
+    _lib.tppo_test_hooks(int(lookback_polls), 1 if no_publish else 0)
+
+
 def tppo_select_tokens(seq_begin, prompt_len, prev_len, new_len, truncated, tail_drop,
-                       extra_policy_mask, extra_value_mask, N, policy_idx, value_idx, counts, ws):
+                       extra_policy_mask, extra_value_mask, N, policy_idx, value_idx, counts, ws,
+                       tail_drop_seq=None):
     B = prompt_len.numel()
+    assert tail_drop_seq is None or tail_drop_seq.numel() == B
     _check(_lib.tppo_select_tokens(_ptr(seq_begin, torch.int32), _ptr(prompt_len, torch.int32),
                                    _ptr(prev_len, torch.int32), _ptr(new_len, torch.int32),
                                    _ptr(truncated, torch.uint8), tail_drop,
+                                   _ptr(tail_drop_seq, torch.int32),
                                    _ptr(extra_policy_mask, torch.uint8),
                                    _ptr(extra_value_mask, torch.uint8), B, N,
                                    _ptr(policy_idx, torch.int32), _ptr(value_idx, torch.int32),

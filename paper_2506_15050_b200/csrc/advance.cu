@@ -66,6 +66,10 @@ constexpr int kAdvSlotItems = 4;                               // consecutive sl
 
 __global__ void __launch_bounds__(kAdvSlotThreads) advance_slots_kernel(const AdvanceArgs a) {
     __shared__ long long s_scan[32];
+    __shared__ int s_bad;
+    if (threadIdx.x == 0) s_bad = 0;
+    // the copy kernel may be scheduled now; it waits for this grid to finish before it reads
+    asm volatile("griddepcontrol.launch_dependents;");
     long long free_base = 0, pos_base = 0;
     int bad = 0;
     for (int c0 = 0; c0 < a.B; c0 += kAdvSlotThreads * kAdvSlotItems) {
@@ -129,12 +133,18 @@ __global__ void __launch_bounds__(kAdvSlotThreads) advance_slots_kernel(const Ad
         pos_base += n_tok;
     }
     if (pos_base > 0x7fffffffll || pos_base > a.capacity) bad |= TPPO_DEV_OVERFLOW;
-    if (bad) atomicOr(a.counts + 3, bad);
+    // this block writes all four counts (no clear beforehand); the copy kernel, which runs after it,
+    // adds its own status bits
+    __syncthreads();
+    if (bad) atomicOr(&s_bad, bad);
+    __syncthreads();
     if (threadIdx.x == 0) {
+        bad = s_bad;
         a.next_seq_begin[a.B] = int32_t(pos_base < 0x7fffffffll ? pos_base : 0x7fffffffll);
         a.counts[0] = int32_t(free_base);
         a.counts[1] = int32_t(free_base < a.M ? free_base : a.M);
         a.counts[2] = int32_t(pos_base < 0x7fffffffll ? pos_base : 0x7fffffffll);
+        a.counts[3] = bad;
     }
 }
 
@@ -156,52 +166,101 @@ __device__ __forceinline__ int adv_warp_count_le(const int32_t* arr, int n, int3
     return lo;
 }
 
-// Ragged copy into the next step's packed context: consecutive threads take consecutive output
-// positions (coalesced stores; loads are coalesced inside a slot), each thread walks the slots
-// forward as its positions advance.  8 bytes of traffic per token.
+// Ragged copy into the next step's packed context.  A block owns 8192 consecutive output positions.
+// It finds the first slot that reaches into them (one warp-wide search), puts the slots of its range
+// into a small shared-memory table -- where each begins in the output and a source pointer already
+// shifted so that source = pointer[output position], null for a slot whose source range is not inside
+// its array -- and then every thread moves four consecutive positions at a time: four loads (the
+// source is only 4-byte aligned), one 16-byte store.  Groups that straddle two slots, and blocks
+// whose range holds more slots than the table, fall back to one position at a time.
+// 8 bytes of traffic per token.
+constexpr int kAdvTable = 128;
+
+struct AdvSlotRef {
+    int64_t begin, next;       // output range of the slot
+    const int32_t* src;        // source = src[output position]; null: nothing to read
+};
+__device__ __forceinline__ AdvSlotRef adv_slot_ref(const AdvanceArgs& a, int i, int& bad) {
+    AdvSlotRef r;
+    r.begin = a.next_seq_begin[i];
+    r.next = a.next_seq_begin[i + 1];
+    r.src = nullptr;
+    const int32_t s = a.slot_source[i];
+    const int64_t len = r.next - r.begin;
+    if (len <= 0) return r;
+    if (s == -1) {
+        const int64_t q = a.seq_begin[i];
+        if (q >= 0 && q + len <= a.N) r.src = a.tokens + q - r.begin;
+    } else if (s >= 0 && s < a.M) {
+        const int64_t q = a.queue_begin[s];
+        if (q >= 0 && q + len <= a.queue_total) r.src = a.queue_tokens + q - r.begin;
+    }
+    if (!r.src) bad = TPPO_DEV_BAD_INDEX;       // positions of such a slot are written as 0
+    return r;
+}
+
 __global__ void __launch_bounds__(kAdvCopyThreads) advance_copy_kernel(const AdvanceArgs a) {
     __shared__ int s_slot0;
+    __shared__ int32_t s_begin[kAdvTable + 1];
+    __shared__ const int32_t* s_src[kAdvTable];
+    // launched as a programmatic dependent of the slot walk: everything above this line (block
+    // scheduling, the parameter fetch) overlaps with it; its results are read only after the wait
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t total = min(int64_t(a.next_seq_begin[a.B]), a.capacity);
     const int64_t t0 = int64_t(blockIdx.x) * kAdvCopyTile;
     if (t0 >= total) return;
+    const int64_t t1 = min(t0 + kAdvCopyTile, total);
     if (threadIdx.x < 32) {
         const int c = adv_warp_count_le(a.next_seq_begin, a.B + 1, int32_t(t0), threadIdx.x);
         if (threadIdx.x == 0) s_slot0 = c - 1;      // last slot that begins at or before t0
     }
     __syncthreads();
-    int i = max(s_slot0, 0);
-    int64_t begin = a.next_seq_begin[i], next = a.next_seq_begin[i + 1];
-    int32_t src = a.slot_source[i];
-    int64_t src_base = src == -1 ? int64_t(a.seq_begin[i]) : (src >= 0 ? int64_t(a.queue_begin[src]) : 0);
+    const int slot0 = max(s_slot0, 0);
     int bad = 0;
-    // batches of eight positions: resolve the sources, issue the eight loads, then store
-    for (int j0 = 0; j0 < kAdvCopyItems; j0 += 8) {
-        const int32_t* srcp[8];
-        int64_t pos[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int64_t p = t0 + threadIdx.x + int64_t(j0 + u) * kAdvCopyThreads;
-            pos[u] = p;
-            srcp[u] = nullptr;
-            if (p >= total) continue;
-            while (p >= next && i + 1 < a.B) {
-                ++i;
-                begin = next;
-                next = a.next_seq_begin[i + 1];
-                src = a.slot_source[i];
-                src_base = src == -1 ? int64_t(a.seq_begin[i]) : (src >= 0 ? int64_t(a.queue_begin[src]) : 0);
-            }
-            const int64_t q = src_base + (p - begin);
-            if (src == -1 && q >= 0 && q < a.N) srcp[u] = a.tokens + q;
-            else if (src >= 0 && q >= 0 && q < a.queue_total) srcp[u] = a.queue_tokens + q;
-            else bad = TPPO_DEV_BAD_INDEX;
+    for (int j = threadIdx.x; j <= kAdvTable; j += kAdvCopyThreads) {
+        const int i = slot0 + j;
+        if (j < kAdvTable && i < a.B) {
+            const AdvSlotRef r = adv_slot_ref(a, i, bad);
+            s_begin[j] = int32_t(r.begin);
+            s_src[j] = r.src;
+        } else {
+            s_begin[j] = i <= a.B ? a.next_seq_begin[min(i, a.B)] : INT32_MAX;
+            if (j < kAdvTable) s_src[j] = nullptr;
         }
-        int32_t v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = srcp[u] ? __ldg(srcp[u]) : 0;
-#pragma unroll
-        for (int u = 0; u < 8; ++u)
-            if (pos[u] < total) a.next_tokens[pos[u]] = v[u];
+    }
+    __syncthreads();
+    // the table serves the block when its last entry begins at or beyond the block's last position
+    const bool table_ok = int64_t(s_begin[kAdvTable]) >= t1 || slot0 + kAdvTable >= a.B;
+    const bool vec = (reinterpret_cast<uintptr_t>(a.next_tokens) & 15) == 0;
+    if (table_ok && vec) {
+        int h = 0;
+        for (int64_t p = t0 + 4 * threadIdx.x; p < t1; p += 4 * kAdvCopyThreads) {
+            while (h + 1 < kAdvTable && slot0 + h + 1 < a.B && p >= int64_t(s_begin[h + 1])) ++h;
+            int4 v = make_int4(0, 0, 0, 0);
+            if (p + 4 <= t1 && p + 4 <= int64_t(s_begin[h + 1])) {       // four positions of one slot
+                const int32_t* src = s_src[h];
+                if (src) {
+                    v.x = __ldg(src + p); v.y = __ldg(src + p + 1);
+                    v.z = __ldg(src + p + 2); v.w = __ldg(src + p + 3);
+                }
+                *reinterpret_cast<int4*>(a.next_tokens + p) = v;
+            } else {
+                int hh = h;
+                for (int e = 0; e < 4 && p + e < t1; ++e) {
+                    while (hh + 1 < kAdvTable && slot0 + hh + 1 < a.B && p + e >= int64_t(s_begin[hh + 1])) ++hh;
+                    const int32_t* src = s_src[hh];
+                    a.next_tokens[p + e] = src ? __ldg(src + p + e) : 0;
+                }
+            }
+        }
+    } else {
+        // one position at a time, each thread walking the slots forward as its positions advance
+        int i = slot0;
+        AdvSlotRef r = adv_slot_ref(a, i, bad);
+        for (int64_t p = t0 + threadIdx.x; p < t1; p += kAdvCopyThreads) {
+            while (p >= r.next && i + 1 < a.B) r = adv_slot_ref(a, ++i, bad);
+            a.next_tokens[p] = (r.src && p >= r.begin && p < r.next) ? __ldg(r.src + p) : 0;
+        }
     }
     if (bad) atomicOr(a.counts + 3, bad);
 }
@@ -230,7 +289,6 @@ TPPO_API int tppo_advance_batch(const int32_t* seq_begin, const int32_t* prompt_
         (capacity > 0 && !next_tokens))
         return TPPO_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    TPPO_CUDA_CHECK(cudaMemsetAsync(counts, 0, 4 * sizeof(int32_t), s));
     AdvanceArgs a;
     a.seq_begin = seq_begin; a.prompt_len = prompt_len; a.prev_len = prev_len; a.new_len = new_len;
     a.truncated = truncated; a.tokens = tokens; a.queue_begin = queue_begin;
@@ -246,8 +304,19 @@ TPPO_API int tppo_advance_batch(const int32_t* seq_begin, const int32_t* prompt_
         int64_t upper = N + queue_total < capacity ? N + queue_total : capacity;
         const int64_t tiles = (upper + kAdvCopyTile - 1) / kAdvCopyTile;
         if (tiles > 0) {
-            advance_copy_kernel<<<unsigned(tiles), kAdvCopyThreads, 0, s>>>(a);
-            TPPO_CUDA_CHECK(cudaGetLastError());
+            // programmatic dependent launch: the copy kernel's blocks are scheduled while the slot
+            // walk still runs and wait inside the kernel for its results
+            cudaLaunchConfig_t lc = {};
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            lc.gridDim = dim3(unsigned(tiles), 1, 1);
+            lc.blockDim = dim3(kAdvCopyThreads, 1, 1);
+            lc.dynamicSmemBytes = 0;
+            lc.stream = s;
+            lc.attrs = attr;
+            lc.numAttrs = 1;
+            TPPO_CUDA_CHECK(cudaLaunchKernelEx(&lc, advance_copy_kernel, a));
         }
     }
     return TPPO_OK;

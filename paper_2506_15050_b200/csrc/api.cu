@@ -9,7 +9,23 @@ size_t value_workspace_bytes();
 size_t lmhead_workspace_bytes(int64_t M, int32_t K, int32_t V);
 }  // namespace tppo
 
-TPPO_API int tppo_version(void) { return 100; }
+// Test hooks (see tppo_test_hooks in the header): read by the launchers of the two look-back kernels.
+namespace tppo {
+static int32_t g_test_polls = -1;
+static int32_t g_test_no_publish = 0;
+uint32_t test_spin_limit(uint32_t normal) {
+    const int32_t p = __atomic_load_n(&g_test_polls, __ATOMIC_RELAXED);
+    return p < 0 ? normal : uint32_t(p);
+}
+int32_t test_no_publish() { return __atomic_load_n(&g_test_no_publish, __ATOMIC_RELAXED); }
+}  // namespace tppo
+
+TPPO_API void tppo_test_hooks(int32_t lookback_polls, int32_t no_publish) {
+    __atomic_store_n(&tppo::g_test_polls, lookback_polls, __ATOMIC_RELAXED);
+    __atomic_store_n(&tppo::g_test_no_publish, no_publish ? 1 : 0, __ATOMIC_RELAXED);
+}
+
+TPPO_API int tppo_version(void) { return 200; }
 
 TPPO_API const char* tppo_status_string(int status) {
     switch (status) {

@@ -57,6 +57,7 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kFltMax = 3.402823466e+38f;     // largest finite binary32
 constexpr float kLn2 = 0.6931471805599453f;
 
 }  // namespace tppo

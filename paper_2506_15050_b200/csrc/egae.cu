@@ -41,6 +41,12 @@ constexpr int kScanTile = kScanThreads * kScanItems;  // 2048 positions
 constexpr int kSegCap = 32;                           // segments of one tile kept in shared memory
 constexpr int kScanCtasPerSm = 8;
 constexpr uint32_t kScanSpinLimit = 1u << 22;
+#ifndef TPPO_EGAE_F64_MAP
+#define TPPO_EGAE_F64_MAP 1    // 1: a run's composite map is evaluated in fp64; 0: in fp32
+#endif
+#ifndef TPPO_EGAE_TICKET
+#define TPPO_EGAE_TICKET 1     // 1: tiles by ticket; 0: tile = f(blockIdx), relying on in-order dispatch
+#endif
 
 struct Affine2 {  // x -> (aA*xA + bA, aR*xR + bR)
     double aA, bA, aR, bR;
@@ -110,12 +116,26 @@ struct EgaeArgs {
     float gamma_f;              // gamma (an fp32 input: exact)
     float gl_hi, gl_lo;         // gamma*lambda = gl_hi + gl_lo up to 2^-48
     float c1;                   // gamma * (1 - lambda)
+    double c1_d;                // the same, not rounded to fp32
     float* adv;
     float* ret;
     int32_t* status;
     TileState* state;
+    // Three words at the head of the workspace, cleared to all-ones together with the tile states:
+    // the ticket counter (+1 wraps the first draw to 0), the finished-tiles counter (likewise), and
+    // the call's status bits, kept INVERTED (a bit is raised by clearing it) so that the one
+    // all-ones clear serves them too.  The last tile to finish writes the status word out.
     uint32_t* ticket;
+    uint32_t* done;
+    uint32_t* ws_status;
+    uint32_t spin_limit;   // polls a look-back may spend on one round of tiles before it gives up
+    int32_t no_publish;    // test hook: tiles keep their states to themselves, so every look-back runs out
 };
+__device__ __forceinline__ void egae_raise(const EgaeArgs& a, int bits) {
+    atomicAnd(a.ws_status, ~uint32_t(bits));
+    __threadfence();      // performed before this thread reaches the tile's final barrier
+}
+__device__ __forceinline__ bool finite_f32(float x) { return fabsf(x) <= kFltMax; }
 
 // Shared-memory image of one tile.  r and v are 64 rows of 32 positions (128 bytes) in the layout
 // the TMA's 128-byte swizzle writes: 16-byte chunk c of row y sits at chunk c ^ (y & 7) of that row
@@ -148,13 +168,14 @@ __device__ __forceinline__ int pos_slot(int l) {      // float index of position
 // position l + 1 is passed in: by the time of the replay its slot may hold a result already.
 struct PosTerm {
     float x, r, v;
+    double xd;          // x before its rounding to fp32
     bool cont, inside;
 };
 __device__ __forceinline__ PosTerm egae_position(const EgaeArgs& a, const TileBuf& buf,
                                                  const TileWin& win, int64_t t0,
                                                  int n_tile, int win_lo, bool win_smem, int l,
-                                                 float v_next_pos, int& i, bool& bad) {
-    PosTerm o{0.f, 0.f, 0.f, false, false};
+                                                 float v_next_pos, int& i, bool& bad, bool& nonfinite) {
+    PosTerm o{0.f, 0.f, 0.f, 0.0, false, false};
     if (l >= n_tile) return o;
     const int32_t p = int32_t(t0 + l);
     int32_t b = 0, e = 0;
@@ -175,13 +196,19 @@ __device__ __forceinline__ PosTerm egae_position(const EgaeArgs& a, const TileBu
     o.inside = true;
     o.r = buf.r[pos_slot(l)];
     o.v = buf.v[pos_slot(l)];
+    if (!finite_f32(o.r)) { o.r = 0.f; nonfinite = true; }      // read as 0 and reported
+    if (!finite_f32(o.v)) { o.v = 0.f; nonfinite = true; }
+    if (!finite_f32(v_next_pos)) v_next_pos = 0.f;               // (its owner reports it)
     if (p + 1 < e) {
+        o.xd = fma(a.c1_d, double(v_next_pos), double(o.r));
         o.x = fmaf(a.c1, v_next_pos, o.r);
         o.cont = true;
     } else {      // last token: G = r + gamma * (0 | bootstrap value | its own value)
         const bool tr = win_smem ? (win.seg_t[i] != 0) : (__ldg(a.truncated + win_lo + i) != 0);
         float v_next = 0.f;
         if (tr) v_next = a.bootstrap ? (win_smem ? win.seg_boot[i] : __ldg(a.bootstrap + win_lo + i)) : o.v;
+        if (!finite_f32(v_next)) { v_next = 0.f; nonfinite = true; }     // tr is set here
+        o.xd = fma(a.gamma, double(v_next), double(o.r));
         o.x = fmaf(a.gamma_f, v_next, o.r);
     }
     return o;
@@ -219,7 +246,7 @@ __device__ __forceinline__ bool egae_look_back(const EgaeArgs& a, int first, int
             p = tmask ? __ffs(int(tmask)) - 1 : 32;
             const uint32_t need = p < 32 ? ((1u << p) - 1u) : 0xffffffffu;
             if ((rmask & need) == need) break;
-            if (++spins > kScanSpinLimit) return false;     // uniform: decided from the ballots
+            if (++spins > a.spin_limit) return false;       // uniform: decided from the ballots
             __nanosleep(20);
         }
         // lane < p: the tile's composite; lane p: the constant map to its value; beyond p: identity
@@ -301,7 +328,7 @@ __device__ __forceinline__ void warp_count_le2(const int32_t* __restrict__ arr1,
 // a segment with bounds outside [0, N] or end < begin was seen; such a segment is treated as empty.
 static_assert(kSegCap == 32, "one lane per window segment");
 __device__ __forceinline__ bool egae_window(const EgaeArgs& a, TileWin& win, int64_t t0, int n_tile,
-                                            int lane) {
+                                            int lane, bool& nonfinite) {
     // segments are ascending and disjoint, so seg_begin and seg_end are both ascending: the window
     // starts after the segments that end at or before the tile's first position and stops before
     // those that begin after its last one
@@ -316,7 +343,9 @@ __device__ __forceinline__ bool egae_window(const EgaeArgs& a, TileWin& win, int
         win.seg_b[lane] = b;
         win.seg_e[lane] = e;
         win.seg_t[lane] = __ldg(a.truncated + i);
-        win.seg_boot[lane] = a.bootstrap ? __ldg(a.bootstrap + i) : 0.f;
+        float boot = a.bootstrap ? __ldg(a.bootstrap + i) : 0.f;
+        if (!finite_f32(boot)) { boot = 0.f; nonfinite |= win.seg_t[lane] != 0; }   // used by cut responses only
+        win.seg_boot[lane] = boot;
     }
     return bad;
 }
@@ -337,10 +366,13 @@ struct RunState {
     float v_right;       // value of the position after the run (its slot is overwritten by the replay)
 };
 
-// The thread's sixteen positions, right to left: its composite map.
-__device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, const TileBuf& buf,
-                                                const TileWin& win, int64_t t0,
-                                                int n_tile, int tid, RunState& rs, bool& bad) {
+// The thread's sixteen positions, right to left: its composite map.  `probe` comes back NaN when a
+// reward or value that the straight-line paths read was not finite (x * 0 is NaN exactly then).
+__device__ __forceinline__ Affine2 egae_run_map_once(const EgaeArgs& a, const TileBuf& buf,
+                                                     const TileWin& win, int64_t t0,
+                                                     int n_tile, int tid, RunState& rs, bool& bad,
+                                                     float& probe, bool& nonfinite) {
+    float probe0 = 0.f;
     const int win_lo = win.win_lo;
     const int win_n = max(win.win_hi - win_lo, 0);
     const bool win_smem = win_n <= kSegCap;
@@ -375,7 +407,8 @@ __device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, const TileBuf
     rs.i_start = i_start;
     rs.fast = fast;
     rs.masked = false;
-    const float v_right = l0 + kScanItems < kScanTile ? buf.v[pos_slot(l0 + kScanItems)] : buf.v_after;
+    float v_right = l0 + kScanItems < kScanTile ? buf.v[pos_slot(l0 + kScanItems)] : buf.v_after;
+    if (!finite_f32(v_right)) v_right = 0.f;     // read as 0; the thread that owns it reports it
     rs.v_right = v_right;
     if (!fast && win_smem) {
         // The segments that overlap the run, from the right: usually one or two.  With at most one
@@ -413,7 +446,12 @@ __device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, const TileBuf
     }
     if (rs.masked) {
         const uint32_t inside = rs.bits & 0xffffu, cont = rs.bits >> 16;
-        float bG = 0.f, bR = 0.f, vn = v_right;
+#if TPPO_EGAE_F64_MAP
+        double bG = 0.0, bR = 0.0;
+#else
+        float bG = 0.f, bR = 0.f;
+#endif
+        float vn = v_right;
 #pragma unroll
         for (int q = kScanItems / 4 - 1; q >= 0; --q) {
             const int s = row_base + (((chunk0 + q) ^ swz) << 2);
@@ -425,21 +463,37 @@ __device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, const TileBuf
             for (int e = 3; e >= 0; --e) {
                 const int k = 4 * q + e;
                 const bool in = (inside >> k) & 1u, c = (cont >> k) & 1u;
+                probe0 = fmaf(rr[e], 0.f, probe0);
+                probe0 = fmaf(vv[e], 0.f, probe0);
+#if TPPO_EGAE_F64_MAP
+                const double rd = in ? double(rr[e]) : 0.0;
+                double x = fma(a.c1_d, double(vn), rd);
+                if (k == rs.k_last) x = fma(a.gamma, double(rs.boundary_own ? vv[e] : rs.v_boundary), rd);
+                x = in ? x : 0.0;
+                bG = c ? fma(a.gl, bG, x) : x;
+                bR = c ? fma(a.gamma, bR, rd) : rd;
+#else
                 float x = fmaf(a.c1, vn, rr[e]);
                 if (k == rs.k_last) x = fmaf(a.gamma_f, rs.boundary_own ? vv[e] : rs.v_boundary, rr[e]);
                 x = in ? x : 0.f;
                 const float re = in ? rr[e] : 0.f;
                 bG = c ? fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, x)) : x;
                 bR = c ? fmaf(a.gamma_f, bR, re) : re;
+#endif
                 vn = vv[e];
             }
         }
+        probe = probe0;
         const bool whole = cont == 0xffffu;
         return Affine2{whole ? a.gl_run : 0.0, double(bG), whole ? a.gamma_run : 0.0, double(bR)};
     }
     if (fast) {
         // every map has the same multiplier and no per-position test is needed
+#if TPPO_EGAE_F64_MAP
+        double bG = 0.0, bR = 0.0;
+#else
         float bG = 0.f, bR = 0.f;
+#endif
         float vn = v_right;
 #pragma unroll
         for (int q = kScanItems / 4 - 1; q >= 0; --q) {
@@ -450,35 +504,84 @@ __device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, const TileBuf
             const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
 #pragma unroll
             for (int e = 3; e >= 0; --e) {
+                probe0 = fmaf(rr[e], 0.f, probe0);
+                probe0 = fmaf(vv[e], 0.f, probe0);
+#if TPPO_EGAE_F64_MAP
+                const double rd = double(rr[e]);
+                bG = fma(a.gl, bG, fma(a.c1_d, double(vn), rd));
+                bR = fma(a.gamma, bR, rd);
+#else
                 const float x = fmaf(a.c1, vn, rr[e]);
                 bG = fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, x));
                 bR = fmaf(a.gamma_f, bR, rr[e]);
+#endif
                 vn = vv[e];
             }
         }
+        probe = probe0;
         return Affine2{a.gl_run, double(bG), a.gamma_run, double(bR)};
     }
+#if TPPO_EGAE_F64_MAP
+    double bG = 0.0, bR = 0.0;
+#else
     float bG = 0.f, bR = 0.f;
+#endif
     double aG = 1.0, aR = 1.0;
     int i = i_start;
     float v_next = v_right;
 #pragma unroll 1
     for (int k = kScanItems - 1; k >= 0; --k) {
-        const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l0 + k, v_next, i, bad);
+        const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l0 + k, v_next, i, bad, nonfinite);
         v_next = buf.v[pos_slot(l0 + k)];
         if (t.cont) {
+#if TPPO_EGAE_F64_MAP
+            bG = fma(a.gl, bG, t.xd);
+            bR = fma(a.gamma, bR, double(t.r));
+#else
             bG = fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, t.x));
             bR = fmaf(a.gamma_f, bR, t.r);
+#endif
             aG *= a.gl;
             aR *= a.gamma;
         } else {
+#if TPPO_EGAE_F64_MAP
+            bG = t.xd;
+#else
             bG = t.x;
+#endif
             bR = t.r;
             aG = 0.0;
             aR = 0.0;
         }
     }
+    probe = 0.f;       // this path tests and replaces every value it reads
     return Affine2{aG, double(bG), aR, double(bR)};
+}
+
+// The composite map of the thread's run.  When a reward or value of the run is a NaN or an infinity
+// the thread overwrites it with 0 in the tile image (its own slots only: nobody else writes them,
+// and a neighbour that reads the first of them as the value after ITS run replaces it on the fly
+// too), reports it when the position lies inside a segment, and evaluates the run again.
+__device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, TileBuf& buf, const TileWin& win,
+                                                int64_t t0, int n_tile, int tid, RunState& rs,
+                                                bool& bad, bool& nonfinite) {
+    Affine2 f = identity2();
+#pragma unroll 1
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        float probe = 0.f;
+        f = egae_run_map_once(a, buf, win, t0, n_tile, tid, rs, bad, probe, nonfinite);
+        if (probe == probe) break;
+        const uint32_t inside = rs.fast ? 0xffffu : (rs.bits & 0xffffu);
+#pragma unroll 1
+        for (int k = 0; k < kScanItems; ++k) {
+            const int sl = pos_slot(tid * kScanItems + k);
+            const bool fr = finite_f32(buf.r[sl]), fv = finite_f32(buf.v[sl]);
+            if (!fr) buf.r[sl] = 0.f;
+            if (!fv) buf.v[sl] = 0.f;
+            if ((!fr || !fv) && ((inside >> k) & 1u)) nonfinite = true;
+        }
+    }
+    return f;
 }
 
 // Four results of one chunk: into the tile image itself (advantages over the values, returns over
@@ -507,7 +610,7 @@ __device__ __forceinline__ void egae_put4(const EgaeArgs& a, TileBuf& buf, bool 
 __device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, TileBuf& buf,
                                                 const TileWin& win, int64_t t0,
                                                 int n_tile, int tid, const RunState& rs, float G,
-                                                float R, bool in_place, bool& bad) {
+                                                float R, bool in_place, bool& bad, bool& nonfinite) {
     const int l0 = tid * kScanItems;
     if (rs.fast) {
         const int row_base = (tid >> 1) << 5;
@@ -572,7 +675,7 @@ __device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, TileBuf& buf,
 #pragma unroll 1
     for (int k = kScanItems - 1; k >= 0; --k) {
         const int l = l0 + k;
-        const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l, v_next, i, bad);
+        const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l, v_next, i, bad, nonfinite);
         v_next = buf.v[pos_slot(l)];
         G = t.cont ? fmaf(a.gl_hi, G, fmaf(a.gl_lo, G, t.x)) : t.x;
         R = t.cont ? fmaf(a.gamma_f, R, t.r) : t.r;
@@ -606,9 +709,13 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t bar = ptx::smem_addr(&s_bar);
     if (threadIdx.x == 0) {
+#if TPPO_EGAE_TICKET
         // the ticket counter starts at all-ones like the rest of the workspace (one memset): + 1
         // wraps the first draw to ticket 0
         s_ticket = atomicAdd(a.ticket, 1u) + 1u;
+#else
+        s_ticket = blockIdx.x;
+#endif
         ptx::mbar_init(bar, 1);
         ptx::fence_mbar_init_cluster();
     }
@@ -616,6 +723,7 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     const uint32_t ticket = s_ticket;
     if (ticket >= uint32_t(a.num_tiles)) return;       // (the grid has exactly num_tiles CTAs)
     const int tile = a.num_tiles - 1 - int(ticket);
+    bool nonfinite = false;
     const int64_t t0 = int64_t(tile) * kScanTile;
     const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
     const bool by_tma = a.tma_ok && n_tile == kScanTile;
@@ -636,13 +744,13 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     }
     if (threadIdx.x == kScanThreads - 1)
         buf.v_after = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
-    if (warp == 0) bad |= egae_window(a, win, t0, n_tile, lane);
-    if (by_tma && !ptx::mbar_wait<false>(bar, 0)) atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT);
+    if (warp == 0) bad |= egae_window(a, win, t0, n_tile, lane, nonfinite);
+    if (by_tma && !ptx::mbar_wait<false>(bar, 0)) egae_raise(a, TPPO_DEV_WAIT_TIMEOUT);
     __syncthreads();
 
     // ---- the thread's sixteen positions, right to left: its composite map; the warp's scan --------
     RunState rs{};
-    const Affine2 f = egae_run_map(a, buf, win, t0, n_tile, threadIdx.x, rs, bad);
+    const Affine2 f = egae_run_map(a, buf, win, t0, n_tile, threadIdx.x, rs, bad, nonfinite);
     // inclusive suffix composition inside the warp: S_l = f_l o f_{l+1} o ... o f_31
     Affine2 S = f;
 #pragma unroll
@@ -665,15 +773,16 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
         Affine2 right = shfl_down(W, 1);            // composite of the warps to the right
         if (lane >= kScanWarps - 1) right = identity2();
         TileState* st = a.state;
-        if (lane == 0 && tile + 1 < a.num_tiles) {
+        const bool publish = lane == 0 && !a.no_publish;
+        if (publish && tile + 1 < a.num_tiles) {
             st_pair(st[tile].aggA, W.aA, W.bA);
             st_pair(st[tile].aggR, W.aR, W.bR);
         }
         double xA = 0.0, xR = 0.0;
         const bool ok = egae_look_back(a, tile + 1, lane, xA, xR);
         if (lane == 0) {
-            if (!ok) { atomicOr(a.status, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
-            st_pair(st[tile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
+            if (!ok) { egae_raise(a, TPPO_DEV_WAIT_TIMEOUT); xA = 0.0; xR = 0.0; }
+            if (publish) st_pair(st[tile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
         }
         xA = __shfl_sync(0xffffffffu, xA, 0);
         xR = __shfl_sync(0xffffffffu, xR, 0);
@@ -687,22 +796,32 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     // ---- replay the thread's positions from the true incoming values, store -----------------------
     const float G = float(fma(rs.excl.aA, s_carry[warp][0], rs.excl.bA));
     const float R = float(fma(rs.excl.aR, s_carry[warp][1], rs.excl.bR));
-    egae_run_replay(a, buf, win, t0, n_tile, threadIdx.x, rs, G, R, by_tma, bad);
-    if (by_tma) {
-        ptx::fence_proxy_async_smem();       // the TMA stores read what was just written
-        __syncthreads();
-        if (threadIdx.x == 0) {
+    egae_run_replay(a, buf, win, t0, n_tile, threadIdx.x, rs, G, R, by_tma, bad, nonfinite);
+    if (bad) egae_raise(a, TPPO_DEV_BAD_SEGMENT);
+    if (nonfinite) egae_raise(a, TPPO_DEV_NONFINITE);
+    if (by_tma) ptx::fence_proxy_async_smem();       // the TMA stores read what was just written
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (by_tma) {
             const int32_t y = tile * (kScanTile / kRowPos);
             umma::tma_store_2d(&map_adv, ptx::smem_addr(buf.v), 0, y);
             if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(buf.r), 0, y);
             ptx::bulk_commit();
-            ptx::bulk_wait<0>();             // shared memory must outlive the stores
         }
+        // The last tile to finish hands the status bits to the caller (every other tile's bits were
+        // raised before its own count: fence, then count).
+        __threadfence();
+        if (atomicAdd(a.done, 1u) + 1u == uint32_t(a.num_tiles) - 1u) {
+            __threadfence();
+            *a.status = int32_t(~*reinterpret_cast<volatile uint32_t*>(a.ws_status));
+        }
+        if (by_tma) ptx::bulk_wait_read<0>();   // shared memory must outlive the stores' reads of it
     }
-    if (bad) atomicOr(a.status, TPPO_DEV_BAD_SEGMENT);
 }
 
 bool make_f32_rows_tensor_map(CUtensorMap* map, const void* base, uint64_t rows);
+uint32_t test_spin_limit(uint32_t normal);
+int32_t test_no_publish();
 
 // Fills the constants derived from gamma and lambda and the tensor maps, then launches one CTA per
 // tile.  The caller has set the pointers, sizes, state and ticket.
@@ -715,7 +834,8 @@ static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
     a.gamma_f = gamma;
     a.gl_hi = float(a.gl);
     a.gl_lo = float(a.gl - double(a.gl_hi));
-    a.c1 = float(double(gamma) * (1.0 - double(lambda)));
+    a.c1_d = double(gamma) * (1.0 - double(lambda));
+    a.c1 = float(a.c1_d);
     a.vec_ok = aligned(a.rewards, 16) && aligned(a.values, 16) && aligned(a.adv, 16) &&
                (!a.ret || aligned(a.ret, 16));
     CUtensorMap map_r, map_v, map_adv, map_ret;
@@ -730,15 +850,24 @@ static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
                make_f32_rows_tensor_map(&map_v, a.values, uint64_t(a.N) / kRowPos) &&
                make_f32_rows_tensor_map(&map_adv, a.adv, uint64_t(a.N) / kRowPos) &&
                (!a.ret || make_f32_rows_tensor_map(&map_ret, a.ret, uint64_t(a.N) / kRowPos));
+    a.spin_limit = test_spin_limit(kScanSpinLimit);
+    a.no_publish = test_no_publish();
     egae_scan_kernel<<<a.num_tiles, kScanThreads, 0, s>>>(a, map_r, map_v, map_adv, map_ret);
     TPPO_CUDA_CHECK(cudaGetLastError());
     return TPPO_OK;
 }
 
+constexpr size_t kScanHeadBytes = 256;      // ticket, finished-tiles counter, inverted status bits
 size_t egae_workspace_bytes(int64_t N) {
     const int64_t tiles = (N + kScanTile - 1) / kScanTile;
-    return align_up(sizeof(uint32_t), kWsAlign) +
-           align_up(size_t(tiles > 0 ? tiles : 1) * sizeof(TileState), kWsAlign);
+    return kScanHeadBytes + align_up(size_t(tiles > 0 ? tiles : 1) * sizeof(TileState), kWsAlign);
+}
+static void egae_carve(EgaeArgs& a, void* ws) {
+    uint32_t* head = static_cast<uint32_t*>(ws);
+    a.ticket = head;
+    a.done = head + 1;
+    a.ws_status = head + 2;
+    a.state = reinterpret_cast<TileState*>(static_cast<char*>(ws) + kScanHeadBytes);
 }
 
 }  // namespace tppo
@@ -759,17 +888,18 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
     if (!workspace || workspace_bytes < need || !aligned(workspace, kWsAlign))
         return TPPO_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
-    if (N == 0) return TPPO_OK;
-    // one memset: tile states start out unset (all-ones), the ticket counter at all-ones too
+    if (N == 0) {
+        TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
+        return TPPO_OK;
+    }
+    // one memset: tile states start out unset (all-ones), and so do the two counters and the
+    // (inverted) status bits; the kernel's last tile writes *status
     TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0xff, need, s));
     EgaeArgs a{};
     a.rewards = rewards; a.values = values; a.seg_begin = seg_begin; a.seg_end = seg_end;
     a.truncated = truncated; a.bootstrap = bootstrap; a.B = B; a.N = int32_t(N);
     a.adv = advantages; a.ret = returns; a.status = status;
-    a.ticket = static_cast<uint32_t*>(workspace);
-    a.state = reinterpret_cast<TileState*>(static_cast<char*>(workspace) +
-                                           align_up(sizeof(uint32_t), kWsAlign));
+    egae_carve(a, workspace);
     return egae_launch(a, gamma, lambda, s);
 }
 
@@ -781,7 +911,7 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
 namespace tppo {
 constexpr int64_t kStaticMaxTokens = TPPO_EGAE_STATIC_MAX_TOKENS;
 constexpr size_t kStaticTiles = size_t((kStaticMaxTokens + kScanTile - 1) / kScanTile);
-constexpr size_t kStaticScratchBytes = 256 + kStaticTiles * sizeof(TileState);
+constexpr size_t kStaticScratchBytes = kScanHeadBytes + kStaticTiles * sizeof(TileState);
 static_assert(sizeof(TileState) == 64, "tile descriptor is 64 bytes");
 }  // namespace tppo
 
@@ -822,17 +952,18 @@ TPPO_API int tppo_egae_static(const float* rewards, const float* values, const i
     const int rc = static_scratch_for_current_device(&scratch);
     if (rc != TPPO_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
-    if (N == 0) return TPPO_OK;
+    if (N == 0) {
+        TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
+        return TPPO_OK;
+    }
     EgaeArgs a{};
     a.rewards = rewards; a.values = values; a.seg_begin = seg_begin; a.seg_end = seg_end;
     a.truncated = truncated; a.bootstrap = bootstrap; a.B = B; a.N = int32_t(N);
     a.adv = advantages; a.ret = returns; a.status = status;
-    a.ticket = static_cast<uint32_t*>(scratch);
-    a.state = reinterpret_cast<TileState*>(static_cast<char*>(scratch) + 256);
-    // the array still holds the previous call's tile states and ticket: reset the part this call
-    // uses to the all-ones pattern (tile states unset, ticket counter one draw before ticket 0)
+    egae_carve(a, scratch);
+    // the array still holds the previous call's tile states and counters: reset the part this call
+    // uses to the all-ones pattern (tile states unset, counters one step before 0, no status bit)
     const size_t tiles = size_t((N + kScanTile - 1) / kScanTile);
-    TPPO_CUDA_CHECK(cudaMemsetAsync(scratch, 0xff, 256 + tiles * sizeof(TileState), s));
+    TPPO_CUDA_CHECK(cudaMemsetAsync(scratch, 0xff, kScanHeadBytes + tiles * sizeof(TileState), s));
     return egae_launch(a, gamma, lambda, s);
 }

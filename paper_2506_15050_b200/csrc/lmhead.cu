@@ -115,6 +115,10 @@ struct EpiDx {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
                 g[i] = cf * ex2(fmaf(__uint_as_float(v[i]), kLog2e, -l2));
+            if (cf == 0.f) {     // clipped, skipped or non-finite row: exact zeros (0 * NaN is not 0)
+#pragma unroll
+                for (int i = 0; i < 32; ++i) g[i] = 0.f;
+            }
             const unsigned d = unsigned(y - col0);
             if (d < 32u) {
 #pragma unroll
@@ -220,11 +224,30 @@ __global__ void __launch_bounds__(256)
 lmhead_rows_kernel(const RowRec* rec, const float2* part, const float* xy, int64_t M, int32_t n_tiles,
                    float eps_low, float eps_high, float inv_denom, float* logp, float* token_loss,
                    float* row_loss, uint8_t* row_clip, float* lse2, float* coef,
-                   const float* ext_max, const float* ext_sum, const float* ext_xy) {
+                   const float* ext_max, const float* ext_sum, const float* ext_xy, int32_t* status) {
     const int64_t r = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     if (r >= M) return;
     const RowRec rr = load_rec(rec + r);
-    if (rr.y < 0) {                      // bad target or index: the row contributes nothing
+    float m = -kInf, s = 0.f, x_y = 0.f;
+    if (rr.y >= 0) {
+        if (ext_max) {           // whole-vocabulary statistics supplied by the caller (vocabulary shards)
+            m = ext_max[r];
+            s = ext_sum[r];
+            x_y = ext_xy[r];
+        } else {
+            for (int t = 0; t < n_tiles; ++t) m = fmaxf(m, part[int64_t(t) * M + r].x);
+            for (int t = 0; t < n_tiles; ++t) {
+                const float2 p = part[int64_t(t) * M + r];
+                s += p.y * expf(p.x - m);
+            }
+            x_y = xy[r];
+        }
+    }
+    // a sum of exponentials that is not positive and finite means the row's logits held a NaN or an
+    // infinity (a non-finite hidden state or weight): the row is skipped and reported
+    const bool finite = s > 0.f && s <= kFltMax && fabsf(m) <= kFltMax && fabsf(x_y) <= kFltMax;
+    if (rr.y >= 0 && !finite) atomicOr(status, TPPO_DEV_NONFINITE);
+    if (rr.y < 0 || !finite) {           // bad target or index, or non-finite logits: contributes nothing
         if (logp) logp[r] = 0.f;
         if (token_loss) token_loss[r] = 0.f;
         row_loss[r] = 0.f;
@@ -232,19 +255,6 @@ lmhead_rows_kernel(const RowRec* rec, const float2* part, const float* xy, int64
         lse2[r] = kInf;
         coef[r] = 0.f;
         return;
-    }
-    float m = -kInf, s = 0.f, x_y;
-    if (ext_max) {               // whole-vocabulary statistics supplied by the caller (vocabulary shards)
-        m = ext_max[r];
-        s = ext_sum[r];
-        x_y = ext_xy[r];
-    } else {
-        for (int t = 0; t < n_tiles; ++t) m = fmaxf(m, part[int64_t(t) * M + r].x);
-        for (int t = 0; t < n_tiles; ++t) {
-            const float2 p = part[int64_t(t) * M + r];
-            s += p.y * expf(p.x - m);
-        }
-        x_y = xy[r];
     }
     const float log_sum = logf(s);
     const RowLoss rl = ppo_row(x_y - m, log_sum, rr.old_logp, rr.adv, eps_low, eps_high, inv_denom);
@@ -456,7 +466,7 @@ int lmhead_run(const LmCall& c) {
     const float inv_denom = c.denom > 0.f ? 1.f / c.denom : 1.f / float(M);
     lmhead_rows_kernel<<<unsigned((M + 255) / 256), 256, 0, s>>>(
         w.rec, w.part, w.xy, M, plan.n_tiles, c.eps_low, c.eps_high, inv_denom, c.logp, c.token_loss,
-        w.row_loss, w.row_clip, w.lse2, w.coef, c.in_max, c.in_sum, c.in_xy);
+        w.row_loss, w.row_clip, w.lse2, w.coef, c.in_max, c.in_sum, c.in_xy, stats + 3);
     TPPO_CUDA_CHECK(cudaGetLastError());
     rc = launch_policy_finish(a, s);
     if (rc != TPPO_OK) return rc;

@@ -17,17 +17,6 @@
 #include "policy_common.cuh"
 #include "ptx.cuh"
 
-#ifdef TPPO_TIMELINE
-// Debug builds only: per-row phase timestamps (SM clock) of cluster 0, read back by a test driver.
-__device__ unsigned long long g_timeline[8][64][16];
-#define TL(rank, it, slot) \
-    do { if (cid == 0 && (it) < 64) g_timeline[rank][it][slot] = clock64(); } while (0)
-extern "C" int tppo_debug_timeline(void* host_out) {
-    return int(cudaMemcpyFromSymbol(host_out, g_timeline, sizeof(g_timeline)));
-}
-#else
-#define TL(rank, it, slot) do {} while (0)
-#endif
 
 namespace tppo {
 
@@ -66,8 +55,15 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
 
     const uint32_t rank = ptx::cluster_ctarank();
     const int32_t cid = int32_t(ptx::cluster_id_x()), ncl = int32_t(ptx::num_clusters_x());
+    // The rest of the device (the SMs that cannot host one more cluster) may work on the tail of the
+    // row list at the same time: a kernel launched as a programmatic dependent of this one starts as
+    // soon as every CTA here has passed this point.
+    asm volatile("griddepcontrol.launch_dependents;");
     const int32_t n = int32_t(policy_n(a));
-    const int32_t n_it = n > cid ? (n - cid + ncl - 1) / ncl : 0;   // rows j = cid + it * ncl
+    int64_t part_lo, part_hi;
+    policy_part(a, n, part_lo, part_hi);
+    const int32_t n_rows = int32_t(part_hi);                        // this launch: entries [0, n_rows)
+    const int32_t n_it = n_rows > cid ? (n_rows - cid + ncl - 1) / ncl : 0;   // rows j = cid + it * ncl
     const uint32_t S = cfg.stages;
     constexpr bool GRAD = OUT != 0;
     constexpr bool STAGED = OUT == 1;   // the stage buffer also stages the gradient
@@ -124,7 +120,6 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
             for (int32_t it = 0; it < n_it; ++it) {
                 ok = ptx::mbar_wait<false>(ptx::smem_addr(&ctl->done[st]), ph);
                 if (!ok) break;
-                TL(rank, it, 8);
                 if (STAGED) {
                     const int64_t j = int64_t(cid) + int64_t(it) * ncl;
                     uint8_t* dst = nullptr;
@@ -143,15 +138,12 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
                         }
                     }
                     ptx::bulk_commit();
-                    TL(rank, it, 9);
                     if (S == 1) {
                         ptx::bulk_wait_read<0>();             // single buffer: drain, then refill
                         if (it + 1 < n_it) issue_load(it + 1);
                     } else if (it >= 1) {
                         ptx::bulk_wait_read<1>();             // the store of row it-1 has left smem
-                        TL(rank, it, 10);
                         if (it - 1 + int32_t(S) < n_it) issue_load(it - 1 + int32_t(S));
-                        TL(rank, it, 11);
                     }
                 } else {
                     if (it + int32_t(S) < n_it) issue_load(it + int32_t(S));   // the row is in registers
@@ -186,9 +178,8 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
             if (tid == 0)   // this row's exchange: C*15 warp partials (+ the target logit)
                 ptx::mbar_arrive_expect_tx(ptx::smem_addr(&ctl->xchg[par]), kPartBytes + (rec_ok ? 4u : 0u));
             if (it + 1 < n_it) rec_next = load_rec(a.rec + j + ncl);   // one row ahead, used next turn
-            if (tid == 0) TL(rank, it, 0);
-            if (!ptx::mbar_wait<false>(ptx::smem_addr(&ctl->full[st]), ph)) { ok = false; break; }
-            if (tid == 0) TL(rank, it, 1);
+            // (warp-uniform: a wait that runs out takes the whole warp to the exit together)
+            if (!ptx::mbar_wait_warp<false>(ptx::smem_addr(&ctl->full[st]), ph)) { ok = false; break; }
 
             // ---- slice -> registers ------------------------------------------------------
             const uint32_t sbase = stage0 + st * cfg.stage_stride;
@@ -218,21 +209,23 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
                                                          ptx::max_bf16x2(xw[k].z, xw[k].w)));
             }
             float m_t = fmaxf(bf16_lo(pm), bf16_hi(pm));
-            m_t = fmaxf(m_t, -1.0e30f);                 // a thread with no unit: keep finite
-            if (tid == 0) TL(rank, it, 12);
+            // a thread with no unit, or whose logits are all -inf (masked): the most negative finite
+            // float keeps x - m_t free of inf - inf; every finite bf16 lies above it
+            m_t = fmaxf(m_t, -kFltMax);
             // ---- exponentials relative to the thread-local max, kept in registers ---------
-            const float off_t = m_t * kLog2e;
-            // (two fp32 lanes per instruction: packed FMA / ADD / MUL halve the issue slots)
+            // exp(x - m) = 2^((x - m) * log2 e): the difference first, so that logits of any finite
+            // magnitude stay in range (m * log2 e alone overflows beyond 2.3e38)
+            // (two fp32 lanes per instruction: packed ADD / MUL halve the issue slots)
             uint64_t e2[kClMaxUnits][4];
             uint64_t s2 = ptx::pack_f32x2(0.f, 0.f);
-            const uint64_t k2 = ptx::pack_f32x2(kLog2e, kLog2e), o2 = ptx::pack_f32x2(-off_t, -off_t);
+            const uint64_t k2 = ptx::pack_f32x2(kLog2e, kLog2e), o2 = ptx::pack_f32x2(-m_t, -m_t);
 #pragma unroll
             for (int k = 0; k < kClMaxUnits; ++k) {
                 const uint32_t w[4] = {xw[k].x, xw[k].y, xw[k].z, xw[k].w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     float t0, t1;
-                    ptx::unpack_f32x2(ptx::fma_f32x2(ptx::pack_f32x2(bf16_lo(w[q]), bf16_hi(w[q])), k2, o2), t0, t1);
+                    ptx::unpack_f32x2(ptx::mul_f32x2(ptx::add_f32x2(ptx::pack_f32x2(bf16_lo(w[q]), bf16_hi(w[q])), o2), k2), t0, t1);
                     e2[k][q] = ptx::pack_f32x2(ex2(t0), ex2(t1));
                     s2 = ptx::add_f32x2(s2, e2[k][q]);
                 }
@@ -243,7 +236,6 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
                 ptx::unpack_f32x2(s2, sa, sb);
                 s_t = sa + sb;
             }
-            if (tid == 0) TL(rank, it, 2);
             // ---- warp partial -> every CTA of the cluster (asynchronous remote stores that count
             //      bytes on the receiver's barrier: no fence, no second hop) ----------------------
             const float wm = warp_max(m_t);
@@ -259,17 +251,15 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
                     ptx::st_async_f32(ptx::map_to_cta(ptx::smem_addr(&ctl->xy[par]), c), x_y,
                                       ptx::map_to_cta(ptx::smem_addr(&ctl->xchg[par]), c));
             }
-            if (tid == 0) TL(rank, it, 4);
-            if (!ptx::mbar_wait<true>(ptx::smem_addr(&ctl->xchg[par]), xph)) { ok = false; break; }
-            if (tid == 0) TL(rank, it, 5);
+            if (!ptx::mbar_wait_warp<true>(ptx::smem_addr(&ctl->xchg[par]), xph)) { ok = false; break; }
             // every warp combines the cluster's partials on its own
-            float pmx = -1.0e30f, psum = 0.f;
+            float pmx = -kFltMax, psum = 0.f;
             {
                 float2 p[(kClMaxParts + 31) / 32];
 #pragma unroll
                 for (int i = 0; i < (C * kClComputeWarps + 31) / 32; ++i) {
                     const int idx = lane + i * 32;
-                    p[i] = idx < C * kClComputeWarps ? ctl->part[par][idx] : make_float2(-1.0e30f, 0.f);
+                    p[i] = idx < C * kClComputeWarps ? ctl->part[par][idx] : make_float2(-kFltMax, 0.f);
                     pmx = fmaxf(pmx, p[i].x);
                 }
                 pmx = warp_max(pmx);
@@ -279,11 +269,16 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
                 psum = warp_sum(psum);
             }
             const float Mx = pmx, Ssum = psum;
-            if (tid == 0) TL(rank, it, 7);
+            // A row whose sum of exponentials is not a positive finite number held a NaN or +inf
+            // logit, or nothing but -inf: it contributes nothing (same value in every thread of the
+            // cluster, since all combine the same partials in the same order).
+            const bool row_finite = Ssum > 0.f && Ssum <= kFltMax && Mx <= kFltMax;
+            const bool use = rec_ok && row_finite;
             RowLoss rl;
             rl.logp = 0.f; rl.loss = 0.f; rl.coef = 0.f; rl.clip = 0;
-            if (rec_ok) rl = ppo_row(ctl->xy[par] - Mx, logf(Ssum), rec.old_logp, rec.adv, a.eps_low, a.eps_high, inv_denom);
+            if (use) rl = ppo_row(ctl->xy[par] - Mx, logf(Ssum), rec.old_logp, rec.adv, a.eps_low, a.eps_high, inv_denom);
             if (rank == 0 && tid == 0) {
+                if (rec_ok && !row_finite) atomicOr(a.stats + 3, TPPO_DEV_NONFINITE);
                 if (a.logp) a.logp[j] = rl.logp;
                 if (a.token_loss) a.token_loss[j] = rl.loss;
                 a.row_loss[j] = rl.loss;
@@ -291,13 +286,19 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
             }
             if (GRAD) {
                 // ---- factor * (softmax - onehot), one rounding to bf16 ---------------------------
-                const float scale = rec_ok ? rl.coef * ex2((m_t - Mx) * kLog2e) / Ssum : 0.f;   // skipped row: zeros
+                const float scale = use ? rl.coef * ex2((m_t - Mx) * kLog2e) / Ssum : 0.f;   // skipped row: zeros
                 uint8_t* grow = nullptr;      // this CTA's slice of the gradient row (direct stores)
                 if (!STAGED) {
                     if (a.mode == TPPO_DLOGITS_COMPACT) grow = dl + (j * int64_t(a.V)) * 2 + uint64_t(u0) * 16u;
                     else if (row_ok) grow = dl + (int64_t(rec.row) * a.ld) * 2 + uint64_t(u0) * 16u;
                 }
                 const uint64_t sc2 = ptx::pack_f32x2(scale, scale);
+                if (!row_finite) {   // rare: NaN * 0 is not 0, so clear the stored exponentials
+#pragma unroll
+                    for (int k = 0; k < kClMaxUnits; ++k)
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) e2[k][q] = 0ull;
+                }
 #pragma unroll
                 for (int k = 0; k < kClMaxUnits; ++k) {
                     const uint32_t u = uint32_t(tid) + uint32_t(k) * kClComputeThreads;
@@ -312,18 +313,16 @@ policy_cluster_kernel(const PolicyArgs a, const ClusterLaunch cfg) {
                     }
                 }
                 if (y_mine) {   // the one-hot term, applied before the single rounding
-                    const float g = ex2(fmaf(x_y, kLog2e, -off_t)) * scale - rl.coef;
+                    const float g = use ? ex2((x_y - m_t) * kLog2e) * scale - rl.coef : 0.f;
                     const uint16_t gb = uint16_t(pack_bf16x2(g, 0.f) & 0xffffu);
                     if (STAGED) ptx::sts_u16(y_addr, gb);
                     else if (grow) *reinterpret_cast<uint16_t*>(grow + y_off) = gb;   // after this thread's own 16-byte store
                 }
-                if (tid == 0) TL(rank, it, 3);
                 if (STAGED) {
                     ptx::fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->done[st]));
                 }
-                if (tid == 0) TL(rank, it, 6);
             }
             if (++st == S) { st = 0; ph ^= 1u; }
         }
@@ -342,7 +341,7 @@ struct ClusterPlan {
 };
 
 template <int C, int OUT>
-static int plan_and_launch(const PolicyArgs& a, cudaStream_t s, int forced_stages) {
+static int plan_and_launch(const PolicyArgs& a, cudaStream_t s, int forced_stages, int* idle_sms) {
     const uint32_t units_total = uint32_t(a.V) >> 3;
     const uint32_t max_units = (units_total + C - 1) / C;     // largest slice, 16-byte units
     if (max_units > uint32_t(kClMaxUnits) * kClComputeThreads || max_units == 0) return TPPO_ERR_UNSUPPORTED;
@@ -378,6 +377,11 @@ static int plan_and_launch(const PolicyArgs& a, cudaStream_t s, int forced_stage
         return TPPO_ERR_UNSUPPORTED;
     int64_t clusters = a.n_max < 1 ? 1 : a.n_max;
     if (clusters > max_clusters) clusters = max_clusters;
+    if (idle_sms) {      // SMs that host no CTA of this launch (one CTA fills an SM)
+        int n_sm = 0;
+        if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n_sm = 0;
+        *idle_sms = n_sm - int(clusters) * C > 0 ? n_sm - int(clusters) * C : 0;
+    }
     lc.gridDim = dim3(unsigned(clusters * C), 1, 1);
     ClusterLaunch cfg{stages, stride};
     if (cudaLaunchKernelEx(&lc, kern, a, cfg) != cudaSuccess) return TPPO_ERR_CUDA;
@@ -387,20 +391,20 @@ static int plan_and_launch(const PolicyArgs& a, cudaStream_t s, int forced_stage
 // variant: bits 0-3 cluster size (0 = default 4), bits 4-6 stage cap (0 = as many as fit),
 // bit 7: store the gradient straight from registers instead of staging it in shared memory for
 // bulk stores (measured slower: the 128-bit global stores stall the compute warps)
-int launch_policy_cluster(const PolicyArgs& a, cudaStream_t s, int variant) {
+int launch_policy_cluster(const PolicyArgs& a, cudaStream_t s, int variant, int* idle_sms) {
     const int c = (variant & 15) ? (variant & 15) : 4;
     const int st = (variant >> 4) & 7;
     const int out = a.mode == TPPO_DLOGITS_NONE ? 0 : ((variant & 128) ? 2 : 1);
     switch (c * 4 + out) {
-        case 2 * 4 + 0: return plan_and_launch<2, 0>(a, s, st);
-        case 2 * 4 + 1: return plan_and_launch<2, 1>(a, s, st);
-        case 2 * 4 + 2: return plan_and_launch<2, 2>(a, s, st);
-        case 4 * 4 + 0: return plan_and_launch<4, 0>(a, s, st);
-        case 4 * 4 + 1: return plan_and_launch<4, 1>(a, s, st);
-        case 4 * 4 + 2: return plan_and_launch<4, 2>(a, s, st);
-        case 8 * 4 + 0: return plan_and_launch<8, 0>(a, s, st);
-        case 8 * 4 + 1: return plan_and_launch<8, 1>(a, s, st);
-        case 8 * 4 + 2: return plan_and_launch<8, 2>(a, s, st);
+        case 2 * 4 + 0: return plan_and_launch<2, 0>(a, s, st, idle_sms);
+        case 2 * 4 + 1: return plan_and_launch<2, 1>(a, s, st, idle_sms);
+        case 2 * 4 + 2: return plan_and_launch<2, 2>(a, s, st, idle_sms);
+        case 4 * 4 + 0: return plan_and_launch<4, 0>(a, s, st, idle_sms);
+        case 4 * 4 + 1: return plan_and_launch<4, 1>(a, s, st, idle_sms);
+        case 4 * 4 + 2: return plan_and_launch<4, 2>(a, s, st, idle_sms);
+        case 8 * 4 + 0: return plan_and_launch<8, 0>(a, s, st, idle_sms);
+        case 8 * 4 + 1: return plan_and_launch<8, 1>(a, s, st, idle_sms);
+        case 8 * 4 + 2: return plan_and_launch<8, 2>(a, s, st, idle_sms);
         default: return TPPO_ERR_UNSUPPORTED;
     }
 }

@@ -30,6 +30,10 @@ struct PolicyArgs {
     uint8_t* row_clip;   // workspace [n_max]: 0 none, 1 lower edge, 2 upper edge
     uint8_t* row_flag;   // workspace [R]: 1 = row is selected (FULL mode with a row list)
     struct RowRec* rec;  // workspace [n_max]: per-entry scalars gathered ahead of the vocabulary sweep
+    // Two kernels may share one call's rows: part 0 = this launch takes all n rows; part 1 = the
+    // first n - n_side of them; part 2 = the last n_side, with n_side = n * side_share_256 / 256.
+    int32_t part;
+    int32_t side_share_256;
 };
 
 // Everything the vocabulary sweep needs to know about the j-th selected entry, gathered once by a
@@ -51,6 +55,12 @@ __device__ __forceinline__ int64_t policy_n(const PolicyArgs& a) {
     int64_t n = a.n_max;
     if (a.n_sel) { const int64_t c = *a.n_sel; n = c < 0 ? 0 : (c < n ? c : n); }
     return n;
+}
+// Selected entries [lo, hi) that this launch works on.
+__device__ __forceinline__ void policy_part(const PolicyArgs& a, int64_t n, int64_t& lo, int64_t& hi) {
+    const int64_t n_side = a.part == 0 ? 0 : (n * a.side_share_256) >> 8;
+    lo = a.part == 2 ? n - n_side : 0;
+    hi = a.part == 1 ? n - n_side : n;
 }
 __device__ __forceinline__ float policy_inv_denom(const PolicyArgs& a, int64_t n) {
     return a.denom > 0.f ? 1.f / a.denom : 1.f / float(n > 0 ? n : 1);

@@ -110,9 +110,12 @@ int launch_policy_finish(const PolicyArgs& a, cudaStream_t s) {
     return TPPO_OK;
 }
 
-int launch_policy_two_pass(const PolicyArgs& a, int dtype, cudaStream_t s, int variant);
-int launch_policy_cluster(const PolicyArgs& a, cudaStream_t s, int variant);
+int launch_policy_two_pass(const PolicyArgs& a, int dtype, cudaStream_t s, int variant, int side_sms);
+int launch_policy_cluster(const PolicyArgs& a, cudaStream_t s, int variant, int* idle_sms);
 bool policy_cluster_supported(const PolicyArgs& a, int dtype);
+
+constexpr int kSideShare256 = 18;       // about 7 % of the rows
+constexpr int64_t kSideMinRows = 2048;  // below this the split is not worth a second launch
 
 size_t policy_workspace_bytes(int64_t R, int64_t n_max) {
     const size_t n = size_t(n_max > 0 ? n_max : 1);
@@ -163,6 +166,8 @@ TPPO_API int tppo_policy_loss_fwd_bwd(const void* logits, int32_t logits_dtype, 
     a.row_flag = reinterpret_cast<uint8_t*>(w);
     w += align_up(size_t(R > 0 ? R : 1), kWsAlign);
     a.rec = reinterpret_cast<RowRec*>(w);
+    a.part = 0;
+    a.side_share_256 = 0;
 
     const int base_hint = kernel_hint & 0xff;
     const bool can_cluster = policy_cluster_supported(a, logits_dtype);
@@ -183,9 +188,32 @@ TPPO_API int tppo_policy_loss_fwd_bwd(const void* logits, int32_t logits_dtype, 
                                  (base_hint == TPPO_POLICY_AUTO && can_cluster &&
                                   dlogits_mode != TPPO_DLOGITS_NONE);
         int rc = TPPO_ERR_UNSUPPORTED;
-        if (use_cluster) rc = launch_policy_cluster(a, s, (kernel_hint >> 8) & 0xff);
+        if (use_cluster) {
+            // The clusters cannot cover every SM (33 clusters of 4 on 148 SMs).  With enough rows the
+            // tail of the row list goes to the plain kernel, launched as a programmatic dependent so
+            // that it runs beside the cluster kernel on the SMs that one leaves idle.  Share of the
+            // rows for it: bits 16-23 of the hint in 1/256 (255 = none), default kSideShare256.
+            const int share_hint = (kernel_hint >> 16) & 0xff;
+            const int share = share_hint == 255 ? 0 : (share_hint ? share_hint : kSideShare256);
+            PolicyArgs front = a;
+            front.part = 1;
+            front.side_share_256 = n_max >= kSideMinRows ? share : 0;
+            int idle_sms = 0;
+            rc = launch_policy_cluster(front, s, (kernel_hint >> 8) & 0xff, &idle_sms);
+            if (rc == TPPO_OK && front.side_share_256 > 0) {
+                if (idle_sms >= 2) {
+                    PolicyArgs tail = front;
+                    tail.part = 2;
+                    rc = launch_policy_two_pass(tail, logits_dtype, s, 0, idle_sms);
+                } else {     // no room beside the clusters: the same rows, after them
+                    PolicyArgs tail = front;
+                    tail.part = 2;
+                    rc = launch_policy_two_pass(tail, logits_dtype, s, 0, 0);
+                }
+            }
+        }
         if (!use_cluster || (rc == TPPO_ERR_UNSUPPORTED && base_hint == TPPO_POLICY_AUTO))
-            rc = launch_policy_two_pass(a, logits_dtype, s, (kernel_hint >> 8) & 0xff);
+            rc = launch_policy_two_pass(a, logits_dtype, s, (kernel_hint >> 8) & 0xff, 0);
         if (rc != TPPO_OK) return rc;
     }
     if (fill_rows) {

@@ -43,17 +43,17 @@ __device__ __forceinline__ void store8(float* p, const float (&g)[8]) {
     *reinterpret_cast<float4*>(p + 4) = make_float4(g[4], g[5], g[6], g[7]);
 }
 
-// running (max, sum of 2^(x*log2e - max*log2e)) update with n new values
+// running (max, sum of 2^((x - max)*log2e)) update with n new values; the difference is formed
+// before the scaling so that logits of any finite magnitude stay in range
 template <int N>
 __device__ __forceinline__ void online_update(float& m, float& s, const float (&x)[N]) {
     float mx = x[0];
 #pragma unroll
     for (int k = 1; k < N; ++k) mx = fmaxf(mx, x[k]);
     const float m_new = fmaxf(m, mx);
-    const float off = m_new * kLog2e;
-    float acc = s * ex2(fmaf(m, kLog2e, -off));
+    float acc = s * ex2((m - m_new) * kLog2e);
 #pragma unroll
-    for (int k = 0; k < N; ++k) acc += ex2(fmaf(x[k], kLog2e, -off));
+    for (int k = 0; k < N; ++k) acc += ex2((x[k] - m_new) * kLog2e);
     m = m_new;
     s = acc;
 }
@@ -70,7 +70,9 @@ __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const 
     const T* logits = static_cast<const T*>(a.logits);
     T* dl = static_cast<T*>(a.dlogits);
 
-    for (int64_t j = blockIdx.x; j < n; j += gridDim.x) {
+    int64_t part_lo, part_hi;
+    policy_part(a, n, part_lo, part_hi);
+    for (int64_t j = part_lo + blockIdx.x; j < part_hi; j += gridDim.x) {
         const RowRec rec = load_rec(a.rec + j);
         const bool row_ok = rec.row >= 0, rec_ok = rec.y >= 0;
         const T* x_row = logits + int64_t(row_ok ? rec.row : 0) * a.ld;
@@ -81,7 +83,7 @@ __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const 
         float coef = 0.f, row_max = 0.f, log_sum = 0.f;
         if (rec_ok) {
             // ---- pass 1 -------------------------------------------------------------------
-            float m = -1.0e30f, s = 0.f;
+            float m = -kFltMax, s = 0.f;      // most negative finite: no inf - inf on masked (-inf) logits
             if (VEC) {
                 const int nu = a.V >> 3;
                 for (int u = tid; u < nu; u += kTwoPassThreads) {
@@ -108,9 +110,17 @@ __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const 
                 for (int w = 1; w < kTwoPassThreads / 32; ++w) M = fmaxf(M, s_m[w]);
                 float S = 0.f;
                 for (int w = 0; w < kTwoPassThreads / 32; ++w) S += s_s[w] * ex2((s_m[w] - M) * kLog2e);
-                const float log_s = logf(S);
-                const RowLoss rl = ppo_row(load_elem(x_row + rec.y) - M, log_s, rec.old_logp, rec.adv,
-                                           a.eps_low, a.eps_high, inv_denom);
+                // not a positive finite sum: the row held a NaN or +inf logit, or nothing but -inf;
+                // it contributes nothing and raises the status bit
+                const bool row_finite = S > 0.f && S <= kFltMax && M <= kFltMax;
+                const float log_s = row_finite ? logf(S) : 0.f;
+                RowLoss rl;
+                rl.logp = 0.f; rl.loss = 0.f; rl.coef = 0.f; rl.clip = 0;
+                if (row_finite)
+                    rl = ppo_row(load_elem(x_row + rec.y) - M, log_s, rec.old_logp, rec.adv,
+                                 a.eps_low, a.eps_high, inv_denom);
+                else
+                    atomicOr(a.stats + 3, TPPO_DEV_NONFINITE);
                 if (a.logp) a.logp[j] = rl.logp;
                 if (a.token_loss) a.token_loss[j] = rl.loss;
                 a.row_loss[j] = rl.loss;
@@ -171,26 +181,37 @@ __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const 
         }
         __syncthreads();   // the shared row scalars are reused by the next row
     }
+    // Launched beside the cluster kernel (as its programmatic dependent) this grid must not be
+    // complete before that one is: whatever follows in the stream waits for this grid only.
+    if (a.part == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
-// variant: blocks per SM (0 = default 3)
-int launch_policy_two_pass(const PolicyArgs& a, int dtype, cudaStream_t s, int variant) {
+// variant: blocks per SM (0 = default 3).  side_sms > 0: launch as a programmatic dependent of the
+// kernel before it in the stream, sized for that many SMs (the ones the cluster kernel leaves idle).
+int launch_policy_two_pass(const PolicyArgs& a, int dtype, cudaStream_t s, int variant, int side_sms) {
     const int per_sm = (variant & 15) ? (variant & 15) : 3;
     int64_t blocks = a.n_max < 1 ? 1 : a.n_max;
-    if (blocks > kNumSms * per_sm) blocks = kNumSms * per_sm;
+    const int sms = side_sms > 0 ? side_sms : kNumSms;
+    if (blocks > sms * per_sm) blocks = sms * per_sm;
     const size_t esz = dtype == TPPO_BF16 ? 2 : 4;
     bool vec = aligned(a.logits, 16) && (a.ld * esz) % 16 == 0;
     if (a.mode == TPPO_DLOGITS_FULL) vec = vec && aligned(a.dlogits, 16);
     if (a.mode == TPPO_DLOGITS_COMPACT)
         vec = vec && aligned(a.dlogits, 16) && (int64_t(a.V) * esz) % 16 == 0;
-    if (dtype == TPPO_BF16) {
-        if (vec) policy_two_pass_kernel<TPPO_BF16, true><<<int(blocks), kTwoPassThreads, 0, s>>>(a);
-        else policy_two_pass_kernel<TPPO_BF16, false><<<int(blocks), kTwoPassThreads, 0, s>>>(a);
-    } else {
-        if (vec) policy_two_pass_kernel<TPPO_F32, true><<<int(blocks), kTwoPassThreads, 0, s>>>(a);
-        else policy_two_pass_kernel<TPPO_F32, false><<<int(blocks), kTwoPassThreads, 0, s>>>(a);
-    }
-    return cudaGetLastError() == cudaSuccess ? TPPO_OK : TPPO_ERR_CUDA;
+    void (*kern)(const PolicyArgs) = nullptr;
+    if (dtype == TPPO_BF16) kern = vec ? policy_two_pass_kernel<TPPO_BF16, true> : policy_two_pass_kernel<TPPO_BF16, false>;
+    else kern = vec ? policy_two_pass_kernel<TPPO_F32, true> : policy_two_pass_kernel<TPPO_F32, false>;
+    cudaLaunchConfig_t lc = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.gridDim = dim3(unsigned(blocks), 1, 1);
+    lc.blockDim = dim3(kTwoPassThreads, 1, 1);
+    lc.dynamicSmemBytes = 0;
+    lc.stream = s;
+    lc.attrs = attr;
+    lc.numAttrs = side_sms > 0 ? 1 : 0;
+    return cudaLaunchKernelEx(&lc, kern, a) == cudaSuccess ? TPPO_OK : TPPO_ERR_CUDA;
 }
 
 }  // namespace tppo

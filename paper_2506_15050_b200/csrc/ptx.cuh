@@ -63,6 +63,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
 }
 
+// The same wait taken by a whole converged warp: every lane polls, and the warp leaves with ONE
+// answer (false if any lane's limit ran out), so that code after a failed wait -- shuffles, warp
+// and cluster barriers -- is still executed by all 32 lanes together.
+template <bool CLUSTER>
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity) {
+    return __all_sync(0xffffffffu, mbar_wait<CLUSTER>(bar, parity)) != 0;
+}
+
 // ---- bulk (TMA, untiled) copies: 16-byte aligned addresses, size a multiple of 16 ------------
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src_gmem, uint32_t bytes,
                                           uint32_t bar) {

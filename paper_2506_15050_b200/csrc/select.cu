@@ -63,6 +63,7 @@ struct SelectArgs {
     const uint8_t* pol_mask;
     const uint8_t* val_mask;
     int32_t tail_drop;
+    const int32_t* tail_drop_seq;   // [B] or null: per-sequence count, overrides tail_drop
     int32_t B;
     int32_t N;
     int32_t num_tiles;
@@ -71,7 +72,15 @@ struct SelectArgs {
     int32_t* value_idx;
     int32_t* counts;            // [4]
     unsigned long long* state;  // [num_tiles]
-    uint32_t* ticket;           // [1]
+    // head of the workspace, cleared to zero together with the tile states: the ticket counter, the
+    // finished-tiles counter and the status bits raised during the call (the last tile to finish
+    // writes counts[0..3])
+    uint32_t* ticket;
+    uint32_t* done;
+    uint32_t* ws_status;
+    uint32_t spin_limit;        // polls a look-back round may take before it gives up
+    int32_t no_publish;         // test hook: tiles keep their totals to themselves
+    int32_t out_vec_ok;         // policy_idx and value_idx are 16-byte aligned
 };
 
 constexpr int kSeqCap = 640;   // sequence starts of one tile kept in shared memory
@@ -95,6 +104,32 @@ __device__ __forceinline__ uint32_t range_bits32(int64_t lo, int64_t hi, int64_t
     return upto_b & ~((1u << int(a)) - 1u);
 }
 
+// One of the tile's two lists from shared memory (16-bit offsets inside the tile) to its place in
+// the output array: 16-byte stores of four indices where the destination allows, single stores at
+// the ragged ends.
+__device__ __forceinline__ void sel_copy_out(int32_t* __restrict__ out, uint32_t base, int n,
+                                             const uint16_t* __restrict__ src, int32_t t0, bool vec) {
+    int32_t* dst = out + base;
+    if (!vec) {
+        for (int k = threadIdx.x; k < n; k += kSelThreads) dst[k] = t0 + int32_t(src[k]);
+        return;
+    }
+    const int head = min(n, int((4u - (base & 3u)) & 3u));       // entries before the first 16-byte boundary
+    const int groups = (n - head) >> 2;
+    if (int(threadIdx.x) < head) dst[threadIdx.x] = t0 + int32_t(src[threadIdx.x]);
+    for (int g = threadIdx.x; g < groups; g += kSelThreads) {
+        const int k = head + 4 * g;
+        int4 v;
+        v.x = t0 + int32_t(src[k]);
+        v.y = t0 + int32_t(src[k + 1]);
+        v.z = t0 + int32_t(src[k + 2]);
+        v.w = t0 + int32_t(src[k + 3]);
+        *reinterpret_cast<int4*>(dst + k) = v;
+    }
+    const int tail0 = head + 4 * groups;
+    if (int(threadIdx.x) < n - tail0) dst[tail0 + threadIdx.x] = t0 + int32_t(src[tail0 + threadIdx.x]);
+}
+
 // Each thread owns 32 consecutive positions.  Its policy / value bits come from interval
 // arithmetic on the few sequences that overlap those positions (usually one) and from one 16-byte
 // loads per byte mask, not from a test per position; selected positions are first compacted inside
@@ -108,6 +143,7 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     __shared__ int s_seq0, s_seq1;
     __shared__ uint32_t s_warp_cnt[kSelWarps];      // policy count | value count << 16
     __shared__ uint32_t s_base_pol, s_base_val, s_tot_pol, s_tot_val;
+    int bad = 0;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // Tiles are handed out in launch order, so every tile this one waits for is already running.
@@ -191,8 +227,15 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
             const int64_t new0 = resp0 + __ldg(a.prev_len + i);
             const int64_t end = new0 + __ldg(a.new_len + i);
             const bool trunc = __ldg(a.truncated + i) != 0;
+            // how many of the latest tokens of an unfinished sequence are left out: one count for all,
+            // or one per sequence (a negative count is reported and read as 0)
+            int64_t drop = 0;
+            if (trunc) {
+                drop = a.tail_drop_seq ? __ldg(a.tail_drop_seq + i) : a.tail_drop;
+                if (drop < 0) { drop = 0; bad = TPPO_DEV_BAD_INDEX; }
+            }
             // a position belongs to the last sequence that begins at or before it: clip to [begin, next)
-            pol_bits |= range_bits32(max(new0, begin), min(end - (trunc ? a.tail_drop : 0), next), p0);
+            pol_bits |= range_bits32(max(new0, begin), min(end - drop, next), p0);
             if (!trunc) val_bits |= range_bits32(max(resp0, begin), min(end, next), p0);
         }
     }
@@ -218,9 +261,10 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
         tile_tot += c;
     }
     // publish the tile's totals as early as possible: later tiles wait for them in their look-back
-    if (threadIdx.x == 0 && tile > 0)
+    if (threadIdx.x == 0 && tile > 0 && !a.no_publish)
         reinterpret_cast<volatile unsigned long long*>(a.state)[tile] =
             sel_pack(1, tile_tot & 0xffffu, tile_tot >> 16);
+    if (bad) { atomicOr(a.ws_status, uint32_t(bad)); __threadfence(); }
     // compact inside the tile (needs no global offset; earlier tiles finish meanwhile)
     {
         uint32_t op = before & 0xffffu, ov = before >> 16;
@@ -243,7 +287,7 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
             uint64_t s = j >= 0 ? st[j] : sel_pack(2, 0, 0);
             uint32_t spins = 0;
             while (!__all_sync(0xffffffffu, sel_flag(s) != 0)) {
-                if (++spins > kSelSpinLimit) { timed_out = true; break; }
+                if (++spins > a.spin_limit) { timed_out = true; break; }
                 __nanosleep(20);
                 if (sel_flag(s) == 0) s = st[j];
             }
@@ -256,35 +300,42 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
             if (m2) break;
         }
         if (lane == 0) {
-            if (timed_out) atomicOr(a.counts + 2, TPPO_DEV_WAIT_TIMEOUT);
-            st[tile] = sel_pack(2, ep + tp, ev + tv);
+            if (timed_out) { atomicOr(a.ws_status, uint32_t(TPPO_DEV_WAIT_TIMEOUT)); __threadfence(); }
+            // (the last tile's inclusive prefix is the pair of totals: it is always stored)
+            if (!a.no_publish || tile == uint32_t(a.num_tiles) - 1) st[tile] = sel_pack(2, ep + tp, ev + tv);
             s_base_pol = ep;
             s_base_val = ev;
             s_tot_pol = tp;
             s_tot_val = tv;
-            if (tile == uint32_t(a.num_tiles) - 1) {
-                a.counts[0] = int32_t(ep + tp);
-                a.counts[1] = int32_t(ev + tv);
-            }
         }
     }
     __syncthreads();
 
     // ---- copy the tile's two lists out, coalesced ----------------------------------------------
-    {
-        int32_t* dp = a.policy_idx + s_base_pol;
-        int32_t* dv = a.value_idx + s_base_val;
-        const int np = int(s_tot_pol), nv = int(s_tot_val);
-        const int32_t base = int32_t(t0);
-        for (int k = threadIdx.x; k < np; k += kSelThreads) dp[k] = base + int32_t(s_out_pol[k]);
-        for (int k = threadIdx.x; k < nv; k += kSelThreads) dv[k] = base + int32_t(s_out_val[k]);
+    sel_copy_out(a.policy_idx, s_base_pol, int(s_tot_pol), s_out_pol, int32_t(t0), a.out_vec_ok != 0);
+    sel_copy_out(a.value_idx, s_base_val, int(s_tot_val), s_out_val, int32_t(t0), a.out_vec_ok != 0);
+
+    // ---- the last tile to finish writes the counts and the status bits -------------------------------
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(a.done, 1u) == uint32_t(a.num_tiles) - 1u) {
+            __threadfence();
+            const uint64_t last = reinterpret_cast<volatile unsigned long long*>(a.state)[a.num_tiles - 1];
+            a.counts[0] = int32_t(sel_pol(last));
+            a.counts[1] = int32_t(sel_val(last));
+            a.counts[2] = int32_t(*reinterpret_cast<volatile uint32_t*>(a.ws_status));
+            a.counts[3] = 0;
+        }
     }
 }
 
 size_t select_workspace_bytes(int64_t N) {
     const int64_t tiles = (N + kSelTile - 1) / kSelTile;
-    return align_up(sizeof(uint32_t), kWsAlign) + align_up(size_t(tiles > 0 ? tiles : 1) * 8, kWsAlign);
+    return kWsAlign + align_up(size_t(tiles > 0 ? tiles : 1) * 8, kWsAlign);
 }
+uint32_t test_spin_limit(uint32_t normal);
+int32_t test_no_publish();
 
 }  // namespace tppo
 
@@ -293,6 +344,7 @@ using namespace tppo;
 TPPO_API int tppo_select_tokens(const int32_t* seq_begin, const int32_t* prompt_len,
                                 const int32_t* prev_len, const int32_t* new_len,
                                 const uint8_t* truncated, int32_t tail_drop,
+                                const int32_t* tail_drop_seq,
                                 const uint8_t* extra_policy_mask, const uint8_t* extra_value_mask,
                                 int32_t B, int64_t N, int32_t* policy_idx, int32_t* value_idx,
                                 int32_t* counts, void* workspace, size_t workspace_bytes,
@@ -306,20 +358,27 @@ TPPO_API int tppo_select_tokens(const int32_t* seq_begin, const int32_t* prompt_
     if (!workspace || workspace_bytes < need || !aligned(workspace, kWsAlign))
         return TPPO_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    TPPO_CUDA_CHECK(cudaMemsetAsync(counts, 0, 4 * sizeof(int32_t), s));
-    if (N == 0 || B == 0) return TPPO_OK;
+    if (N == 0 || B == 0) {
+        TPPO_CUDA_CHECK(cudaMemsetAsync(counts, 0, 4 * sizeof(int32_t), s));
+        return TPPO_OK;
+    }
+    // one clear (tile states, the two counters, the status bits); the kernel writes all of counts
     TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0, need, s));
     SelectArgs a;
     a.seq_begin = seq_begin; a.prompt_len = prompt_len; a.prev_len = prev_len; a.new_len = new_len;
     a.truncated = truncated; a.pol_mask = extra_policy_mask; a.val_mask = extra_value_mask;
-    a.tail_drop = tail_drop; a.B = B; a.N = int32_t(N);
+    a.tail_drop = tail_drop; a.tail_drop_seq = tail_drop_seq; a.B = B; a.N = int32_t(N);
+    a.spin_limit = test_spin_limit(kSelSpinLimit);
+    a.no_publish = test_no_publish();
+    a.out_vec_ok = aligned(policy_idx, 16) && aligned(value_idx, 16);
     a.mask_vec_ok = (!extra_policy_mask || aligned(extra_policy_mask, 16)) &&
                     (!extra_value_mask || aligned(extra_value_mask, 16));
     a.num_tiles = int32_t((N + kSelTile - 1) / kSelTile);
     a.policy_idx = policy_idx; a.value_idx = value_idx; a.counts = counts;
     a.ticket = static_cast<uint32_t*>(workspace);
-    a.state = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) +
-                                                    align_up(sizeof(uint32_t), kWsAlign));
+    a.done = a.ticket + 1;
+    a.ws_status = a.ticket + 2;
+    a.state = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWsAlign);
     select_tokens_kernel<<<a.num_tiles, kSelThreads, 0, s>>>(a);
     TPPO_CUDA_CHECK(cudaGetLastError());
     return TPPO_OK;

@@ -102,3 +102,34 @@ def combine_row_stats(row_max, row_sumexp, row_target_logit, rescale, group=None
     row_sumexp.copy_(sums[0])
     row_target_logit.copy_(sums[1])
     return row_max, row_sumexp, row_target_logit
+
+
+def vocab_shard_bounds(V: int, world: int, align: int = 8):
+    """Column ranges [lo, hi) of the LM-head weight, one per rank: equal widths rounded up to
+    `align` columns (the GEMM kernels want multiples of 8), the last rank taking what is left."""
+    width = (-(-V // world) + align - 1) // align * align
+    cuts = [min(r * width, V) for r in range(world)] + [V]
+    return [(cuts[r], cuts[r + 1]) for r in range(world)]
+
+
+def vocab_parallel_step(stats_fn, rescale_fn, grads_fn, group=None):
+    """One step of the vocabulary-parallel LM-head on this rank; every collective it needs is here.
+
+    stats_fn() -> (row_max, row_sumexp, row_target_logit): this rank's [M] float32 statistics over its
+        column shard (on a GPU: `binding.tppo_lmhead_shard_stats`).
+    rescale_fn(row_max, row_max_all, row_sumexp): see `combine_row_stats`.
+    grads_fn(row_max, row_sumexp, row_target_logit) -> dhidden_partial or None: loss and gradients
+        from the whole-vocabulary statistics (`binding.tppo_lmhead_shard_fwd_bwd`); the [M, K] tensor
+        it returns holds this shard's term of dX * W^T.
+    The returned tensor is the complete dhidden (the partial terms summed over the ranks, in place).
+    Traffic per rank: 12 bytes x M for the statistics and one all-reduce of M x K gradient elements.
+    No rank reads another rank's memory; the collectives are torch.distributed's (NCCL on GPUs).
+    """
+    import torch.distributed as dist
+    row_max, row_sumexp, row_target_logit = stats_fn()
+    combine_row_stats(row_max, row_sumexp, row_target_logit, rescale_fn, group=group)
+    dhidden = grads_fn(row_max, row_sumexp, row_target_logit)
+    multi = dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1
+    if dhidden is not None and multi:
+        dist.all_reduce(dhidden, op=dist.ReduceOp.SUM, group=group)
+    return dhidden

@@ -35,7 +35,7 @@ def run_egae(B, rewards, values, seg_begin, seg_end, truncated, bootstrap, gamma
     return adv[:N].cpu().numpy(), (None if ret is None else ret[:N].cpu().numpy()), int(status.item())
 
 
-def run_select(c, tail_drop=0, pm=None, vm=None, N=None):
+def run_select(c, tail_drop=0, pm=None, vm=None, N=None, tail_drop_seq=None, strict=True):
     from paper_2506_15050_b200 import binding as b
     N = int(c["seq_begin"][-1]) if N is None else N
     sb = dev(c["seq_begin"], torch.int32)
@@ -47,10 +47,12 @@ def run_select(c, tail_drop=0, pm=None, vm=None, N=None):
     ws = b.workspace(b.OP_SELECT_TOKENS, N, len(c["prompt_len"]), 0, 0, DEV)
     ws.fill_(0xAB)
     b.tppo_select_tokens(sb, pl, pv, nl, tr, tail_drop, dev(pm, torch.uint8), dev(vm, torch.uint8),
-                         N, pol, val, counts, ws)
+                         N, pol, val, counts, ws, tail_drop_seq=dev(tail_drop_seq, torch.int32))
     torch.cuda.synchronize()
     cn = counts.cpu().numpy()
     pol, val = pol.cpu().numpy(), val.cpu().numpy()
+    if not strict:       # a call that is expected to give up: whatever was written, anywhere in the lists
+        return pol[pol != -7], val[val != -7], cn
     assert np.all(pol[cn[0]:] == -7) and np.all(val[cn[1]:] == -7)   # nothing past the counts
     return pol[:cn[0]], val[:cn[1]], cn
 
@@ -114,17 +116,25 @@ def run_value(values, old_values, returns, value_idx, xi_low, xi_high, denom=0.0
 
 
 def adv_close(gpu, ref, seg_begin, seg_end, rtol=1e-5):
-    """|gpu-ref| <= rtol * max(|ref|, s) with s = max(1, max |ref| over the segment): the relative
-    bound for fp32 advantages, made meaningful where the exact value is 0."""
+    """Largest |gpu - ref| / tol over the segments, tol = rtol * max(|ref|, 1) element by element:
+    the relative bound for fp32 advantages and returns, with a floor of 1 only where the exact
+    value is 0 or tiny (the last token of a cut response with gamma = 1 has advantage exactly 0).
+    Positions outside every segment must be exactly 0."""
     worst = 0.0
     inside = np.zeros(len(ref), bool)
     for b, e in zip(seg_begin, seg_end):
         if e <= b:
             continue
         inside[b:e] = True
-        s = max(1.0, float(np.max(np.abs(ref[b:e]))))
-        tol = rtol * np.maximum(np.abs(ref[b:e]), s)
         err = np.abs(gpu[b:e].astype(np.float64) - ref[b:e])
-        worst = max(worst, float(np.max(err / tol)))
+        worst = max(worst, float(np.max(err / (rtol * np.maximum(np.abs(ref[b:e]), 1.0)))))
     assert np.all(gpu[~inside] == 0.0)
     return worst
+
+
+def worst_relative_error(gpu, ref, floor=1.0):
+    """Largest |gpu - ref| / |ref| over the elements with |ref| >= floor (reported by the tests)."""
+    big = np.abs(ref) >= floor
+    if not big.any():
+        return 0.0
+    return float(np.max(np.abs(gpu[big].astype(np.float64) - ref[big]) / np.abs(ref[big])))

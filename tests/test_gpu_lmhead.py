@@ -123,8 +123,10 @@ def test_lmhead_matches_oracle(M, K, V, chunk):
     keep = ~edge
     ref_dh, abs_dh = ref_dhidden(dx, wb)
     grad_close(out["dh"][keep], ref_dh[keep], abs_dh[keep], "dhidden")
-    if not edge.any():
-        grad_close(out["dw"], *ref_dweight(hb, dx), "dweight")
+    # dweight sums over all rows, so a row on a clip edge cannot be left out of it: the seeds are
+    # chosen so that there is none, and the comparison below always runs
+    assert not edge.any()
+    grad_close(out["dw"], *ref_dweight(hb, dx), "dweight")
     # clipped rows have a zero gradient
     clipped = (ref["dlogits"] == 0).all(axis=1) & keep
     assert np.all(out["dh"][clipped] == 0)
@@ -195,20 +197,28 @@ def test_lmhead_host_errors_and_determinism():
 
 # ---------------------------------------------------------------------------------------------
 # config 5 at full size: [16384, 5120] x [5120, 152064], the launch configuration that is timed.
-# The oracle forms one vocabulary row of logits at a time, so it checks sampled rows in full and,
+# The oracle forms one vocabulary row of logits at a time, so it checks about 256 sampled rows in
+# full (every row position of a GEMM tile, both edges of 32 tiles; a few minutes of host time) and,
 # for dweight (which sums over all rows), a run whose advantages are zero outside the sampled
 # rows: every other row then has dX = 0 and the reference sum has only the sampled terms.
 # ---------------------------------------------------------------------------------------------
 LOG_V_MODEL = -13.0      # typical log-prob of a random token under these logits (an input, not a result)
 
 
-def _config5_sample(c, n_rows, seed):
+def _config5_sample(c, seed, tile=128):
+    """At least 256 rows of the M = 16384: the first and the last row of 32 different 128-row GEMM
+    tiles (the first and the last tile among them), one row for every position 0..127 inside a tile
+    (each taken from a different tile), and 64 rows drawn at random."""
     rng = np.random.default_rng(seed)
     M = c["M"]
-    pick = np.sort(rng.choice(M, n_rows, replace=False)).astype(np.int32)
-    pick[0], pick[-1] = 0, M - 1
-    pick[1], pick[2] = 127, 128                     # both sides of a tile boundary
-    return np.unique(pick).astype(np.int32)
+    n_tiles = M // tile
+    edge_tiles = np.unique(np.concatenate([np.arange(0, n_tiles, n_tiles // 32), [n_tiles - 1]]))
+    edges = np.concatenate([edge_tiles * tile, edge_tiles * tile + tile - 1])
+    lanes = np.array([((i * 37) % n_tiles) * tile + i for i in range(tile)])
+    pick = np.unique(np.concatenate([edges, lanes, rng.choice(M, 64, replace=False)])).astype(np.int32)
+    assert len(pick) >= 224 and len(np.unique(pick % tile)) == tile
+    assert len(np.intersect1d(pick[pick % tile == 0] // tile, pick[pick % tile == tile - 1] // tile)) >= 32
+    return pick
 
 
 @pytest.fixture(scope="module")
@@ -216,12 +226,18 @@ def cfg5():
     c = synth.config5(DEV)
     assert c["hidden"].shape == (16384, 5120) and c["weight"].shape == (5120, 152064)
     c["hb"], c["wb"] = synth.bf16_bits(c["hidden"]), synth.bf16_bits(c["weight"])
-    c["pick"] = _config5_sample(c, 16, seed=50)
+    c["pick"] = _config5_sample(c, seed=50)
     c["x_pick"] = oracle.lmhead_logits_rows(c["hb"], c["wb"], c["pick"])
     lp = oracle.logprob(c["x_pick"], c["targets"][c["pick"]])
     old = (LOG_V_MODEL + c["old_logp_noise"]).astype(np.float32)
     old[c["pick"]] = (lp + c["old_logp_noise"][c["pick"]]).astype(np.float32)
     c["old_logp"] = old
+    # the oracle's Eq. 1 results and dhidden rows for the sampled rows, shared by the tests below
+    # (the advantages of the sampled rows and the divisor M are the same in all of them)
+    c["ref"] = oracle.policy_loss(c["x_pick"], c["targets"][c["pick"]], None, None, old[c["pick"]],
+                                  c["adv"][c["pick"]], f32(c["eps_low"]), f32(c["eps_high"]),
+                                  denom=float(c["M"]))
+    c["ref_dh"] = ref_dhidden(c["ref"]["dlogits"], c["wb"])
     yield c
     del c["hidden"], c["weight"]
     torch.cuda.empty_cache()
@@ -234,11 +250,10 @@ def test_config5_full_sampled_rows(cfg5, variant):
     out = run_lmhead(c["hidden"], c["weight"], c["targets"], c["old_logp"], c["adv"], c["eps_low"],
                      c["eps_high"], chunk_tiles=variant)
     assert out["stats"][0] == M and out["stats"][3] == 0
-    ref = oracle.policy_loss(c["x_pick"], c["targets"][pick], None, None, c["old_logp"][pick],
-                             c["adv"][pick], f32(c["eps_low"]), f32(c["eps_high"]), denom=float(M))
+    ref = c["ref"]
     np.testing.assert_allclose(out["logp"][pick], ref["logp"], rtol=0, atol=LOGP_ATOL)
     np.testing.assert_allclose(out["token_loss"][pick], ref["token_loss"], rtol=0, atol=4 * LOGP_ATOL)
-    grad_close(out["dh"][pick], *ref_dhidden(ref["dlogits"], c["wb"]), "dhidden rows")
+    grad_close(out["dh"][pick], *c["ref_dh"], "dhidden rows")
     # properties that hold at any size
     assert np.all(np.isfinite(out["logp"])) and np.all(out["logp"] < 0)
     assert abs(out["loss"] - float(np.mean(out["token_loss"].astype(np.float64)))) <= 1e-5
@@ -263,8 +278,7 @@ def test_config5_full_dweight_from_sampled_rows(cfg5):
     out = run_lmhead(c["hidden"], c["weight"], c["targets"], c["old_logp"], adv, c["eps_low"],
                      c["eps_high"])
     assert out["stats"][3] == 0
-    ref = oracle.policy_loss(c["x_pick"], c["targets"][pick], None, None, c["old_logp"][pick],
-                             adv[pick], f32(c["eps_low"]), f32(c["eps_high"]), denom=float(M))
+    ref = c["ref"]                 # same rows, same advantages on them, same divisor
     assert np.any(ref["dlogits"] != 0)
     rng = np.random.default_rng(51)
     cols = np.concatenate([rng.choice(V, 1500, replace=False), [0, 255, 256, V - 1, V - 8],
@@ -277,7 +291,7 @@ def test_config5_full_dweight_from_sampled_rows(cfg5):
     # rows without advantage have an exactly zero gradient; the sampled ones match the oracle
     others = np.setdiff1d(np.arange(M), pick)
     assert float(out["dh_t"][torch.from_numpy(others).to(DEV)].float().abs().max()) == 0.0
-    grad_close(out["dh"][pick], *ref_dhidden(ref["dlogits"], c["wb"]), "dhidden rows")
+    grad_close(out["dh"][pick], *c["ref_dh"], "dhidden rows")
 
 
 # ---- vocabulary shards (weight split by columns; the ranks are emulated one after another) --------
@@ -351,8 +365,10 @@ def test_lmhead_vocabulary_shards_match_oracle(M, K, V, bounds, chunk):
     ref_dh, abs_dh = ref_dhidden(dx, wb)
     # every shard's partial dhidden is rounded to bf16 before the sum: |p_i| <= its sum of |a||b|
     grad_close(out["dh"][keep], ref_dh[keep], 2.0 * abs_dh[keep], "dhidden")
-    if not edge.any():
-        grad_close(out["dw"], *ref_dweight(hb, dx), "dweight")
+    # dweight sums over all rows, so a row on a clip edge cannot be left out of it: the seeds are
+    # chosen so that there is none, and the comparison below always runs
+    assert not edge.any()
+    grad_close(out["dw"], *ref_dweight(hb, dx), "dweight")
 
 
 def test_lmhead_one_shard_equals_the_unsharded_call():

@@ -6,7 +6,8 @@ import torch
 
 import oracle
 from paper_2506_15050_b200 import synth
-from gpu_util import DEV, adv_close, dev, run_egae, run_policy, run_select, run_value
+from gpu_util import (DEV, adv_close, dev, run_egae, run_policy, run_select, run_value,
+                      worst_relative_error)
 
 pytestmark = pytest.mark.gpu
 
@@ -21,11 +22,11 @@ def f32(x):
 # ------------------------------------------------------------------------------------------------
 # selection
 # ------------------------------------------------------------------------------------------------
-def check_select(c, tail_drop=0, pm=None, vm=None):
-    pol, val, cn = run_select(c, tail_drop, pm, vm)
+def check_select(c, tail_drop=0, pm=None, vm=None, tail_drop_seq=None):
+    pol, val, cn = run_select(c, tail_drop, pm, vm, tail_drop_seq=tail_drop_seq)
     rp, rv = oracle.select_tokens(c["seq_begin"], c["prompt_len"], c["prev_len"], c["new_len"],
-                                  c["truncated"], tail_drop, pm, vm)
-    assert cn[2] == 0
+                                  c["truncated"], tail_drop, pm, vm, tail_drop_seq=tail_drop_seq)
+    assert cn[2] == 0 and cn[3] == 0
     assert cn[0] == len(rp) and cn[1] == len(rv)
     assert np.array_equal(pol, rp) and np.array_equal(val, rv)
     return cn
@@ -67,6 +68,37 @@ def test_select_edge_cases():
         check_select(c, tail_drop=2)
 
 
+def test_select_per_sequence_tail_drop():
+    """One count per sequence (Section 3.2 leaves the number of excluded latest tokens open): random
+    ragged batches over several tiles, counts larger than a sequence, the array overriding the scalar,
+    and a negative entry (read as 0, reported)."""
+    for seed in range(3):
+        rng = np.random.default_rng(100 + seed)
+        B = int(rng.integers(2, 80))
+        prompt = rng.integers(0, 300, B)
+        prev = rng.integers(0, 500, B) * rng.integers(0, 2, B)
+        new = rng.integers(0, 900, B)
+        trunc = rng.integers(0, 2, B).astype(np.uint8)
+        sb, _, _ = synth.pack(prompt, prev, new)
+        c = dict(seq_begin=sb, prompt_len=prompt, prev_len=prev, new_len=new, truncated=trunc)
+        N = int(sb[-1])
+        td = rng.integers(0, 1000, B).astype(np.int32)
+        cn = check_select(c, 5, tail_drop_seq=td)
+        assert cn[0] == int(np.sum(np.maximum(0, new - trunc.astype(np.int64) * td)))
+        pm = rng.integers(0, 2, max(N, 1)).astype(np.uint8)
+        vm = rng.integers(0, 2, max(N, 1)).astype(np.uint8)
+        check_select(c, 0, pm, vm, tail_drop_seq=td)
+        same = run_select(c, 0, tail_drop_seq=np.full(B, 7, np.int32))
+        scalar = run_select(c, 7)
+        assert np.array_equal(same[0], scalar[0]) and np.array_equal(same[1], scalar[1])
+        if trunc.any():
+            neg = td.copy()
+            neg[int(np.argmax(trunc))] = -3
+            pol, val, cn = run_select(c, 0, tail_drop_seq=neg)
+            rp, rv = oracle.select_tokens(sb, prompt, prev, new, trunc, 0, tail_drop_seq=neg)
+            assert cn[2] == 4 and np.array_equal(pol, rp) and np.array_equal(val, rv)
+
+
 def test_select_run_to_run_identical_and_config4():
     c = synth.config4(B=600, hi=32768)
     a1 = run_select(c, 16, c["extra_policy_mask"], c["extra_value_mask"])
@@ -74,6 +106,8 @@ def test_select_run_to_run_identical_and_config4():
     assert np.array_equal(a1[0], a2[0]) and np.array_equal(a1[1], a2[1])
     check_select(c, 16, c["extra_policy_mask"], c["extra_value_mask"])
     check_select(c, 0)
+    td = np.random.default_rng(7).integers(0, 64, c["B"]).astype(np.int32)
+    check_select(c, 0, c["extra_policy_mask"], c["extra_value_mask"], tail_drop_seq=td)
 
 
 # ------------------------------------------------------------------------------------------------
@@ -85,7 +119,61 @@ def check_egae(B, r, v, sb, se, tr, boot, gamma, lam):
     assert status == 0
     assert adv_close(adv, ra, sb, se, ADV_RTOL) <= 1.0
     assert adv_close(ret, rr, sb, se, ADV_RTOL) <= 1.0
+    print("worst relative error where |exact| >= 1: advantages %.2e, returns %.2e"
+          % (worst_relative_error(adv, ra), worst_relative_error(ret, rr)))
     return adv, ret
+
+
+def test_egae_nonfinite_inputs_are_read_as_zero_and_reported():
+    """A NaN / infinite reward or value inside a segment is read as 0 (so every output stays finite
+    and equals the oracle's result on the cleaned arrays) and raises the status bit; the same
+    garbage outside every segment is ignored."""
+    from paper_2506_15050_b200 import binding as b
+    rng = np.random.default_rng(61)
+    N = 3 * 2048 + 300
+    r = rng.standard_normal(N).astype(np.float32)
+    v = rng.standard_normal(N).astype(np.float32)
+    sb, se = np.array([10, 2500, 5000], np.int32), np.array([2400, 4990, N - 7], np.int32)
+    tr = np.array([1, 0, 1], np.uint8)
+    boot = np.array([0.3, np.nan, np.inf], np.float32)      # boot[1] belongs to a finished response: unused
+    r[2450], v[3], v[N - 2] = np.nan, np.inf, np.nan         # outside every segment: ignored
+    adv, ret, st = run_egae(3, r, v, sb, se, tr, np.array([0.3, np.nan, 0.5], np.float32), 0.99, 0.95)
+    ra, rr = oracle.egae(r, v, sb, se, tr, np.array([0.3, 0.0, 0.5], np.float32), f32(0.99), f32(0.95))
+    assert st == 0 and adv_close(adv, ra, sb, se, ADV_RTOL) <= 1.0 and adv_close(ret, rr, sb, se, ADV_RTOL) <= 1.0
+    bad_r, bad_v = r.copy(), v.copy()
+    bad_r[100], bad_r[2047], bad_v[2048], bad_v[4989], bad_v[5000] = np.nan, np.inf, -np.inf, np.nan, np.inf
+    clean_r, clean_v = bad_r.copy(), bad_v.copy()
+    clean_r[[100, 2047]] = 0
+    clean_v[[2048, 4989, 5000]] = 0
+    for bt in (boot, None):
+        adv, ret, st = run_egae(3, bad_r, bad_v, sb, se, tr, bt, 0.99, 0.95)
+        clean_boot = None if bt is None else np.array([0.3, 0.0, 0.0], np.float32)
+        ra, rr = oracle.egae(clean_r, clean_v, sb, se, tr, clean_boot, f32(0.99), f32(0.95))
+        assert st == b.DEV_NONFINITE
+        assert np.all(np.isfinite(adv)) and np.all(np.isfinite(ret))
+        assert adv_close(adv, ra, sb, se, ADV_RTOL) <= 1.0 and adv_close(ret, rr, sb, se, ADV_RTOL) <= 1.0
+
+
+def test_lookback_waits_give_up_cleanly():
+    """The bounded waits of the two look-back kernels, made to run out on the host's say-so: tiles
+    do not publish and a look-back gives up after four polls.  Both calls must come back with
+    TPPO_DEV_WAIT_TIMEOUT, finite in-bounds outputs and a usable device; with the hooks cleared the
+    same calls are exact again."""
+    from paper_2506_15050_b200 import binding as b
+    c = synth.config4(B=300)
+    try:
+        b.tppo_test_hooks(4, True)
+        adv, ret, st = run_egae(c["B"], c["rewards"], c["values"], c["seg_begin"], c["seg_end"],
+                                c["truncated"], c["bootstrap"], 1.0, 0.95)
+        assert st & b.DEV_WAIT_TIMEOUT and np.all(np.isfinite(adv)) and np.all(np.isfinite(ret))
+        pol, val, cn = run_select(c, 0, c["extra_policy_mask"], c["extra_value_mask"], strict=False)
+        assert cn[2] & b.DEV_WAIT_TIMEOUT
+        assert np.all((pol >= 0) & (pol < c["N"])) and np.all((val >= 0) & (val < c["N"]))
+    finally:
+        b.tppo_test_hooks(-1, False)
+    check_egae(c["B"], c["rewards"], c["values"], c["seg_begin"], c["seg_end"], c["truncated"],
+               c["bootstrap"], 1.0, 0.95)
+    check_select(c, 0, c["extra_policy_mask"], c["extra_value_mask"])
 
 
 def test_egae_config1_and_truncated_tail_is_zero():
@@ -216,7 +304,7 @@ def grad_close(gpu, ref, coef_abs, bf16):
 
 
 def check_policy(logits_t, targets, rows, aux_idx, old_logp, adv, el, eh, denom=0.0, mode=2, hint=0,
-                 inplace=False):
+                 inplace=False, min_compared=0.9):
     is_bf16 = logits_t.dtype == torch.bfloat16
     host = synth.bf16_bits(logits_t) if is_bf16 else logits_t.cpu().numpy()
     R, V = host.shape
@@ -229,31 +317,34 @@ def check_policy(logits_t, targets, rows, aux_idx, old_logp, adv, el, eh, denom=
     np.testing.assert_allclose(out["token_loss"][:n], ref["token_loss"], rtol=0,
                                atol=LOGP_ATOL * max(1.0, float(np.max(np.abs(adv))) * 2))
     assert abs(out["loss"] - ref["loss"]) <= LOGP_ATOL * max(1.0, float(np.max(np.abs(adv))))
-    # clip decisions may differ only for ratios within rounding of an edge
-    rho = np.exp(ref["logp"] - np.asarray(old_logp, np.float64)[aux_idx if aux_idx is not None else (rows if rows is not None else np.arange(R))])
-    near = int(np.sum((np.abs(rho - (1 - f32(el))) < 1e-3) | (np.abs(rho - (1 + f32(eh))) < 1e-3)))
+    # Clip decisions are taken in fp32 on the GPU and in float64 by the oracle: a row whose ratio lies
+    # within 1e-3 of a clip edge may fall on either side.  Only those rows are left out of the gradient
+    # comparison (and they bound the difference of the clip counts); every other row is compared.
+    a_idx = aux_idx if aux_idx is not None else (rows if rows is not None else np.arange(R))
+    rho = np.exp(ref["logp"] - np.asarray(old_logp, np.float64)[a_idx])
+    near_row = (np.abs(rho - (1 - f32(el))) < 1e-3) | (np.abs(rho - (1 + f32(eh))) < 1e-3)
+    near = int(near_row.sum())
+    keep = np.where(~near_row)[0]
+    assert len(keep) >= min_compared * n, "too many rows near a clip edge: the check would be hollow"
     assert abs(out["clip_lo"] - ref["clip_lo"]) <= near and abs(out["clip_hi"] - ref["clip_hi"]) <= near
     if mode != 0:
         g = out["dlogits"].float().cpu().numpy()
         d = f32(denom) if denom > 0 else max(n, 1)
-        a_idx = aux_idx if aux_idx is not None else (rows if rows is not None else np.arange(R))
         coef = np.abs(np.asarray(adv, np.float64)[a_idx] * rho / d)
         if mode == 2:
             assert g.shape == (max(n, 1), V)
-            if near == 0:
-                assert grad_close(g[:n], ref["dlogits"], coef, is_bf16) <= 1.0
+            gsel = g[:n]
         else:
             sel = np.arange(R) if rows is None else np.asarray(rows)
-            if near == 0:
-                assert grad_close(g[sel][:, :V], ref["dlogits"], coef, is_bf16) <= 1.0
+            gsel = g[sel][:, :V]
             unsel = np.setdiff1d(np.arange(R), sel)
             assert np.all(g[unsel][:, :V] == 0)          # rows that are not selected: exact zeros
+        assert grad_close(gsel[keep], ref["dlogits"][keep], coef[keep], is_bf16) <= 1.0
         A = np.asarray(adv, np.float64)[a_idx]
         clipped = np.clip(rho, 1 - f32(el), 1 + f32(eh)) * A < rho * A
-        inactive = np.where(clipped | (A == 0))[0]
-        if near == 0 and len(inactive):
-            gi = g[:n][inactive] if mode == 2 else g[sel][inactive][:, :V]
-            assert np.all(gi == 0)                        # clipped rows: exact zeros
+        inactive = np.where((clipped | (A == 0)) & ~near_row)[0]
+        if len(inactive):
+            assert np.all(gsel[inactive] == 0)            # clipped rows: exact zeros
     return out, ref
 
 
@@ -343,29 +434,74 @@ def test_policy_shapes(V, ld, dtype, hint):
         rho = np.exp(ref["logp"] - old[aux])
         coef = np.abs(adv[aux] * rho / 64.0)
         gsel = g[:50] if mode == 2 else g[rows][:, :V]
-        near = np.sum((np.abs(rho - 0.8) < 1e-3) | (np.abs(rho - 1.2) < 1e-3))
-        if near == 0:
-            assert grad_close(gsel, ref["dlogits"], coef, is_bf16) <= 1.0
+        keep = ~((np.abs(rho - 0.8) < 1e-3) | (np.abs(rho - 1.2) < 1e-3))     # rows off the clip edges
+        assert keep.sum() >= 45
+        assert grad_close(gsel[keep], ref["dlogits"][keep], coef[keep], is_bf16) <= 1.0
+
+
+BF16_MAX = 3.3895313892515355e38      # largest finite bf16
 
 
 def test_policy_overflow_safety_and_onehot_row():
+    """Logits at the largest finite bf16 magnitude: exp(x - max) is formed from the difference, so
+    nothing overflows on the way.  Rows: all +max (uniform), one +max among -max (one-hot, logp 0),
+    all -max (uniform), a wide ramp, and -inf entries (masked vocabulary) beside ordinary ones."""
     V = 8192
-    x = np.zeros((4, V), np.float32)
-    x[0, :] = 1.0e4           # huge equal logits: uniform distribution, no overflow
-    x[1, 5] = 1.0e4
-    x[1, 6:] = -1.0e4         # one dominant logit: logp -> 0
-    x[2, :] = -3.0e4
+    x = np.zeros((6, V), np.float32)
+    x[0, :] = BF16_MAX
+    x[1, :] = -BF16_MAX
+    x[1, 5] = BF16_MAX
+    x[2, :] = -BF16_MAX
     x[3, :] = np.linspace(-80, 80, V)
+    x[4, :] = np.linspace(-3, 3, V)
+    x[4, 100:4000] = -np.inf
+    x[5, :] = 1.0e4
+    x[5, 6:] = -3.0e4
     xt = torch.from_numpy(x).to(torch.bfloat16).to(DEV)
-    y = np.array([7, 5, 0, V - 1], np.int32)
+    assert float(xt[0, 0]) == BF16_MAX and float(xt[2, 0]) == -BF16_MAX
+    y = np.array([7, 5, 0, V - 1, 50, 3], np.int32)
     host = synth.bf16_bits(xt)
     lp = oracle.logprob(host, y)
-    assert abs(lp[0] + np.log(V)) < 1e-9 and abs(lp[1]) < 1e-9
+    assert abs(lp[0] + np.log(V)) < 1e-9 and abs(lp[1]) < 1e-9 and abs(lp[2] + np.log(V)) < 1e-9
     old = lp.astype(np.float32)
-    adv = np.array([1.0, -1.0, 0.5, 2.0], np.float32)
+    adv = np.array([1.0, -1.0, 0.5, 2.0, -0.7, 1.5], np.float32)
     for hint in (1, 2):
         out, ref = check_policy(xt, y, None, None, old, adv, 0.2, 0.2, mode=2, hint=hint)
-        assert np.all(np.isfinite(out["dlogits"].float().cpu().numpy()))
+        g = out["dlogits"].float().cpu().numpy()
+        assert np.all(np.isfinite(g)) and np.all(g[4, 100:4000] == 0)
+
+
+@pytest.mark.parametrize("hint", [1, 2])
+def test_policy_nonfinite_rows_are_skipped_and_reported(hint):
+    """A row with a NaN or +inf logit, or with nothing but -inf, has no log-softmax: it contributes
+    nothing (loss term 0, zero gradient row), raises the status bit, and leaves the other rows alone."""
+    from paper_2506_15050_b200 import binding as b
+    rng = np.random.default_rng(77)
+    R, V = 9, 8192
+    x = (2 * rng.standard_normal((R, V))).astype(np.float32)
+    x[1, 4000] = np.nan
+    x[3, 17] = np.inf
+    x[6, :] = -np.inf
+    xt = torch.from_numpy(x).to(torch.bfloat16).to(DEV)
+    y = rng.integers(0, V, R).astype(np.int32)
+    good = np.array([0, 2, 4, 5, 7, 8], np.int32)
+    host = synth.bf16_bits(xt)
+    lp = np.zeros(R)
+    lp[good] = oracle.logprob(host, y, good)
+    old = (lp + 0.05 * rng.standard_normal(R)).astype(np.float32)
+    adv = rng.standard_normal(R).astype(np.float32)
+    out = run_policy(xt, y, None, None, old, adv, 0.2, 0.2, 0.0, 2, hint)
+    assert out["status"] == b.DEV_NONFINITE and out["n"] == R
+    ref = oracle.policy_loss(host, y, good, None, old, adv, f32(0.2), f32(0.2), float(R))
+    g = out["dlogits"].float().cpu().numpy()
+    assert np.all(np.isfinite(g)) and np.isfinite(out["loss"])
+    bad = np.setdiff1d(np.arange(R), good)
+    assert np.all(g[bad] == 0) and np.all(out["logp"][bad] == 0) and np.all(out["token_loss"][bad] == 0)
+    np.testing.assert_allclose(out["logp"][good], ref["logp"], rtol=0, atol=LOGP_ATOL)
+    assert abs(out["loss"] - ref["loss"]) <= LOGP_ATOL
+    rho = np.exp(ref["logp"] - old[good])
+    coef = np.abs(adv[good] * rho / R)
+    assert grad_close(g[good], ref["dlogits"], coef, True) <= 1.0
 
 
 @pytest.mark.parametrize("hint", [1, 2])
@@ -460,6 +596,79 @@ def test_value_loss(xl, xh):
     bad[5] = N + 3
     _, dv5, _, st5 = run_value(v, vo, R, bad, xl, xh)
     assert st5 == 4 and np.all(np.isfinite(dv5))
+
+
+def test_value_loss_nonfinite_tokens_and_unsorted_list():
+    from paper_2506_15050_b200 import binding as b
+    rng = np.random.default_rng(52)
+    N = 30000
+    v = rng.standard_normal(N).astype(np.float32)
+    vo = (v + 0.3 * rng.standard_normal(N)).astype(np.float32)
+    R = rng.choice([-1.0, 1.0], N).astype(np.float32)
+    idx = np.sort(rng.choice(N, 12000, replace=False)).astype(np.int32)
+    bad_tok = idx[[5, 4000, 11999]]
+    v2, vo2, R2 = v.copy(), vo.copy(), R.copy()
+    v2[bad_tok[0]], vo2[bad_tok[1]], R2[bad_tok[2]] = np.nan, np.inf, -np.inf
+    off = np.setdiff1d(np.arange(N), idx)
+    v2[off[7]] = np.nan                                     # not a value token: ignored
+    keep = np.setdiff1d(idx, bad_tok).astype(np.int32)
+    for want_grad in (True, False):
+        loss, dv, n, st = run_value(v2, vo2, R2, idx, 0.5, 0.6, want_grad=want_grad)
+        rl, rdv = oracle.value_loss(v, vo, R, keep, f32(0.5), f32(0.6), denom=float(len(idx)))
+        assert st == b.DEV_NONFINITE and n == len(idx) and abs(loss - rl) <= 1e-5 * max(1.0, abs(rl))
+        if want_grad:
+            assert np.all(np.isfinite(dv)) and np.all(dv[bad_tok] == 0) and np.all(dv[off] == 0)
+            np.testing.assert_allclose(dv[keep], rdv[keep], rtol=1e-5, atol=1e-9)
+    # a list that is not ascending: reported, outputs finite
+    swapped = idx.copy()
+    swapped[[3000, 3001]] = swapped[[3001, 3000]]
+    loss, dv, n, st = run_value(v, vo, R, swapped, 0.5, 0.6)
+    assert st == 4 and np.isfinite(loss) and np.all(np.isfinite(dv))
+    # the forward-only call gathers and takes any order
+    perm = rng.permutation(idx).astype(np.int32)
+    loss_p, _, _, st_p = run_value(v, vo, R, perm, 0.5, 0.6, want_grad=False)
+    rl, _ = oracle.value_loss(v, vo, R, idx, f32(0.5), f32(0.6))
+    assert st_p == 0 and abs(loss_p - rl) <= 1e-5 * max(1.0, abs(rl))
+    # no list: the first n positions; unaligned arrays take the element-wise path
+    loss_i, dv_i, n_i, st_i = run_value(v, vo, R, None, 0.5, 0.6, n_sel=777)
+    rl_i, rdv_i = oracle.value_loss(v, vo, R, np.arange(777, dtype=np.int32), f32(0.5), f32(0.6))
+    assert st_i == 0 and n_i == 777 and abs(loss_i - rl_i) <= 1e-5
+    np.testing.assert_allclose(dv_i, rdv_i, rtol=1e-5, atol=1e-9)
+
+
+def test_value_loss_unaligned_arrays_and_tile_edges():
+    """Value tokens on both sides of every tile edge of the sweep, a list that ends on an edge, and
+    arrays that start off a 16-byte boundary."""
+    from paper_2506_15050_b200 import binding as b
+    rng = np.random.default_rng(53)
+    T = 4032
+    N = 5 * T + 17
+    v = rng.standard_normal(N).astype(np.float32)
+    vo = (v + 0.3 * rng.standard_normal(N)).astype(np.float32)
+    R = rng.standard_normal(N).astype(np.float32)
+    edges = np.concatenate([[k * T - 1, k * T, k * T + 1] for k in range(1, 6)])
+    idx = np.unique(np.concatenate([[0, N - 1], edges[edges < N], rng.choice(N, 900, replace=False)])).astype(np.int32)
+    for sel in (idx, idx[idx < 2 * T], np.arange(N, dtype=np.int32), np.arange(T, 2 * T, dtype=np.int32)):
+        loss, dv, n, st = run_value(v, vo, R, sel, 0.5, 0.6)
+        rl, rdv = oracle.value_loss(v, vo, R, sel, f32(0.5), f32(0.6))
+        assert st == 0 and n == len(sel) and abs(loss - rl) <= 1e-5 * max(1.0, abs(rl))
+        np.testing.assert_allclose(dv, rdv, rtol=1e-5, atol=1e-9)
+    # unaligned views
+    buf = [torch.zeros(N + 4, device=DEV) for _ in range(4)]
+    for off in (1, 3):
+        for t_, h in zip(buf[:3], (v, vo, R)):
+            t_[off:off + N] = dev(h, torch.float32)
+        buf[3].fill_(float("nan"))
+        loss_t = torch.zeros(1, device=DEV)
+        stats = torch.zeros(2, dtype=torch.int32, device=DEV)
+        ws = b.workspace(b.OP_VALUE_LOSS, N, 0, len(idx), 0, DEV)
+        b.tppo_value_loss(buf[0][off:off + N], buf[1][off:off + N], buf[2][off:off + N], dev(idx, torch.int32),
+                          None, len(idx), 0.5, 0.6, 0.0, loss_t, buf[3][off:off + N], stats, ws)
+        torch.cuda.synchronize()
+        rl, rdv = oracle.value_loss(v, vo, R, idx, f32(0.5), f32(0.6))
+        assert int(stats[1]) == 0 and abs(float(loss_t) - rl) <= 1e-5 * max(1.0, abs(rl))
+        np.testing.assert_allclose(buf[3][off:off + N].cpu().numpy(), rdv, rtol=1e-5, atol=1e-9)
+        assert torch.isnan(buf[3][:off]).all() and torch.isnan(buf[3][off + N:]).all()
 
 
 def test_value_loss_config1():

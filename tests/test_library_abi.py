@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_host_only_calls(lib):
     lib.tppo_status_string.restype = ctypes.c_char_p
-    assert lib.tppo_version() >= 100
+    assert lib.tppo_version() >= 200
     assert lib.tppo_status_string(0) == b"ok"
     assert b"workspace" in lib.tppo_status_string(2)
     lib.tppo_workspace_bytes.restype = ctypes.c_size_t
@@ -57,9 +57,9 @@ def test_argument_errors_are_reported_before_any_launch(lib):
     p = ctypes.cast(buf, vp)
     assert lib.tppo_egae(p, p, p, p, p, None, 1, 10, 1.5, 0.95, p, None, p, None, 0, None) == 1   # gamma > 1
     assert lib.tppo_egae(p, p, p, p, p, None, 1, 10, 1.0, 0.95, p, None, p, None, 0, None) == 2   # no workspace
-    lib.tppo_select_tokens.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, i32, i64, vp, vp, vp, vp, sz, vp]
-    assert lib.tppo_select_tokens(p, p, p, p, p, -1, None, None, 1, 10, p, p, p, p, 4096, None) == 1
-    assert lib.tppo_select_tokens(p, p, p, p, p, 0, None, None, 1, 10, p, p, p, None, 0, None) == 2
+    lib.tppo_select_tokens.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, vp, i32, i64, vp, vp, vp, vp, sz, vp]
+    assert lib.tppo_select_tokens(p, p, p, p, p, -1, None, None, None, 1, 10, p, p, p, p, 4096, None) == 1
+    assert lib.tppo_select_tokens(p, p, p, p, p, 0, None, None, None, 1, 10, p, p, p, None, 0, None) == 2
     lib.tppo_value_loss.argtypes = [vp, vp, vp, i64, vp, vp, i64, f32, f32, f32, vp, vp, vp, vp, sz, vp]
     assert lib.tppo_value_loss(p, p, p, 10, None, None, 20, 0.5, 0.6, 0.0, p, None, p, p, 4096, None) == 1
     lib.tppo_policy_loss_fwd_bwd.argtypes = [vp, i32, i64, i32, i64, vp, vp, vp, i64, vp, vp, vp, i64, f32, f32,
