@@ -116,6 +116,21 @@ def logprob(logits, targets, rows=None):
     return out
 
 
+def logprob_stats(logits, targets, rows=None, aux_idx=None, old_logp=None):
+    """Forward-only statistics: dict(logp[n], entropy[n], mean_entropy, mean_kl)."""
+    a, code, ld = _logits_view(logits)
+    t = _arr(targets, np.int32)
+    rw = _arr(rows, np.int32)
+    ax = _arr(aux_idx, np.int32)
+    ol = _arr(old_logp, np.float32)
+    n = a.shape[0] if rw is None else rw.shape[0]
+    logp, ent = np.empty(n, np.float64), np.empty(n, np.float64)
+    means = np.zeros(2, np.float64)
+    lib().oracle_logprob_stats(_p(a), C.c_int(code), C.c_int32(a.shape[1]), C.c_int64(ld), _p(t),
+                               _p(rw), _p(ax), C.c_int64(n), _p(ol), _p(logp), _p(ent), _p(means))
+    return dict(logp=logp, entropy=ent, mean_entropy=float(means[0]), mean_kl=float(means[1]))
+
+
 def policy_loss(logits, targets, rows, aux_idx, old_logp, adv, eps_low, eps_high,
                 denom=0.0, want_dlogits=True):
     """Returns dict(logp, token_loss, loss, clip_lo, clip_hi, dlogits[n,V] or None)."""

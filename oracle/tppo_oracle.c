@@ -12,8 +12,8 @@
  *
  * Parity pins (see tests/test_oracle_*.py): brute-force sums of Eq. 2/6, the gamma=lambda=1
  * telescoped closed form, a hand-derived 3-token example, scipy's IIR filter, exhaustive mask
- * enumeration, scipy logsumexp, finite differences and float64 autograd of Eq. 1 / Eq. 4-5.
- * No function here is "parity unpinned".
+ * enumeration, scipy logsumexp, finite differences and float64 autograd of Eq. 1 / Eq. 4-5,
+ * torch's float64 softmax entropy.  No function here is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -173,6 +173,47 @@ void oracle_logprob(const void *logits, int dtype, int32_t V, int64_t ld,
         row_max_and_logsum(logits, dtype, ld, row, V, &m, &log_sum);
         logp[j] = (logit_at(logits, dtype, ld, row, targets[row]) - m) - log_sum;
     }
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Statistics of the forward-only sweep that produces the old-policy log-probs (the step of
+ * Algorithm 1 that snapshots pi_theta_old): per selected row the log-prob of its target and
+ * the entropy of its softmax,
+ *     H = - sum_v p_v log p_v,   p_v = softmax_v,   log p_v = (x_v - m) - log S,
+ * a vocabulary entry of probability 0 (x_v = -inf) contributing 0; and over the selected rows
+ * the means of H and of old_logp - logp (the usual sample estimate of KL(pi_old || pi_theta)).
+ * aux_idx[j] (NULL: the logits row) indexes old_logp, which may be NULL (mean_kl = 0).
+ * ---------------------------------------------------------------------------------------- */
+void oracle_logprob_stats(const void *logits, int dtype, int32_t V, int64_t ld,
+                          const int32_t *targets, const int32_t *rows, const int32_t *aux_idx,
+                          int64_t n, const float *old_logp,
+                          double *logp, double *entropy, double *means /* [2] */)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t j = 0; j < n; ++j) {
+        const int64_t row = rows ? rows[j] : j;
+        double m, log_sum;
+        row_max_and_logsum(logits, dtype, ld, row, V, &m, &log_sum);
+        logp[j] = (logit_at(logits, dtype, ld, row, targets[row]) - m) - log_sum;
+        double H = 0.0;
+        for (int32_t v = 0; v < V; ++v) {
+            const double lp = (logit_at(logits, dtype, ld, row, v) - m) - log_sum;
+            const double p = exp(lp);
+            if (p > 0.0) H -= p * lp;
+        }
+        entropy[j] = H;
+    }
+    double sum_h = 0.0, sum_kl = 0.0;
+    for (int64_t j = 0; j < n; ++j) {
+        sum_h += entropy[j];
+        if (old_logp) {
+            const int64_t row = rows ? rows[j] : j;
+            const int64_t a = aux_idx ? aux_idx[j] : row;
+            sum_kl += (double)old_logp[a] - logp[j];
+        }
+    }
+    means[0] = n > 0 ? sum_h / (double)n : 0.0;
+    means[1] = n > 0 ? sum_kl / (double)n : 0.0;
 }
 
 /* ------------------------------------------------------------------------------------------

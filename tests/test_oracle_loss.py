@@ -74,6 +74,47 @@ def test_logprob_and_gradient_at_the_largest_magnitudes():
     np.testing.assert_allclose(oracle.logprob(np.full((1, V), 2.0 ** 100), y[:1]), [-np.log(V)], atol=1e-12)
 
 
+def test_entropy_and_kl_statistics():
+    """Forward-only statistics against torch's float64 softmax (-sum p log p), closed forms (uniform
+    row: log V; one-hot row: 0; two equal maxima among -inf: log 2), bounds, shift invariance, and
+    the KL estimate against its definition mean(old_logp - logp) with an index map."""
+    rng = np.random.default_rng(11)
+    R, V = 12, 257
+    x = (3.0 * rng.standard_normal((R, V))).astype(np.float32)
+    y = rng.integers(0, V, R).astype(np.int32)
+    out = oracle.logprob_stats(x, y)
+    xt = torch.tensor(x, dtype=torch.float64)
+    lp = torch.log_softmax(xt, dim=1)
+    ref_h = -(lp.exp() * lp).sum(dim=1).numpy()
+    np.testing.assert_allclose(out["entropy"], ref_h, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(out["logp"], lp[torch.arange(R), torch.tensor(y).long()].numpy(), atol=1e-12)
+    assert abs(out["mean_entropy"] - ref_h.mean()) < 1e-12 and out["mean_kl"] == 0.0
+    assert np.all(out["entropy"] > 0) and np.all(out["entropy"] < np.log(V))
+    np.testing.assert_allclose(oracle.logprob_stats(x + np.float32(16.0), y)["entropy"], out["entropy"], atol=1e-4)
+    # closed forms
+    special = np.full((3, V), -np.inf, np.float32)
+    special[0, :] = 0.7                       # uniform
+    special[1, 5] = 2.0                       # one-hot: every other entry has probability 0
+    special[2, [3, 200]] = -1.5               # two equal entries
+    h = oracle.logprob_stats(special, np.array([0, 5, 3], np.int32))
+    np.testing.assert_allclose(h["entropy"], [np.log(V), 0.0, np.log(2.0)], atol=1e-12)
+    np.testing.assert_allclose(h["logp"], [-np.log(V), 0.0, -np.log(2.0)], atol=1e-12)
+    # rows, index map and the KL estimate
+    rows = np.array([7, 2, 9, 0], np.int32)
+    aux = np.array([1, 30, 5, 12], np.int32)
+    old = rng.standard_normal(40).astype(np.float32)
+    sub = oracle.logprob_stats(x, y, rows, aux, old)
+    np.testing.assert_allclose(sub["entropy"], ref_h[rows], atol=1e-12)
+    assert abs(sub["mean_kl"] - np.mean(old[aux].astype(np.float64) - sub["logp"])) < 1e-12
+    on_policy = out["logp"].astype(np.float32)
+    assert abs(oracle.logprob_stats(x, y, None, None, on_policy)["mean_kl"]) < 1e-7
+    # bf16 storage
+    xb = torch.from_numpy(x).to(torch.bfloat16)
+    bits = xb.view(torch.int16).numpy().view(np.uint16)
+    lpb = torch.log_softmax(xb.double(), dim=1)
+    np.testing.assert_allclose(oracle.logprob_stats(bits, y)["entropy"], -(lpb.exp() * lpb).sum(dim=1).numpy(), atol=1e-12)
+
+
 def torch_policy_loss(x, y, old, adv, el, eh, denom):
     """Eq. 1 restated with autograd as an independent comparator (float64)."""
     xt = torch.tensor(x, dtype=torch.float64, requires_grad=True)
