@@ -121,10 +121,11 @@ size_t tppo_workspace_bytes(int op, int64_t N, int32_t B, int64_t n_max, int32_t
  * A reward, value or used bootstrap value inside a segment that is a NaN or an infinity is read as
  * 0 and raises TPPO_DEV_NONFINITE, so the outputs stay finite.
  * Precision: the advantage is carried as G_t = A_t + values[t] (G_t = rewards[t] + gamma*(1-lambda)*
- * V(s_{t+1}) + gamma*lambda*G_{t+1}, so successive values never cancel); runs of 16 consecutive
- * positions are evaluated in fp32 (gamma*lambda split into two floats, exact to 2^-48), everything
- * carried across runs, warps and tiles is fp64.  The error of a result is a few units of 2^-24 of
- * the largest |G| or |R| of its run and does not grow with the length of a response.  N < 2^31.
+ * V(s_{t+1}) + gamma*lambda*G_{t+1}, so successive values never cancel).  Everything carried across
+ * runs of 16 consecutive positions, warps and tiles is fp64 (the composite map of each run
+ * included); inside a run the results are evaluated in fp32 from the entering value rounded once.
+ * The error of a result is that rounding plus at most 16 fp32 roundings at the magnitude of |G| or
+ * |R| inside its run; it does not grow with the length of a response.  N < 2^31.
  * Arrays that are 16-byte aligned take the fast path (TMA copies); others are still handled.
  * The first call in a process looks up the driver's tensor-map encoder (without it every tile takes
  * the slower plain-load path; no error).
@@ -240,6 +241,32 @@ int tppo_policy_loss_fwd_bwd(const void *logits, int32_t logits_dtype,
                              float *logp, float *token_loss, float *loss, int32_t *stats,
                              void *dlogits, int32_t dlogits_mode, int32_t kernel_hint,
                              void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Forward-only sweep with statistics: the log-probs of the old-policy snapshot (the step of
+ * Algorithm 1 that sets pi_theta_old before the updates; the same gather as above, one read of each
+ * selected row, no gradient) together with two diagnostics taken from the same pass.  For the j-th
+ * selected row r = rows[j] (j < n = min(*n_sel, n_max)), a = aux_idx[j]:
+ *     logp[j]    = x[r, y] - log sum_v exp(x[r, v]),          y = targets[r]
+ *     entropy[j] = - sum_v p_v log p_v,  p = softmax(x[r, :])  (an entry of probability 0 adds 0)
+ *     means[0]   = (1/n) sum_j entropy[j]
+ *     means[1]   = (1/n) sum_j (old_logp[a] - logp[j])         (sample estimate of KL(pi_old || pi))
+ *   logits, targets, rows, n_sel, n_max, aux_idx, aux_len: as in tppo_policy_loss_fwd_bwd
+ *   old_logp   fp32 [aux_len] or NULL (means[1] is then 0 and aux_idx is not used)
+ *   logp       [n_max] fp32 out;  entropy [n_max] fp32 out or NULL;  means [2] fp32 out
+ *   stats      [4] int32 out: n, 0, 0, status bits
+ *   workspace  tppo_workspace_bytes(TPPO_OP_POLICY_LOSS, R, 0, n_max, V) bytes
+ * A row with a bad index or target, or whose logits hold a NaN or +inf (or nothing but -inf), gets
+ * logp = entropy = 0, is left out of both sums (n still divides) and raises its status bit.
+ * Fixed-order reductions: run-to-run identical.
+ */
+int tppo_policy_logprob_stats(const void *logits, int32_t logits_dtype,
+                              int64_t R, int32_t V, int64_t ld,
+                              const int32_t *targets,
+                              const int32_t *rows, const int32_t *n_sel, int64_t n_max,
+                              const int32_t *aux_idx, const float *old_logp, int64_t aux_len,
+                              float *logp, float *entropy, float *means, int32_t *stats,
+                              void *workspace, size_t workspace_bytes, void *stream);
 
 /* kernel_hint values of tppo_policy_loss_fwd_bwd */
 enum {

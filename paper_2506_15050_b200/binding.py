@@ -48,6 +48,9 @@ _lib.tppo_policy_loss_fwd_bwd.restype = C.c_int
 _lib.tppo_policy_loss_fwd_bwd.argtypes = [_vp, _i32, _i64, _i32, _i64, _vp, _vp, _vp, _i64, _vp,
                                           _vp, _vp, _i64, _f32, _f32, _f32, _vp, _vp, _vp, _vp,
                                           _vp, _i32, _i32, _vp, _sz, _vp]
+_lib.tppo_policy_logprob_stats.restype = C.c_int
+_lib.tppo_policy_logprob_stats.argtypes = [_vp, _i32, _i64, _i32, _i64, _vp, _vp, _vp, _i64, _vp, _vp, _i64,
+                                           _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.tppo_value_loss.restype = C.c_int
 _lib.tppo_value_loss.argtypes = [_vp, _vp, _vp, _i64, _vp, _vp, _i64, _f32, _f32, _f32, _vp, _vp,
                                  _vp, _vp, _sz, _vp]
@@ -176,6 +179,20 @@ def tppo_policy_loss_fwd_bwd(logits, targets, rows, n_sel, n_max, aux_idx, old_l
         eps_low, eps_high, denom, _ptr(logp, torch.float32), _ptr(token_loss, torch.float32),
         _ptr(loss, torch.float32), _ptr(stats, torch.int32),
         None if dlogits is None else dlogits.data_ptr(), dlogits_mode, kernel_hint,
+        _ptr(ws), ws.numel(), _stream()))
+
+
+def tppo_policy_logprob_stats(logits, targets, rows, n_sel, n_max, aux_idx, old_logp, logp, entropy,
+                              means, stats, ws, V=None):
+    assert logits.is_cuda and logits.dim() == 2 and logits.stride(1) == 1
+    dt = {torch.bfloat16: BF16, torch.float32: F32}[logits.dtype]
+    R, ld = logits.shape[0], logits.stride(0)
+    V = logits.shape[1] if V is None else V
+    _check(_lib.tppo_policy_logprob_stats(
+        logits.data_ptr(), dt, R, V, ld, _ptr(targets, torch.int32), _ptr(rows, torch.int32),
+        _ptr(n_sel, torch.int32), n_max, _ptr(aux_idx, torch.int32), _ptr(old_logp, torch.float32),
+        0 if old_logp is None else old_logp.numel(), _ptr(logp, torch.float32),
+        _ptr(entropy, torch.float32), _ptr(means, torch.float32), _ptr(stats, torch.int32),
         _ptr(ws), ws.numel(), _stream()))
 
 

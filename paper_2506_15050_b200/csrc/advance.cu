@@ -199,7 +199,7 @@ __device__ __forceinline__ AdvSlotRef adv_slot_ref(const AdvanceArgs& a, int i, 
     return r;
 }
 
-__global__ void __launch_bounds__(kAdvCopyThreads) advance_copy_kernel(const AdvanceArgs a) {
+__global__ void __launch_bounds__(kAdvCopyThreads, 6) advance_copy_kernel(const AdvanceArgs a) {
     __shared__ int s_slot0;
     __shared__ int32_t s_begin[kAdvTable + 1];
     __shared__ const int32_t* s_src[kAdvTable];
@@ -233,23 +233,43 @@ __global__ void __launch_bounds__(kAdvCopyThreads) advance_copy_kernel(const Adv
     const bool table_ok = int64_t(s_begin[kAdvTable]) >= t1 || slot0 + kAdvTable >= a.B;
     const bool vec = (reinterpret_cast<uintptr_t>(a.next_tokens) & 15) == 0;
     if (table_ok && vec) {
+        // two groups of four positions per trip, all eight loads issued before the first store
+        const int n_slots = min(kAdvTable, a.B - slot0);          // table entries in use
+        const int32_t e1 = int32_t(t1);
         int h = 0;
-        for (int64_t p = t0 + 4 * threadIdx.x; p < t1; p += 4 * kAdvCopyThreads) {
-            while (h + 1 < kAdvTable && slot0 + h + 1 < a.B && p >= int64_t(s_begin[h + 1])) ++h;
-            int4 v = make_int4(0, 0, 0, 0);
-            if (p + 4 <= t1 && p + 4 <= int64_t(s_begin[h + 1])) {       // four positions of one slot
-                const int32_t* src = s_src[h];
-                if (src) {
-                    v.x = __ldg(src + p); v.y = __ldg(src + p + 1);
-                    v.z = __ldg(src + p + 2); v.w = __ldg(src + p + 3);
+        constexpr int kStep = 4 * kAdvCopyThreads;
+        for (int32_t p0 = int32_t(t0) + 4 * threadIdx.x; p0 < e1; p0 += 2 * kStep) {
+            int4 v[2];
+            bool whole[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int32_t p = p0 + u * kStep;
+                v[u] = make_int4(0, 0, 0, 0);
+                whole[u] = false;
+                if (p >= e1) continue;
+                while (h + 1 < n_slots && p >= s_begin[h + 1]) ++h;
+                whole[u] = p + 4 <= e1 && p + 4 <= s_begin[h + 1];      // four positions of one slot
+                if (whole[u]) {
+                    const int32_t* src = s_src[h];
+                    if (src) {
+                        v[u].x = __ldg(src + p); v[u].y = __ldg(src + p + 1);
+                        v[u].z = __ldg(src + p + 2); v[u].w = __ldg(src + p + 3);
+                    }
                 }
-                *reinterpret_cast<int4*>(a.next_tokens + p) = v;
-            } else {
-                int hh = h;
-                for (int e = 0; e < 4 && p + e < t1; ++e) {
-                    while (hh + 1 < kAdvTable && slot0 + hh + 1 < a.B && p + e >= int64_t(s_begin[hh + 1])) ++hh;
-                    const int32_t* src = s_src[hh];
-                    a.next_tokens[p + e] = src ? __ldg(src + p + e) : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int32_t p = p0 + u * kStep;
+                if (p >= e1) continue;
+                if (whole[u]) {
+                    *reinterpret_cast<int4*>(a.next_tokens + p) = v[u];
+                } else {        // the group straddles two slots or the end: one position at a time
+                    int hh = 0;
+                    for (int e = 0; e < 4 && p + e < e1; ++e) {
+                        while (hh + 1 < n_slots && p + e >= s_begin[hh + 1]) ++hh;
+                        const int32_t* src = s_src[hh];
+                        a.next_tokens[p + e] = src ? __ldg(src + p + e) : 0;
+                    }
                 }
             }
         }

@@ -8,15 +8,18 @@
 // are affine in the value at the next position: every position carries a map x -> a*x + b, with
 // a = 0 on the last token of a segment and outside every segment.  Maps compose associatively.
 //
-// Precision.  A thread owns sixteen consecutive positions and runs them sequentially in fp32 (the
-// multiplier gamma*lambda, the only factor that is raised to high powers, is split into two floats
-// so that it is exact to 2^-48); everything that crosses threads -- the thread composites, the warp
-// scan, the tile composites and the look-back -- is fp64, and the value entering a thread's run is
-// rounded to fp32 once.  The rounding error of a result is a few units of 2^-24 of the largest
-// |G| or |R| in its run; nothing accumulates over the length of a segment.
+// Precision.  A thread owns sixteen consecutive positions (its run).  The composite map of a run,
+// and everything that crosses threads -- the warp scan, the tile composites, the look-back -- is
+// fp64: the value that enters a run is exact to double rounding however long the segment is.  (With
+// fp32 run composites, each run's rounding, small as it is, added up over the hundreds of runs of a
+// long response: 2.5e-5 absolute on zero-mean dense rewards over 9000 tokens.)  The results of a run
+// are then replayed from that entering value, rounded to fp32 once, sequentially in fp32 (the
+// multiplier gamma*lambda split into two floats, exact to 2^-48).  The error of a result is thus the
+// rounding of the entering value plus at most sixteen fp32 roundings at the magnitude of |G| or |R|
+// inside its own run; nothing accumulates over the length of a segment.
 //
-// Tiles of 2048 positions are taken by ticket from the END of the arrays backwards, so the tiles a
-// tile looks back at (those to its right) hold earlier tickets and are running or done.  A tile
+// Tiles of 2048 positions are worked on from the END of the arrays backwards, so the tiles a
+// tile looks back at (those to its right) were started earlier and are running or done.  A tile
 // composes its positions right to left, publishes the composite, and obtains the value entering
 // from its right-hand neighbour by decoupled look-back over the tiles behind it.  A composite whose
 // `a` has become 0 (a segment ended inside the range) ends the look-back early.  The inputs of a
@@ -34,18 +37,24 @@
 
 namespace tppo {
 
-constexpr int kScanThreads = 128;
+constexpr int kScanThreads = 128;     // (256-thread tiles of 4096 positions measured 5 % slower)
 constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kScanItems = 16;
 constexpr int kScanTile = kScanThreads * kScanItems;  // 2048 positions
 constexpr int kSegCap = 32;                           // segments of one tile kept in shared memory
-constexpr int kScanCtasPerSm = 8;
+constexpr int kScanCtasPerSm = 1024 / kScanThreads;
+constexpr int kScanBoxRows = 64;                      // rows of 32 positions per TMA box
+constexpr int kScanBoxes = kScanTile / (kScanBoxRows * 32);
+static_assert(kScanTile % (kScanBoxRows * 32) == 0, "a tile is a whole number of TMA boxes");
 constexpr uint32_t kScanSpinLimit = 1u << 22;
-#ifndef TPPO_EGAE_F64_MAP
-#define TPPO_EGAE_F64_MAP 1    // 1: a run's composite map is evaluated in fp64; 0: in fp32
-#endif
+// Tile order.  0 (default): block b takes tile num_tiles-1-b.  A tile only ever waits for tiles to
+// its right, i.e. for blocks with smaller indices, and thread blocks are dispatched in index order, so
+// those are running or done; should that ever not hold, the bounded wait gives up and the call
+// reports TPPO_DEV_WAIT_TIMEOUT instead of hanging.  1: tiles are drawn from an atomic ticket
+// counter instead, which needs no assumption about dispatch order (measured 1.3 us slower at
+// 17.5 M tokens: one L2 round trip and one barrier more in every tile's life).
 #ifndef TPPO_EGAE_TICKET
-#define TPPO_EGAE_TICKET 1     // 1: tiles by ticket; 0: tile = f(blockIdx), relying on in-order dispatch
+#define TPPO_EGAE_TICKET 0
 #endif
 
 struct Affine2 {  // x -> (aA*xA + bA, aR*xR + bR)
@@ -121,20 +130,11 @@ struct EgaeArgs {
     float* ret;
     int32_t* status;
     TileState* state;
-    // Three words at the head of the workspace, cleared to all-ones together with the tile states:
-    // the ticket counter (+1 wraps the first draw to 0), the finished-tiles counter (likewise), and
-    // the call's status bits, kept INVERTED (a bit is raised by clearing it) so that the one
-    // all-ones clear serves them too.  The last tile to finish writes the status word out.
-    uint32_t* ticket;
-    uint32_t* done;
-    uint32_t* ws_status;
+    uint32_t* ticket;      // head of the workspace, cleared to all-ones with the tile states (+1 wraps to 0)
     uint32_t spin_limit;   // polls a look-back may spend on one round of tiles before it gives up
     int32_t no_publish;    // test hook: tiles keep their states to themselves, so every look-back runs out
 };
-__device__ __forceinline__ void egae_raise(const EgaeArgs& a, int bits) {
-    atomicAnd(a.ws_status, ~uint32_t(bits));
-    __threadfence();      // performed before this thread reaches the tile's final barrier
-}
+__device__ __forceinline__ void egae_raise(const EgaeArgs& a, int bits) { atomicOr(a.status, bits); }
 __device__ __forceinline__ bool finite_f32(float x) { return fabsf(x) <= kFltMax; }
 
 // Shared-memory image of one tile.  r and v are 64 rows of 32 positions (128 bytes) in the layout
@@ -446,11 +446,7 @@ __device__ __forceinline__ Affine2 egae_run_map_once(const EgaeArgs& a, const Ti
     }
     if (rs.masked) {
         const uint32_t inside = rs.bits & 0xffffu, cont = rs.bits >> 16;
-#if TPPO_EGAE_F64_MAP
         double bG = 0.0, bR = 0.0;
-#else
-        float bG = 0.f, bR = 0.f;
-#endif
         float vn = v_right;
 #pragma unroll
         for (int q = kScanItems / 4 - 1; q >= 0; --q) {
@@ -465,21 +461,12 @@ __device__ __forceinline__ Affine2 egae_run_map_once(const EgaeArgs& a, const Ti
                 const bool in = (inside >> k) & 1u, c = (cont >> k) & 1u;
                 probe0 = fmaf(rr[e], 0.f, probe0);
                 probe0 = fmaf(vv[e], 0.f, probe0);
-#if TPPO_EGAE_F64_MAP
                 const double rd = in ? double(rr[e]) : 0.0;
                 double x = fma(a.c1_d, double(vn), rd);
                 if (k == rs.k_last) x = fma(a.gamma, double(rs.boundary_own ? vv[e] : rs.v_boundary), rd);
                 x = in ? x : 0.0;
                 bG = c ? fma(a.gl, bG, x) : x;
                 bR = c ? fma(a.gamma, bR, rd) : rd;
-#else
-                float x = fmaf(a.c1, vn, rr[e]);
-                if (k == rs.k_last) x = fmaf(a.gamma_f, rs.boundary_own ? vv[e] : rs.v_boundary, rr[e]);
-                x = in ? x : 0.f;
-                const float re = in ? rr[e] : 0.f;
-                bG = c ? fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, x)) : x;
-                bR = c ? fmaf(a.gamma_f, bR, re) : re;
-#endif
                 vn = vv[e];
             }
         }
@@ -489,11 +476,7 @@ __device__ __forceinline__ Affine2 egae_run_map_once(const EgaeArgs& a, const Ti
     }
     if (fast) {
         // every map has the same multiplier and no per-position test is needed
-#if TPPO_EGAE_F64_MAP
         double bG = 0.0, bR = 0.0;
-#else
-        float bG = 0.f, bR = 0.f;
-#endif
         float vn = v_right;
 #pragma unroll
         for (int q = kScanItems / 4 - 1; q >= 0; --q) {
@@ -506,26 +489,16 @@ __device__ __forceinline__ Affine2 egae_run_map_once(const EgaeArgs& a, const Ti
             for (int e = 3; e >= 0; --e) {
                 probe0 = fmaf(rr[e], 0.f, probe0);
                 probe0 = fmaf(vv[e], 0.f, probe0);
-#if TPPO_EGAE_F64_MAP
                 const double rd = double(rr[e]);
                 bG = fma(a.gl, bG, fma(a.c1_d, double(vn), rd));
                 bR = fma(a.gamma, bR, rd);
-#else
-                const float x = fmaf(a.c1, vn, rr[e]);
-                bG = fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, x));
-                bR = fmaf(a.gamma_f, bR, rr[e]);
-#endif
                 vn = vv[e];
             }
         }
         probe = probe0;
         return Affine2{a.gl_run, double(bG), a.gamma_run, double(bR)};
     }
-#if TPPO_EGAE_F64_MAP
     double bG = 0.0, bR = 0.0;
-#else
-    float bG = 0.f, bR = 0.f;
-#endif
     double aG = 1.0, aR = 1.0;
     int i = i_start;
     float v_next = v_right;
@@ -534,21 +507,12 @@ __device__ __forceinline__ Affine2 egae_run_map_once(const EgaeArgs& a, const Ti
         const PosTerm t = egae_position(a, buf, win, t0, n_tile, win_lo, win_smem, l0 + k, v_next, i, bad, nonfinite);
         v_next = buf.v[pos_slot(l0 + k)];
         if (t.cont) {
-#if TPPO_EGAE_F64_MAP
             bG = fma(a.gl, bG, t.xd);
             bR = fma(a.gamma, bR, double(t.r));
-#else
-            bG = fmaf(a.gl_hi, bG, fmaf(a.gl_lo, bG, t.x));
-            bR = fmaf(a.gamma_f, bR, t.r);
-#endif
             aG *= a.gl;
             aR *= a.gamma;
         } else {
-#if TPPO_EGAE_F64_MAP
             bG = t.xd;
-#else
-            bG = t.x;
-#endif
             bR = t.r;
             aG = 0.0;
             aR = 0.0;
@@ -690,9 +654,8 @@ __device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, TileBuf& buf,
     }
 }
 
-// One CTA per tile of 2048 positions; tiles are taken by ticket, from the END of the arrays
-// backwards, so the tiles a tile looks back at (those to its right) hold earlier tickets and are
-// running or done.  The latencies of a tile (ticket, copy, window search, look-back) are covered by
+// One CTA per tile of 2048 positions, from the END of the arrays backwards, so the tiles a tile
+// looks back at (those to its right) were started earlier and are running or done.  The latencies of a tile (ticket, copy, window search, look-back) are covered by
 // the other CTAs resident on the SM.  A whole tile's results are written over its inputs in shared
 // memory and leave by two TMA stores.
 __global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm)
@@ -733,8 +696,12 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     if (by_tma) {
         if (threadIdx.x == 0) {
             ptx::mbar_arrive_expect_tx(bar, 2 * kScanTile * uint32_t(sizeof(float)));
-            umma::tma_load_2d(ptx::smem_addr(buf.r), &map_r, bar, 0, int32_t(t0 / kRowPos));
-            umma::tma_load_2d(ptx::smem_addr(buf.v), &map_v, bar, 0, int32_t(t0 / kRowPos));
+#pragma unroll
+            for (int bx = 0; bx < kScanBoxes; ++bx) {
+                const int32_t y = int32_t(t0 / kRowPos) + bx * kScanBoxRows;
+                umma::tma_load_2d(ptx::smem_addr(buf.r + bx * kScanBoxRows * kRowPos), &map_r, bar, 0, y);
+                umma::tma_load_2d(ptx::smem_addr(buf.v + bx * kScanBoxRows * kRowPos), &map_v, bar, 0, y);
+            }
         }
     } else {
         for (int k = threadIdx.x; k < n_tile; k += kScanThreads) {
@@ -799,23 +766,19 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     egae_run_replay(a, buf, win, t0, n_tile, threadIdx.x, rs, G, R, by_tma, bad, nonfinite);
     if (bad) egae_raise(a, TPPO_DEV_BAD_SEGMENT);
     if (nonfinite) egae_raise(a, TPPO_DEV_NONFINITE);
-    if (by_tma) ptx::fence_proxy_async_smem();       // the TMA stores read what was just written
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        if (by_tma) {
-            const int32_t y = tile * (kScanTile / kRowPos);
-            umma::tma_store_2d(&map_adv, ptx::smem_addr(buf.v), 0, y);
-            if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(buf.r), 0, y);
+    if (by_tma) {
+        ptx::fence_proxy_async_smem();       // the TMA stores read what was just written
+        __syncthreads();
+        if (threadIdx.x == 0) {
+#pragma unroll
+            for (int bx = 0; bx < kScanBoxes; ++bx) {
+                const int32_t y = tile * (kScanTile / kRowPos) + bx * kScanBoxRows;
+                umma::tma_store_2d(&map_adv, ptx::smem_addr(buf.v + bx * kScanBoxRows * kRowPos), 0, y);
+                if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(buf.r + bx * kScanBoxRows * kRowPos), 0, y);
+            }
             ptx::bulk_commit();
+            ptx::bulk_wait_read<0>();   // shared memory must outlive the stores' reads of it
         }
-        // The last tile to finish hands the status bits to the caller (every other tile's bits were
-        // raised before its own count: fence, then count).
-        __threadfence();
-        if (atomicAdd(a.done, 1u) + 1u == uint32_t(a.num_tiles) - 1u) {
-            __threadfence();
-            *a.status = int32_t(~*reinterpret_cast<volatile uint32_t*>(a.ws_status));
-        }
-        if (by_tma) ptx::bulk_wait_read<0>();   // shared memory must outlive the stores' reads of it
     }
 }
 
@@ -857,16 +820,13 @@ static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
     return TPPO_OK;
 }
 
-constexpr size_t kScanHeadBytes = 256;      // ticket, finished-tiles counter, inverted status bits
+constexpr size_t kScanHeadBytes = 256;      // the ticket counter
 size_t egae_workspace_bytes(int64_t N) {
     const int64_t tiles = (N + kScanTile - 1) / kScanTile;
     return kScanHeadBytes + align_up(size_t(tiles > 0 ? tiles : 1) * sizeof(TileState), kWsAlign);
 }
 static void egae_carve(EgaeArgs& a, void* ws) {
-    uint32_t* head = static_cast<uint32_t*>(ws);
-    a.ticket = head;
-    a.done = head + 1;
-    a.ws_status = head + 2;
+    a.ticket = static_cast<uint32_t*>(ws);
     a.state = reinterpret_cast<TileState*>(static_cast<char*>(ws) + kScanHeadBytes);
 }
 
@@ -888,12 +848,11 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
     if (!workspace || workspace_bytes < need || !aligned(workspace, kWsAlign))
         return TPPO_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (N == 0) {
-        TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
-        return TPPO_OK;
-    }
-    // one memset: tile states start out unset (all-ones), and so do the two counters and the
-    // (inverted) status bits; the kernel's last tile writes *status
+    TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
+    if (N == 0) return TPPO_OK;
+    // tile states start out unset (all-ones), the ticket counter at all-ones too.  (Letting the last
+    // tile to finish hand over the status bits instead of clearing them here was measured: the fence
+    // and counter at the end of every tile cost 9 us at 17.5 M tokens, a 4-byte clear nothing.)
     TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0xff, need, s));
     EgaeArgs a{};
     a.rewards = rewards; a.values = values; a.seg_begin = seg_begin; a.seg_end = seg_end;
@@ -952,17 +911,15 @@ TPPO_API int tppo_egae_static(const float* rewards, const float* values, const i
     const int rc = static_scratch_for_current_device(&scratch);
     if (rc != TPPO_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (N == 0) {
-        TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
-        return TPPO_OK;
-    }
+    TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
+    if (N == 0) return TPPO_OK;
     EgaeArgs a{};
     a.rewards = rewards; a.values = values; a.seg_begin = seg_begin; a.seg_end = seg_end;
     a.truncated = truncated; a.bootstrap = bootstrap; a.B = B; a.N = int32_t(N);
     a.adv = advantages; a.ret = returns; a.status = status;
     egae_carve(a, scratch);
-    // the array still holds the previous call's tile states and counters: reset the part this call
-    // uses to the all-ones pattern (tile states unset, counters one step before 0, no status bit)
+    // the array still holds the previous call's tile states and ticket: reset the part this call
+    // uses to the all-ones pattern (tile states unset, ticket counter one draw before ticket 0)
     const size_t tiles = size_t((N + kScanTile - 1) / kScanTile);
     TPPO_CUDA_CHECK(cudaMemsetAsync(scratch, 0xff, kScanHeadBytes + tiles * sizeof(TileState), s));
     return egae_launch(a, gamma, lambda, s);

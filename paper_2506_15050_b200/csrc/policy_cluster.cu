@@ -14,6 +14,10 @@
 // the row is in registers), or over its slice in shared memory, from where the producer warp sends
 // it out with bulk stores.  Each logit crosses the HBM interface exactly once in each direction.
 // No multicast is used: every CTA issues plain copies of its own slice.
+//
+// Thirty-three clusters of four fill 132 of the 148 SMs.  On large row lists the host gives the
+// last rows of the list to the plain two-pass kernel, launched as a programmatic dependent of this
+// one, so that it runs on the remaining SMs at the same time (policy_loss.cu).
 #include "policy_common.cuh"
 #include "ptx.cuh"
 

@@ -114,7 +114,7 @@ int launch_policy_two_pass(const PolicyArgs& a, int dtype, cudaStream_t s, int v
 int launch_policy_cluster(const PolicyArgs& a, cudaStream_t s, int variant, int* idle_sms);
 bool policy_cluster_supported(const PolicyArgs& a, int dtype);
 
-constexpr int kSideShare256 = 18;       // about 7 % of the rows
+constexpr int kSideShare256 = 22;       // 8.6 % of the rows: both launches then end together at V = 152064
 constexpr int64_t kSideMinRows = 2048;  // below this the split is not worth a second launch
 
 size_t policy_workspace_bytes(int64_t R, int64_t n_max) {

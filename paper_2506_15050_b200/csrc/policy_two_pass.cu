@@ -21,6 +21,24 @@ __device__ __forceinline__ void store_elem(uint16_t* p, float v) {
 }
 __device__ __forceinline__ void store_elem(float* p, float v) { *p = v; }
 
+// The same in two steps, so that several loads can be issued before the first is used.
+template <typename T> struct RawUnit;
+template <> struct RawUnit<uint16_t> { uint4 w; };
+template <> struct RawUnit<float> { float4 a, b; };
+__device__ __forceinline__ RawUnit<uint16_t> load_raw(const uint16_t* p) {
+    return RawUnit<uint16_t>{*reinterpret_cast<const uint4*>(p)};
+}
+__device__ __forceinline__ RawUnit<float> load_raw(const float* p) {
+    return RawUnit<float>{*reinterpret_cast<const float4*>(p), *reinterpret_cast<const float4*>(p + 4)};
+}
+__device__ __forceinline__ void widen8(const RawUnit<uint16_t>& r, float (&x)[8]) {
+    x[0] = bf16_lo(r.w.x); x[1] = bf16_hi(r.w.x); x[2] = bf16_lo(r.w.y); x[3] = bf16_hi(r.w.y);
+    x[4] = bf16_lo(r.w.z); x[5] = bf16_hi(r.w.z); x[6] = bf16_lo(r.w.w); x[7] = bf16_hi(r.w.w);
+}
+__device__ __forceinline__ void widen8(const RawUnit<float>& r, float (&x)[8]) {
+    x[0] = r.a.x; x[1] = r.a.y; x[2] = r.a.z; x[3] = r.a.w; x[4] = r.b.x; x[5] = r.b.y; x[6] = r.b.z; x[7] = r.b.w;
+}
+
 // 8 consecutive elements from a 16-byte aligned address
 __device__ __forceinline__ void load8(const uint16_t* p, float (&x)[8]) {
     const uint4 w = *reinterpret_cast<const uint4*>(p);
@@ -86,7 +104,22 @@ __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const 
             float m = -kFltMax, s = 0.f;      // most negative finite: no inf - inf on masked (-inf) logits
             if (VEC) {
                 const int nu = a.V >> 3;
-                for (int u = tid; u < nu; u += kTwoPassThreads) {
+                // four independent 16-byte loads per thread and trip: a single load in flight per
+                // thread leaves the sweep bound by memory latency
+                constexpr int kDeep = 4;
+                int u = tid;
+                for (; u + (kDeep - 1) * kTwoPassThreads < nu; u += kDeep * kTwoPassThreads) {
+                    RawUnit<T> raw[kDeep];
+#pragma unroll
+                    for (int d = 0; d < kDeep; ++d) raw[d] = load_raw(x_row + (int64_t(u + d * kTwoPassThreads) << 3));
+#pragma unroll
+                    for (int d = 0; d < kDeep; ++d) {
+                        float x[8];
+                        widen8(raw[d], x);
+                        online_update<8>(m, s, x);
+                    }
+                }
+                for (; u < nu; u += kTwoPassThreads) {
                     float x[8];
                     load8(x_row + (int64_t(u) << 3), x);
                     online_update<8>(m, s, x);
@@ -155,7 +188,27 @@ __global__ void __launch_bounds__(kTwoPassThreads) policy_two_pass_kernel(const 
             } else if (VEC) {
                 const int nu = a.V >> 3;
                 const int yu = rec.y >> 3, yk = rec.y & 7;
-                for (int u = tid; u < nu; u += kTwoPassThreads) {
+                constexpr int kDeep = 4;
+                int u = tid;
+                for (; u + (kDeep - 1) * kTwoPassThreads < nu; u += kDeep * kTwoPassThreads) {
+                    RawUnit<T> raw[kDeep];
+#pragma unroll
+                    for (int d = 0; d < kDeep; ++d) raw[d] = load_raw(x_row + (int64_t(u + d * kTwoPassThreads) << 3));
+#pragma unroll
+                    for (int d = 0; d < kDeep; ++d) {
+                        const int ud = u + d * kTwoPassThreads;
+                        float x[8], g[8];
+                        widen8(raw[d], x);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) g[k] = coef * ex2(fmaf(x[k] - row_max, kLog2e, -off));
+                        if (ud == yu) {
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) if (k == yk) g[k] -= coef;
+                        }
+                        store8(g_row + (int64_t(ud) << 3), g);
+                    }
+                }
+                for (; u < nu; u += kTwoPassThreads) {
                     float x[8], g[8];
                     load8(x_row + (int64_t(u) << 3), x);
 #pragma unroll

@@ -12,6 +12,14 @@ constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kSelItems = 32;                                  // positions per thread
 constexpr int kSelTile = kSelThreads * kSelItems;              // 8192 positions per tile
 constexpr uint32_t kSelSpinLimit = 1u << 22;
+// Tile order.  0 (default): block b takes tile b; thread blocks are dispatched in index order, so the
+// tiles a tile waits for (smaller indices) are running or done, and should that ever not hold the
+// bounded wait gives up with TPPO_DEV_WAIT_TIMEOUT instead of hanging.  1: tiles are drawn from an
+// atomic ticket counter, which needs no assumption about dispatch order (measured 6 us slower at
+// 17.5 M positions: an L2 round trip at the head of every tile's chain of latencies).
+#ifndef TPPO_SEL_TICKET
+#define TPPO_SEL_TICKET 0
+#endif
 
 // tile state word: [63:62] flag (1 = tile total, 2 = inclusive prefix), [61:31] policy count,
 // [30:0] value count.  One 64-bit store publishes flag and payload together.
@@ -72,12 +80,7 @@ struct SelectArgs {
     int32_t* value_idx;
     int32_t* counts;            // [4]
     unsigned long long* state;  // [num_tiles]
-    // head of the workspace, cleared to zero together with the tile states: the ticket counter, the
-    // finished-tiles counter and the status bits raised during the call (the last tile to finish
-    // writes counts[0..3])
-    uint32_t* ticket;
-    uint32_t* done;
-    uint32_t* ws_status;
+    uint32_t* ticket;           // head of the workspace, cleared to zero together with the tile states
     uint32_t spin_limit;        // polls a look-back round may take before it gives up
     int32_t no_publish;         // test hook: tiles keep their totals to themselves
     int32_t out_vec_ok;         // policy_idx and value_idx are 16-byte aligned
@@ -146,8 +149,12 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     int bad = 0;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // Tiles are handed out in launch order, so every tile this one waits for is already running.
+    // A tile only waits for tiles with smaller indices.
+#if TPPO_SEL_TICKET
     if (threadIdx.x == 0) s_tile = atomicAdd(a.ticket, 1u);
+#else
+    if (threadIdx.x == 0) s_tile = blockIdx.x;
+#endif
     __syncthreads();
     const uint32_t tile = s_tile;
     if (tile >= uint32_t(a.num_tiles)) return;
@@ -264,7 +271,7 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     if (threadIdx.x == 0 && tile > 0 && !a.no_publish)
         reinterpret_cast<volatile unsigned long long*>(a.state)[tile] =
             sel_pack(1, tile_tot & 0xffffu, tile_tot >> 16);
-    if (bad) { atomicOr(a.ws_status, uint32_t(bad)); __threadfence(); }
+    if (bad) atomicOr(a.counts + 2, bad);
     // compact inside the tile (needs no global offset; earlier tiles finish meanwhile)
     {
         uint32_t op = before & 0xffffu, ov = before >> 16;
@@ -300,13 +307,16 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
             if (m2) break;
         }
         if (lane == 0) {
-            if (timed_out) { atomicOr(a.ws_status, uint32_t(TPPO_DEV_WAIT_TIMEOUT)); __threadfence(); }
-            // (the last tile's inclusive prefix is the pair of totals: it is always stored)
-            if (!a.no_publish || tile == uint32_t(a.num_tiles) - 1) st[tile] = sel_pack(2, ep + tp, ev + tv);
+            if (timed_out) atomicOr(a.counts + 2, TPPO_DEV_WAIT_TIMEOUT);
+            if (!a.no_publish) st[tile] = sel_pack(2, ep + tp, ev + tv);
             s_base_pol = ep;
             s_base_val = ev;
             s_tot_pol = tp;
             s_tot_val = tv;
+            if (tile == uint32_t(a.num_tiles) - 1) {
+                a.counts[0] = int32_t(ep + tp);
+                a.counts[1] = int32_t(ev + tv);
+            }
         }
     }
     __syncthreads();
@@ -314,20 +324,6 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     // ---- copy the tile's two lists out, coalesced ----------------------------------------------
     sel_copy_out(a.policy_idx, s_base_pol, int(s_tot_pol), s_out_pol, int32_t(t0), a.out_vec_ok != 0);
     sel_copy_out(a.value_idx, s_base_val, int(s_tot_val), s_out_val, int32_t(t0), a.out_vec_ok != 0);
-
-    // ---- the last tile to finish writes the counts and the status bits -------------------------------
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        if (atomicAdd(a.done, 1u) == uint32_t(a.num_tiles) - 1u) {
-            __threadfence();
-            const uint64_t last = reinterpret_cast<volatile unsigned long long*>(a.state)[a.num_tiles - 1];
-            a.counts[0] = int32_t(sel_pol(last));
-            a.counts[1] = int32_t(sel_val(last));
-            a.counts[2] = int32_t(*reinterpret_cast<volatile uint32_t*>(a.ws_status));
-            a.counts[3] = 0;
-        }
-    }
 }
 
 size_t select_workspace_bytes(int64_t N) {
@@ -358,11 +354,10 @@ TPPO_API int tppo_select_tokens(const int32_t* seq_begin, const int32_t* prompt_
     if (!workspace || workspace_bytes < need || !aligned(workspace, kWsAlign))
         return TPPO_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (N == 0 || B == 0) {
-        TPPO_CUDA_CHECK(cudaMemsetAsync(counts, 0, 4 * sizeof(int32_t), s));
-        return TPPO_OK;
-    }
-    // one clear (tile states, the two counters, the status bits); the kernel writes all of counts
+    TPPO_CUDA_CHECK(cudaMemsetAsync(counts, 0, 4 * sizeof(int32_t), s));
+    if (N == 0 || B == 0) return TPPO_OK;
+    // (Handing the counts and status bits over by the last tile to finish, to save the 16-byte clear
+    // above, was measured: the fence and counter at the end of every tile cost 6 us at 17.5 M tokens.)
     TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0, need, s));
     SelectArgs a;
     a.seq_begin = seq_begin; a.prompt_len = prompt_len; a.prev_len = prev_len; a.new_len = new_len;
@@ -376,8 +371,6 @@ TPPO_API int tppo_select_tokens(const int32_t* seq_begin, const int32_t* prompt_
     a.num_tiles = int32_t((N + kSelTile - 1) / kSelTile);
     a.policy_idx = policy_idx; a.value_idx = value_idx; a.counts = counts;
     a.ticket = static_cast<uint32_t*>(workspace);
-    a.done = a.ticket + 1;
-    a.ws_status = a.ticket + 2;
     a.state = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWsAlign);
     select_tokens_kernel<<<a.num_tiles, kSelThreads, 0, s>>>(a);
     TPPO_CUDA_CHECK(cudaGetLastError());
