@@ -41,9 +41,13 @@ from paper_2506_15050_b200 import synth  # noqa: E402
 METRIC = "selected tokens/s, fused logprob+PPO loss fwd+bwd, V=152064 bf16; % HBM peak"
 UNIT = "selected tokens/s"
 ALGO_BYTES_PER_TOKEN = 2 * 2 * synth.V_QWEN       # bf16 row read once + bf16 gradient row written once
-# dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the sweep kernel at 2048 rows
-# (1194.38 MB; the full workload is too large to capture), per row; traffic is proportional to rows.
-NCU_TRAFFIC_BYTES_PER_TOKEN = 1194.38e6 / 2048
+# dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture at 2048 rows (the full workload is too
+# large to capture) of the two kernels that share the rows of a policy-loss call: policy_cluster_kernel
+# 569.41 + 517.59 MB on 1872 rows, policy_two_pass_kernel (side launch) 53.58 + 12.89 MB on 176 rows;
+# per row, scaled by rows.  (Reads are exactly one pass over the logits; of the writes about 90 MB were
+# still in L2 when the capture ended, at any row count, so the scaled figure understates full-size
+# writes by about 7 %.)  profiles/policy_cluster_kernel_cfg3.md has the command.
+NCU_TRAFFIC_BYTES_PER_TOKEN = (569.413376e6 + 517.587200e6 + 53.582080e6 + 12.886528e6) / 2048
 
 
 def measured_peaks():
@@ -65,15 +69,55 @@ def measured_tensor_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons while the timed region runs: NVML from a thread every
+    2 ms (read-only queries), or `nvidia-smi -lms` when the NVML binding is not importable.  A timed
+    region of a few tens of milliseconds still gets its samples this way."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index: int):
         self.index, self.rows, self.proc = index, [], None
+        self.sm, self.reasons, self.sm_max = [], set(), None
+        self.stop_flag, self.thread, self.nvml = threading.Event(), None, None
+
+    def _nvml_loop(self):
+        n, h = self.nvml
+        bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+                "sw_power_cap": 0x4}
+        get_reasons = getattr(n, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            getattr(n, "nvmlDeviceGetCurrentClocksThrottleReasons")
+        while not self.stop_flag.is_set():
+            try:
+                self.sm.append(float(n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM)))
+                r = int(get_reasons(h))
+                for name, bit in bits.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
 
     def start(self):
+        try:
+            import pynvml as n
+            n.nvmlInit()
+            # torch's device index is an index into CUDA_VISIBLE_DEVICES
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = self.index
+            if vis:
+                ent = vis.split(",")[self.index].strip()
+                phys = int(ent) if ent.isdigit() else None
+            h = n.nvmlDeviceGetHandleByIndex(phys) if phys is not None else \
+                n.nvmlDeviceGetHandleByUUID(ent.encode())
+            self.sm_max = float(n.nvmlDeviceGetMaxClockInfo(h, n.NVML_CLOCK_SM))
+            self.nvml = (n, h)
+            self.thread = threading.Thread(target=self._nvml_loop, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
@@ -88,24 +132,28 @@ class ClockSampler:
             self.rows.append([x.strip() for x in line.split(",")])
 
     def stop(self):
+        if self.nvml is not None:
+            self.stop_flag.set()
+            self.thread.join(timeout=1.0)
+            return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.sm_max,
+                    "reasons": sorted(self.reasons), "samples": len(self.sm), "source": "nvml, every 2 ms"}
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.15)
         self.proc.terminate()
         sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows:
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
             except (ValueError, IndexError):
                 continue
-            for name, v in zip(names, r[2:6]):
+            for name, v in zip(self.NAMES, r[2:6]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None,
                 "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "source": "nvidia-smi -lms 100"}
 
 
 def spawn_ranks(n_gpus: int) -> int:
@@ -227,17 +275,25 @@ class Step:
                                self.vstats, self.ws_val)
 
     def run(self, events=None):
+        """One step.  With `events` (a list), five CUDA events are recorded around the four calls and
+        appended as one tuple: the calls' device times come out of the same run that is timed."""
+        if events is None:
+            self.egae()
+            self.select()
+            self.policy()
+            self.value()
+            return
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        ev[0].record()
         self.egae()
+        ev[1].record()
         self.select()
-        if events is not None:
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            self.policy()
-            e1.record()
-            events.append((e0, e1))
-        else:
-            self.policy()
+        ev[2].record()
+        self.policy()
+        ev[3].record()
         self.value()
+        ev[4].record()
+        events.append(tuple(ev))
 
     KERNELS_PER_STEP = 6   # egae scan, select, policy prepare + sweep + finish, value loss
 
@@ -477,7 +533,7 @@ def main():
     ap.add_argument("--hint", type=int, default=0, help="kernel_hint passed to the policy loss")
     ap.add_argument("--rows", type=int, default=16384,
                     help="rows of the loss micro-batch (smaller only for profiler captures)")
-    ap.add_argument("--workload", default="cfg3", choices=["cfg3", "lmhead", "cfg4", "stub"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg3", "lmhead", "cfg4", "configs", "stub"])
     ap.add_argument("--lmhead-calls", type=int, default=5)
     ap.add_argument("--lm-shards", type=int, default=1,
                     help="with --workload lmhead: also time one rank of this many vocabulary shards")
@@ -488,6 +544,8 @@ def main():
     ap.add_argument("--no-small", action="store_true", help="skip the config-4 small-kernel measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--graph-steps", type=int, default=50,
+                    help="steps of the extra measurement that replays the step as one CUDA graph (0: skip)")
     args = ap.parse_args()
 
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
@@ -512,6 +570,9 @@ def main():
         return
     if args.workload == "cfg4":
         run_cfg4_workload(args, rank, world, local, dev, warmup)
+        return
+    if args.workload == "configs":
+        run_config_table(args, dev)
         return
     st = Step(dev, seed=2 + rank, rows=args.rows)      # every rank holds its own batch
     st.hint = args.hint
@@ -555,12 +616,41 @@ def main():
     n_val = int(st.counts[1].item())
     assert n_tok == st.n and int(st.stats[3].item()) == 0 and int(st.status.item()) == 0
     value = world * n_tok / (ms_step * 1e-3)
-    pol = time_stats([a.elapsed_time(b) for a, b in events])
+    pol = time_stats([e[2].elapsed_time(e[3]) for e in events])
+    calls_us = {name: time_stats([e[k].elapsed_time(e[k + 1]) * 1e3 for e in events])
+                for k, name in enumerate(("egae", "select", "policy", "value"))}
     pol_ms = pol["mean"]
     peak, peak_kind = measured_peaks()
     algo_bytes = n_tok * ALGO_BYTES_PER_TOKEN
     achieved = algo_bytes / (pol_ms * 1e-3) / 1e9
     traffic = n_tok * NCU_TRAFFIC_BYTES_PER_TOKEN if (st.V == synth.V_QWEN and NCU_TRAFFIC_BYTES_PER_TOKEN) else None
+
+    # ---- the same step captured once into a CUDA graph and replayed: what the launch gaps between
+    #      the step's fourteen stream operations cost (reported beside the headline, not as it) ------
+    graph = None
+    if args.graph_steps > 0:
+        try:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                st.run()
+            for _ in range(3):
+                g.replay()
+            barrier()
+            gm = [torch.cuda.Event(enable_timing=True)]
+            gm[0].record()
+            for _ in range(args.graph_steps):
+                g.replay()
+                gm.append(torch.cuda.Event(enable_timing=True))
+                gm[-1].record()
+            barrier()
+            gs = time_stats([a.elapsed_time(b) for a, b in zip(gm[:-1], gm[1:])])
+            assert int(st.counts[0].item()) == n_tok and int(st.stats[3].item()) == 0
+            graph = {"ms_per_step": gs, "value_at_mean": world * n_tok / (gs["mean"] * 1e-3),
+                     "steps": args.graph_steps}
+            del g
+        except Exception as e:      # capture is an extra: the headline above does not depend on it
+            graph = {"error": repr(e)[:200]}
+            torch.cuda.synchronize()
 
     # ---- end to end: host buffers in, losses out, copies inside the timed region ---------------
     e2e = None
@@ -657,6 +747,7 @@ def main():
             "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
             "config": workload_config(st.N, st.n, n_val, args.hint),
+            "step_calls_us": calls_us, "cuda_graph_replay": graph,
             "roofline": roofline,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": Step.KERNELS_PER_STEP * args.steps,
             "clocks": clocks, "small_kernels": small_kernels, "lmhead_variant": lmhead}))
@@ -967,6 +1058,123 @@ def measure_cfg4(dev, steps, warmup):
             "advance": {"freed": int(an[0]), "context_tokens": int(an[2])},
             "timing": "CUDA events around each C-ABI call (its memset and kernels)",
             "kernels": kernels, "clocks": clocks}
+
+
+def _time_call(f, reps, warm=3):
+    """Mean / median / min device time of one call (ms), CUDA events around every repetition."""
+    for _ in range(warm):
+        f()
+    torch.cuda.synchronize()
+    ev = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); f(); e1.record()
+        ev.append((e0, e1))
+    torch.cuda.synchronize()
+    return time_stats([a.elapsed_time(b_) for a, b_ in ev])
+
+
+def run_config_table(args, dev):
+    """The benchmark configurations that are not the bench line, one after another (configs 1, 2 and
+    4; config 3 is the default workload, config 5 `--workload lmhead`): GPU time of the hot path on
+    each, and the oracle on the host cores on the whole of the small ones and a bounded sample of
+    the large one.  Prints one JSON object; fills the per-config table of the benchmark spec."""
+    import oracle
+    from paper_2506_15050_b200 import binding as b
+    f32 = lambda x: float(np.float32(x))
+    t = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).to(dev)
+    out = {"cores": oracle.num_threads()}
+
+    def path(c, logits, rows_sel, mode):
+        """Device buffers and one closure that runs EGAE, selection, policy loss, value loss."""
+        N, B, V = c["N"], c["B"], c["V"]
+        r, v, ov = t(c["rewards"], torch.float32), t(c["values"], torch.float32), t(c["old_values"], torch.float32)
+        sb, se, tr = t(c["seg_begin"], torch.int32), t(c["seg_end"], torch.int32), t(c["truncated"], torch.uint8)
+        sq = t(c["seq_begin"], torch.int32)
+        pl, pv, nl = (t(c[k], torch.int32) for k in ("prompt_len", "prev_len", "new_len"))
+        tg = t(c["targets"], torch.int32)
+        adv, ret = torch.zeros(N, device=dev), torch.zeros(N, device=dev)
+        pol, val = torch.zeros(N, dtype=torch.int32, device=dev), torch.zeros(N, dtype=torch.int32, device=dev)
+        cnt, st = torch.zeros(4, dtype=torch.int32, device=dev), torch.zeros(1, dtype=torch.int32, device=dev)
+        logp, loss, vloss = torch.zeros(N, device=dev), torch.zeros(1, device=dev), torch.zeros(1, device=dev)
+        stats, vstats = torch.zeros(4, dtype=torch.int32, device=dev), torch.zeros(2, dtype=torch.int32, device=dev)
+        old = torch.zeros(N, device=dev)
+        dl = torch.empty_like(logits) if mode == b.DLOGITS_FULL else torch.empty((rows_sel, V), dtype=logits.dtype, device=dev)
+        dv = torch.zeros(N, device=dev)
+        w1, w2 = b.workspace(b.OP_EGAE, N, B, 0, 0, dev), b.workspace(b.OP_SELECT_TOKENS, N, B, 0, 0, dev)
+        w3, w4 = b.workspace(b.OP_POLICY_LOSS, N, 0, N, V, dev), b.workspace(b.OP_VALUE_LOSS, N, 0, N, 0, dev)
+
+        def small():
+            b.tppo_egae(r, v, sb, se, tr, None, c["gamma"], c["lam"], adv, ret, st, w1)
+            b.tppo_select_tokens(sq, pl, pv, nl, tr, 0, None, None, N, pol, val, cnt, w2)
+
+        def policy():
+            b.tppo_policy_loss_fwd_bwd(logits, tg, pol[:rows_sel], cnt[0:1], rows_sel, None, old, adv,
+                                       c["eps_low"], c["eps_high"], 0.0, logp, None, loss, stats, dl, mode, w3)
+
+        def value():
+            b.tppo_value_loss(v, ov, ret, val, cnt[1:2], N, c["xi_low"], c["xi_high"], 0.0, vloss, dv, vstats, w4)
+
+        small()
+        b.tppo_policy_loss_fwd_bwd(logits, tg, pol, cnt[0:1], N, None, old, adv, 0.2, 0.2, 0.0, logp, None, loss,
+                                   stats, None, b.DLOGITS_NONE, w3)       # old-policy log-probs
+        torch.cuda.synchronize()
+        idx = pol[:int(cnt[0])].long()
+        old[idx] = logp[:len(idx)] + t(c["old_logp_noise"], torch.float32)[idx]
+        return small, policy, value, cnt, stats
+
+    # ---- config 1 -----------------------------------------------------------------------------------
+    c1 = synth.config1()
+    small, policy, value, cnt, stats = path(c1, t(c1["logits"], torch.float32), 170, b.DLOGITS_COMPACT)
+    step = lambda: (small(), policy(), value())
+    g = _time_call(step, 200)
+    w0 = time.perf_counter()
+    for _ in range(20):
+        a_, r_ = oracle.egae(c1["rewards"], c1["values"], c1["seg_begin"], c1["seg_end"], c1["truncated"], None, 1.0, f32(0.95))
+        p_, v_ = oracle.select_tokens(c1["seq_begin"], c1["prompt_len"], c1["prev_len"], c1["new_len"], c1["truncated"])
+        oracle.policy_loss(c1["logits"], c1["targets"], p_, None, np.zeros(c1["N"], np.float32), a_.astype(np.float32), f32(0.2), f32(0.2))
+        oracle.value_loss(c1["values"], c1["old_values"], r_.astype(np.float32), v_, f32(0.5), f32(0.6))
+    o = (time.perf_counter() - w0) / 20
+    out["cfg1"] = {"n_selected": int(cnt[0]), "gpu_step_us": {k: v * 1e3 for k, v in g.items()},
+                   "oracle_step_ms": o * 1e3, "note": "whole path, V=1000 fp32; latency-bound (13 launches)"}
+    # ---- config 2 -----------------------------------------------------------------------------------
+    c2 = synth.config2(dev)
+    res2 = {}
+    for name, mode in (("compact", b.DLOGITS_COMPACT), ("full_zero_filled", b.DLOGITS_FULL)):
+        small, policy, value, cnt, stats = path(c2, c2["logits"], 4096, mode)
+        g = _time_call(policy, 30)
+        n = int(cnt[0])
+        algo = n * ALGO_BYTES_PER_TOKEN + (0 if mode == b.DLOGITS_COMPACT else (c2["N"] - n) * 2 * c2["V"])
+        res2[name] = {"policy_call_ms": g, "algorithmic_bytes": algo, "GB/s": algo / (g["mean"] * 1e-3) / 1e9,
+                      "selected_tokens_per_s": n / (g["mean"] * 1e-3)}
+        assert n == 4096 and int(stats[3]) == 0
+        del small, policy, value
+        torch.cuda.empty_cache()
+    rows = 256
+    host = synth.bf16_bits(c2["logits"][:rows])
+    w0 = time.perf_counter()
+    oracle.policy_loss(host, c2["targets"], np.arange(rows, dtype=np.int32), None, np.zeros(c2["N"], np.float32),
+                       np.ones(c2["N"], np.float32), f32(0.2), f32(0.2), 4096.0)
+    o = time.perf_counter() - w0
+    out["cfg2"] = {"n_selected": 4096, "gpu": res2,
+                   "oracle": {"sample_rows": rows, "seconds": o, "selected_tokens_per_s": rows / o,
+                              "scaled_to_4096_rows_s": o * 4096 / rows}}
+    del c2
+    torch.cuda.empty_cache()
+    # ---- config 4 -----------------------------------------------------------------------------------
+    m = measure_cfg4(dev, 30, 3)
+    c4 = synth.config4()
+    w0 = time.perf_counter()
+    oracle.egae(c4["rewards"], c4["values"], c4["seg_begin"], c4["seg_end"], c4["truncated"], c4["bootstrap"], 1.0, f32(0.95))
+    w1 = time.perf_counter()
+    oracle.select_tokens(c4["seq_begin"], c4["prompt_len"], c4["prev_len"], c4["new_len"], c4["truncated"], 0,
+                         c4["extra_policy_mask"], c4["extra_value_mask"])
+    w2 = time.perf_counter()
+    out["cfg4"] = {"tokens": c4["N"], "gpu_us": {k: v["us"] for k, v in m["kernels"].items()},
+                   "gpu_frac_of_measured_hbm": {k: v["frac"] for k, v in m["kernels"].items()},
+                   "oracle_egae_s": w1 - w0, "oracle_select_s": w2 - w1,
+                   "oracle_egae_tokens_per_s": c4["N"] / (w1 - w0), "oracle_select_tokens_per_s": c4["N"] / (w2 - w1)}
+    print(json.dumps(out))
 
 
 def run_cfg4_workload(args, rank, world, local, dev, warmup):

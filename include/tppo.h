@@ -283,12 +283,7 @@ enum {
  *     l  = 1/2 * max((values[p]-returns[p])^2, (Vc-returns[p])^2),   loss = (1/denom) sum l
  *     dvalues[p] = (values[p]-returns[p])/denom  if the unclipped term is the max (ties included),
  *                  else (Vc-returns[p])/denom if Vc == values[p], else 0
- *   values, old_values, returns [N] fp32
- *   value_idx [n_max] int32 or NULL for 0..n_max-1.  With dvalues the list must be strictly ascending
- *             with entries in [0, N), the order tppo_select_tokens writes (the kernel then sweeps
- *             the positions in order and writes every entry of dvalues itself); every adjacent pair
- *             is checked, and a list that is not ascending raises TPPO_DEV_BAD_INDEX and leaves loss
- *             and dvalues unspecified (finite, in bounds).  Without dvalues any distinct entries do.
+ *   values, old_values, returns [N] fp32; value_idx [n_max] int32 (distinct) or NULL for 0..n_max-1
  *   loss [1] fp32 out; dvalues [N] fp32 out (zero off the value tokens) or NULL
  *   stats [2] int32 out: n, status bits
  * A value token whose value, old value or return is a NaN or an infinity contributes nothing (loss
@@ -407,9 +402,12 @@ int tppo_lmhead_shard_fwd_bwd(const void *hidden, const void *weight_shard,
  *   slot_source  [B] int32 out
  *   counts       [4] int32 out: freed slots, refilled slots, context tokens of the next step, device
  *                status bits (TPPO_DEV_OVERFLOW when the context exceeds `capacity` or 2^31-1: the
- *                excess is not written; TPPO_DEV_BAD_INDEX for negative lengths or reads outside
- *                `tokens` / `queue_tokens`, which are skipped)
- * No workspace.  Bit-exact and run-to-run identical.
+ *                excess is not written; TPPO_DEV_BAD_INDEX for negative lengths and for a slot whose
+ *                source range does not lie inside `tokens` / `queue_tokens`: its context is then
+ *                written as zeros, nothing outside the arrays is read)
+ * No workspace and no clear beforehand: the slot walk writes all four counts itself, and the copy
+ * kernel is launched as its programmatic dependent (scheduled while the walk still runs, reading its
+ * results only after it has finished).  Bit-exact and run-to-run identical.
  */
 int tppo_advance_batch(const int32_t *seq_begin, const int32_t *prompt_len,
                        const int32_t *prev_len, const int32_t *new_len,

@@ -37,12 +37,23 @@
 
 namespace tppo {
 
-constexpr int kScanThreads = 128;     // (256-thread tiles of 4096 positions measured 5 % slower)
+#ifndef TPPO_SCAN_ITEMS
+#define TPPO_SCAN_ITEMS 16
+#endif
+constexpr int kScanItems = TPPO_SCAN_ITEMS;           // consecutive positions per thread (its run): 16 or 32
+constexpr int kScanTile = 2048;                       // positions per tile (4096 measured 5 % slower)
+constexpr int kScanThreads = kScanTile / kScanItems;
 constexpr int kScanWarps = kScanThreads / 32;
-constexpr int kScanItems = 16;
-constexpr int kScanTile = kScanThreads * kScanItems;  // 2048 positions
+constexpr int kScanChunks = kScanItems / 4;           // 16-byte chunks of a run
+constexpr int kThreadsPerRow = 32 / kScanItems;       // a row of the tile image holds 32 positions
+constexpr uint32_t kRunMask = kScanItems == 32 ? 0xffffffffu : ((1u << (kScanItems & 31)) - 1u);
+static_assert(kScanItems == 8 || kScanItems == 16 || kScanItems == 32, "a run is a quarter, half or whole row");
+__device__ __forceinline__ uint32_t bits_below(int k) { return k >= 32 ? 0xffffffffu : ((1u << k) - 1u); }
 constexpr int kSegCap = 32;                           // segments of one tile kept in shared memory
-constexpr int kScanCtasPerSm = 1024 / kScanThreads;
+#ifndef TPPO_SCAN_CTAS
+#define TPPO_SCAN_CTAS (TPPO_SCAN_ITEMS == 16 ? 8 : (TPPO_SCAN_ITEMS == 8 ? 4 : 12))
+#endif
+constexpr int kScanCtasPerSm = TPPO_SCAN_CTAS;   // registers resp. shared memory allow no more
 constexpr int kScanBoxRows = 64;                      // rows of 32 positions per TMA box
 constexpr int kScanBoxes = kScanTile / (kScanBoxRows * 32);
 static_assert(kScanTile % (kScanBoxRows * 32) == 0, "a tile is a whole number of TMA boxes");
@@ -359,7 +370,7 @@ struct RunState {
     // a segment (bits 0-15), which of them continue into the next position (bits 16-31), and for the
     // one last token, its position (or -1) and the value its TD residual bootstraps from
     bool masked;
-    uint32_t bits;
+    uint32_t inside, cont;
     int k_last;
     float v_boundary;
     bool boundary_own;   // the boundary value is the last token's own value (no bootstrap array)
@@ -378,8 +389,8 @@ __device__ __forceinline__ Affine2 egae_run_map_once(const EgaeArgs& a, const Ti
     const bool win_smem = win_n <= kSegCap;
     const int l0 = tid * kScanItems;        // first position of this thread inside the tile
     // its four chunks: row tid/2, chunks 4*(tid&1) + q, stored at chunk ^ (row & 7)
-    const int row_base = (tid >> 1) << 5;
-    const int chunk0 = (tid & 1) << 2, swz = (tid >> 1) & 7;
+    const int row_base = (tid / kThreadsPerRow) << 5;
+    const int chunk0 = (tid % kThreadsPerRow) * kScanChunks, swz = (tid / kThreadsPerRow) & 7;
     const int l_last = min(l0 + kScanItems, n_tile) - 1;
     int i_start = -1;
     if (l_last >= l0) {
@@ -425,7 +436,7 @@ __device__ __forceinline__ Affine2 egae_run_map_once(const EgaeArgs& a, const Ti
             if (e <= p0 && e > b) break;      // ascending and disjoint: the earlier ones end earlier still
             const int lo = int(max(b, p0) - p0), hi = int(min(e, p0 + kScanItems) - p0);
             if (hi <= lo) continue;
-            const uint32_t m = ((1u << hi) - 1u) & ~((1u << lo) - 1u);
+            const uint32_t m = bits_below(hi) & ~bits_below(lo);
             inside |= m;
             cont |= m;
             if (e <= p0 + kScanItems) {       // the segment's last token lies in the run
@@ -441,15 +452,16 @@ __device__ __forceinline__ Affine2 egae_run_map_once(const EgaeArgs& a, const Ti
                 }
             }
         }
-        rs.bits = inside | (cont << 16);
+        rs.inside = inside;
+        rs.cont = cont;
         rs.masked = n_last <= 1;
     }
     if (rs.masked) {
-        const uint32_t inside = rs.bits & 0xffffu, cont = rs.bits >> 16;
+        const uint32_t inside = rs.inside, cont = rs.cont;
         double bG = 0.0, bR = 0.0;
         float vn = v_right;
 #pragma unroll
-        for (int q = kScanItems / 4 - 1; q >= 0; --q) {
+        for (int q = kScanChunks - 1; q >= 0; --q) {
             const int s = row_base + (((chunk0 + q) ^ swz) << 2);
             const float4 r4 = *reinterpret_cast<const float4*>(buf.r + s);
             const float4 v4 = *reinterpret_cast<const float4*>(buf.v + s);
@@ -471,7 +483,7 @@ __device__ __forceinline__ Affine2 egae_run_map_once(const EgaeArgs& a, const Ti
             }
         }
         probe = probe0;
-        const bool whole = cont == 0xffffu;
+        const bool whole = cont == kRunMask;
         return Affine2{whole ? a.gl_run : 0.0, double(bG), whole ? a.gamma_run : 0.0, double(bR)};
     }
     if (fast) {
@@ -479,7 +491,7 @@ __device__ __forceinline__ Affine2 egae_run_map_once(const EgaeArgs& a, const Ti
         double bG = 0.0, bR = 0.0;
         float vn = v_right;
 #pragma unroll
-        for (int q = kScanItems / 4 - 1; q >= 0; --q) {
+        for (int q = kScanChunks - 1; q >= 0; --q) {
             const int s = row_base + (((chunk0 + q) ^ swz) << 2);
             const float4 r4 = *reinterpret_cast<const float4*>(buf.r + s);
             const float4 v4 = *reinterpret_cast<const float4*>(buf.v + s);
@@ -535,7 +547,7 @@ __device__ __forceinline__ Affine2 egae_run_map(const EgaeArgs& a, TileBuf& buf,
         float probe = 0.f;
         f = egae_run_map_once(a, buf, win, t0, n_tile, tid, rs, bad, probe, nonfinite);
         if (probe == probe) break;
-        const uint32_t inside = rs.fast ? 0xffffu : (rs.bits & 0xffffu);
+        const uint32_t inside = rs.fast ? kRunMask : rs.inside;
 #pragma unroll 1
         for (int k = 0; k < kScanItems; ++k) {
             const int sl = pos_slot(tid * kScanItems + k);
@@ -577,11 +589,11 @@ __device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, TileBuf& buf,
                                                 float R, bool in_place, bool& bad, bool& nonfinite) {
     const int l0 = tid * kScanItems;
     if (rs.fast) {
-        const int row_base = (tid >> 1) << 5;
-        const int chunk0 = (tid & 1) << 2, swz = (tid >> 1) & 7;
+        const int row_base = (tid / kThreadsPerRow) << 5;
+        const int chunk0 = (tid % kThreadsPerRow) * kScanChunks, swz = (tid / kThreadsPerRow) & 7;
         float vn = rs.v_right;
 #pragma unroll
-        for (int q = kScanItems / 4 - 1; q >= 0; --q) {
+        for (int q = kScanChunks - 1; q >= 0; --q) {
             const int s = row_base + (((chunk0 + q) ^ swz) << 2);
             const float4 r4 = *reinterpret_cast<const float4*>(buf.r + s);
             const float4 v4 = *reinterpret_cast<const float4*>(buf.v + s);
@@ -602,12 +614,12 @@ __device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, TileBuf& buf,
         return;
     }
     if (rs.masked) {
-        const int row_base = (tid >> 1) << 5;
-        const int chunk0 = (tid & 1) << 2, swz = (tid >> 1) & 7;
-        const uint32_t inside = rs.bits & 0xffffu, cont = rs.bits >> 16;
+        const int row_base = (tid / kThreadsPerRow) << 5;
+        const int chunk0 = (tid % kThreadsPerRow) * kScanChunks, swz = (tid / kThreadsPerRow) & 7;
+        const uint32_t inside = rs.inside, cont = rs.cont;
         float vn = rs.v_right;
 #pragma unroll
-        for (int q = kScanItems / 4 - 1; q >= 0; --q) {
+        for (int q = kScanChunks - 1; q >= 0; --q) {
             const int s = row_base + (((chunk0 + q) ^ swz) << 2);
             const float4 r4 = *reinterpret_cast<const float4*>(buf.r + s);
             const float4 v4 = *reinterpret_cast<const float4*>(buf.v + s);
@@ -782,6 +794,185 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     }
 }
 
+// ---- the same scan as a software pipeline ------------------------------------------------------------
+// In the kernel above a tile's life is a chain of latencies, and the longest link is the look-back:
+// the right-hand neighbours of a tile are worked on at the same moment, so a tile that has just
+// published its composite waits for theirs, three of its four warps idle at a barrier.  Here a CTA
+// stays resident and takes tile after tile (by ticket), two tile images in shared memory, and looks
+// back for tile k-1 only AFTER it has composed the maps of tile k: by then the neighbours'
+// composites have long been published (one round of loads, no waiting), and while warp 0 looks back
+// the other warps draw the ticket after next and search the segment window of the next tile.  The
+// copy of tile k+1 is issued as soon as the results of tile k-1 have left its buffer.
+//   iteration k:  wait copy(k) | maps(k), warp scan | publish composite(k); look-back(k-1) ||
+//                 ticket(k+2), window(k+1) | replay(k-1), store | issue copy(k+1)
+constexpr int kPipeCtasPerSm = 6;
+constexpr int kPipeRing = 4;          // ring of tile numbers / segment windows: tiles k-1, k, k+1, k+2
+constexpr uint32_t kTileBytes = 2 * kScanTile * uint32_t(sizeof(float));
+
+__global__ void __launch_bounds__(kScanThreads, kPipeCtasPerSm)
+egae_pipe_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
+                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_adv,
+                 const __grid_constant__ CUtensorMap map_ret) {
+    __shared__ TileBuf s_buf[2];
+    __shared__ TileWin s_win[kPipeRing];
+    __shared__ __align__(8) uint64_t s_full[2];      // the inputs of the tile in buffer b have arrived
+    __shared__ int s_tile[kPipeRing];                // tile taken for pipeline step k (ring), -1: none left
+    __shared__ Affine2 s_warp[kScanWarps];
+    __shared__ Affine2 s_right[2][kScanWarps];       // composite of the warps to the right of each warp
+    __shared__ Affine2 s_whole[2];                   // composite of the whole tile
+    __shared__ double s_carry[kScanWarps][2];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    bool bad = false, nonfinite = false, late = false;
+
+    auto draw = [&]() -> int {       // the next tile from the end of the arrays, or -1
+        const uint32_t t = atomicAdd(a.ticket, 1u) + 1u;      // the counter starts at all-ones
+        return t < uint32_t(a.num_tiles) ? a.num_tiles - 1 - int(t) : -1;
+    };
+    auto tile_len = [&](int tile) { return int(min(int64_t(kScanTile), int64_t(a.N) - int64_t(tile) * kScanTile)); };
+    auto issue_copy = [&](int k, int tile) {     // one thread; whole, aligned tiles only
+        if (!(a.tma_ok && tile_len(tile) == kScanTile)) return;
+        const uint32_t bar = ptx::smem_addr(&s_full[k & 1]);
+        TileBuf& buf = s_buf[k & 1];
+        ptx::mbar_arrive_expect_tx(bar, kTileBytes);
+#pragma unroll
+        for (int bx = 0; bx < kScanBoxes; ++bx) {
+            const int32_t y = tile * (kScanTile / kRowPos) + bx * kScanBoxRows;
+            umma::tma_load_2d(ptx::smem_addr(buf.r + bx * kScanBoxRows * kRowPos), &map_r, bar, 0, y);
+            umma::tma_load_2d(ptx::smem_addr(buf.v + bx * kScanBoxRows * kRowPos), &map_v, bar, 0, y);
+        }
+    };
+
+    if (tid == 0) {
+        ptx::mbar_init(ptx::smem_addr(&s_full[0]), 1);
+        ptx::mbar_init(ptx::smem_addr(&s_full[1]), 1);
+        ptx::fence_mbar_init_cluster();
+        const int t0 = draw();
+        const int t1 = t0 >= 0 ? draw() : -1;
+        s_tile[0] = t0; s_tile[1] = t1; s_tile[2] = -1; s_tile[3] = -1;
+        if (t0 >= 0) issue_copy(0, t0);
+        if (t1 >= 0) issue_copy(1, t1);
+    }
+    __syncthreads();
+    if (warp == 0 && s_tile[0] >= 0)
+        bad |= egae_window(a, s_win[0], int64_t(s_tile[0]) * kScanTile, tile_len(s_tile[0]), lane, nonfinite);
+
+    RunState cur{}, prev{};
+    int prev_tile = -1;
+    for (int k = 0;; ++k) {
+        __syncthreads();                                                  // tile numbers and windows of this step are visible
+        const int tile = s_tile[k & (kPipeRing - 1)];
+        const int64_t t0 = int64_t(tile < 0 ? 0 : tile) * kScanTile;
+        const int n_tile = tile < 0 ? 0 : tile_len(tile);
+        const bool by_tma = tile >= 0 && a.tma_ok && n_tile == kScanTile;
+        TileBuf& buf = s_buf[k & 1];
+        const TileWin& win = s_win[k & (kPipeRing - 1)];
+        if (tile >= 0) {
+            if (by_tma) {
+                if (!ptx::mbar_wait<false>(ptx::smem_addr(&s_full[k & 1]), uint32_t(k >> 1) & 1u)) late = true;
+            } else {      // a ragged or unaligned tile: plain loads
+                for (int q = tid; q < n_tile; q += kScanThreads) {
+                    buf.r[pos_slot(q)] = __ldg(a.rewards + t0 + q);
+                    buf.v[pos_slot(q)] = __ldg(a.values + t0 + q);
+                }
+            }
+            if (tid == kScanThreads - 1) buf.v_after = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
+        }
+        __syncthreads();
+        if (tile >= 0) {
+            // the thread's run, right to left: its composite map; the warp's scan
+            const Affine2 f = egae_run_map(a, buf, win, t0, n_tile, tid, cur, bad, nonfinite);
+            Affine2 S = f;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const Affine2 o = shfl_down(S, d);
+                if (lane + d < 32) S = compose(S, o);
+            }
+            cur.excl = shfl_down(S, 1);
+            if (lane == 31) cur.excl = identity2();
+            if (lane == 0) s_warp[warp] = S;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            if (tile >= 0) {          // composite of the tile: published at once, kept for the look-back one step on
+                Affine2 W = lane < kScanWarps ? s_warp[lane] : identity2();
+#pragma unroll
+                for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
+                Affine2 right = shfl_down(W, 1);
+                if (lane >= kScanWarps - 1) right = identity2();
+                if (lane < kScanWarps) s_right[k & 1][lane] = right;
+                if (lane == 0) {
+                    s_whole[k & 1] = W;
+                    if (!a.no_publish && tile + 1 < a.num_tiles) {
+                        st_pair(a.state[tile].aggA, W.aA, W.bA);
+                        st_pair(a.state[tile].aggR, W.aR, W.bR);
+                    }
+                }
+                __syncwarp();
+            }
+            if (prev_tile >= 0) {     // the value entering the tile of the step before
+                double xA = 0.0, xR = 0.0;
+                const bool ok = egae_look_back(a, prev_tile + 1, lane, xA, xR);
+                if (lane == 0) {
+                    if (!ok) { late = true; xA = 0.0; xR = 0.0; }
+                    const Affine2 W = s_whole[(k - 1) & 1];
+                    if (!a.no_publish) st_pair(a.state[prev_tile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
+                }
+                xA = __shfl_sync(0xffffffffu, xA, 0);
+                xR = __shfl_sync(0xffffffffu, xR, 0);
+                if (lane < kScanWarps) {
+                    const Affine2 right = s_right[(k - 1) & 1][lane];
+                    s_carry[lane][0] = fma(right.aA, xA, right.bA);
+                    s_carry[lane][1] = fma(right.aR, xR, right.bR);
+                }
+            }
+        } else if (warp == 1) {       // the tile after next
+            if (lane == 0) {
+                const bool more = tile >= 0 && s_tile[(k + 1) & (kPipeRing - 1)] >= 0;
+                s_tile[(k + 2) & (kPipeRing - 1)] = more ? draw() : -1;
+            }
+        } else if (warp == 2) {       // the segment window of the next tile
+            const int nt = s_tile[(k + 1) & (kPipeRing - 1)];
+            if (tile >= 0 && nt >= 0)
+                bad |= egae_window(a, s_win[(k + 1) & (kPipeRing - 1)], int64_t(nt) * kScanTile, tile_len(nt), lane, nonfinite);
+        }
+        __syncthreads();
+        if (prev_tile >= 0) {
+            // replay the positions of the step before from their true incoming values, store
+            const int64_t pt0 = int64_t(prev_tile) * kScanTile;
+            const int pn = tile_len(prev_tile);
+            const bool p_tma = a.tma_ok && pn == kScanTile;
+            TileBuf& pbuf = s_buf[(k - 1) & 1];
+            const float G = float(fma(prev.excl.aA, s_carry[warp][0], prev.excl.bA));
+            const float R = float(fma(prev.excl.aR, s_carry[warp][1], prev.excl.bR));
+            egae_run_replay(a, pbuf, s_win[(k - 1) & (kPipeRing - 1)], pt0, pn, tid, prev, G, R, p_tma, bad, nonfinite);
+            if (p_tma) ptx::fence_proxy_async_smem();       // the TMA stores read what was just written
+            __syncthreads();
+            if (tid == 0) {
+                if (p_tma) {
+#pragma unroll
+                    for (int bx = 0; bx < kScanBoxes; ++bx) {
+                        const int32_t y = prev_tile * (kScanTile / kRowPos) + bx * kScanBoxRows;
+                        umma::tma_store_2d(&map_adv, ptx::smem_addr(pbuf.v + bx * kScanBoxRows * kRowPos), 0, y);
+                        if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(pbuf.r + bx * kScanBoxRows * kRowPos), 0, y);
+                    }
+                    ptx::bulk_commit();
+                    ptx::bulk_wait_read<0>();       // the buffer is free once the stores have read it
+                }
+                // ... and takes the inputs of tile k+1 (tiles 0 and 1 were requested at the start)
+                const int nt = s_tile[(k + 1) & (kPipeRing - 1)];
+                if (tile >= 0 && nt >= 0) issue_copy(k + 1, nt);
+            }
+        }
+        if (tile < 0) break;
+        prev = cur;
+        prev_tile = tile;
+    }
+    if (bad) egae_raise(a, TPPO_DEV_BAD_SEGMENT);
+    if (nonfinite) egae_raise(a, TPPO_DEV_NONFINITE);
+    if (late) egae_raise(a, TPPO_DEV_WAIT_TIMEOUT);
+}
+
 bool make_f32_rows_tensor_map(CUtensorMap* map, const void* base, uint64_t rows);
 uint32_t test_spin_limit(uint32_t normal);
 int32_t test_no_publish();
@@ -815,7 +1006,16 @@ static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
                (!a.ret || make_f32_rows_tensor_map(&map_ret, a.ret, uint64_t(a.N) / kRowPos));
     a.spin_limit = test_spin_limit(kScanSpinLimit);
     a.no_publish = test_no_publish();
-    egae_scan_kernel<<<a.num_tiles, kScanThreads, 0, s>>>(a, map_r, map_v, map_adv, map_ret);
+#ifndef TPPO_EGAE_PIPE
+#define TPPO_EGAE_PIPE 0
+#endif
+    // enough tiles to fill the device several times over: resident CTAs that take tile after tile;
+    // otherwise one CTA per tile
+    if (TPPO_EGAE_PIPE && a.tma_ok && a.num_tiles >= 4 * kNumSms * kPipeCtasPerSm) {
+        egae_pipe_kernel<<<kNumSms * kPipeCtasPerSm, kScanThreads, 0, s>>>(a, map_r, map_v, map_adv, map_ret);
+    } else {
+        egae_scan_kernel<<<a.num_tiles, kScanThreads, 0, s>>>(a, map_r, map_v, map_adv, map_ret);
+    }
     TPPO_CUDA_CHECK(cudaGetLastError());
     return TPPO_OK;
 }
