@@ -26,6 +26,7 @@
 // whole tile arrive by two tiled TMA copies (rows of 32 positions, 128-byte swizzle: the four
 // 16-byte chunks a thread owns then sit in different bank groups from its neighbours'); there is no
 // per-thread staging code.
+#include <algorithm>
 #include <cstddef>
 #include <cstring>
 
@@ -89,7 +90,8 @@ struct TileState {
     double aggA[2];    // (a, b) of the tile's composite for the advantage recurrence
     double aggR[2];    // (a, b) of the tile's composite for the return recurrence
     double inc[2];     // A and R at the tile's first position
-    double pad[2];
+    int32_t win_lo, win_hi;   // segments [win_lo, win_hi) may touch the tile (written by the clearing kernel)
+    int32_t pad[2];
 };
 static_assert(sizeof(TileState) == 64, "tile state is four 16-byte pairs");
 constexpr unsigned long long kUnset = 0xffffffffffffffffull;
@@ -141,6 +143,7 @@ struct EgaeArgs {
     float* ret;
     int32_t* status;
     TileState* state;
+    int32_t after_clear;   // launched as the programmatic dependent of the kernel that clears status and states
     uint32_t* ticket;      // head of the workspace, cleared to all-ones with the tile states (+1 wraps to 0)
     uint32_t spin_limit;   // polls a look-back may spend on one round of tiles before it gives up
     int32_t no_publish;    // test hook: tiles keep their states to themselves, so every look-back runs out
@@ -344,7 +347,12 @@ __device__ __forceinline__ bool egae_window(const EgaeArgs& a, TileWin& win, int
     // starts after the segments that end at or before the tile's first position and stops before
     // those that begin after its last one
     int lo, hi;
-    warp_count_le2(a.seg_end, int32_t(t0), a.seg_begin, int32_t(t0 + n_tile - 1), a.B, lane, lo, hi);
+    if (a.after_clear) {      // found for every tile by the clearing kernel
+        const int2 w = __ldcg(reinterpret_cast<const int2*>(&a.state[t0 / kScanTile].win_lo));
+        lo = w.x; hi = w.y;
+    } else {
+        warp_count_le2(a.seg_end, int32_t(t0), a.seg_begin, int32_t(t0 + n_tile - 1), a.B, lane, lo, hi);
+    }
     if (lane == 0) { win.win_lo = lo; win.win_hi = hi; }
     bool bad = false;
     if (hi - lo <= kSegCap && lane < hi - lo) {
@@ -687,6 +695,7 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
 #if TPPO_EGAE_TICKET
         // the ticket counter starts at all-ones like the rest of the workspace (one memset): + 1
         // wraps the first draw to ticket 0
+        if (a.after_clear) asm volatile("griddepcontrol.wait;" ::: "memory");
         s_ticket = atomicAdd(a.ticket, 1u) + 1u;
 #else
         s_ticket = blockIdx.x;
@@ -723,8 +732,13 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     }
     if (threadIdx.x == kScanThreads - 1)
         buf.v_after = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
-    if (warp == 0) bad |= egae_window(a, win, t0, n_tile, lane, nonfinite);
-    if (by_tma && !ptx::mbar_wait<false>(bar, 0)) egae_raise(a, TPPO_DEV_WAIT_TIMEOUT);
+    if (warp == 0) {
+        // the segment window was found by the kernel launched just before this one, which lets this
+        // one start at once (programmatic dependent launch): its end is awaited here
+        if (a.after_clear) asm volatile("griddepcontrol.wait;" ::: "memory");
+        bad |= egae_window(a, win, t0, n_tile, lane, nonfinite);
+    }
+    const bool copy_late = by_tma && !ptx::mbar_wait<false>(bar, 0);      // reported once the status word may be touched
     __syncthreads();
 
     // ---- the thread's sixteen positions, right to left: its composite map; the warp's scan --------
@@ -740,6 +754,10 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     rs.excl = shfl_down(S, 1);   // composite of the lanes to the right
     if (lane == 31) rs.excl = identity2();
     if (lane == 0) s_warp[warp] = S;
+    // Everything above read inputs only.  The status word and the tile states are cleared by the
+    // small kernel launched just before this one, which lets this one start at once (programmatic
+    // dependent launch): its end is awaited here, before the first word of either is touched.
+    if (a.after_clear) asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();                                                      // (A)
 
     // ---- tile composite, look-back, per-warp carries (warp 0) ------------------------------------
@@ -778,6 +796,7 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     egae_run_replay(a, buf, win, t0, n_tile, threadIdx.x, rs, G, R, by_tma, bad, nonfinite);
     if (bad) egae_raise(a, TPPO_DEV_BAD_SEGMENT);
     if (nonfinite) egae_raise(a, TPPO_DEV_NONFINITE);
+    if (copy_late) egae_raise(a, TPPO_DEV_WAIT_TIMEOUT);
     if (by_tma) {
         ptx::fence_proxy_async_smem();       // the TMA stores read what was just written
         __syncthreads();
@@ -794,34 +813,48 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     }
 }
 
-// ---- the same scan as a software pipeline ------------------------------------------------------------
-// In the kernel above a tile's life is a chain of latencies, and the longest link is the look-back:
-// the right-hand neighbours of a tile are worked on at the same moment, so a tile that has just
-// published its composite waits for theirs, three of its four warps idle at a barrier.  Here a CTA
-// stays resident and takes tile after tile (by ticket), two tile images in shared memory, and looks
-// back for tile k-1 only AFTER it has composed the maps of tile k: by then the neighbours'
-// composites have long been published (one round of loads, no waiting), and while warp 0 looks back
-// the other warps draw the ticket after next and search the segment window of the next tile.  The
-// copy of tile k+1 is issued as soon as the results of tile k-1 have left its buffer.
-//   iteration k:  wait copy(k) | maps(k), warp scan | publish composite(k); look-back(k-1) ||
-//                 ticket(k+2), window(k+1) | replay(k-1), store | issue copy(k+1)
-constexpr int kPipeCtasPerSm = 6;
-constexpr int kPipeRing = 4;          // ring of tile numbers / segment windows: tiles k-1, k, k+1, k+2
+// ---- the same scan by resident CTAs with specialised warps ---------------------------------------------
+// In the kernel above a tile's life is a chain of latencies (copy, maps, publish, look-back, replay,
+// store), three of its four warps wait at barriers while warp 0 looks back, and registers allow
+// eight tiles per SM: the SM's issue slots and the DRAM are both idle two thirds of the time.  Here a
+// CTA stays resident, takes tile after tile by ticket, holds three tile images, and splits the work
+// of a step between its warps so that the latencies of different tiles overlap:
+//   step k, first half:   compute warps  maps of tile k, warp scans
+//                         chain warp     look-back for tile k-1 (its neighbours published their
+//                                        composites a step ago: one round of loads), value entering
+//                                        it published, carries of its warps
+//                         mover warp     results of tile k-2 stored, its image reused for the copy of
+//                                        tile k+1 (needed one whole step later)
+//           second half:  compute warps  replay of tile k-1 into its image
+//                         chain warp     composite of tile k from the warps' composites, published
+//                         mover warp     ticket for step k+2, segment window of tile k+1
+// Forward progress: tickets are drawn by running CTAs only and a tile waits only for tiles with
+// lower tickets; a CTA publishes the composite of its tile k after the look-back of its tile k-1,
+// which has a lower ticket, so the lowest unfinished ticket never waits for a higher one.
+constexpr int kResThreads = kScanThreads + 64;     // compute warps + chain warp + mover warp
+constexpr int kResCtasPerSm = 4;
+constexpr int kResBufs = 3;
+constexpr int kResRing = 8;                        // tile numbers of steps k-2 .. k+2
 constexpr uint32_t kTileBytes = 2 * kScanTile * uint32_t(sizeof(float));
+struct ResShared {
+    TileBuf buf[kResBufs];
+    TileWin win[4];                                // steps k-1, k, k+1
+    uint64_t full[kResBufs];                       // the inputs of the tile in image b have arrived
+    int tile[kResRing];                            // tile of step k (ring), -1: none left
+    Affine2 warp_comp[kScanWarps];                 // composites of the warps of tile k
+    Affine2 right[kScanWarps];                     // of tile k: composite of the warps to the right of each warp
+    Affine2 whole;                                 // of tile k: the tile's composite
+    double carry[kScanWarps][2];                   // of tile k-1: values entering each warp
+};
+constexpr size_t kResSmemBytes = sizeof(ResShared) + 1024;      // + room to align the images
 
-__global__ void __launch_bounds__(kScanThreads, kPipeCtasPerSm)
-egae_pipe_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
-                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_adv,
-                 const __grid_constant__ CUtensorMap map_ret) {
-    __shared__ TileBuf s_buf[2];
-    __shared__ TileWin s_win[kPipeRing];
-    __shared__ __align__(8) uint64_t s_full[2];      // the inputs of the tile in buffer b have arrived
-    __shared__ int s_tile[kPipeRing];                // tile taken for pipeline step k (ring), -1: none left
-    __shared__ Affine2 s_warp[kScanWarps];
-    __shared__ Affine2 s_right[2][kScanWarps];       // composite of the warps to the right of each warp
-    __shared__ Affine2 s_whole[2];                   // composite of the whole tile
-    __shared__ double s_carry[kScanWarps][2];
-
+__global__ void __launch_bounds__(kResThreads, kResCtasPerSm)
+egae_resident_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
+                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_adv,
+                     const __grid_constant__ CUtensorMap map_ret) {
+    extern __shared__ unsigned char res_smem_raw[];
+    ResShared& sh = *reinterpret_cast<ResShared*>(
+        (reinterpret_cast<uintptr_t>(res_smem_raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     bool bad = false, nonfinite = false, late = false;
 
@@ -830,143 +863,178 @@ egae_pipe_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
         return t < uint32_t(a.num_tiles) ? a.num_tiles - 1 - int(t) : -1;
     };
     auto tile_len = [&](int tile) { return int(min(int64_t(kScanTile), int64_t(a.N) - int64_t(tile) * kScanTile)); };
-    auto issue_copy = [&](int k, int tile) {     // one thread; whole, aligned tiles only
-        if (!(a.tma_ok && tile_len(tile) == kScanTile)) return;
-        const uint32_t bar = ptx::smem_addr(&s_full[k & 1]);
-        TileBuf& buf = s_buf[k & 1];
-        ptx::mbar_arrive_expect_tx(bar, kTileBytes);
+    auto whole_tile = [&](int tile) { return tile_len(tile) == kScanTile; };       // copied and stored by TMA
+    // one lane: the copy of a whole tile into image b; another lane fetches the value after the tile
+    auto request = [&](int b, int tile) {
+        TileBuf& buf = sh.buf[b];
+        if (lane == 0 && whole_tile(tile)) {
+            const uint32_t bar = ptx::smem_addr(&sh.full[b]);
+            ptx::mbar_arrive_expect_tx(bar, kTileBytes);
 #pragma unroll
-        for (int bx = 0; bx < kScanBoxes; ++bx) {
-            const int32_t y = tile * (kScanTile / kRowPos) + bx * kScanBoxRows;
-            umma::tma_load_2d(ptx::smem_addr(buf.r + bx * kScanBoxRows * kRowPos), &map_r, bar, 0, y);
-            umma::tma_load_2d(ptx::smem_addr(buf.v + bx * kScanBoxRows * kRowPos), &map_v, bar, 0, y);
+            for (int bx = 0; bx < kScanBoxes; ++bx) {
+                const int32_t y = tile * (kScanTile / kRowPos) + bx * kScanBoxRows;
+                umma::tma_load_2d(ptx::smem_addr(buf.r + bx * kScanBoxRows * kRowPos), &map_r, bar, 0, y);
+                umma::tma_load_2d(ptx::smem_addr(buf.v + bx * kScanBoxRows * kRowPos), &map_v, bar, 0, y);
+            }
+        }
+        if (lane == 1) {
+            const int64_t after = int64_t(tile) * kScanTile + tile_len(tile);
+            buf.v_after = after < a.N ? __ldg(a.values + after) : 0.f;
         }
     };
 
-    if (tid == 0) {
-        ptx::mbar_init(ptx::smem_addr(&s_full[0]), 1);
-        ptx::mbar_init(ptx::smem_addr(&s_full[1]), 1);
-        ptx::fence_mbar_init_cluster();
-        const int t0 = draw();
-        const int t1 = t0 >= 0 ? draw() : -1;
-        s_tile[0] = t0; s_tile[1] = t1; s_tile[2] = -1; s_tile[3] = -1;
-        if (t0 >= 0) issue_copy(0, t0);
-        if (t1 >= 0) issue_copy(1, t1);
+    // the ticket counter, the tile states and the segment windows are written by the kernel launched
+    // just before this one
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (warp == kScanWarps + 1) {
+        int t0 = -1, t1 = -1;
+        if (lane == 0) {
+#pragma unroll
+            for (int b = 0; b < kResBufs; ++b) ptx::mbar_init(ptx::smem_addr(&sh.full[b]), 1);
+            ptx::fence_mbar_init_cluster();
+            t0 = draw();
+            t1 = t0 >= 0 ? draw() : -1;
+            sh.tile[0] = t0; sh.tile[1] = t1;
+#pragma unroll
+            for (int i = 2; i < kResRing; ++i) sh.tile[i] = -1;
+        }
+        t0 = __shfl_sync(0xffffffffu, t0, 0);
+        if (t0 >= 0) {
+            request(0, t0);
+            bad |= egae_window(a, sh.win[0], int64_t(t0) * kScanTile, tile_len(t0), lane, nonfinite);
+        }
     }
     __syncthreads();
-    if (warp == 0 && s_tile[0] >= 0)
-        bad |= egae_window(a, s_win[0], int64_t(s_tile[0]) * kScanTile, tile_len(s_tile[0]), lane, nonfinite);
 
-    RunState cur{}, prev{};
-    int prev_tile = -1;
-    for (int k = 0;; ++k) {
-        __syncthreads();                                                  // tile numbers and windows of this step are visible
-        const int tile = s_tile[k & (kPipeRing - 1)];
-        const int64_t t0 = int64_t(tile < 0 ? 0 : tile) * kScanTile;
-        const int n_tile = tile < 0 ? 0 : tile_len(tile);
-        const bool by_tma = tile >= 0 && a.tma_ok && n_tile == kScanTile;
-        TileBuf& buf = s_buf[k & 1];
-        const TileWin& win = s_win[k & (kPipeRing - 1)];
-        if (tile >= 0) {
-            if (by_tma) {
-                if (!ptx::mbar_wait<false>(ptx::smem_addr(&s_full[k & 1]), uint32_t(k >> 1) & 1u)) late = true;
-            } else {      // a ragged or unaligned tile: plain loads
-                for (int q = tid; q < n_tile; q += kScanThreads) {
-                    buf.r[pos_slot(q)] = __ldg(a.rewards + t0 + q);
-                    buf.v[pos_slot(q)] = __ldg(a.values + t0 + q);
-                }
-            }
-            if (tid == kScanThreads - 1) buf.v_after = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
-        }
-        __syncthreads();
-        if (tile >= 0) {
-            // the thread's run, right to left: its composite map; the warp's scan
-            const Affine2 f = egae_run_map(a, buf, win, t0, n_tile, tid, cur, bad, nonfinite);
-            Affine2 S = f;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const Affine2 o = shfl_down(S, d);
-                if (lane + d < 32) S = compose(S, o);
-            }
-            cur.excl = shfl_down(S, 1);
-            if (lane == 31) cur.excl = identity2();
-            if (lane == 0) s_warp[warp] = S;
-        }
-        __syncthreads();
-        if (warp == 0) {
-            if (tile >= 0) {          // composite of the tile: published at once, kept for the look-back one step on
-                Affine2 W = lane < kScanWarps ? s_warp[lane] : identity2();
-#pragma unroll
-                for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
-                Affine2 right = shfl_down(W, 1);
-                if (lane >= kScanWarps - 1) right = identity2();
-                if (lane < kScanWarps) s_right[k & 1][lane] = right;
-                if (lane == 0) {
-                    s_whole[k & 1] = W;
-                    if (!a.no_publish && tile + 1 < a.num_tiles) {
-                        st_pair(a.state[tile].aggA, W.aA, W.bA);
-                        st_pair(a.state[tile].aggR, W.aR, W.bR);
+    // Each kind of warp runs its own loop (its registers hold only what its own work needs); all
+    // loops make the same two barrier calls per step and leave after the same step, which every
+    // thread reads from the ring of tile numbers.
+    auto step_barrier = [] { asm volatile("bar.sync 0, %0;" ::"n"(kResThreads) : "memory"); };
+    struct Step { int tile, ptile, pptile, ntile; bool done; };
+    auto step_of = [&](int k) {
+        Step st;
+        st.tile = sh.tile[k & (kResRing - 1)];
+        st.ptile = k >= 1 ? sh.tile[(k - 1) & (kResRing - 1)] : -1;
+        st.pptile = k >= 2 ? sh.tile[(k - 2) & (kResRing - 1)] : -1;
+        st.ntile = sh.tile[(k + 1) & (kResRing - 1)];
+        st.done = st.tile < 0 && st.ptile < 0 && st.pptile < 0;
+        return st;
+    };
+    // images: step k in k % 3, step k-1 in (k+2) % 3, steps k+1 and k-2 in (k+1) % 3
+
+    if (warp < kScanWarps) {
+        // ---- compute warps: maps of tile k | replay of tile k-1 --------------------------------------
+        RunState cur{}, prev{};
+        uint32_t phases = 0;      // bit b: parity of the phase barrier b completes next (a ragged tile arms none)
+#pragma unroll 1
+        for (int k = 0;; ++k) {
+            const Step st = step_of(k);
+            if (st.done) break;
+            if (st.tile >= 0) {
+                const int bk = k % kResBufs;
+                TileBuf& buf = sh.buf[bk];
+                const int64_t t0 = int64_t(st.tile) * kScanTile;
+                const int n_tile = tile_len(st.tile);
+                if (n_tile == kScanTile) {
+                    if (!ptx::mbar_wait<false>(ptx::smem_addr(&sh.full[bk]), (phases >> bk) & 1u)) late = true;
+                    phases ^= 1u << bk;
+                } else {      // the ragged tile: plain loads, then a barrier among the compute warps
+                    for (int q = tid; q < n_tile; q += kScanThreads) {
+                        buf.r[pos_slot(q)] = __ldg(a.rewards + t0 + q);
+                        buf.v[pos_slot(q)] = __ldg(a.values + t0 + q);
                     }
+                    asm volatile("bar.sync 1, %0;" ::"n"(kScanThreads) : "memory");
                 }
-                __syncwarp();
+                const Affine2 f = egae_run_map(a, buf, sh.win[k & 3], t0, n_tile, tid, cur, bad, nonfinite);
+                Affine2 S = f;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const Affine2 o = shfl_down(S, d);
+                    if (lane + d < 32) S = compose(S, o);
+                }
+                cur.excl = shfl_down(S, 1);
+                if (lane == 31) cur.excl = identity2();
+                if (lane == 0) sh.warp_comp[warp] = S;
             }
-            if (prev_tile >= 0) {     // the value entering the tile of the step before
+            step_barrier();
+            if (st.ptile >= 0) {
+                const int64_t pt0 = int64_t(st.ptile) * kScanTile;
+                const int pn = tile_len(st.ptile);
+                const bool p_tma = pn == kScanTile;
+                const float G = float(fma(prev.excl.aA, sh.carry[warp][0], prev.excl.bA));
+                const float R = float(fma(prev.excl.aR, sh.carry[warp][1], prev.excl.bR));
+                egae_run_replay(a, sh.buf[(k + 2) % kResBufs], sh.win[(k - 1) & 3], pt0, pn, tid, prev, G, R, p_tma, bad, nonfinite);
+                if (p_tma) ptx::fence_proxy_async_smem();       // the TMA stores read what was just written
+            }
+            prev = cur;
+            step_barrier();
+        }
+    } else if (warp == kScanWarps) {
+        // ---- chain warp: look-back for tile k-1 | composite of tile k ----------------------------------
+#pragma unroll 1
+        for (int k = 0;; ++k) {
+            const Step st = step_of(k);
+            if (st.done) break;
+            if (st.ptile >= 0) {     // the value entering the tile of the step before
                 double xA = 0.0, xR = 0.0;
-                const bool ok = egae_look_back(a, prev_tile + 1, lane, xA, xR);
+                const bool ok = egae_look_back(a, st.ptile + 1, lane, xA, xR);
                 if (lane == 0) {
                     if (!ok) { late = true; xA = 0.0; xR = 0.0; }
-                    const Affine2 W = s_whole[(k - 1) & 1];
-                    if (!a.no_publish) st_pair(a.state[prev_tile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
+                    const Affine2 W = sh.whole;
+                    if (!a.no_publish) st_pair(a.state[st.ptile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
                 }
                 xA = __shfl_sync(0xffffffffu, xA, 0);
                 xR = __shfl_sync(0xffffffffu, xR, 0);
                 if (lane < kScanWarps) {
-                    const Affine2 right = s_right[(k - 1) & 1][lane];
-                    s_carry[lane][0] = fma(right.aA, xA, right.bA);
-                    s_carry[lane][1] = fma(right.aR, xR, right.bR);
+                    const Affine2 right = sh.right[lane];
+                    sh.carry[lane][0] = fma(right.aA, xA, right.bA);
+                    sh.carry[lane][1] = fma(right.aR, xR, right.bR);
                 }
             }
-        } else if (warp == 1) {       // the tile after next
-            if (lane == 0) {
-                const bool more = tile >= 0 && s_tile[(k + 1) & (kPipeRing - 1)] >= 0;
-                s_tile[(k + 2) & (kPipeRing - 1)] = more ? draw() : -1;
-            }
-        } else if (warp == 2) {       // the segment window of the next tile
-            const int nt = s_tile[(k + 1) & (kPipeRing - 1)];
-            if (tile >= 0 && nt >= 0)
-                bad |= egae_window(a, s_win[(k + 1) & (kPipeRing - 1)], int64_t(nt) * kScanTile, tile_len(nt), lane, nonfinite);
-        }
-        __syncthreads();
-        if (prev_tile >= 0) {
-            // replay the positions of the step before from their true incoming values, store
-            const int64_t pt0 = int64_t(prev_tile) * kScanTile;
-            const int pn = tile_len(prev_tile);
-            const bool p_tma = a.tma_ok && pn == kScanTile;
-            TileBuf& pbuf = s_buf[(k - 1) & 1];
-            const float G = float(fma(prev.excl.aA, s_carry[warp][0], prev.excl.bA));
-            const float R = float(fma(prev.excl.aR, s_carry[warp][1], prev.excl.bR));
-            egae_run_replay(a, pbuf, s_win[(k - 1) & (kPipeRing - 1)], pt0, pn, tid, prev, G, R, p_tma, bad, nonfinite);
-            if (p_tma) ptx::fence_proxy_async_smem();       // the TMA stores read what was just written
-            __syncthreads();
-            if (tid == 0) {
-                if (p_tma) {
+            step_barrier();
+            if (st.tile >= 0) {      // composite of the tile from its warps' composites, published
+                Affine2 W = lane < kScanWarps ? sh.warp_comp[lane] : identity2();
 #pragma unroll
-                    for (int bx = 0; bx < kScanBoxes; ++bx) {
-                        const int32_t y = prev_tile * (kScanTile / kRowPos) + bx * kScanBoxRows;
-                        umma::tma_store_2d(&map_adv, ptx::smem_addr(pbuf.v + bx * kScanBoxRows * kRowPos), 0, y);
-                        if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(pbuf.r + bx * kScanBoxRows * kRowPos), 0, y);
+                for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
+                Affine2 right = shfl_down(W, 1);
+                if (lane >= kScanWarps - 1) right = identity2();
+                if (lane < kScanWarps) sh.right[lane] = right;
+                if (lane == 0) {
+                    sh.whole = W;
+                    if (!a.no_publish && st.tile + 1 < a.num_tiles) {
+                        st_pair(a.state[st.tile].aggA, W.aA, W.bA);
+                        st_pair(a.state[st.tile].aggR, W.aR, W.bR);
                     }
-                    ptx::bulk_commit();
-                    ptx::bulk_wait_read<0>();       // the buffer is free once the stores have read it
                 }
-                // ... and takes the inputs of tile k+1 (tiles 0 and 1 were requested at the start)
-                const int nt = s_tile[(k + 1) & (kPipeRing - 1)];
-                if (tile >= 0 && nt >= 0) issue_copy(k + 1, nt);
             }
+            step_barrier();
         }
-        if (tile < 0) break;
-        prev = cur;
-        prev_tile = tile;
+    } else {
+        // ---- mover warp: results of tile k-2 out, inputs of tile k+1 in | next ticket and window ------
+#pragma unroll 1
+        for (int k = 0;; ++k) {
+            const Step st = step_of(k);
+            if (st.done) break;
+            const int bn = (k + 1) % kResBufs;
+            if (st.pptile >= 0 && whole_tile(st.pptile) && lane == 0) {
+                TileBuf& obuf = sh.buf[bn];
+#pragma unroll
+                for (int bx = 0; bx < kScanBoxes; ++bx) {
+                    const int32_t y = st.pptile * (kScanTile / kRowPos) + bx * kScanBoxRows;
+                    umma::tma_store_2d(&map_adv, ptx::smem_addr(obuf.v + bx * kScanBoxRows * kRowPos), 0, y);
+                    if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(obuf.r + bx * kScanBoxRows * kRowPos), 0, y);
+                }
+                ptx::bulk_commit();
+                ptx::bulk_wait_read<0>();       // the image is free once the stores have read it
+            }
+            __syncwarp();
+            if (st.ntile >= 0) request(bn, st.ntile);
+            step_barrier();
+            if (lane == 0) sh.tile[(k + 2) & (kResRing - 1)] = (st.tile >= 0 && st.ntile >= 0) ? draw() : -1;
+            if (st.ntile >= 0)
+                bad |= egae_window(a, sh.win[(k + 1) & 3], int64_t(st.ntile) * kScanTile, tile_len(st.ntile), lane, nonfinite);
+            step_barrier();
+        }
     }
     if (bad) egae_raise(a, TPPO_DEV_BAD_SEGMENT);
     if (nonfinite) egae_raise(a, TPPO_DEV_NONFINITE);
@@ -979,6 +1047,58 @@ int32_t test_no_publish();
 
 // Fills the constants derived from gamma and lambda and the tensor maps, then launches one CTA per
 // tile.  The caller has set the pointers, sizes, state and ticket.
+constexpr size_t kScanHeadBytes = 256;      // the ticket counter
+
+// Number of entries of the ascending array arr[0..n) that are <= key.
+template <bool LDG>
+__device__ __forceinline__ int count_le(const int32_t* __restrict__ arr, int n, int32_t key) {
+    int lo = 0, hi = n;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if ((LDG ? __ldg(arr + mid) : arr[mid]) <= key) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// Launched just before the scan, which is its programmatic dependent and starts beside it: status
+// word to 0, ticket counter to all-ones, and one thread per tile sets the tile's state to unset
+// (all-ones) and finds its segment window, so that a tile of the scan reads its window instead of
+// searching for it: the search (three dependent rounds of global loads by one warp) was the longest
+// latency of a tile's first phase, longer than the copy of its inputs.  Here a block first copies the
+// segment bounds into shared memory (2 x 4 x B bytes, one round of loads) and searches there; bounds
+// that do not fit are searched in global memory.
+constexpr int kClearThreads = 128;
+constexpr int kClearSmemMaxB = 12288;       // 96 KB of segment bounds
+__global__ void __launch_bounds__(kClearThreads) egae_clear_kernel(int32_t* status, uint4* head,
+                                                                   TileState* state, int num_tiles,
+                                                                   const int32_t* seg_begin,
+                                                                   const int32_t* seg_end, int B,
+                                                                   int64_t N, int in_smem) {
+    extern __shared__ int32_t s_bounds[];      // seg_end[0..B), seg_begin[0..B)
+    asm volatile("griddepcontrol.launch_dependents;");
+    const int tile = blockIdx.x * blockDim.x + threadIdx.x;
+    if (tile == 0) *status = 0;
+    if (tile < int(kScanHeadBytes / 16)) head[tile] = make_uint4(~0u, ~0u, ~0u, ~0u);
+    if (in_smem) {
+        for (int i = threadIdx.x; i < B; i += kClearThreads) {
+            s_bounds[i] = __ldg(seg_end + i);
+            s_bounds[B + i] = __ldg(seg_begin + i);
+        }
+        __syncthreads();
+    }
+    if (tile >= num_tiles) return;
+    const int64_t t0 = int64_t(tile) * kScanTile;
+    const int64_t t_last = min(t0 + kScanTile, N) - 1;
+    const int lo = in_smem ? count_le<false>(s_bounds, B, int32_t(t0)) : count_le<true>(seg_end, B, int32_t(t0));
+    const int hi = in_smem ? count_le<false>(s_bounds + B, B, int32_t(t_last))
+                           : count_le<true>(seg_begin, B, int32_t(t_last));
+    uint4* st = reinterpret_cast<uint4*>(state + tile);
+    st[0] = make_uint4(~0u, ~0u, ~0u, ~0u);
+    st[1] = make_uint4(~0u, ~0u, ~0u, ~0u);
+    st[2] = make_uint4(~0u, ~0u, ~0u, ~0u);
+    st[3] = make_uint4(uint32_t(lo), uint32_t(hi), 0u, 0u);
+}
+
 static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
     a.num_tiles = int32_t((int64_t(a.N) + kScanTile - 1) / kScanTile);
     a.gamma = double(gamma);
@@ -1006,21 +1126,33 @@ static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
                (!a.ret || make_f32_rows_tensor_map(&map_ret, a.ret, uint64_t(a.N) / kRowPos));
     a.spin_limit = test_spin_limit(kScanSpinLimit);
     a.no_publish = test_no_publish();
-#ifndef TPPO_EGAE_PIPE
-#define TPPO_EGAE_PIPE 0
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(a.num_tiles));
+    cfg.blockDim = dim3(kScanThreads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = a.after_clear ? 1 : 0;
+#ifndef TPPO_EGAE_RESIDENT_MIN_TILES
+#define TPPO_EGAE_RESIDENT_MIN_TILES (2 * kNumSms * kResCtasPerSm)
 #endif
-    // enough tiles to fill the device several times over: resident CTAs that take tile after tile;
-    // otherwise one CTA per tile
-    if (TPPO_EGAE_PIPE && a.tma_ok && a.num_tiles >= 4 * kNumSms * kPipeCtasPerSm) {
-        egae_pipe_kernel<<<kNumSms * kPipeCtasPerSm, kScanThreads, 0, s>>>(a, map_r, map_v, map_adv, map_ret);
-    } else {
-        egae_scan_kernel<<<a.num_tiles, kScanThreads, 0, s>>>(a, map_r, map_v, map_adv, map_ret);
+    // enough whole tiles to keep resident CTAs busy for several steps each: warp-specialised resident
+    // CTAs; otherwise one CTA per tile
+    if (a.after_clear && a.tma_ok && a.num_tiles >= TPPO_EGAE_RESIDENT_MIN_TILES) {
+        TPPO_CUDA_CHECK(cudaFuncSetAttribute(egae_resident_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             int(kResSmemBytes)));
+        cfg.gridDim = dim3(unsigned(std::min(a.num_tiles, kNumSms * kResCtasPerSm)));
+        cfg.blockDim = dim3(kResThreads);
+        cfg.dynamicSmemBytes = kResSmemBytes;
+        TPPO_CUDA_CHECK(cudaLaunchKernelEx(&cfg, egae_resident_kernel, a, map_r, map_v, map_adv, map_ret));
+        return TPPO_OK;
     }
-    TPPO_CUDA_CHECK(cudaGetLastError());
+    TPPO_CUDA_CHECK(cudaLaunchKernelEx(&cfg, egae_scan_kernel, a, map_r, map_v, map_adv, map_ret));
     return TPPO_OK;
 }
 
-constexpr size_t kScanHeadBytes = 256;      // the ticket counter
 size_t egae_workspace_bytes(int64_t N) {
     const int64_t tiles = (N + kScanTile - 1) / kScanTile;
     return kScanHeadBytes + align_up(size_t(tiles > 0 ? tiles : 1) * sizeof(TileState), kWsAlign);
@@ -1048,13 +1180,32 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
     if (!workspace || workspace_bytes < need || !aligned(workspace, kWsAlign))
         return TPPO_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
-    if (N == 0) return TPPO_OK;
-    // tile states start out unset (all-ones), the ticket counter at all-ones too.  (Letting the last
-    // tile to finish hand over the status bits instead of clearing them here was measured: the fence
-    // and counter at the end of every tile cost 9 us at 17.5 M tokens, a 4-byte clear nothing.)
-    TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0xff, need, s));
+    if (N == 0) {
+        TPPO_CUDA_CHECK(cudaMemsetAsync(status, 0, sizeof(int32_t), s));
+        return TPPO_OK;
+    }
+    // Tile states start out unset (all-ones), the ticket counter at all-ones too, the status at 0:
+    // one small kernel writes them, and the scan starts beside it as its programmatic dependent,
+    // copying tiles in and composing maps until it first needs either.  (Two memsets in front of a
+    // plain launch cost about 5 us more at 17.5 M tokens; letting the last tile to finish hand over
+    // the status bits, to save the clear altogether, cost 9 us for the fence and counter at every
+    // tile's end.)
+    {
+        static_assert(kScanHeadBytes / 16 <= kClearThreads, "the first block writes the head");
+        const int tiles = int((N + kScanTile - 1) / kScanTile);
+        const int in_smem = B <= kClearSmemMaxB;
+        const size_t smem = in_smem ? size_t(2) * size_t(B) * sizeof(int32_t) : 0;
+        if (smem > 48 * 1024)       // (an attribute of the function on the current device; the call is cheap)
+            TPPO_CUDA_CHECK(cudaFuncSetAttribute(egae_clear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 2 * kClearSmemMaxB * int(sizeof(int32_t))));
+        egae_clear_kernel<<<(tiles + kClearThreads - 1) / kClearThreads, kClearThreads, smem, s>>>(
+            status, static_cast<uint4*>(workspace),
+            reinterpret_cast<TileState*>(static_cast<char*>(workspace) + kScanHeadBytes), tiles,
+            seg_begin, seg_end, B, N, in_smem);
+        TPPO_CUDA_CHECK(cudaGetLastError());
+    }
     EgaeArgs a{};
+    a.after_clear = 1;
     a.rewards = rewards; a.values = values; a.seg_begin = seg_begin; a.seg_end = seg_end;
     a.truncated = truncated; a.bootstrap = bootstrap; a.B = B; a.N = int32_t(N);
     a.adv = advantages; a.ret = returns; a.status = status;

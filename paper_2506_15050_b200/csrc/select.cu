@@ -3,6 +3,7 @@
 // arithmetic on the sequences that overlap them, ranks come from popcounts and a warp / tile
 // prefix, a decoupled look-back chain links the tiles, and every selected position is written once
 // in ascending order.  Integer work throughout: the result is bit-exact and run-to-run identical.
+#include <algorithm>
 #include "common.cuh"
 
 namespace tppo {
@@ -151,6 +152,7 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // A tile only waits for tiles with smaller indices.
 #if TPPO_SEL_TICKET
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // the counter is cleared by the kernel before
     if (threadIdx.x == 0) s_tile = atomicAdd(a.ticket, 1u);
 #else
     if (threadIdx.x == 0) s_tile = blockIdx.x;
@@ -267,6 +269,10 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
         if (w < warp) before += c;
         tile_tot += c;
     }
+    // Everything above read inputs only.  The counts and the tile states are cleared by the small
+    // kernel launched just before this one, which lets this one start at once (programmatic
+    // dependent launch): its end is awaited here, before the first word of either is touched.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // publish the tile's totals as early as possible: later tiles wait for them in their look-back
     if (threadIdx.x == 0 && tile > 0 && !a.no_publish)
         reinterpret_cast<volatile unsigned long long*>(a.state)[tile] =
@@ -326,6 +332,14 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     sel_copy_out(a.value_idx, s_base_val, int(s_tot_val), s_out_val, int32_t(t0), a.out_vec_ok != 0);
 }
 
+// Clears the counts and the workspace of one call; the selection kernel is its programmatic dependent.
+__global__ void __launch_bounds__(256) select_clear_kernel(int32_t* counts, uint4* ws, size_t n16) {
+    asm volatile("griddepcontrol.launch_dependents;");
+    if (blockIdx.x == 0 && threadIdx.x < 4) counts[threadIdx.x] = 0;
+    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n16; i += size_t(gridDim.x) * blockDim.x)
+        ws[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
 size_t select_workspace_bytes(int64_t N) {
     const int64_t tiles = (N + kSelTile - 1) / kSelTile;
     return kWsAlign + align_up(size_t(tiles > 0 ? tiles : 1) * 8, kWsAlign);
@@ -354,11 +368,20 @@ TPPO_API int tppo_select_tokens(const int32_t* seq_begin, const int32_t* prompt_
     if (!workspace || workspace_bytes < need || !aligned(workspace, kWsAlign))
         return TPPO_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    TPPO_CUDA_CHECK(cudaMemsetAsync(counts, 0, 4 * sizeof(int32_t), s));
-    if (N == 0 || B == 0) return TPPO_OK;
-    // (Handing the counts and status bits over by the last tile to finish, to save the 16-byte clear
-    // above, was measured: the fence and counter at the end of every tile cost 6 us at 17.5 M tokens.)
-    TPPO_CUDA_CHECK(cudaMemsetAsync(workspace, 0, need, s));
+    if (N == 0 || B == 0) {
+        TPPO_CUDA_CHECK(cudaMemsetAsync(counts, 0, 4 * sizeof(int32_t), s));
+        return TPPO_OK;
+    }
+    // One small kernel clears the counts and the tile states, and the selection kernel starts beside
+    // it, reading masks and sequence bounds until it first needs either.  (Two memsets in front of a
+    // plain launch cost 6 us more at 17.5 M tokens; handing the counts over by the last tile to
+    // finish, to save the clear altogether, cost 6 us for the fence and counter at every tile's end.)
+    {
+        const size_t n16 = need / 16;
+        const int blocks = int(std::min<size_t>((n16 + 255) / 256, 64));
+        select_clear_kernel<<<blocks, 256, 0, s>>>(counts, static_cast<uint4*>(workspace), n16);
+        TPPO_CUDA_CHECK(cudaGetLastError());
+    }
     SelectArgs a;
     a.seq_begin = seq_begin; a.prompt_len = prompt_len; a.prev_len = prev_len; a.new_len = new_len;
     a.truncated = truncated; a.pol_mask = extra_policy_mask; a.val_mask = extra_value_mask;
@@ -372,7 +395,15 @@ TPPO_API int tppo_select_tokens(const int32_t* seq_begin, const int32_t* prompt_
     a.policy_idx = policy_idx; a.value_idx = value_idx; a.counts = counts;
     a.ticket = static_cast<uint32_t*>(workspace);
     a.state = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWsAlign);
-    select_tokens_kernel<<<a.num_tiles, kSelThreads, 0, s>>>(a);
-    TPPO_CUDA_CHECK(cudaGetLastError());
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(a.num_tiles));
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    TPPO_CUDA_CHECK(cudaLaunchKernelEx(&cfg, select_tokens_kernel, a));
     return TPPO_OK;
 }
