@@ -295,7 +295,9 @@ class Step:
         ev[4].record()
         events.append(tuple(ev))
 
-    KERNELS_PER_STEP = 6   # egae scan, select, policy prepare + sweep + finish, value loss
+    # EGAE clear + scan, selection clear + kernel, policy prepare + cluster sweep + side sweep + finish,
+    # value clear + kernel (a policy call below 2048 rows has no side sweep)
+    KERNELS_PER_STEP = 10
 
 
 class LmHeadStep:
@@ -749,7 +751,7 @@ def main():
             "config": workload_config(st.N, st.n, n_val, args.hint),
             "step_calls_us": calls_us, "cuda_graph_replay": graph,
             "roofline": roofline,
-            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": Step.KERNELS_PER_STEP * args.steps,
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": (Step.KERNELS_PER_STEP - (st.n < 2048)) * args.steps,
             "clocks": clocks, "small_kernels": small_kernels, "lmhead_variant": lmhead}))
     if world > 1:
         import torch.distributed as dist
@@ -946,7 +948,13 @@ def run_lmhead_workload(args, rank, world, local, dev, warmup):
 # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of each small kernel on config 4
 # (profiles/egae_select_value_advance_cfg4.md gives the command); None once a kernel has changed
 # since its counters were taken.
-NCU_CFG4_TRAFFIC = {"egae": None, "select": None, "value": None, "advance": None}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of each call's kernels on this very
+# workload (ncu capture of `python bench.py --workload cfg4 --steps 1 --warmup 3`;
+# profiles/egae_select_value_advance_cfg4.md): the scan kernel, the selection kernel, the value
+# kernel plus the kernel that zero-fills dvalues, the slot walk plus the copy kernel.  None once a
+# kernel has changed since.
+NCU_CFG4_TRAFFIC = {"egae": 140769536 + 94864896, "select": 35140608 + 726784,
+                    "value": 145093888 + 21591040 + 7936 + 7788544, "advance": 43353088 + 1300736 + 78592}
 
 
 def measure_cfg4(dev, steps, warmup):
@@ -1195,7 +1203,7 @@ def run_cfg4_workload(args, rank, world, local, dev, warmup):
                          "traffic": k["egae"]["traffic"], "kernel": "egae_scan_kernel",
                          "kernel_ms": k["egae"]["us"] / 1e3,
                          "algorithmic_bytes_per_launch": k["egae"]["algorithmic_bytes"]},
-            "kernels": k, "gpu_launches": 6 * steps, "clocks": m["clocks"]}))
+            "kernels": k, "gpu_launches": 8 * steps, "clocks": m["clocks"]}))
 
 
 if __name__ == "__main__":

@@ -90,8 +90,7 @@ struct TileState {
     double aggA[2];    // (a, b) of the tile's composite for the advantage recurrence
     double aggR[2];    // (a, b) of the tile's composite for the return recurrence
     double inc[2];     // A and R at the tile's first position
-    int32_t win_lo, win_hi;   // segments [win_lo, win_hi) may touch the tile (written by the clearing kernel)
-    int32_t pad[2];
+    int32_t win[4];    // per 2048-position part of the tile: segments [win[2p], win[2p+1]) may touch it (written by the clearing kernel)
 };
 static_assert(sizeof(TileState) == 64, "tile state is four 16-byte pairs");
 constexpr unsigned long long kUnset = 0xffffffffffffffffull;
@@ -342,13 +341,13 @@ __device__ __forceinline__ void warp_count_le2(const int32_t* __restrict__ arr1,
 // a segment with bounds outside [0, N] or end < begin was seen; such a segment is treated as empty.
 static_assert(kSegCap == 32, "one lane per window segment");
 __device__ __forceinline__ bool egae_window(const EgaeArgs& a, TileWin& win, int64_t t0, int n_tile,
-                                            int lane, bool& nonfinite) {
+                                            int lane, bool& nonfinite, const int32_t* found) {
     // segments are ascending and disjoint, so seg_begin and seg_end are both ascending: the window
     // starts after the segments that end at or before the tile's first position and stops before
     // those that begin after its last one
     int lo, hi;
-    if (a.after_clear) {      // found for every tile by the clearing kernel
-        const int2 w = __ldcg(reinterpret_cast<const int2*>(&a.state[t0 / kScanTile].win_lo));
+    if (found) {      // found for every tile by the clearing kernel
+        const int2 w = __ldcg(reinterpret_cast<const int2*>(found));
         lo = w.x; hi = w.y;
     } else {
         warp_count_le2(a.seg_end, int32_t(t0), a.seg_begin, int32_t(t0 + n_tile - 1), a.B, lane, lo, hi);
@@ -674,101 +673,150 @@ __device__ __forceinline__ void egae_run_replay(const EgaeArgs& a, TileBuf& buf,
     }
 }
 
-// One CTA per tile of 2048 positions, from the END of the arrays backwards, so the tiles a tile
-// looks back at (those to its right) were started earlier and are running or done.  The latencies of a tile (ticket, copy, window search, look-back) are covered by
-// the other CTAs resident on the SM.  A whole tile's results are written over its inputs in shared
-// memory and leave by two TMA stores.
-__global__ void __launch_bounds__(kScanThreads, kScanCtasPerSm)
+// One CTA per tile, from the END of the arrays backwards, so the tiles a tile looks back at (those
+// to its right) were started earlier and are running or done.  A tile is kScanParts parts of 2048
+// positions (one by default); a thread owns one run of sixteen positions in every part.  The
+// latencies of a tile (copy, segment window, look-back) are covered by the other CTAs resident on
+// the SM.  A whole part's results are written over its inputs in shared memory and leave by TMA stores.
+//
+// Measured at 17.5 M tokens against this form (81 us per call), and dropped:
+//  - two parts per tile (the same 128 threads map the right part, then the left part, then one
+//    publication and one look-back per 4096 positions; six tiles per SM): 95 us;
+//  - resident CTAs that take tile after tile by ticket, (a) with two tile images, the look-back for
+//    tile k-1 after the maps of tile k: 92 us -- the copy of tile k+1 cannot start before the replay
+//    of tile k-1 has left its image, so every step waits for a copy; (b) with three images and
+//    specialised warps (four compute warps, a warp that looks back and publishes, a warp that moves
+//    tiles, draws tickets and fetches windows), four CTAs per SM: 82 us, and 90 us when the look-back
+//    warp runs ahead of the others -- the steps of the resident CTAs lock into one another through
+//    the look-back, and each step then lasts as long as the slowest neighbour's.
+// In-kernel clock stamps of a debug build: a tile lives about 20 k cycles (start to first barrier 2.6 k,
+// window + copy 3.9 k, maps and warp scans 3.1 k, compose + publish 0.9 k, look-back 5.8 k, carries
+// 0.9 k, replay + store 2.8 k); every variant above has fewer warps per SM in the two compute phases,
+// and those run at one instruction per six cycles and warp.
+#ifndef TPPO_SCAN_PARTS
+#define TPPO_SCAN_PARTS 1
+#endif
+constexpr int kScanParts = TPPO_SCAN_PARTS;
+constexpr int kScan2CtasPerSm = 6;
+template <int H>
+__global__ void __launch_bounds__(kScanThreads, H == 1 ? kScanCtasPerSm : kScan2CtasPerSm)
 egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
                  const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_adv,
                  const __grid_constant__ CUtensorMap map_ret) {
-    __shared__ TileBuf buf;
-    __shared__ TileWin win;
-    __shared__ __align__(8) uint64_t s_bar;      // the tile's inputs have arrived
+    constexpr int kWarpsAll = H * kScanWarps;       // "warps" of the tile, left to right: part p, warp w -> p * 4 + w
+    static_assert(kWarpsAll <= 32, "one lane per warp composite");
+    __shared__ TileBuf buf[H];
+    __shared__ TileWin win[H];
+    __shared__ __align__(8) uint64_t s_bar[H];      // the part's inputs have arrived
     __shared__ uint32_t s_ticket;
-    __shared__ Affine2 s_warp[kScanWarps];
-    __shared__ double s_carry[kScanWarps][2];
+    __shared__ Affine2 s_warp[kWarpsAll];
+    __shared__ double s_carry[kWarpsAll][2];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t bar = ptx::smem_addr(&s_bar);
     if (threadIdx.x == 0) {
 #if TPPO_EGAE_TICKET
-        // the ticket counter starts at all-ones like the rest of the workspace (one memset): + 1
-        // wraps the first draw to ticket 0
+        // the ticket counter starts at all-ones like the rest of the workspace: + 1 wraps the first
+        // draw to ticket 0
         if (a.after_clear) asm volatile("griddepcontrol.wait;" ::: "memory");
         s_ticket = atomicAdd(a.ticket, 1u) + 1u;
 #else
         s_ticket = blockIdx.x;
 #endif
-        ptx::mbar_init(bar, 1);
+#pragma unroll
+        for (int p = 0; p < H; ++p) ptx::mbar_init(ptx::smem_addr(&s_bar[p]), 1);
         ptx::fence_mbar_init_cluster();
     }
     __syncthreads();
     const uint32_t ticket = s_ticket;
     if (ticket >= uint32_t(a.num_tiles)) return;       // (the grid has exactly num_tiles CTAs)
     const int tile = a.num_tiles - 1 - int(ticket);
-    bool nonfinite = false;
-    const int64_t t0 = int64_t(tile) * kScanTile;
-    const int n_tile = int(min(int64_t(kScanTile), int64_t(a.N) - t0));
-    const bool by_tma = a.tma_ok && n_tile == kScanTile;
-    bool bad = false;
+    const int64_t tile0 = int64_t(tile) * (H * kScanTile);
+    bool bad = false, nonfinite = false, copy_late = false;
+    int n_part[H];
+    bool by_tma[H];
+#pragma unroll
+    for (int p = 0; p < H; ++p) {
+        const int64_t left = int64_t(a.N) - (tile0 + int64_t(p) * kScanTile);
+        n_part[p] = int(max(int64_t(0), min(int64_t(kScanTile), left)));
+        by_tma[p] = a.tma_ok && n_part[p] == kScanTile;
+    }
 
-    // ---- inputs: two TMA copies for a whole tile, plain loads for a ragged or unaligned one ------
-    if (by_tma) {
-        if (threadIdx.x == 0) {
+    // ---- inputs: TMA copies for a whole part (rightmost first), plain loads for a ragged or unaligned one
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int p = H - 1; p >= 0; --p) {
+            if (!by_tma[p]) continue;
+            const uint32_t bar = ptx::smem_addr(&s_bar[p]);
             ptx::mbar_arrive_expect_tx(bar, 2 * kScanTile * uint32_t(sizeof(float)));
 #pragma unroll
             for (int bx = 0; bx < kScanBoxes; ++bx) {
-                const int32_t y = int32_t(t0 / kRowPos) + bx * kScanBoxRows;
-                umma::tma_load_2d(ptx::smem_addr(buf.r + bx * kScanBoxRows * kRowPos), &map_r, bar, 0, y);
-                umma::tma_load_2d(ptx::smem_addr(buf.v + bx * kScanBoxRows * kRowPos), &map_v, bar, 0, y);
+                const int32_t y = int32_t((tile0 + int64_t(p) * kScanTile) / kRowPos) + bx * kScanBoxRows;
+                umma::tma_load_2d(ptx::smem_addr(buf[p].r + bx * kScanBoxRows * kRowPos), &map_r, bar, 0, y);
+                umma::tma_load_2d(ptx::smem_addr(buf[p].v + bx * kScanBoxRows * kRowPos), &map_v, bar, 0, y);
             }
         }
-    } else {
-        for (int k = threadIdx.x; k < n_tile; k += kScanThreads) {
-            buf.r[pos_slot(k)] = __ldg(a.rewards + t0 + k);
-            buf.v[pos_slot(k)] = __ldg(a.values + t0 + k);
+    }
+#pragma unroll
+    for (int p = 0; p < H; ++p) {
+        const int64_t t0 = tile0 + int64_t(p) * kScanTile;
+        if (!by_tma[p]) {
+            for (int k = threadIdx.x; k < n_part[p]; k += kScanThreads) {
+                buf[p].r[pos_slot(k)] = __ldg(a.rewards + t0 + k);
+                buf[p].v[pos_slot(k)] = __ldg(a.values + t0 + k);
+            }
         }
+        if (threadIdx.x == kScanThreads - 1)
+            buf[p].v_after = (t0 + n_part[p] < a.N) ? __ldg(a.values + t0 + n_part[p]) : 0.f;
     }
-    if (threadIdx.x == kScanThreads - 1)
-        buf.v_after = (t0 + n_tile < a.N) ? __ldg(a.values + t0 + n_tile) : 0.f;
-    if (warp == 0) {
-        // the segment window was found by the kernel launched just before this one, which lets this
-        // one start at once (programmatic dependent launch): its end is awaited here
+    if (warp < H) {
+        // warp p fetches the segment window of part p.  With a clearing kernel in front (which lets
+        // this kernel start at once: programmatic dependent launch) the windows were found there:
+        // its end is awaited here
         if (a.after_clear) asm volatile("griddepcontrol.wait;" ::: "memory");
-        bad |= egae_window(a, win, t0, n_tile, lane, nonfinite);
+        if (n_part[warp] > 0)
+            bad |= egae_window(a, win[warp], tile0 + int64_t(warp) * kScanTile, n_part[warp], lane, nonfinite,
+                               a.after_clear ? a.state[tile].win + 2 * warp : nullptr);
     }
-    const bool copy_late = by_tma && !ptx::mbar_wait<false>(bar, 0);      // reported once the status word may be touched
+    if (by_tma[H - 1] && !ptx::mbar_wait<false>(ptx::smem_addr(&s_bar[H - 1]), 0)) copy_late = true;
     __syncthreads();
 
-    // ---- the thread's sixteen positions, right to left: its composite map; the warp's scan --------
-    RunState rs{};
-    const Affine2 f = egae_run_map(a, buf, win, t0, n_tile, threadIdx.x, rs, bad, nonfinite);
-    // inclusive suffix composition inside the warp: S_l = f_l o f_{l+1} o ... o f_31
-    Affine2 S = f;
+    // ---- per part, right to left: the thread's sixteen positions, right to left: its composite map;
+    //      the warp's scan
+    RunState rs[H];
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const Affine2 o = shfl_down(S, d);
-        if (lane + d < 32) S = compose(S, o);
+    for (int p = H - 1; p >= 0; --p) {
+        if (p < H - 1 && by_tma[p] && !ptx::mbar_wait<false>(ptx::smem_addr(&s_bar[p]), 0)) copy_late = true;
+        rs[p] = RunState{};
+        Affine2 S = identity2();
+        if (n_part[p] > 0) {
+            S = egae_run_map(a, buf[p], win[p], tile0 + int64_t(p) * kScanTile, n_part[p], threadIdx.x, rs[p],
+                             bad, nonfinite);
+            // inclusive suffix composition inside the warp: S_l = f_l o f_{l+1} o ... o f_31
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const Affine2 o = shfl_down(S, d);
+                if (lane + d < 32) S = compose(S, o);
+            }
+        }
+        rs[p].excl = shfl_down(S, 1);   // composite of the lanes to the right
+        if (lane == 31) rs[p].excl = identity2();
+        if (lane == 0) s_warp[p * kScanWarps + warp] = S;
     }
-    rs.excl = shfl_down(S, 1);   // composite of the lanes to the right
-    if (lane == 31) rs.excl = identity2();
-    if (lane == 0) s_warp[warp] = S;
-    // Everything above read inputs only.  The status word and the tile states are cleared by the
-    // small kernel launched just before this one, which lets this one start at once (programmatic
-    // dependent launch): its end is awaited here, before the first word of either is touched.
+    // Everything above read inputs only (and the windows).  The status word and the tile states are
+    // cleared by the kernel in front: its end is awaited here by every thread, before the first word
+    // of either is touched.
     if (a.after_clear) asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();                                                      // (A)
 
     // ---- tile composite, look-back, per-warp carries (warp 0) ------------------------------------
     if (warp == 0) {
-        // lane w < 4 holds warp w's composite; suffix-compose them, so that lane w ends with
-        // W_w o ... o W_3 and lane 0 with the tile's composite
-        Affine2 W = lane < kScanWarps ? s_warp[lane] : identity2();
+        // lane j < kWarpsAll holds the composite of "warp" j; suffix-compose them, so that lane j
+        // ends with W_j o ... o W_last and lane 0 with the tile's composite
+        Affine2 W = lane < kWarpsAll ? s_warp[lane] : identity2();
 #pragma unroll
-        for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
+        for (int d = 1; d < kWarpsAll; d <<= 1) W = compose(W, shfl_down(W, d));
         Affine2 right = shfl_down(W, 1);            // composite of the warps to the right
-        if (lane >= kScanWarps - 1) right = identity2();
+        if (lane >= kWarpsAll - 1) right = identity2();
         TileState* st = a.state;
         const bool publish = lane == 0 && !a.no_publish;
         if (publish && tile + 1 < a.num_tiles) {
@@ -783,7 +831,7 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
         }
         xA = __shfl_sync(0xffffffffu, xA, 0);
         xR = __shfl_sync(0xffffffffu, xR, 0);
-        if (lane < kScanWarps) {
+        if (lane < kWarpsAll) {
             s_carry[lane][0] = fma(right.aA, xA, right.bA);
             s_carry[lane][1] = fma(right.aR, xR, right.bR);
         }
@@ -791,254 +839,39 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     __syncthreads();                                                      // (B)
 
     // ---- replay the thread's positions from the true incoming values, store -----------------------
-    const float G = float(fma(rs.excl.aA, s_carry[warp][0], rs.excl.bA));
-    const float R = float(fma(rs.excl.aR, s_carry[warp][1], rs.excl.bR));
-    egae_run_replay(a, buf, win, t0, n_tile, threadIdx.x, rs, G, R, by_tma, bad, nonfinite);
+#pragma unroll
+    for (int p = H - 1; p >= 0; --p) {
+        if (n_part[p] <= 0) continue;
+        const double* c = s_carry[p * kScanWarps + warp];
+        const float G = float(fma(rs[p].excl.aA, c[0], rs[p].excl.bA));
+        const float R = float(fma(rs[p].excl.aR, c[1], rs[p].excl.bR));
+        egae_run_replay(a, buf[p], win[p], tile0 + int64_t(p) * kScanTile, n_part[p], threadIdx.x, rs[p], G, R,
+                        by_tma[p], bad, nonfinite);
+    }
     if (bad) egae_raise(a, TPPO_DEV_BAD_SEGMENT);
     if (nonfinite) egae_raise(a, TPPO_DEV_NONFINITE);
     if (copy_late) egae_raise(a, TPPO_DEV_WAIT_TIMEOUT);
-    if (by_tma) {
+    bool any_tma = false;
+#pragma unroll
+    for (int p = 0; p < H; ++p) any_tma |= by_tma[p];
+    if (any_tma) {
         ptx::fence_proxy_async_smem();       // the TMA stores read what was just written
         __syncthreads();
         if (threadIdx.x == 0) {
 #pragma unroll
-            for (int bx = 0; bx < kScanBoxes; ++bx) {
-                const int32_t y = tile * (kScanTile / kRowPos) + bx * kScanBoxRows;
-                umma::tma_store_2d(&map_adv, ptx::smem_addr(buf.v + bx * kScanBoxRows * kRowPos), 0, y);
-                if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(buf.r + bx * kScanBoxRows * kRowPos), 0, y);
+            for (int p = 0; p < H; ++p) {
+                if (!by_tma[p]) continue;
+#pragma unroll
+                for (int bx = 0; bx < kScanBoxes; ++bx) {
+                    const int32_t y = int32_t((tile0 + int64_t(p) * kScanTile) / kRowPos) + bx * kScanBoxRows;
+                    umma::tma_store_2d(&map_adv, ptx::smem_addr(buf[p].v + bx * kScanBoxRows * kRowPos), 0, y);
+                    if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(buf[p].r + bx * kScanBoxRows * kRowPos), 0, y);
+                }
             }
             ptx::bulk_commit();
             ptx::bulk_wait_read<0>();   // shared memory must outlive the stores' reads of it
         }
     }
-}
-
-// ---- the same scan by resident CTAs with specialised warps ---------------------------------------------
-// In the kernel above a tile's life is a chain of latencies (copy, maps, publish, look-back, replay,
-// store), three of its four warps wait at barriers while warp 0 looks back, and registers allow
-// eight tiles per SM: the SM's issue slots and the DRAM are both idle two thirds of the time.  Here a
-// CTA stays resident, takes tile after tile by ticket, holds three tile images, and splits the work
-// of a step between its warps so that the latencies of different tiles overlap:
-//   step k, first half:   compute warps  maps of tile k, warp scans
-//                         chain warp     look-back for tile k-1 (its neighbours published their
-//                                        composites a step ago: one round of loads), value entering
-//                                        it published, carries of its warps
-//                         mover warp     results of tile k-2 stored, its image reused for the copy of
-//                                        tile k+1 (needed one whole step later)
-//           second half:  compute warps  replay of tile k-1 into its image
-//                         chain warp     composite of tile k from the warps' composites, published
-//                         mover warp     ticket for step k+2, segment window of tile k+1
-// Forward progress: tickets are drawn by running CTAs only and a tile waits only for tiles with
-// lower tickets; a CTA publishes the composite of its tile k after the look-back of its tile k-1,
-// which has a lower ticket, so the lowest unfinished ticket never waits for a higher one.
-constexpr int kResThreads = kScanThreads + 64;     // compute warps + chain warp + mover warp
-constexpr int kResCtasPerSm = 4;
-constexpr int kResBufs = 3;
-constexpr int kResRing = 8;                        // tile numbers of steps k-2 .. k+2
-constexpr uint32_t kTileBytes = 2 * kScanTile * uint32_t(sizeof(float));
-struct ResShared {
-    TileBuf buf[kResBufs];
-    TileWin win[4];                                // steps k-1, k, k+1
-    uint64_t full[kResBufs];                       // the inputs of the tile in image b have arrived
-    int tile[kResRing];                            // tile of step k (ring), -1: none left
-    Affine2 warp_comp[kScanWarps];                 // composites of the warps of tile k
-    Affine2 right[kScanWarps];                     // of tile k: composite of the warps to the right of each warp
-    Affine2 whole;                                 // of tile k: the tile's composite
-    double carry[kScanWarps][2];                   // of tile k-1: values entering each warp
-};
-constexpr size_t kResSmemBytes = sizeof(ResShared) + 1024;      // + room to align the images
-
-__global__ void __launch_bounds__(kResThreads, kResCtasPerSm)
-egae_resident_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
-                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_adv,
-                     const __grid_constant__ CUtensorMap map_ret) {
-    extern __shared__ unsigned char res_smem_raw[];
-    ResShared& sh = *reinterpret_cast<ResShared*>(
-        (reinterpret_cast<uintptr_t>(res_smem_raw) + 1023) & ~uintptr_t(1023));
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    bool bad = false, nonfinite = false, late = false;
-
-    auto draw = [&]() -> int {       // the next tile from the end of the arrays, or -1
-        const uint32_t t = atomicAdd(a.ticket, 1u) + 1u;      // the counter starts at all-ones
-        return t < uint32_t(a.num_tiles) ? a.num_tiles - 1 - int(t) : -1;
-    };
-    auto tile_len = [&](int tile) { return int(min(int64_t(kScanTile), int64_t(a.N) - int64_t(tile) * kScanTile)); };
-    auto whole_tile = [&](int tile) { return tile_len(tile) == kScanTile; };       // copied and stored by TMA
-    // one lane: the copy of a whole tile into image b; another lane fetches the value after the tile
-    auto request = [&](int b, int tile) {
-        TileBuf& buf = sh.buf[b];
-        if (lane == 0 && whole_tile(tile)) {
-            const uint32_t bar = ptx::smem_addr(&sh.full[b]);
-            ptx::mbar_arrive_expect_tx(bar, kTileBytes);
-#pragma unroll
-            for (int bx = 0; bx < kScanBoxes; ++bx) {
-                const int32_t y = tile * (kScanTile / kRowPos) + bx * kScanBoxRows;
-                umma::tma_load_2d(ptx::smem_addr(buf.r + bx * kScanBoxRows * kRowPos), &map_r, bar, 0, y);
-                umma::tma_load_2d(ptx::smem_addr(buf.v + bx * kScanBoxRows * kRowPos), &map_v, bar, 0, y);
-            }
-        }
-        if (lane == 1) {
-            const int64_t after = int64_t(tile) * kScanTile + tile_len(tile);
-            buf.v_after = after < a.N ? __ldg(a.values + after) : 0.f;
-        }
-    };
-
-    // the ticket counter, the tile states and the segment windows are written by the kernel launched
-    // just before this one
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (warp == kScanWarps + 1) {
-        int t0 = -1, t1 = -1;
-        if (lane == 0) {
-#pragma unroll
-            for (int b = 0; b < kResBufs; ++b) ptx::mbar_init(ptx::smem_addr(&sh.full[b]), 1);
-            ptx::fence_mbar_init_cluster();
-            t0 = draw();
-            t1 = t0 >= 0 ? draw() : -1;
-            sh.tile[0] = t0; sh.tile[1] = t1;
-#pragma unroll
-            for (int i = 2; i < kResRing; ++i) sh.tile[i] = -1;
-        }
-        t0 = __shfl_sync(0xffffffffu, t0, 0);
-        if (t0 >= 0) {
-            request(0, t0);
-            bad |= egae_window(a, sh.win[0], int64_t(t0) * kScanTile, tile_len(t0), lane, nonfinite);
-        }
-    }
-    __syncthreads();
-
-    // Each kind of warp runs its own loop (its registers hold only what its own work needs); all
-    // loops make the same two barrier calls per step and leave after the same step, which every
-    // thread reads from the ring of tile numbers.
-    auto step_barrier = [] { asm volatile("bar.sync 0, %0;" ::"n"(kResThreads) : "memory"); };
-    struct Step { int tile, ptile, pptile, ntile; bool done; };
-    auto step_of = [&](int k) {
-        Step st;
-        st.tile = sh.tile[k & (kResRing - 1)];
-        st.ptile = k >= 1 ? sh.tile[(k - 1) & (kResRing - 1)] : -1;
-        st.pptile = k >= 2 ? sh.tile[(k - 2) & (kResRing - 1)] : -1;
-        st.ntile = sh.tile[(k + 1) & (kResRing - 1)];
-        st.done = st.tile < 0 && st.ptile < 0 && st.pptile < 0;
-        return st;
-    };
-    // images: step k in k % 3, step k-1 in (k+2) % 3, steps k+1 and k-2 in (k+1) % 3
-
-    if (warp < kScanWarps) {
-        // ---- compute warps: maps of tile k | replay of tile k-1 --------------------------------------
-        RunState cur{}, prev{};
-        uint32_t phases = 0;      // bit b: parity of the phase barrier b completes next (a ragged tile arms none)
-#pragma unroll 1
-        for (int k = 0;; ++k) {
-            const Step st = step_of(k);
-            if (st.done) break;
-            if (st.tile >= 0) {
-                const int bk = k % kResBufs;
-                TileBuf& buf = sh.buf[bk];
-                const int64_t t0 = int64_t(st.tile) * kScanTile;
-                const int n_tile = tile_len(st.tile);
-                if (n_tile == kScanTile) {
-                    if (!ptx::mbar_wait<false>(ptx::smem_addr(&sh.full[bk]), (phases >> bk) & 1u)) late = true;
-                    phases ^= 1u << bk;
-                } else {      // the ragged tile: plain loads, then a barrier among the compute warps
-                    for (int q = tid; q < n_tile; q += kScanThreads) {
-                        buf.r[pos_slot(q)] = __ldg(a.rewards + t0 + q);
-                        buf.v[pos_slot(q)] = __ldg(a.values + t0 + q);
-                    }
-                    asm volatile("bar.sync 1, %0;" ::"n"(kScanThreads) : "memory");
-                }
-                const Affine2 f = egae_run_map(a, buf, sh.win[k & 3], t0, n_tile, tid, cur, bad, nonfinite);
-                Affine2 S = f;
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const Affine2 o = shfl_down(S, d);
-                    if (lane + d < 32) S = compose(S, o);
-                }
-                cur.excl = shfl_down(S, 1);
-                if (lane == 31) cur.excl = identity2();
-                if (lane == 0) sh.warp_comp[warp] = S;
-            }
-            step_barrier();
-            if (st.ptile >= 0) {
-                const int64_t pt0 = int64_t(st.ptile) * kScanTile;
-                const int pn = tile_len(st.ptile);
-                const bool p_tma = pn == kScanTile;
-                const float G = float(fma(prev.excl.aA, sh.carry[warp][0], prev.excl.bA));
-                const float R = float(fma(prev.excl.aR, sh.carry[warp][1], prev.excl.bR));
-                egae_run_replay(a, sh.buf[(k + 2) % kResBufs], sh.win[(k - 1) & 3], pt0, pn, tid, prev, G, R, p_tma, bad, nonfinite);
-                if (p_tma) ptx::fence_proxy_async_smem();       // the TMA stores read what was just written
-            }
-            prev = cur;
-            step_barrier();
-        }
-    } else if (warp == kScanWarps) {
-        // ---- chain warp: look-back for tile k-1 | composite of tile k ----------------------------------
-#pragma unroll 1
-        for (int k = 0;; ++k) {
-            const Step st = step_of(k);
-            if (st.done) break;
-            if (st.ptile >= 0) {     // the value entering the tile of the step before
-                double xA = 0.0, xR = 0.0;
-                const bool ok = egae_look_back(a, st.ptile + 1, lane, xA, xR);
-                if (lane == 0) {
-                    if (!ok) { late = true; xA = 0.0; xR = 0.0; }
-                    const Affine2 W = sh.whole;
-                    if (!a.no_publish) st_pair(a.state[st.ptile].inc, fma(W.aA, xA, W.bA), fma(W.aR, xR, W.bR));
-                }
-                xA = __shfl_sync(0xffffffffu, xA, 0);
-                xR = __shfl_sync(0xffffffffu, xR, 0);
-                if (lane < kScanWarps) {
-                    const Affine2 right = sh.right[lane];
-                    sh.carry[lane][0] = fma(right.aA, xA, right.bA);
-                    sh.carry[lane][1] = fma(right.aR, xR, right.bR);
-                }
-            }
-            step_barrier();
-            if (st.tile >= 0) {      // composite of the tile from its warps' composites, published
-                Affine2 W = lane < kScanWarps ? sh.warp_comp[lane] : identity2();
-#pragma unroll
-                for (int d = 1; d < kScanWarps; d <<= 1) W = compose(W, shfl_down(W, d));
-                Affine2 right = shfl_down(W, 1);
-                if (lane >= kScanWarps - 1) right = identity2();
-                if (lane < kScanWarps) sh.right[lane] = right;
-                if (lane == 0) {
-                    sh.whole = W;
-                    if (!a.no_publish && st.tile + 1 < a.num_tiles) {
-                        st_pair(a.state[st.tile].aggA, W.aA, W.bA);
-                        st_pair(a.state[st.tile].aggR, W.aR, W.bR);
-                    }
-                }
-            }
-            step_barrier();
-        }
-    } else {
-        // ---- mover warp: results of tile k-2 out, inputs of tile k+1 in | next ticket and window ------
-#pragma unroll 1
-        for (int k = 0;; ++k) {
-            const Step st = step_of(k);
-            if (st.done) break;
-            const int bn = (k + 1) % kResBufs;
-            if (st.pptile >= 0 && whole_tile(st.pptile) && lane == 0) {
-                TileBuf& obuf = sh.buf[bn];
-#pragma unroll
-                for (int bx = 0; bx < kScanBoxes; ++bx) {
-                    const int32_t y = st.pptile * (kScanTile / kRowPos) + bx * kScanBoxRows;
-                    umma::tma_store_2d(&map_adv, ptx::smem_addr(obuf.v + bx * kScanBoxRows * kRowPos), 0, y);
-                    if (a.ret) umma::tma_store_2d(&map_ret, ptx::smem_addr(obuf.r + bx * kScanBoxRows * kRowPos), 0, y);
-                }
-                ptx::bulk_commit();
-                ptx::bulk_wait_read<0>();       // the image is free once the stores have read it
-            }
-            __syncwarp();
-            if (st.ntile >= 0) request(bn, st.ntile);
-            step_barrier();
-            if (lane == 0) sh.tile[(k + 2) & (kResRing - 1)] = (st.tile >= 0 && st.ntile >= 0) ? draw() : -1;
-            if (st.ntile >= 0)
-                bad |= egae_window(a, sh.win[(k + 1) & 3], int64_t(st.ntile) * kScanTile, tile_len(st.ntile), lane, nonfinite);
-            step_barrier();
-        }
-    }
-    if (bad) egae_raise(a, TPPO_DEV_BAD_SEGMENT);
-    if (nonfinite) egae_raise(a, TPPO_DEV_NONFINITE);
-    if (late) egae_raise(a, TPPO_DEV_WAIT_TIMEOUT);
 }
 
 bool make_f32_rows_tensor_map(CUtensorMap* map, const void* base, uint64_t rows);
@@ -1062,45 +895,67 @@ __device__ __forceinline__ int count_le(const int32_t* __restrict__ arr, int n, 
 
 // Launched just before the scan, which is its programmatic dependent and starts beside it: status
 // word to 0, ticket counter to all-ones, and one thread per tile sets the tile's state to unset
-// (all-ones) and finds its segment window, so that a tile of the scan reads its window instead of
+// (all-ones) and finds the segment window of each of its parts, so that the scan reads a window instead of
 // searching for it: the search (three dependent rounds of global loads by one warp) was the longest
 // latency of a tile's first phase, longer than the copy of its inputs.  Here a block first copies the
 // segment bounds into shared memory (2 x 4 x B bytes, one round of loads) and searches there; bounds
 // that do not fit are searched in global memory.
-constexpr int kClearThreads = 128;
+constexpr int kClearThreads = 256;
 constexpr int kClearSmemMaxB = 12288;       // 96 KB of segment bounds
 __global__ void __launch_bounds__(kClearThreads) egae_clear_kernel(int32_t* status, uint4* head,
                                                                    TileState* state, int num_tiles,
                                                                    const int32_t* seg_begin,
                                                                    const int32_t* seg_end, int B,
-                                                                   int64_t N, int in_smem) {
-    extern __shared__ int32_t s_bounds[];      // seg_end[0..B), seg_begin[0..B)
+                                                                   int64_t N, int in_smem, int parts) {
+    extern __shared__ __align__(16) int32_t s_bounds[];      // seg_end[0..B), seg_begin[0..B)
     asm volatile("griddepcontrol.launch_dependents;");
     const int tile = blockIdx.x * blockDim.x + threadIdx.x;
     if (tile == 0) *status = 0;
     if (tile < int(kScanHeadBytes / 16)) head[tile] = make_uint4(~0u, ~0u, ~0u, ~0u);
     if (in_smem) {
-        for (int i = threadIdx.x; i < B; i += kClearThreads) {
-            s_bounds[i] = __ldg(seg_end + i);
-            s_bounds[B + i] = __ldg(seg_begin + i);
+        // 16-byte loads where the arrays allow it, all of a thread's loads in flight together
+        const bool vec = ((reinterpret_cast<uintptr_t>(seg_end) | reinterpret_cast<uintptr_t>(seg_begin)) & 15) == 0 &&
+                         (B & 3) == 0;
+        if (vec) {
+            const int4* e4 = reinterpret_cast<const int4*>(seg_end);
+            const int4* b4 = reinterpret_cast<const int4*>(seg_begin);
+            int4* se = reinterpret_cast<int4*>(s_bounds);
+            int4* sb = reinterpret_cast<int4*>(s_bounds + B);
+#pragma unroll 4
+            for (int i = threadIdx.x; i < B / 4; i += kClearThreads) {
+                se[i] = __ldg(e4 + i);
+                sb[i] = __ldg(b4 + i);
+            }
+        } else {
+            for (int i = threadIdx.x; i < B; i += kClearThreads) {
+                s_bounds[i] = __ldg(seg_end + i);
+                s_bounds[B + i] = __ldg(seg_begin + i);
+            }
         }
         __syncthreads();
     }
     if (tile >= num_tiles) return;
-    const int64_t t0 = int64_t(tile) * kScanTile;
-    const int64_t t_last = min(t0 + kScanTile, N) - 1;
-    const int lo = in_smem ? count_le<false>(s_bounds, B, int32_t(t0)) : count_le<true>(seg_end, B, int32_t(t0));
-    const int hi = in_smem ? count_le<false>(s_bounds + B, B, int32_t(t_last))
-                           : count_le<true>(seg_begin, B, int32_t(t_last));
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+    for (int p = 0; p < parts; ++p) {       // parts <= 2
+        const int64_t t0 = (int64_t(tile) * parts + p) * kScanTile;
+        if (t0 >= N) break;
+        const int64_t t_last = min(t0 + kScanTile, N) - 1;
+        w[2 * p] = uint32_t(in_smem ? count_le<false>(s_bounds, B, int32_t(t0)) : count_le<true>(seg_end, B, int32_t(t0)));
+        w[2 * p + 1] = uint32_t(in_smem ? count_le<false>(s_bounds + B, B, int32_t(t_last))
+                                        : count_le<true>(seg_begin, B, int32_t(t_last)));
+    }
     uint4* st = reinterpret_cast<uint4*>(state + tile);
     st[0] = make_uint4(~0u, ~0u, ~0u, ~0u);
     st[1] = make_uint4(~0u, ~0u, ~0u, ~0u);
     st[2] = make_uint4(~0u, ~0u, ~0u, ~0u);
-    st[3] = make_uint4(uint32_t(lo), uint32_t(hi), 0u, 0u);
+    st[3] = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+
+
 static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
-    a.num_tiles = int32_t((int64_t(a.N) + kScanTile - 1) / kScanTile);
+    constexpr int parts = kScanParts;
+    a.num_tiles = int32_t((int64_t(a.N) + parts * kScanTile - 1) / (parts * kScanTile));
     a.gamma = double(gamma);
     a.gl = double(gamma) * double(lambda);
     a.gamma_run = 1.0; a.gl_run = 1.0;
@@ -1135,21 +990,7 @@ static int egae_launch(EgaeArgs& a, float gamma, float lambda, cudaStream_t s) {
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = a.after_clear ? 1 : 0;
-#ifndef TPPO_EGAE_RESIDENT_MIN_TILES
-#define TPPO_EGAE_RESIDENT_MIN_TILES (2 * kNumSms * kResCtasPerSm)
-#endif
-    // enough whole tiles to keep resident CTAs busy for several steps each: warp-specialised resident
-    // CTAs; otherwise one CTA per tile
-    if (a.after_clear && a.tma_ok && a.num_tiles >= TPPO_EGAE_RESIDENT_MIN_TILES) {
-        TPPO_CUDA_CHECK(cudaFuncSetAttribute(egae_resident_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             int(kResSmemBytes)));
-        cfg.gridDim = dim3(unsigned(std::min(a.num_tiles, kNumSms * kResCtasPerSm)));
-        cfg.blockDim = dim3(kResThreads);
-        cfg.dynamicSmemBytes = kResSmemBytes;
-        TPPO_CUDA_CHECK(cudaLaunchKernelEx(&cfg, egae_resident_kernel, a, map_r, map_v, map_adv, map_ret));
-        return TPPO_OK;
-    }
-    TPPO_CUDA_CHECK(cudaLaunchKernelEx(&cfg, egae_scan_kernel, a, map_r, map_v, map_adv, map_ret));
+    TPPO_CUDA_CHECK(cudaLaunchKernelEx(&cfg, egae_scan_kernel<kScanParts>, a, map_r, map_v, map_adv, map_ret));
     return TPPO_OK;
 }
 
@@ -1192,7 +1033,8 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
     // tile's end.)
     {
         static_assert(kScanHeadBytes / 16 <= kClearThreads, "the first block writes the head");
-        const int tiles = int((N + kScanTile - 1) / kScanTile);
+        constexpr int parts = kScanParts;
+        const int tiles = int((N + parts * kScanTile - 1) / (parts * kScanTile));
         const int in_smem = B <= kClearSmemMaxB;
         const size_t smem = in_smem ? size_t(2) * size_t(B) * sizeof(int32_t) : 0;
         if (smem > 48 * 1024)       // (an attribute of the function on the current device; the call is cheap)
@@ -1201,7 +1043,7 @@ TPPO_API int tppo_egae(const float* rewards, const float* values, const int32_t*
         egae_clear_kernel<<<(tiles + kClearThreads - 1) / kClearThreads, kClearThreads, smem, s>>>(
             status, static_cast<uint4*>(workspace),
             reinterpret_cast<TileState*>(static_cast<char*>(workspace) + kScanHeadBytes), tiles,
-            seg_begin, seg_end, B, N, in_smem);
+            seg_begin, seg_end, B, N, in_smem, parts);
         TPPO_CUDA_CHECK(cudaGetLastError());
     }
     EgaeArgs a{};

@@ -280,6 +280,8 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     if (bad) atomicOr(a.counts + 2, bad);
     // compact inside the tile (needs no global offset; earlier tiles finish meanwhile)
     {
+        // (one loop over both lists, trip count the larger popcount instead of their sum, measured
+        // slower: 43.3 against 41.0 us per call at 17.5 M tokens)
         uint32_t op = before & 0xffffu, ov = before >> 16;
         uint32_t b = pol_bits;
         while (b) { s_out_pol[op++] = uint16_t(l0 + __ffs(int(b)) - 1); b &= b - 1; }
