@@ -708,26 +708,33 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
     __shared__ TileBuf buf[H];
     __shared__ TileWin win[H];
     __shared__ __align__(8) uint64_t s_bar[H];      // the part's inputs have arrived
+#if TPPO_EGAE_TICKET
     __shared__ uint32_t s_ticket;
+#endif
     __shared__ Affine2 s_warp[kWarpsAll];
     __shared__ double s_carry[kWarpsAll][2];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) {
 #if TPPO_EGAE_TICKET
+    if (threadIdx.x == 0) {
         // the ticket counter starts at all-ones like the rest of the workspace: + 1 wraps the first
         // draw to ticket 0
         if (a.after_clear) asm volatile("griddepcontrol.wait;" ::: "memory");
         s_ticket = atomicAdd(a.ticket, 1u) + 1u;
+    }
+    __syncthreads();
+    const uint32_t ticket = s_ticket;
 #else
-        s_ticket = blockIdx.x;
+    const uint32_t ticket = blockIdx.x;
 #endif
+    // Thread 0 initialises the copy barriers and issues the copies at once; the other threads first
+    // touch a barrier after the block-wide barrier below (one barrier less in every tile's life, and
+    // the copies start that much earlier).
+    if (threadIdx.x == 0) {
 #pragma unroll
         for (int p = 0; p < H; ++p) ptx::mbar_init(ptx::smem_addr(&s_bar[p]), 1);
         ptx::fence_mbar_init_cluster();
     }
-    __syncthreads();
-    const uint32_t ticket = s_ticket;
     if (ticket >= uint32_t(a.num_tiles)) return;       // (the grid has exactly num_tiles CTAs)
     const int tile = a.num_tiles - 1 - int(ticket);
     const int64_t tile0 = int64_t(tile) * (H * kScanTile);
@@ -777,8 +784,8 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
             bad |= egae_window(a, win[warp], tile0 + int64_t(warp) * kScanTile, n_part[warp], lane, nonfinite,
                                a.after_clear ? a.state[tile].win + 2 * warp : nullptr);
     }
-    if (by_tma[H - 1] && !ptx::mbar_wait<false>(ptx::smem_addr(&s_bar[H - 1]), 0)) copy_late = true;
     __syncthreads();
+    if (by_tma[H - 1] && !ptx::mbar_wait<false>(ptx::smem_addr(&s_bar[H - 1]), 0)) copy_late = true;
 
     // ---- per part, right to left: the thread's sixteen positions, right to left: its composite map;
     //      the warp's scan
