@@ -1144,7 +1144,7 @@ def run_config_table(args, dev):
         oracle.value_loss(c1["values"], c1["old_values"], r_.astype(np.float32), v_, f32(0.5), f32(0.6))
     o = (time.perf_counter() - w0) / 20
     out["cfg1"] = {"n_selected": int(cnt[0]), "gpu_step_us": {k: v * 1e3 for k, v in g.items()},
-                   "oracle_step_ms": o * 1e3, "note": "whole path, V=1000 fp32; latency-bound (13 launches)"}
+                   "oracle_step_ms": o * 1e3, "note": "whole path, V=1000 fp32; latency-bound (9 kernel launches, no memsets)"}
     # ---- config 2 -----------------------------------------------------------------------------------
     c2 = synth.config2(dev)
     res2 = {}

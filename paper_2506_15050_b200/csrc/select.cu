@@ -31,38 +31,6 @@ __device__ __forceinline__ uint32_t sel_flag(uint64_t s) { return uint32_t(s >> 
 __device__ __forceinline__ uint32_t sel_pol(uint64_t s) { return uint32_t(s >> 31) & 0x7fffffffu; }
 __device__ __forceinline__ uint32_t sel_val(uint64_t s) { return uint32_t(s) & 0x7fffffffu; }
 
-// Number of entries of the ascending array arr[0..n) that are <= key, found by a whole warp: each
-// round probes 32 evenly spaced entries (one load per lane) and narrows the range 32-fold until at
-// most 128 entries remain, which are read in one go (four independent loads per lane): 4097
-// entries take two dependent rounds.  Every lane returns the same count; an array that is not
-// ascending still yields an in-range answer.
-__device__ __forceinline__ int warp_count_le(const int32_t* __restrict__ arr, int n, int32_t key,
-                                             int lane) {
-    int lo = 0, hi = n;       // the answer lies in [lo, hi]
-    while (hi - lo > 128) {
-        const int span = hi - lo;
-        const int step = (span + 31) >> 5;
-        const int idx = lo + lane * step;
-        const bool le = idx < hi && __ldg(arr + idx) <= key;
-        const uint32_t m = __ballot_sync(0xffffffffu, le);
-        const int c = __ffs(int(~m)) - 1;          // leading run of probes that are <= key
-        if (c < 0) { lo = min(lo + 31 * step + 1, hi); continue; }
-        const int new_hi = min(lo + c * step, hi);
-        if (c > 0) lo = lo + (c - 1) * step + 1;
-        hi = new_hi;
-    }
-    bool le[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int idx = lo + 32 * j + lane;
-        le[j] = idx < hi && __ldg(arr + idx) <= key;
-    }
-    int count = 0;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) count += __popc(__ballot_sync(0xffffffffu, le[j]));
-    return lo + count;
-}
-
 struct SelectArgs {
     const int32_t* seq_begin;
     const int32_t* prompt_len;
@@ -81,6 +49,7 @@ struct SelectArgs {
     int32_t* value_idx;
     int32_t* counts;            // [4]
     unsigned long long* state;  // [num_tiles]
+    const int2* window;         // [num_tiles]: (seq0, seq1) of every tile, found by the clearing kernel
     uint32_t* ticket;           // head of the workspace, cleared to zero together with the tile states
     uint32_t spin_limit;        // polls a look-back round may take before it gives up
     int32_t no_publish;         // test hook: tiles keep their totals to themselves
@@ -144,7 +113,6 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     __shared__ uint16_t s_out_val[kSelTile];
     __shared__ int32_t s_sb[kSeqCap + 1];
     __shared__ uint32_t s_tile;
-    __shared__ int s_seq0, s_seq1;
     __shared__ uint32_t s_warp_cnt[kSelWarps];      // policy count | value count << 16
     __shared__ uint32_t s_base_pol, s_base_val, s_tot_pol, s_tot_val;
     int bad = 0;
@@ -190,15 +158,12 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     const uint32_t own_bits = n_mine >= kSelItems ? 0xffffffffu : ((1u << n_mine) - 1u);
 
     // ---- window of sequences that can touch the tile: [seq0, seq1), seq0 may be -1 -------------
-    if (warp == 0) {
-        const int c = warp_count_le(a.seq_begin, a.B + 1, int32_t(t0), lane);
-        if (lane == 0) s_seq0 = c - 1;
-    } else if (warp == 1) {
-        const int c = warp_count_le(a.seq_begin, a.B + 1, int32_t(t0 + n_tile - 1), lane);
-        if (lane == 0) s_seq1 = c;     // sequences with index < c begin at or before the last position
-    }
-    __syncthreads();
-    const int seq0 = s_seq0, seq1 = s_seq1;
+    // Found for every tile by the small kernel launched just before this one (which also clears the
+    // counts and the tile states and lets this kernel start at once: programmatic dependent launch).
+    // Its end is awaited here; the mask loads above are in flight meanwhile.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int2 w = __ldcg(a.window + tile);
+    const int seq0 = w.x, seq1 = w.y;
     const int first = max(seq0, 0);
     const int n_win = min(seq1, a.B) - first + 1;         // entries first .. min(seq1, B) inclusive
     const bool win_smem = n_win <= kSeqCap + 1;
@@ -269,10 +234,6 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
         if (w < warp) before += c;
         tile_tot += c;
     }
-    // Everything above read inputs only.  The counts and the tile states are cleared by the small
-    // kernel launched just before this one, which lets this one start at once (programmatic
-    // dependent launch): its end is awaited here, before the first word of either is touched.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     // publish the tile's totals as early as possible: later tiles wait for them in their look-back
     if (threadIdx.x == 0 && tile > 0 && !a.no_publish)
         reinterpret_cast<volatile unsigned long long*>(a.state)[tile] =
@@ -334,17 +295,50 @@ __global__ void __launch_bounds__(kSelThreads) select_tokens_kernel(const Select
     sel_copy_out(a.value_idx, s_base_val, int(s_tot_val), s_out_val, int32_t(t0), a.out_vec_ok != 0);
 }
 
-// Clears the counts and the workspace of one call; the selection kernel is its programmatic dependent.
-__global__ void __launch_bounds__(256) select_clear_kernel(int32_t* counts, uint4* ws, size_t n16) {
+// Launched just before the selection kernel, which is its programmatic dependent: clears the
+// counts, the ticket counter and the tile states, and one thread per tile finds the tile's window
+// of sequences -- seq0 = the last sequence that begins at or before the tile's first position (-1:
+// none), seq1 = the number of sequences that begin at or before its last position -- by two searches
+// over the sequence starts staged in shared memory (starts that do not fit are searched in global
+// memory).  A search per tile inside the selection kernel was three dependent rounds of global loads
+// in every tile's life.
+constexpr int kSelClearThreads = 256;
+constexpr int kSelClearSmemMaxB = 24575;      // 96 KB of sequence starts
+template <bool LDG>
+__device__ __forceinline__ int sel_count_le(const int32_t* __restrict__ arr, int n, int32_t key) {
+    int lo = 0, hi = n;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if ((LDG ? __ldg(arr + mid) : arr[mid]) <= key) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+__global__ void __launch_bounds__(kSelClearThreads) select_clear_kernel(
+        int32_t* counts, uint32_t* ticket, unsigned long long* state, int2* window, int num_tiles,
+        const int32_t* seq_begin, int B, int64_t N, int in_smem) {
+    extern __shared__ __align__(16) int32_t s_starts[];      // seq_begin[0..B]
     asm volatile("griddepcontrol.launch_dependents;");
-    if (blockIdx.x == 0 && threadIdx.x < 4) counts[threadIdx.x] = 0;
-    for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n16; i += size_t(gridDim.x) * blockDim.x)
-        ws[i] = make_uint4(0u, 0u, 0u, 0u);
+    const int tile = blockIdx.x * blockDim.x + threadIdx.x;
+    if (tile < 4) counts[tile] = 0;
+    if (tile == 0) *ticket = 0u;
+    if (in_smem) {
+        for (int i = threadIdx.x; i <= B; i += kSelClearThreads) s_starts[i] = __ldg(seq_begin + i);
+        __syncthreads();
+    }
+    if (tile >= num_tiles) return;
+    const int64_t t0 = int64_t(tile) * kSelTile;
+    const int64_t t_last = min(t0 + kSelTile, N) - 1;
+    const int c0 = in_smem ? sel_count_le<false>(s_starts, B + 1, int32_t(t0)) : sel_count_le<true>(seq_begin, B + 1, int32_t(t0));
+    const int c1 = in_smem ? sel_count_le<false>(s_starts, B + 1, int32_t(t_last))
+                           : sel_count_le<true>(seq_begin, B + 1, int32_t(t_last));
+    state[tile] = 0ull;
+    window[tile] = make_int2(c0 - 1, c1);
 }
 
 size_t select_workspace_bytes(int64_t N) {
     const int64_t tiles = (N + kSelTile - 1) / kSelTile;
-    return kWsAlign + align_up(size_t(tiles > 0 ? tiles : 1) * 8, kWsAlign);
+    // head (ticket counter) | tile states | tile windows
+    return kWsAlign + 2 * align_up(size_t(tiles > 0 ? tiles : 1) * 8, kWsAlign);
 }
 uint32_t test_spin_limit(uint32_t normal);
 int32_t test_no_publish();
@@ -378,10 +372,18 @@ TPPO_API int tppo_select_tokens(const int32_t* seq_begin, const int32_t* prompt_
     // it, reading masks and sequence bounds until it first needs either.  (Two memsets in front of a
     // plain launch cost 6 us more at 17.5 M tokens; handing the counts over by the last tile to
     // finish, to save the clear altogether, cost 6 us for the fence and counter at every tile's end.)
+    const int32_t tiles = int32_t((N + kSelTile - 1) / kSelTile);
+    unsigned long long* state = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWsAlign);
+    int2* window = reinterpret_cast<int2*>(static_cast<char*>(workspace) + kWsAlign +
+                                           align_up(size_t(tiles) * 8, kWsAlign));
     {
-        const size_t n16 = need / 16;
-        const int blocks = int(std::min<size_t>((n16 + 255) / 256, 64));
-        select_clear_kernel<<<blocks, 256, 0, s>>>(counts, static_cast<uint4*>(workspace), n16);
+        const int in_smem = B <= kSelClearSmemMaxB;
+        const size_t smem = in_smem ? (size_t(B) + 1) * sizeof(int32_t) : 0;
+        if (smem > 48 * 1024)       // (an attribute of the function on the current device; the call is cheap)
+            TPPO_CUDA_CHECK(cudaFuncSetAttribute(select_clear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (kSelClearSmemMaxB + 1) * int(sizeof(int32_t))));
+        select_clear_kernel<<<(tiles + kSelClearThreads - 1) / kSelClearThreads, kSelClearThreads, smem, s>>>(
+            counts, static_cast<uint32_t*>(workspace), state, window, tiles, seq_begin, B, N, in_smem);
         TPPO_CUDA_CHECK(cudaGetLastError());
     }
     SelectArgs a;
@@ -393,10 +395,11 @@ TPPO_API int tppo_select_tokens(const int32_t* seq_begin, const int32_t* prompt_
     a.out_vec_ok = aligned(policy_idx, 16) && aligned(value_idx, 16);
     a.mask_vec_ok = (!extra_policy_mask || aligned(extra_policy_mask, 16)) &&
                     (!extra_value_mask || aligned(extra_value_mask, 16));
-    a.num_tiles = int32_t((N + kSelTile - 1) / kSelTile);
+    a.num_tiles = tiles;
     a.policy_idx = policy_idx; a.value_idx = value_idx; a.counts = counts;
     a.ticket = static_cast<uint32_t*>(workspace);
-    a.state = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWsAlign);
+    a.state = state;
+    a.window = window;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(unsigned(a.num_tiles));
     cfg.blockDim = dim3(kSelThreads);
