@@ -954,7 +954,8 @@ def run_lmhead_workload(args, rank, world, local, dev, warmup):
 # kernel plus the kernel that zero-fills dvalues, the slot walk plus the copy kernel.  None once a
 # kernel has changed since.
 NCU_CFG4_TRAFFIC = {"egae": 140769536 + 94864896, "select": 35140608 + 726784,
-                    "value": 145093888 + 21591040 + 7936 + 7788544, "advance": 43353088 + 1300736 + 78592}
+                    "value": None,      # the value kernel's launch shape has changed since the capture
+                    "advance": 43353088 + 1300736 + 78592}
 
 
 def measure_cfg4(dev, steps, warmup):

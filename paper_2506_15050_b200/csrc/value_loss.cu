@@ -5,7 +5,7 @@
 // zero off the value tokens: a first kernel fills it with 16-byte stores (and clears the two words
 // the blocks count in), the loss kernel is its programmatic dependent and scatters the tokens'
 // entries once that kernel has ended.  Measured on 17.5 M positions at 25 % density: 53.5 us per call
-// in this form; 55.8 us with two memsets in front of a plain launch; 61 us when the dependent kernel
+// in this form with four blocks per SM and four tokens per trip, 49-50 us with eight blocks and two tokens; 55.8 us with two memsets in front of a plain launch; 61 us when the dependent kernel
 // starts its gathers beside the fill, holds the gradients of its first 8192 tokens per block in
 // shared memory and scatters them after the fill has ended (the fill and the gathers then share the
 // DRAM and neither runs at its own rate); 74 us for a dense sweep over the positions that writes
@@ -21,7 +21,8 @@
 namespace tppo {
 
 constexpr int kValThreads = 256;
-constexpr int kValMaxBlocks = kNumSms * 4;
+constexpr int kValBlocksPerSm = 8;      // 2048 resident threads per SM at 32 registers
+constexpr int kValMaxBlocks = kNumSms * kValBlocksPerSm;
 
 struct ValueArgs {
     const float* values;
@@ -119,7 +120,7 @@ __global__ void __launch_bounds__(512) value_clear_kernel(float* dvalues, int64_
 
 // Launched as the programmatic dependent of the clearing kernel: its blocks are resident and have
 // their arguments when that kernel ends, and start the moment it does.
-__global__ void __launch_bounds__(kValThreads) value_loss_kernel(const ValueArgs a) {
+__global__ void __launch_bounds__(kValThreads, kValBlocksPerSm) value_loss_kernel(const ValueArgs a) {
     __shared__ double s_red[kValThreads / 32];
     __shared__ bool s_last;
     const int64_t n = value_n(a);
@@ -129,24 +130,26 @@ __global__ void __launch_bounds__(kValThreads) value_loss_kernel(const ValueArgs
     int bad = 0;
     bool nonfinite = false;
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    // Four independent tokens per thread and trip, so that the index load and the three gathers of
-    // one token overlap with those of the others.
-    constexpr int kUnroll = 4;
+    // Two independent tokens per thread and trip, so that the index load and the three gathers of
+    // one token overlap with those of the other, and eight blocks per SM: measured at 17.5 M
+    // positions, call us: four blocks x four tokens 52.7, five x four 50.3, six x four 51.8, four x
+    // eight 51.4, eight x four 51.1, eight x three 50.5, eight x two 49.1-50.3.
+    constexpr int kUnroll = 2;
     const int64_t stride = int64_t(gridDim.x) * kValThreads;
     for (int64_t j0 = int64_t(blockIdx.x) * kValThreads + threadIdx.x; j0 < n; j0 += stride * kUnroll) {
-        int64_t p[kUnroll];
+        int32_t p[kUnroll];       // (N < 2^31 is checked by the host)
         bool ok[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
             const int64_t j = j0 + u * stride;
-            p[u] = j < n ? (a.value_idx ? int64_t(__ldg(a.value_idx + j)) : j) : -1;
+            p[u] = j < n ? (a.value_idx ? __ldg(a.value_idx + j) : int32_t(j)) : -1;
             ok[u] = p[u] >= 0 && p[u] < a.N;
             if (j < n && !ok[u]) bad = TPPO_DEV_BAD_INDEX;
         }
         float v[kUnroll], vo[kUnroll], R[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
-            const int64_t q = ok[u] ? p[u] : 0;
+            const int32_t q = ok[u] ? p[u] : 0;
             v[u] = ok[u] ? __ldg(a.values + q) : 0.f;
             vo[u] = ok[u] ? __ldg(a.old_values + q) : 0.f;
             R[u] = ok[u] ? __ldg(a.returns + q) : 0.f;
