@@ -953,9 +953,8 @@ def run_lmhead_workload(args, rank, world, local, dev, warmup):
 # profiles/egae_select_value_advance_cfg4.md): the scan kernel, the selection kernel, the value
 # kernel plus the kernel that zero-fills dvalues, the slot walk plus the copy kernel.  None once a
 # kernel has changed since.
-NCU_CFG4_TRAFFIC = {"egae": 140769536 + 94864896, "select": 35140608 + 726784,
-                    "value": None,      # the value kernel's launch shape has changed since the capture
-                    "advance": 43353088 + 1300736 + 78592}
+NCU_CFG4_TRAFFIC = {"egae": 140726784 + 94525696, "select": 35154688 + 814592,
+                    "value": 145664768 + 22165504 + 7424 + 7357440, "advance": 43357184 + 1402880 + 78592}
 
 
 def measure_cfg4(dev, steps, warmup):
