@@ -954,7 +954,7 @@ def run_lmhead_workload(args, rank, world, local, dev, warmup):
 # kernel plus the kernel that zero-fills dvalues, the slot walk plus the copy kernel.  None once a
 # kernel has changed since.
 NCU_CFG4_TRAFFIC = {"egae": 140726784 + 94525696, "select": 35154688 + 814592,
-                    "value": 145664768 + 22165504 + 7424 + 7357440, "advance": 43357184 + 1402880 + 78592}
+                    "value": 145664768 + 22165504 + 7424 + 7357440, "advance": None}      # the copy kernel has changed since the capture
 
 
 def measure_cfg4(dev, steps, warmup):

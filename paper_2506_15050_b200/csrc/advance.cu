@@ -5,6 +5,7 @@
 // slots, then the packed offsets of the next step's context), then a bandwidth-bound ragged copy
 // moves the kept sequences and the queued prompts into the new packed token buffer.  Integer work
 // throughout: bit-exact and run-to-run identical.
+#include <algorithm>
 #include "common.cuh"
 
 namespace tppo {
@@ -72,20 +73,47 @@ __global__ void __launch_bounds__(kAdvSlotThreads) advance_slots_kernel(const Ad
     asm volatile("griddepcontrol.launch_dependents;");
     long long free_base = 0, pos_base = 0;
     int bad = 0;
+    // a thread's four slots as one 16-byte access per array where the arrays allow it (the scalar
+    // form's stores, 16 bytes apart between lanes, took 4 of the walk's 9 us at 4096 slots)
+    const bool vec = (a.B & 3) == 0 &&
+                     ((reinterpret_cast<uintptr_t>(a.prompt_len) | reinterpret_cast<uintptr_t>(a.prev_len) |
+                       reinterpret_cast<uintptr_t>(a.new_len) | reinterpret_cast<uintptr_t>(a.next_prompt_len) |
+                       reinterpret_cast<uintptr_t>(a.next_prev_len) | reinterpret_cast<uintptr_t>(a.slot_source) |
+                       reinterpret_cast<uintptr_t>(a.next_seq_begin)) & 15) == 0 &&
+                     (reinterpret_cast<uintptr_t>(a.truncated) & 3) == 0;
     for (int c0 = 0; c0 < a.B; c0 += kAdvSlotThreads * kAdvSlotItems) {
         const int i0 = c0 + int(threadIdx.x) * kAdvSlotItems;
         bool valid[kAdvSlotItems], fin[kAdvSlotItems];
         long long p[kAdvSlotItems], q[kAdvSlotItems], n[kAdvSlotItems];
         int my_fin = 0;
+        static_assert(kAdvSlotItems == 4, "one 16-byte access per array and thread");
+        if (vec) {
+            const bool in = i0 < a.B;       // all four or none
+            const uint32_t t4 = in ? __ldg(reinterpret_cast<const uint32_t*>(a.truncated + i0)) : 0u;
+            const int4 z = make_int4(0, 0, 0, 0);
+            const int4 p4 = in ? __ldg(reinterpret_cast<const int4*>(a.prompt_len + i0)) : z;
+            const int4 q4 = in ? __ldg(reinterpret_cast<const int4*>(a.prev_len + i0)) : z;
+            const int4 n4 = in ? __ldg(reinterpret_cast<const int4*>(a.new_len + i0)) : z;
+            const int pp[4] = {p4.x, p4.y, p4.z, p4.w}, qq[4] = {q4.x, q4.y, q4.z, q4.w},
+                      nn[4] = {n4.x, n4.y, n4.z, n4.w};
 #pragma unroll
-        for (int u = 0; u < kAdvSlotItems; ++u) {
-            const int i = i0 + u;
-            valid[u] = i < a.B;
-            fin[u] = valid[u] && __ldg(a.truncated + i) == 0;
-            p[u] = valid[u] ? __ldg(a.prompt_len + i) : 0;
-            q[u] = valid[u] ? __ldg(a.prev_len + i) : 0;
-            n[u] = valid[u] ? __ldg(a.new_len + i) : 0;
-            my_fin += fin[u];
+            for (int u = 0; u < kAdvSlotItems; ++u) {
+                valid[u] = in;
+                fin[u] = in && ((t4 >> (8 * u)) & 0xffu) == 0;
+                p[u] = pp[u]; q[u] = qq[u]; n[u] = nn[u];
+                my_fin += fin[u];
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < kAdvSlotItems; ++u) {
+                const int i = i0 + u;
+                valid[u] = i < a.B;
+                fin[u] = valid[u] && __ldg(a.truncated + i) == 0;
+                p[u] = valid[u] ? __ldg(a.prompt_len + i) : 0;
+                q[u] = valid[u] ? __ldg(a.prev_len + i) : 0;
+                n[u] = valid[u] ? __ldg(a.new_len + i) : 0;
+                my_fin += fin[u];
+            }
         }
         long long n_fin;
         long long rank = free_base + block_exclusive_sum<long long>(my_fin, s_scan, n_fin);
@@ -118,15 +146,30 @@ __global__ void __launch_bounds__(kAdvSlotThreads) advance_slots_kernel(const Ad
         }
         long long n_tok;
         long long begin = pos_base + block_exclusive_sum<long long>(my_len, s_scan, n_tok);
+        if (vec) {
+            if (valid[0]) {
+                int32_t nb[kAdvSlotItems];
 #pragma unroll
-        for (int u = 0; u < kAdvSlotItems; ++u) {
-            if (valid[u]) {
-                const int i = i0 + u;
-                a.next_prompt_len[i] = pl[u];
-                a.next_prev_len[i] = pv[u];
-                a.slot_source[i] = src[u];
-                a.next_seq_begin[i] = int32_t(begin < 0x7fffffffll ? begin : 0x7fffffffll);
-                begin += len[u];
+                for (int u = 0; u < kAdvSlotItems; ++u) {
+                    nb[u] = int32_t(begin < 0x7fffffffll ? begin : 0x7fffffffll);
+                    begin += len[u];
+                }
+                *reinterpret_cast<int4*>(a.next_prompt_len + i0) = make_int4(pl[0], pl[1], pl[2], pl[3]);
+                *reinterpret_cast<int4*>(a.next_prev_len + i0) = make_int4(pv[0], pv[1], pv[2], pv[3]);
+                *reinterpret_cast<int4*>(a.slot_source + i0) = make_int4(src[0], src[1], src[2], src[3]);
+                *reinterpret_cast<int4*>(a.next_seq_begin + i0) = make_int4(nb[0], nb[1], nb[2], nb[3]);
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < kAdvSlotItems; ++u) {
+                if (valid[u]) {
+                    const int i = i0 + u;
+                    a.next_prompt_len[i] = pl[u];
+                    a.next_prev_len[i] = pv[u];
+                    a.slot_source[i] = src[u];
+                    a.next_seq_begin[i] = int32_t(begin < 0x7fffffffll ? begin : 0x7fffffffll);
+                    begin += len[u];
+                }
             }
         }
         free_base += n_fin;
@@ -166,7 +209,8 @@ __device__ __forceinline__ int adv_warp_count_le(const int32_t* arr, int n, int3
     return lo;
 }
 
-// Ragged copy into the next step's packed context.  A block owns 8192 consecutive output positions.
+// Ragged copy into the next step's packed context.  A block owns one stretch of consecutive output
+// positions (an even share of the context, at least 8192).
 // It finds the first slot that reaches into them (one warp-wide search), puts the slots of its range
 // into a small shared-memory table -- where each begins in the output and a source pointer already
 // shifted so that source = pointer[output position], null for a slot whose source range is not inside
@@ -207,9 +251,15 @@ __global__ void __launch_bounds__(kAdvCopyThreads, 6) advance_copy_kernel(const 
     // scheduling, the parameter fetch) overlaps with it; its results are read only after the wait
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t total = min(int64_t(a.next_seq_begin[a.B]), a.capacity);
-    const int64_t t0 = int64_t(blockIdx.x) * kAdvCopyTile;
+    // The grid is sized on the host for what the output buffer can hold, at most one wave of resident
+    // blocks; the context actually written is split evenly between them (one slot search and one
+    // table per block, no ragged last wave), in stretches that are a multiple of four positions so
+    // that the 16-byte stores stay aligned, and of at least a tile.
+    int64_t per = (total + gridDim.x - 1) / gridDim.x;
+    per = max((per + 3) & ~int64_t(3), int64_t(kAdvCopyTile));
+    const int64_t t0 = int64_t(blockIdx.x) * per;
     if (t0 >= total) return;
-    const int64_t t1 = min(t0 + kAdvCopyTile, total);
+    const int64_t t1 = min(t0 + per, total);
     if (threadIdx.x < 32) {
         const int c = adv_warp_count_le(a.next_seq_begin, a.B + 1, int32_t(t0), threadIdx.x);
         if (threadIdx.x == 0) s_slot0 = c - 1;      // last slot that begins at or before t0
@@ -233,16 +283,17 @@ __global__ void __launch_bounds__(kAdvCopyThreads, 6) advance_copy_kernel(const 
     const bool table_ok = int64_t(s_begin[kAdvTable]) >= t1 || slot0 + kAdvTable >= a.B;
     const bool vec = (reinterpret_cast<uintptr_t>(a.next_tokens) & 15) == 0;
     if (table_ok && vec) {
-        // two groups of four positions per trip, all eight loads issued before the first store
+        // kGroups groups of four positions per trip, all their loads issued before the first store
         const int n_slots = min(kAdvTable, a.B - slot0);          // table entries in use
         const int32_t e1 = int32_t(t1);
         int h = 0;
         constexpr int kStep = 4 * kAdvCopyThreads;
-        for (int32_t p0 = int32_t(t0) + 4 * threadIdx.x; p0 < e1; p0 += 2 * kStep) {
-            int4 v[2];
-            bool whole[2];
+        constexpr int kGroups = 2;      // (3, 4 and 6 groups in flight measured the same: 30.2-31.1 us per call)
+        for (int32_t p0 = int32_t(t0) + 4 * threadIdx.x; p0 < e1; p0 += kGroups * kStep) {
+            int4 v[kGroups];
+            bool whole[kGroups];
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
+            for (int u = 0; u < kGroups; ++u) {
                 const int32_t p = p0 + u * kStep;
                 v[u] = make_int4(0, 0, 0, 0);
                 whole[u] = false;
@@ -258,7 +309,7 @@ __global__ void __launch_bounds__(kAdvCopyThreads, 6) advance_copy_kernel(const 
                 }
             }
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
+            for (int u = 0; u < kGroups; ++u) {
                 const int32_t p = p0 + u * kStep;
                 if (p >= e1) continue;
                 if (whole[u]) {
@@ -322,7 +373,8 @@ TPPO_API int tppo_advance_batch(const int32_t* seq_begin, const int32_t* prompt_
         // the number of context tokens is only known on the device: size the grid for the most the
         // output buffer can hold; CTAs past the end return at once
         int64_t upper = N + queue_total < capacity ? N + queue_total : capacity;
-        const int64_t tiles = (upper + kAdvCopyTile - 1) / kAdvCopyTile;
+        int64_t tiles = (upper + kAdvCopyTile - 1) / kAdvCopyTile;
+        tiles = std::min<int64_t>(tiles, int64_t(kNumSms) * 6);       // one wave of resident blocks
         if (tiles > 0) {
             // programmatic dependent launch: the copy kernel's blocks are scheduled while the slot
             // walk still runs and wait inside the kernel for its results
