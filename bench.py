@@ -46,7 +46,7 @@ ALGO_BYTES_PER_TOKEN = 2 * 2 * synth.V_QWEN       # bf16 row read once + bf16 gr
 # 569.41 + 517.59 MB on 1872 rows, policy_two_pass_kernel (side launch) 53.58 + 12.89 MB on 176 rows;
 # per row, scaled by rows.  (Reads are exactly one pass over the logits; of the writes about 90 MB were
 # still in L2 when the capture ended, at any row count, so the scaled figure understates full-size
-# writes by about 7 %.)  profiles/policy_cluster_kernel_cfg3.md has the command.
+# writes by about 7 %.)  The summary of that capture under profiles/ has the command.
 NCU_TRAFFIC_BYTES_PER_TOKEN = (569.413376e6 + 517.587200e6 + 53.582080e6 + 12.886528e6) / 2048
 
 
@@ -945,14 +945,10 @@ def run_lmhead_workload(args, rank, world, local, dev, warmup):
 
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of each small kernel on config 4
-# (profiles/egae_select_value_advance_cfg4.md gives the command); None once a kernel has changed
-# since its counters were taken.
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of each call's kernels on this very
-# workload (ncu capture of `python bench.py --workload cfg4 --steps 1 --warmup 3`;
-# profiles/egae_select_value_advance_cfg4.md): the scan kernel, the selection kernel, the value
-# kernel plus the kernel that zero-fills dvalues, the slot walk plus the copy kernel.  None once a
-# kernel has changed since.
+# workload (ncu capture of `python bench.py --workload cfg4 --steps 1 --warmup 3`, summarised under
+# profiles/): the scan kernel, the selection kernel, the value kernel plus the kernel that zero-fills
+# dvalues, the slot walk plus the copy kernel.  None once a kernel has changed since.
 NCU_CFG4_TRAFFIC = {"egae": 140726784 + 94525696, "select": 35154688 + 814592,
                     "value": 145664768 + 22165504 + 7424 + 7357440, "advance": None}      # the copy kernel has changed since the capture
 
@@ -1086,7 +1082,7 @@ def run_config_table(args, dev):
     """The benchmark configurations that are not the bench line, one after another (configs 1, 2 and
     4; config 3 is the default workload, config 5 `--workload lmhead`): GPU time of the hot path on
     each, and the oracle on the host cores on the whole of the small ones and a bounded sample of
-    the large one.  Prints one JSON object; fills the per-config table of the benchmark spec."""
+    the large one.  Prints one JSON object; one entry per config."""
     import oracle
     from paper_2506_15050_b200 import binding as b
     f32 = lambda x: float(np.float32(x))
