@@ -950,7 +950,7 @@ def run_lmhead_workload(args, rank, world, local, dev, warmup):
 # profiles/): the scan kernel, the selection kernel, the value kernel plus the kernel that zero-fills
 # dvalues, the slot walk plus the copy kernel.  None once a kernel has changed since.
 NCU_CFG4_TRAFFIC = {"egae": 140726784 + 94525696, "select": 35154688 + 814592,
-                    "value": 145664768 + 22165504 + 7424 + 7357440, "advance": None}      # the copy kernel has changed since the capture
+                    "value": 145664768 + 22165504 + 7424 + 7357440, "advance": 43368192 + 1502720 + 80896}
 
 
 def measure_cfg4(dev, steps, warmup):
