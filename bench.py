@@ -949,8 +949,8 @@ def run_lmhead_workload(args, rank, world, local, dev, warmup):
 # workload (ncu capture of `python bench.py --workload cfg4 --steps 1 --warmup 3`, summarised under
 # profiles/): the scan kernel, the selection kernel, the value kernel plus the kernel that zero-fills
 # dvalues, the slot walk plus the copy kernel.  None once a kernel has changed since.
-NCU_CFG4_TRAFFIC = {"egae": 140726784 + 94525696, "select": 35154688 + 814592,
-                    "value": 145664768 + 22165504 + 7424 + 7357440, "advance": 43368192 + 1502720 + 80896}
+NCU_CFG4_TRAFFIC = {"egae": 140728064 + 94136576, "select": 35152896 + 814336,
+                    "value": 145394688 + 21827072 + 7424 + 7879168, "advance": 43362048 + 1535232 + 80896}
 
 
 def measure_cfg4(dev, steps, warmup):

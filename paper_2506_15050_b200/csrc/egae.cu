@@ -763,6 +763,18 @@ egae_scan_kernel(const EgaeArgs a, const __grid_constant__ CUtensorMap map_r,
             }
         }
     }
+    // ... and asks for the inputs of the tile that a block a quarter wave later will take to be
+    // brought into L2 now, so that its copy is served from there (tppo_egae at 17.5 M tokens: none
+    // 81.0 us; 37 / 74 / 148 / 222 / 296 / 444 / 592 / 888 / 1184 / 2368 tiles ahead 77.0 / 76.3 / 76.2 /
+    // 75.6-76.5 / 75.6-75.9 / 76.4 / 76.5-76.8 / 77.8 / 78.1 / 83.6)
+#ifndef TPPO_SCAN_PREFETCH_TILES
+#define TPPO_SCAN_PREFETCH_TILES (2 * kNumSms)
+#endif
+    if (threadIdx.x == 32 && a.tma_ok && TPPO_SCAN_PREFETCH_TILES > 0 && tile >= TPPO_SCAN_PREFETCH_TILES) {
+        const int64_t q0 = int64_t(tile - TPPO_SCAN_PREFETCH_TILES) * (H * kScanTile);
+        ptx::bulk_prefetch_l2(a.rewards + q0, H * kScanTile * uint32_t(sizeof(float)));
+        ptx::bulk_prefetch_l2(a.values + q0, H * kScanTile * uint32_t(sizeof(float)));
+    }
 #pragma unroll
     for (int p = 0; p < H; ++p) {
         const int64_t t0 = tile0 + int64_t(p) * kScanTile;

@@ -82,6 +82,10 @@ __device__ __forceinline__ void bulk_store(void* dst_gmem, uint32_t src_smem, ui
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                  ::"l"(dst_gmem), "r"(src_smem), "r"(bytes) : "memory");
 }
+// Hint: bring `bytes` of global memory (16-byte aligned, a multiple of 16) into L2.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src_gmem, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src_gmem), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() {

@@ -5,6 +5,7 @@
 // in ascending order.  Integer work throughout: the result is bit-exact and run-to-run identical.
 #include <algorithm>
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace tppo {
 
@@ -155,6 +156,17 @@ __global__ void __launch_bounds__(kSelThreads, 6) select_tokens_kernel(const Sel
         if (a.val_mask) {
             vm_bits = 0;
             for (int k = 0; k < n_mine; ++k) vm_bits |= uint32_t(__ldg(a.val_mask + p0 + k) != 0) << k;
+        }
+    }
+    // ... and ask for the mask bytes of a tile that a later block will take to be brought into L2
+#ifndef TPPO_SEL_PREFETCH_TILES
+#define TPPO_SEL_PREFETCH_TILES (2 * kNumSms)
+#endif
+    if (threadIdx.x == 64 && TPPO_SEL_PREFETCH_TILES > 0 && a.mask_vec_ok) {
+        const int64_t q0 = (int64_t(tile) + TPPO_SEL_PREFETCH_TILES) * kSelTile;
+        if (q0 + kSelTile <= a.N) {
+            if (a.pol_mask) ptx::bulk_prefetch_l2(a.pol_mask + q0, kSelTile);
+            if (a.val_mask) ptx::bulk_prefetch_l2(a.val_mask + q0, kSelTile);
         }
     }
     const uint32_t own_bits = n_mine >= kSelItems ? 0xffffffffu : ((1u << n_mine) - 1u);

@@ -129,23 +129,37 @@ __global__ void __launch_bounds__(kValThreads, kValBlocksPerSm) value_loss_kerne
     double acc = 0.0;
     int bad = 0;
     bool nonfinite = false;
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     // Two independent tokens per thread and trip, so that the index load and the three gathers of
     // one token overlap with those of the other, and eight blocks per SM: measured at 17.5 M
     // positions, call us: four blocks x four tokens 52.7, five x four 50.3, six x four 51.8, four x
-    // eight 51.4, eight x four 51.1, eight x three 50.5, eight x two 49.1-50.3.
+    // eight 51.4, eight x four 51.1, eight x three 50.5, eight x two 49.1-50.3.  The indices of a trip
+    // are loaded one trip ahead (those of the first trip before the wait for the clearing kernel,
+    // which writes nothing this kernel reads before it), so that a trip's gathers start at once:
+    // 50.8 -> 48.3-49.3 us.  (Indices two trips ahead plus an L2 prefetch of the next trip's three
+    // gathers: 49.5-50.2, dropped.)
     constexpr int kUnroll = 2;
     const int64_t stride = int64_t(gridDim.x) * kValThreads;
-    for (int64_t j0 = int64_t(blockIdx.x) * kValThreads + threadIdx.x; j0 < n; j0 += stride * kUnroll) {
-        int32_t p[kUnroll];       // (N < 2^31 is checked by the host)
-        bool ok[kUnroll];
+    auto load_indices = [&](int64_t j0, int32_t (&p)[kUnroll]) {       // (N < 2^31 is checked by the host)
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
             const int64_t j = j0 + u * stride;
             p[u] = j < n ? (a.value_idx ? __ldg(a.value_idx + j) : int32_t(j)) : -1;
-            ok[u] = p[u] >= 0 && p[u] < a.N;
-            if (j < n && !ok[u]) bad = TPPO_DEV_BAD_INDEX;
         }
+    };
+    int64_t j0 = int64_t(blockIdx.x) * kValThreads + threadIdx.x;
+    int32_t p_next[kUnroll];
+    load_indices(j0, p_next);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (; j0 < n; j0 += stride * kUnroll) {
+        int32_t p[kUnroll];
+        bool ok[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            p[u] = p_next[u];
+            ok[u] = p[u] >= 0 && p[u] < a.N;
+            if (j0 + u * stride < n && !ok[u]) bad = TPPO_DEV_BAD_INDEX;
+        }
+        load_indices(j0 + stride * kUnroll, p_next);
         float v[kUnroll], vo[kUnroll], R[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
