@@ -703,3 +703,27 @@ def test_select_and_egae_many_tiny_sequences():
     boot = rng.standard_normal(B).astype(np.float32)
     check_egae(B, r, v, seg_b, seg_e, trunc, boot, 0.99, 0.95)
     check_egae(B, r, v, seg_b, seg_e, trunc, None, 1.0, 1.0)
+
+
+# more sequences than the clearing kernels stage in shared memory (12288 segments for the scan,
+# 24575 sequence starts for the selection): their window searches then read the global arrays
+def test_select_and_egae_more_sequences_than_the_clearing_kernels_stage():
+    rng = np.random.default_rng(21)
+    B = 26000
+    prompt = rng.integers(0, 4, B)
+    prev = rng.integers(0, 5, B) * rng.integers(0, 2, B)
+    new = rng.integers(0, 24, B)
+    trunc = rng.integers(0, 2, B).astype(np.uint8)
+    sb, seg_b, seg_e = synth.pack(prompt, prev, new)
+    N = int(sb[-1])
+    assert N > 8 * 8192                          # several tiles of either kernel
+    c = dict(seq_begin=sb, prompt_len=prompt, prev_len=prev, new_len=new, truncated=trunc)
+    pm = rng.integers(0, 2, N).astype(np.uint8)
+    vm = rng.integers(0, 2, N).astype(np.uint8)
+    check_select(c, tail_drop=2)
+    check_select(c, 1, pm, vm)
+    r = rng.standard_normal(N).astype(np.float32)
+    v = rng.standard_normal(N).astype(np.float32)
+    boot = rng.standard_normal(B).astype(np.float32)
+    check_egae(B, r, v, seg_b, seg_e, trunc, boot, 0.99, 0.95)
+    check_egae(B, r, v, seg_b, seg_e, trunc, None, 1.0, 0.9)
