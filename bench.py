@@ -240,6 +240,10 @@ class Step:
         self.ws_val = b.workspace(b.OP_VALUE_LOSS, N, 0, N, 0, dev)
         self.ev = None
         self.hint = 0
+        # EGAE and the token selection read the same inputs and write disjoint outputs: the selection
+        # runs on a second stream beside the scan (both are chains of latencies, not bandwidth)
+        self.side = torch.cuda.Stream(device=dev)
+        self.overlap = True
         self.denom_pol = 0.0      # > 0: selected-token counts of the whole job (several GPUs)
         self.denom_val = 0.0
         # old-policy log-probs (the old-policy snapshot of Algorithm 1): forward-only pass of the same kernel, plus noise
@@ -277,17 +281,31 @@ class Step:
     def run(self, events=None):
         """One step.  With `events` (a list), five CUDA events are recorded around the four calls and
         appended as one tuple: the calls' device times come out of the same run that is timed."""
-        if events is None:
+        timed = events is not None
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)] if timed else None
+        if timed:
+            ev[0].record()
+        if self.overlap:
+            main = torch.cuda.current_stream()
+            fork, join = torch.cuda.Event(), torch.cuda.Event()
+            fork.record(main)
+            self.side.wait_event(fork)
+            with torch.cuda.stream(self.side):
+                self.select()
+                join.record(self.side)
             self.egae()
+            if timed:
+                ev[1].record()
+            main.wait_event(join)       # ev[1] -> ev[2]: what of the selection is left after the scan
+        else:
+            self.egae()
+            if timed:
+                ev[1].record()
             self.select()
+        if not timed:
             self.policy()
             self.value()
             return
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
-        ev[0].record()
-        self.egae()
-        ev[1].record()
-        self.select()
         ev[2].record()
         self.policy()
         ev[3].record()
@@ -542,6 +560,8 @@ def main():
     ap.add_argument("--lm-rows", type=int, default=16384,
                     help="rows of the LM-head workload (smaller only for profiler captures)")
     ap.add_argument("--cfg4-steps", type=int, default=30, help="steps of the small-kernel measurement")
+    ap.add_argument("--serial", action="store_true",
+                    help="run the token selection after EGAE on the same stream instead of beside it")
     ap.add_argument("--no-lmhead", action="store_true")
     ap.add_argument("--no-small", action="store_true", help="skip the config-4 small-kernel measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -577,6 +597,7 @@ def main():
         run_config_table(args, dev)
         return
     st = Step(dev, seed=2 + rank, rows=args.rows)      # every rank holds its own batch
+    st.overlap = not args.serial
     st.hint = args.hint
     if world > 1:
         # token-level mean over the whole job: each rank divides by the global selected-token counts
@@ -619,8 +640,9 @@ def main():
     assert n_tok == st.n and int(st.stats[3].item()) == 0 and int(st.status.item()) == 0
     value = world * n_tok / (ms_step * 1e-3)
     pol = time_stats([e[2].elapsed_time(e[3]) for e in events])
+    sel_name = "select_after_egae (the selection runs beside the scan on a second stream)" if st.overlap else "select"
     calls_us = {name: time_stats([e[k].elapsed_time(e[k + 1]) * 1e3 for e in events])
-                for k, name in enumerate(("egae", "select", "policy", "value"))}
+                for k, name in enumerate(("egae", sel_name, "policy", "value"))}
     pol_ms = pol["mean"]
     peak, peak_kind = measured_peaks()
     algo_bytes = n_tok * ALGO_BYTES_PER_TOKEN
